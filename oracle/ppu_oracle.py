@@ -1,0 +1,540 @@
+"""CPU oracle for the partial-parameter-update training step.
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain reference that the
+tests, the smoke check and the benchmark's CPU-baseline leg compare the CUDA
+library against.  The product never imports it and it imports nothing from the
+product; it shares no layout code, tables or helpers with the CUDA sources.
+
+What it computes, all in numpy (float64 unless a dtype is passed), following
+"Partial Parameter Updates for Efficient Distributed Training":
+
+* the decoder forward pass on all parameters and the loss of Eq. 2.2;
+* the gradient of Algorithm 1 line 9 in two ways: the definition (full
+  backward, then mask to the trainable index set) and the restricted backward
+  of Appendix C.1 (weight gradients only for the trained FFN slice, input
+  gradients through every slice, nothing below the lowest trained layer);
+* the inner AdamW update on the subset (Algorithm 1 line 10, Section 3.1);
+* per-node deltas, the count vector m, the count-normalised average and the
+  outer Nesterov step (Algorithm 1 lines 12-15, Eq. 2.4-2.5);
+* the closed-form parameter and FLOP counts of Table 1 and Appendix C.2.
+
+numpy's matmul is the only library primitive used as a step.  There is no
+blocking, fusion or reordering beyond what the equations state.
+
+Conventions the paper leaves open (all stated again in the design notes):
+weights are stored [out, in] (y = x W^T), so the paper's W in R^{4d x d} is
+W_in and V in R^{d x 4d} is W_out; pre-LayerNorm blocks; GELU in its tanh form;
+rotary positions on adjacent pairs with base 1e4; tied input/output embedding;
+no linear biases; loss = mean over the B*(S-1) predicted tokens; AdamW with
+bias correction and eps = 1e-8; Nesterov in the "buf = mu*buf + g, step with
+g + mu*buf" form with g = -Delta.
+
+Parity pins live in tests/test_oracle_*.py.  Conventions above that no printed
+number fixes (GELU variant, RoPE pairing, eps values, Nesterov form) are
+"parity unpinned" against the authors' own code; every function's arithmetic
+is pinned against finite differences, closed forms or textbook special cases.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+import math
+import numpy as np
+
+
+# --------------------------------------------------------------------------
+# configuration and canonical parameter layout
+# --------------------------------------------------------------------------
+@dataclass
+class Model:
+    n_layer: int
+    d_model: int
+    n_head: int
+    d_ff: int
+    vocab: int
+    ln_eps: float = 1e-5
+    rope_base: float = 1e4
+
+    @property
+    def d_head(self) -> int:
+        return self.d_model // self.n_head
+
+
+@dataclass
+class AdamW:
+    lr: float = 1e-3
+    beta1: float = 0.9
+    beta2: float = 0.95
+    eps: float = 1e-8
+    wd: float = 0.1
+
+
+@dataclass
+class Outer:
+    lr: float = 0.7
+    momentum: float = 0.9
+
+
+def layout(cfg: Model):
+    """Ordered (name, offset, shape) records of the flat parameter vector.
+
+    E [V,d]; per layer ln1_g, ln1_b, W_q, W_k, W_v, W_o (each [d,d], out x in),
+    ln2_g, ln2_b, W_in [F,d], W_out [d,F]; then lnf_g, lnf_b.  W_in / W_out are
+    the paper's W and V of Section 2.2.1.
+    """
+    d, F, V = cfg.d_model, cfg.d_ff, cfg.vocab
+    recs, off = [], 0
+
+    def add(name, shape):
+        nonlocal off
+        recs.append((name, off, tuple(shape)))
+        off += int(np.prod(shape))
+
+    add("E", (V, d))
+    for l in range(cfg.n_layer):
+        p = f"l{l}."
+        add(p + "ln1_g", (d,)); add(p + "ln1_b", (d,))
+        add(p + "W_q", (d, d)); add(p + "W_k", (d, d)); add(p + "W_v", (d, d))
+        add(p + "W_o", (d, d))
+        add(p + "ln2_g", (d,)); add(p + "ln2_b", (d,))
+        add(p + "W_in", (F, d)); add(p + "W_out", (d, F))
+    add("lnf_g", (d,)); add("lnf_b", (d,))
+    return recs
+
+
+def n_params(cfg: Model) -> int:
+    recs = layout(cfg)
+    name, off, shape = recs[-1]
+    return off + int(np.prod(shape))
+
+
+def views(cfg: Model, theta: np.ndarray) -> dict:
+    """name -> reshaped view into theta (no copies)."""
+    return {name: theta[off:off + int(np.prod(shape))].reshape(shape)
+            for name, off, shape in layout(cfg)}
+
+
+# --------------------------------------------------------------------------
+# elementwise pieces
+# --------------------------------------------------------------------------
+_GELU_C = math.sqrt(2.0 / math.pi)
+_GELU_A = 0.044715
+
+
+def gelu(x):
+    return 0.5 * x * (1.0 + np.tanh(_GELU_C * (x + _GELU_A * x * x * x)))
+
+
+def gelu_grad(x):
+    u = _GELU_C * (x + _GELU_A * x * x * x)
+    t = np.tanh(u)
+    du = _GELU_C * (1.0 + 3.0 * _GELU_A * x * x)
+    return 0.5 * (1.0 + t) + 0.5 * x * (1.0 - t * t) * du
+
+
+def layernorm(x, g, b, eps):
+    mu = x.mean(axis=-1, keepdims=True)
+    var = ((x - mu) ** 2).mean(axis=-1, keepdims=True)
+    rstd = 1.0 / np.sqrt(var + eps)
+    xhat = (x - mu) * rstd
+    return xhat * g + b, (xhat, rstd)
+
+
+def layernorm_bwd(dy, g, cache):
+    """Returns dx, dgamma, dbeta."""
+    xhat, rstd = cache
+    dyg = dy * g
+    m1 = dyg.mean(axis=-1, keepdims=True)
+    m2 = (dyg * xhat).mean(axis=-1, keepdims=True)
+    dx = rstd * (dyg - m1 - xhat * m2)
+    red = tuple(range(dy.ndim - 1))
+    return dx, (dy * xhat).sum(axis=red), dy.sum(axis=red)
+
+
+def rope_tables(S, d_head, base, dtype):
+    i = np.arange(d_head // 2, dtype=np.float64)
+    inv = base ** (-2.0 * i / d_head)
+    ang = np.arange(S, dtype=np.float64)[:, None] * inv[None, :]   # [S, dh/2]
+    return np.cos(ang).astype(dtype), np.sin(ang).astype(dtype)
+
+
+def rope(x, cos, sin, inverse=False):
+    """x [B,S,h,dh]; rotates adjacent pairs (2i, 2i+1) by +angle (or -angle)."""
+    x0, x1 = x[..., 0::2], x[..., 1::2]
+    c = cos[None, :, None, :]
+    s = sin[None, :, None, :]
+    if inverse:
+        s = -s
+    out = np.empty_like(x)
+    out[..., 0::2] = x0 * c - x1 * s
+    out[..., 1::2] = x0 * s + x1 * c
+    return out
+
+
+def attention_probs(q, k):
+    """A = softmax_row(q k^T / sqrt(d_h)) with the causal mask s' <= s.
+    q, k [B,S,h,dh] (already rotated) -> [B,h,S,S]."""
+    S, dh = q.shape[1], q.shape[3]
+    causal = np.tril(np.ones((S, S), dtype=bool))
+    sc = np.einsum("bshd,bthd->bhst", q, k) / math.sqrt(dh)
+    sc = np.where(causal[None, None], sc, -np.inf)
+    sc = sc - sc.max(axis=-1, keepdims=True)
+    A = np.exp(sc)
+    return A / A.sum(axis=-1, keepdims=True)
+
+
+# --------------------------------------------------------------------------
+# forward pass and loss (Eq. 2.2; Appendix C.1 forward equations)
+# --------------------------------------------------------------------------
+def forward(cfg: Model, theta: np.ndarray, tokens: np.ndarray, keep=True):
+    """Returns (loss, cache).  tokens int [B,S]; loss is the mean NLL over the
+    B*(S-1) positions that have a next token."""
+    P = views(cfg, theta)
+    dt = theta.dtype
+    B, S = tokens.shape
+    d, h, dh = cfg.d_model, cfg.n_head, cfg.d_head
+    cos, sin = rope_tables(S, dh, cfg.rope_base, dt)
+    keep_probs = keep and B * h * S * S * cfg.n_layer * theta.itemsize <= (1 << 29)
+    x = P["E"][tokens]                                    # [B,S,d]
+    layers = []
+    for l in range(cfg.n_layer):
+        p = f"l{l}."
+        a, ln1 = layernorm(x, P[p + "ln1_g"], P[p + "ln1_b"], cfg.ln_eps)
+        q = rope((a @ P[p + "W_q"].T).reshape(B, S, h, dh), cos, sin)
+        k = rope((a @ P[p + "W_k"].T).reshape(B, S, h, dh), cos, sin)
+        v = (a @ P[p + "W_v"].T).reshape(B, S, h, dh)
+        A = attention_probs(q, k)                         # [B,h,S,S]
+        U = np.einsum("bhst,bthd->bshd", A, v).reshape(B, S, d)
+        x1 = x + U @ P[p + "W_o"].T
+        bb, ln2 = layernorm(x1, P[p + "ln2_g"], P[p + "ln2_b"], cfg.ln_eps)
+        Hd = bb @ P[p + "W_in"].T                         # [B,S,F]
+        Ac = gelu(Hd)
+        x2 = x1 + Ac @ P[p + "W_out"].T
+        if keep:
+            layers.append(dict(a=a, ln1=ln1, q=q, k=k, v=v, U=U, b=bb, ln2=ln2,
+                               Hd=Hd, Ac=Ac, A=A if keep_probs else None))
+        x = x2
+    f, lnf = layernorm(x, P["lnf_g"], P["lnf_b"], cfg.ln_eps)
+    logits = f @ P["E"].T                                 # [B,S,V]
+    z = logits[:, :-1, :]
+    zmax = z.max(axis=-1, keepdims=True)
+    lse = zmax[..., 0] + np.log(np.exp(z - zmax).sum(axis=-1))
+    tgt = tokens[:, 1:]
+    picked = np.take_along_axis(z, tgt[..., None].astype(np.int64), axis=-1)[..., 0]
+    count = B * (S - 1)
+    loss = float((lse - picked).sum() / count)
+    cache = dict(tokens=tokens, layers=layers, f=f, lnf=lnf, logits=logits,
+                 lse=lse, cos=cos, sin=sin) if keep else None
+    return loss, cache
+
+
+def _dlogits(cfg, cache):
+    tokens, logits, lse = cache["tokens"], cache["logits"], cache["lse"]
+    B, S = tokens.shape
+    count = B * (S - 1)
+    dl = np.zeros_like(logits)
+    prob = np.exp(logits[:, :-1, :] - lse[..., None])
+    dl[:, :-1, :] = prob
+    bi, si = np.meshgrid(np.arange(B), np.arange(S - 1), indexing="ij")
+    dl[bi, si, tokens[:, 1:]] -= 1.0
+    dl /= count
+    return dl
+
+
+def _attention_bwd(cfg, L, dU, cache):
+    """Appendix C.1, MHA steps 2-4 (softmax backward in its standard form
+    dS = A * (dA - rowsum(dA * A))).  Returns dq, dk, dv before inverse RoPE
+    is applied to dq, dk."""
+    B, S, h, dh = L["q"].shape
+    dUh = dU.reshape(B, S, h, dh)
+    A = L["A"] if L["A"] is not None else attention_probs(L["q"], L["k"])
+    dv = np.einsum("bhst,bshd->bthd", A, dUh)
+    dA = np.einsum("bshd,bthd->bhst", dUh, L["v"])
+    dS = A * (dA - (dA * A).sum(axis=-1, keepdims=True))
+    dS = dS / math.sqrt(dh)
+    dq = np.einsum("bhst,bthd->bshd", dS, L["k"])
+    dk = np.einsum("bhst,bshd->bthd", dS, L["q"])
+    return dq, dk, dv
+
+
+# --------------------------------------------------------------------------
+# gradients: the definition (full, then mask) and the restricted backward
+# --------------------------------------------------------------------------
+def grad_full(cfg: Model, theta: np.ndarray, tokens: np.ndarray):
+    """(loss, dense gradient of the loss w.r.t. every parameter)."""
+    loss, c = forward(cfg, theta, tokens)
+    P = views(cfg, theta)
+    g = np.zeros_like(theta)
+    G = views(cfg, g)
+    B, S = tokens.shape
+    d = cfg.d_model
+    dl = _dlogits(cfg, c)
+    G["E"] += dl.reshape(B * S, -1).T @ c["f"].reshape(B * S, d)
+    df = dl @ P["E"]
+    gx, dgam, dbet = layernorm_bwd(df, P["lnf_g"], c["lnf"])
+    G["lnf_g"] += dgam; G["lnf_b"] += dbet
+    for l in reversed(range(cfg.n_layer)):
+        p = f"l{l}."
+        L = c["layers"][l]
+        T2 = lambda t: t.reshape(B * S, -1)
+        # FFN (Appendix C.1, MLP steps 1-5 with every slice)
+        G[p + "W_out"] += T2(gx).T @ T2(L["Ac"])
+        dA = gx @ P[p + "W_out"]
+        dH = dA * gelu_grad(L["Hd"])
+        G[p + "W_in"] += T2(dH).T @ T2(L["b"])
+        db = dH @ P[p + "W_in"]
+        dx1, dgam, dbet = layernorm_bwd(db, P[p + "ln2_g"], L["ln2"])
+        G[p + "ln2_g"] += dgam; G[p + "ln2_b"] += dbet
+        g1 = gx + dx1
+        # attention
+        G[p + "W_o"] += T2(g1).T @ T2(L["U"])
+        dU = g1 @ P[p + "W_o"]
+        dq, dk, dv = _attention_bwd(cfg, L, dU, c)
+        dq = rope(dq, c["cos"], c["sin"], inverse=True)
+        dk = rope(dk, c["cos"], c["sin"], inverse=True)
+        a2 = T2(L["a"])
+        G[p + "W_q"] += T2(dq).T @ a2
+        G[p + "W_k"] += T2(dk).T @ a2
+        G[p + "W_v"] += T2(dv).T @ a2
+        da = (dq.reshape(B, S, d) @ P[p + "W_q"] + dk.reshape(B, S, d) @ P[p + "W_k"]
+              + dv.reshape(B, S, d) @ P[p + "W_v"])
+        dx0, dgam, dbet = layernorm_bwd(da, P[p + "ln1_g"], L["ln1"])
+        G[p + "ln1_g"] += dgam; G[p + "ln1_b"] += dbet
+        gx = g1 + dx0
+    np.add.at(G["E"], tokens.reshape(-1), gx.reshape(B * S, d))
+    return loss, g
+
+
+def grad_restricted(cfg: Model, theta: np.ndarray, tokens: np.ndarray, ranges):
+    """Restricted backward of Appendix C.1 for FFN hidden-unit slices.
+
+    ranges[l] = (lo, hi): hidden units of layer l this node trains (lo == hi:
+    none).  Returns (loss, {l: (dW_in[lo:hi, :], dW_out[:, lo:hi])}).
+    Weight gradients are formed for the trained slice only; the input gradient
+    runs through every slice and every head; below the lowest trained layer
+    nothing is computed, and at that layer only its own slice's part.
+    """
+    loss, c = forward(cfg, theta, tokens)
+    P = views(cfg, theta)
+    B, S = tokens.shape
+    trained = [l for l in range(cfg.n_layer) if ranges[l][1] > ranges[l][0]]
+    out = {}
+    if not trained:
+        return loss, out
+    l0 = min(trained)
+    dl = _dlogits(cfg, c)
+    df = dl @ P["E"]
+    gx, _, _ = layernorm_bwd(df, P["lnf_g"], c["lnf"])
+    T2 = lambda t: t.reshape(B * S, -1)
+    for l in reversed(range(l0, cfg.n_layer)):
+        p = f"l{l}."
+        L = c["layers"][l]
+        lo, hi = ranges[l]
+        if l == l0:
+            dA_n = gx @ P[p + "W_out"][:, lo:hi]
+            dH_n = dA_n * gelu_grad(L["Hd"][..., lo:hi])
+            out[l] = (T2(dH_n).T @ T2(L["b"]), T2(gx).T @ T2(L["Ac"][..., lo:hi]))
+            break
+        dA = gx @ P[p + "W_out"]
+        dH = dA * gelu_grad(L["Hd"])
+        if hi > lo:
+            out[l] = (T2(dH[..., lo:hi]).T @ T2(L["b"]),
+                      T2(gx).T @ T2(L["Ac"][..., lo:hi]))
+        db = dH @ P[p + "W_in"]
+        dx1, _, _ = layernorm_bwd(db, P[p + "ln2_g"], L["ln2"])
+        g1 = gx + dx1
+        dU = g1 @ P[p + "W_o"]
+        dq, dk, dv = _attention_bwd(cfg, L, dU, c)
+        dq = rope(dq, c["cos"], c["sin"], inverse=True)
+        dk = rope(dk, c["cos"], c["sin"], inverse=True)
+        d = cfg.d_model
+        da = (dq.reshape(B, S, d) @ P[p + "W_q"] + dk.reshape(B, S, d) @ P[p + "W_k"]
+              + dv.reshape(B, S, d) @ P[p + "W_v"])
+        dx0, _, _ = layernorm_bwd(da, P[p + "ln1_g"], L["ln1"])
+        gx = g1 + dx0
+    return loss, out
+
+
+# --------------------------------------------------------------------------
+# index sets, count vector (Algorithm 1 notation; Section 2.2.1)
+# --------------------------------------------------------------------------
+def slice_ranges(cfg: Model, n_slices: int, replica: int):
+    """MLP-only slicing: node k takes slice n = k mod N, hidden units
+    [n F/N, (n+1) F/N) of every layer."""
+    n = replica % n_slices
+    w = cfg.d_ff // n_slices
+    return [(n * w, (n + 1) * w)] * cfg.n_layer
+
+
+def layer_ranges(cfg: Model, stride: int, replica: int):
+    """Whole-FFN assignment: node with index n = k mod stride trains the full
+    FFN of the blocks l with l mod stride == n."""
+    n = replica % stride
+    return [(0, cfg.d_ff) if l % stride == n else (0, 0) for l in range(cfg.n_layer)]
+
+
+def train_index(cfg: Model, ranges, train_non_mlp=False) -> np.ndarray:
+    """Flat indices of I_k^train in a fixed order: for each layer the W_in rows
+    block, then the W_out column block (row-major over [d, hi-lo]); when
+    train_non_mlp is set, every non-FFN parameter follows (the paper's
+    MLP-only slicing trains those on all nodes)."""
+    recs = {name: (off, shape) for name, off, shape in layout(cfg)}
+    d, F = cfg.d_model, cfg.d_ff
+    parts = []
+    for l in range(cfg.n_layer):
+        lo, hi = ranges[l]
+        if hi <= lo:
+            continue
+        off_in, _ = recs[f"l{l}.W_in"]
+        parts.append(off_in + np.arange(lo * d, hi * d, dtype=np.int64))
+        off_out, _ = recs[f"l{l}.W_out"]
+        rows = np.arange(d, dtype=np.int64)[:, None] * F
+        cols = np.arange(lo, hi, dtype=np.int64)[None, :]
+        parts.append((off_out + rows + cols).reshape(-1))
+    if train_non_mlp:
+        for name, off, shape in layout(cfg):
+            if name.endswith("W_in") or name.endswith("W_out"):
+                continue
+            parts.append(off + np.arange(int(np.prod(shape)), dtype=np.int64))
+    return np.concatenate(parts) if parts else np.zeros(0, dtype=np.int64)
+
+
+def count_vector(n_total: int, index_sets) -> np.ndarray:
+    """m[i] = number of listed nodes whose train set contains i."""
+    m = np.zeros(n_total, dtype=np.int64)
+    for idx in index_sets:
+        m[idx] += 1
+    return m
+
+
+# --------------------------------------------------------------------------
+# inner optimizer (Algorithm 1 line 10; AdamW, Section 3.1)
+# --------------------------------------------------------------------------
+def adamw_update(p, g, m, v, t, hp: AdamW):
+    """One decoupled-weight-decay Adam step on arrays of equal shape; t is the
+    1-based step count.  Returns new (p, m, v)."""
+    m = hp.beta1 * m + (1.0 - hp.beta1) * g
+    v = hp.beta2 * v + (1.0 - hp.beta2) * g * g
+    mhat = m / (1.0 - hp.beta1 ** t)
+    vhat = v / (1.0 - hp.beta2 ** t)
+    p = p - hp.lr * (mhat / (np.sqrt(vhat) + hp.eps) + hp.wd * p)
+    return p, m, v
+
+
+class Replica:
+    """One node k of Algorithm 1: its train index set, its values of the
+    trainable parameters, and its AdamW state.  Frozen parameters are read
+    from the global vector and never written."""
+
+    def __init__(self, cfg: Model, theta_global: np.ndarray, ranges,
+                 train_non_mlp=False):
+        self.cfg = cfg
+        self.ranges = list(ranges)
+        self.train_non_mlp = train_non_mlp
+        self.idx = train_index(cfg, ranges, train_non_mlp)
+        self.theta_sub = theta_global[self.idx].copy()     # theta_k^(t,0) <- theta^(t)
+        self.m = np.zeros_like(self.theta_sub)
+        self.v = np.zeros_like(self.theta_sub)
+        self.t = 0
+        self.last_loss = None
+        self.last_grad = None
+
+    def materialise(self, theta_global):
+        th = theta_global.copy()
+        th[self.idx] = self.theta_sub
+        return th
+
+    def gradient(self, theta_global, tokens, mode="restricted"):
+        """g_k[I_train] of Algorithm 1 line 9, in the order of self.idx."""
+        th = self.materialise(theta_global)
+        if mode == "masked_full" or self.train_non_mlp:
+            loss, g = grad_full(self.cfg, th, tokens)
+            return loss, g[self.idx]
+        loss, sl = grad_restricted(self.cfg, th, tokens, self.ranges)
+        parts = []
+        for l in range(self.cfg.n_layer):
+            if l in sl:
+                parts.append(sl[l][0].reshape(-1))
+                parts.append(sl[l][1].reshape(-1))
+        g = np.concatenate(parts) if parts else np.zeros(0, dtype=th.dtype)
+        return loss, g
+
+    def local_step(self, theta_global, tokens, hp: AdamW, mode="restricted"):
+        loss, g = self.gradient(theta_global, tokens, mode)
+        self.t += 1
+        self.theta_sub, self.m, self.v = adamw_update(self.theta_sub, g, self.m,
+                                                      self.v, self.t, hp)
+        self.last_loss, self.last_grad = loss, g
+        return loss
+
+
+# --------------------------------------------------------------------------
+# outer synchronisation (Algorithm 1 lines 12-15; Eq. 2.4-2.5)
+# --------------------------------------------------------------------------
+def outer_sync(theta, buf, replicas, hp: Outer):
+    """Dense definition.  Delta_k is theta_k^(t,H) - theta^(t) on I_k^train and
+    0 elsewhere; Delta = sum_k Delta_k / m with 0/0 := 0; the outer optimizer
+    is SGD with Nesterov momentum on the pseudo-gradient g = -Delta.  Every
+    listed replica restarts from the new global parameters.
+    Returns (theta_new, buf_new, m)."""
+    n = theta.shape[0]
+    total = np.zeros(n, dtype=theta.dtype)
+    for r in replicas:
+        dk = np.zeros(n, dtype=theta.dtype)
+        dk[r.idx] = r.theta_sub - theta[r.idx]
+        total += dk
+    m = count_vector(n, [r.idx for r in replicas])
+    delta = np.where(m > 0, total / np.maximum(m, 1), 0.0)
+    g = -delta
+    buf_new = hp.momentum * buf + g
+    theta_new = theta - hp.lr * (g + hp.momentum * buf_new)
+    for r in replicas:
+        r.theta_sub = theta_new[r.idx].copy()
+    return theta_new, buf_new, m
+
+
+def outer_elementwise(theta, buf, ends, hp: Outer):
+    """The same outer step for a sample of parameter positions.  theta, buf:
+    values at the sampled positions; ends: one array per owning replica with
+    NaN where that replica does not train the position."""
+    total = np.zeros_like(theta)
+    m = np.zeros(theta.shape, dtype=np.int64)
+    for e in ends:
+        own = ~np.isnan(e)
+        total[own] += e[own] - theta[own]
+        m += own
+    delta = np.where(m > 0, total / np.maximum(m, 1), 0.0)
+    g = -delta
+    buf_new = hp.momentum * buf + g
+    return theta - hp.lr * (g + hp.momentum * buf_new), buf_new
+
+
+# --------------------------------------------------------------------------
+# closed forms: Table 1 parameter counts and Appendix C.2 FLOPs
+# --------------------------------------------------------------------------
+def trainable_params(cfg: Model, rho_mlp: float, rho_attn: float = 1.0) -> int:
+    """Parameters a node trains under the paper's slicing: all non-MLP
+    parameters (with only a rho_attn fraction of the Q/K/V projections) plus a
+    rho_mlp fraction of every FFN."""
+    d, F, V, L = cfg.d_model, cfg.d_ff, cfg.vocab, cfg.n_layer
+    ffn = 2 * d * F
+    qkv = 3 * d * d
+    other = V * d + L * (d * d + 4 * d) + 2 * d
+    return int(round(other + L * (rho_attn * qkv + rho_mlp * ffn)))
+
+
+def flops_forward(cfg: Model, B: int, S: int) -> float:
+    H, Dff, V, L = cfg.d_model, cfg.d_ff, cfg.vocab, cfg.n_layer
+    emb = B * S * H
+    mha = 8 * B * S * H * H + 4 * B * S * S * H
+    ffn = 4 * B * S * H * Dff
+    outp = 2 * B * S * H * V + 3 * B * S * V
+    return emb + L * (mha + ffn) + outp
+
+
+def flops_backward(cfg: Model, B: int, S: int, rho_mlp: float, rho_attn: float) -> float:
+    H, Dff, V, L = cfg.d_model, cfg.d_ff, cfg.vocab, cfg.n_layer
+    emb = B * S * H
+    mha = 8 * B * S * S * H + (10 + 6 * rho_attn) * B * S * H * H
+    ffn = 4 * B * S * H * Dff + 4 * rho_mlp * B * S * H * Dff
+    outp = 2 * B * S * H * V + 3 * B * S * V
+    return 2 * emb + L * (mha + ffn) + 2 * outp

@@ -1,0 +1,174 @@
+"""Pins for the CPU oracle: each checks it against something other than itself
+(printed values of the paper, closed forms, finite differences, library
+routines for textbook special cases, brute force on tiny inputs)."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ppu_oracle as O
+from paper_2509_22418_b200 import synth
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rows(name):
+    out = []
+    for line in open(os.path.join(GOLD, name)):
+        line = line.strip()
+        if line and not line.startswith("#"):
+            out.append([float(x) for x in line.split()])
+    return out
+
+
+def tiny():
+    cfg = O.Model(2, 64, 4, 256, 512)
+    th = synth.init_params(7, O.layout(cfg)).astype(np.float64)
+    tok = synth.tokens(7, 0, 0, 0, 4, 64, cfg.vocab)
+    return cfg, th, tok
+
+
+def micro():
+    cfg = O.Model(2, 16, 2, 32, 24)
+    rng = np.random.default_rng(3)
+    th = rng.normal(0, 0.3, O.n_params(cfg))
+    tok = rng.integers(0, cfg.vocab, (2, 6)).astype(np.int32)
+    return cfg, th, tok
+
+
+# ---- closed forms printed by the paper -----------------------------------
+def test_table1_trainable_parameter_column():
+    cfg = O.Model(24, 2048, 16, 8192, 32000)
+    for rho_mlp, rho_attn, printed in _rows("table1_trainable_params.txt"):
+        got = O.trainable_params(cfg, rho_mlp, rho_attn) / 1e9
+        digits = 1 if printed == 1.3 else 2
+        assert round(got, digits) == printed, (rho_mlp, rho_attn, got)
+    assert O.trainable_params(cfg, 1, 1) == O.n_params(cfg)
+
+
+def test_flops_saving_claim_and_rho_one_identity():
+    cfg = O.Model(24, 2048, 16, 8192, 32000)
+    for rho_mlp, rho_attn, S, V, pct, tol in _rows("flops_saving.txt"):
+        S = int(S)
+        full = O.flops_forward(cfg, 16, S) + O.flops_backward(cfg, 16, S, 1, 1)
+        part = O.flops_forward(cfg, 16, S) + O.flops_backward(cfg, 16, S, rho_mlp, rho_attn)
+        assert abs(100 * (1 - part / full) - pct) <= tol
+    # rho = 1: backward = 2 x forward for the layer stack and the output head
+    B, S = 16, 1024
+    emb = B * S * cfg.d_model
+    fwd = O.flops_forward(cfg, B, S) - emb
+    bwd = O.flops_backward(cfg, B, S, 1, 1) - 2 * emb
+    assert bwd == 2 * fwd
+
+
+# ---- finite differences ----------------------------------------------------
+def test_full_gradient_matches_central_differences():
+    cfg, th, tok = micro()
+    loss, g = O.grad_full(cfg, th, tok)
+    rng = np.random.default_rng(0)
+    for name, off, shape in O.layout(cfg):
+        n = int(np.prod(shape))
+        for i in off + rng.choice(n, size=min(n, 6), replace=False):
+            e = 1e-5
+            tp, tm = th.copy(), th.copy()
+            tp[i] += e
+            tm[i] -= e
+            fd = (O.forward(cfg, tp, tok, keep=False)[0]
+                  - O.forward(cfg, tm, tok, keep=False)[0]) / (2 * e)
+            assert abs(fd - g[i]) <= 1e-6 * max(1.0, abs(fd)) + 1e-9, (name, i, fd, g[i])
+
+
+def test_restricted_gradient_matches_central_differences():
+    cfg, th, tok = micro()
+    ranges = [(8, 16), (8, 16)]
+    r = O.Replica(cfg, th, ranges)
+    loss, g = r.gradient(th, tok, "restricted")
+    rng = np.random.default_rng(1)
+    for j in rng.choice(len(r.idx), size=40, replace=False):
+        i, e = r.idx[j], 1e-5
+        tp, tm = th.copy(), th.copy()
+        tp[i] += e
+        tm[i] -= e
+        fd = (O.forward(cfg, tp, tok, keep=False)[0]
+              - O.forward(cfg, tm, tok, keep=False)[0]) / (2 * e)
+        assert abs(fd - g[j]) <= 1e-6 * max(1.0, abs(fd)) + 1e-9
+
+
+# ---- invariants of the method --------------------------------------------
+@pytest.mark.parametrize("ranges_fn", [
+    lambda cfg: O.slice_ranges(cfg, 4, 1),
+    lambda cfg: O.layer_ranges(cfg, 2, 1),      # lowest trained layer is 1
+    lambda cfg: [(64, 192), (0, 64)],
+])
+def test_restricted_equals_masked_full(ranges_fn):
+    cfg, th, tok = tiny()
+    r = O.Replica(cfg, th, ranges_fn(cfg))
+    l1, g1 = r.gradient(th, tok, "restricted")
+    l2, g2 = r.gradient(th, tok, "masked_full")
+    assert l1 == l2
+    assert np.abs(g1 - g2).max() <= 1e-12 * max(1.0, np.abs(g2).max())
+    assert np.abs(g2).max() > 0
+
+
+def test_frozen_parameters_bit_identical_and_only_subset_moves():
+    cfg, th, tok = tiny()
+    hp = O.AdamW()
+    r = O.Replica(cfg, th, O.slice_ranges(cfg, 4, 2))
+    th0 = th.copy()
+    for h in range(3):
+        r.local_step(th, synth.tokens(7, 2, 0, h, 4, 64, cfg.vocab), hp)
+    assert np.array_equal(th, th0)                      # global vector never written
+    after = r.materialise(th)
+    mask = np.zeros(len(th), bool)
+    mask[r.idx] = True
+    assert np.array_equal(after[~mask], th0[~mask])
+    assert np.all(after[mask] != th0[mask])
+    # outer step: positions no replica trains keep their exact bits
+    th1, buf1, m = O.outer_sync(th, np.zeros_like(th), [r], O.Outer())
+    assert np.array_equal(th1[m == 0], th0[m == 0])
+    assert np.all(buf1[m == 0] == 0)
+
+
+def test_mlp_is_additive_over_slices_and_dx_sums_all_slices():
+    rng = np.random.default_rng(5)
+    d, F, N, T = 8, 32, 4, 5
+    W, V = rng.normal(size=(F, d)), rng.normal(size=(d, F))
+    x, G = rng.normal(size=(T, d)), rng.normal(size=(T, d))
+    y = O.gelu(x @ W.T) @ V.T
+    w = F // N
+    y_s = sum(O.gelu(x @ W[n * w:(n + 1) * w].T) @ V[:, n * w:(n + 1) * w].T for n in range(N))
+    assert np.allclose(y, y_s, rtol=0, atol=1e-12)
+    dx = ((G @ V) * O.gelu_grad(x @ W.T)) @ W
+    dx_s = sum(((G @ V[:, n * w:(n + 1) * w]) * O.gelu_grad(x @ W[n * w:(n + 1) * w].T))
+               @ W[n * w:(n + 1) * w] for n in range(N))
+    assert np.allclose(dx, dx_s, rtol=0, atol=1e-12)
+
+
+def test_count_vector_and_shared_slices():
+    cfg, th, tok = tiny()
+    K, N = 8, 4
+    reps = [O.Replica(cfg, th, O.slice_ranges(cfg, N, k)) for k in range(K)]
+    m = O.count_vector(len(th), [r.idx for r in reps])
+    V = O.views(cfg, m)
+    for l in range(cfg.n_layer):
+        assert np.all(V[f"l{l}.W_in"] == K // N) and np.all(V[f"l{l}.W_out"] == K // N)
+    assert np.all(V["E"] == 0) and np.all(V["l0.W_q"] == 0)
+    assert np.array_equal(reps[1].idx, reps[1 + N].idx)
+    # replicas 1 and 5 move their shared slice by +a and +3a: the average is +2a
+    a = 1e-3
+    reps[1].theta_sub += a
+    reps[5].theta_sub += 3 * a
+    th1, _, _ = O.outer_sync(th, np.zeros_like(th), reps, O.Outer(lr=1.0, momentum=0.0))
+    assert np.allclose(th1[reps[1].idx] - th[reps[1].idx], 2 * a, rtol=1e-9)
+    paper_m = O.count_vector(len(th), [O.train_index(cfg, O.slice_ranges(cfg, N, k), True)
+                                       for k in range(K)])
+    Vp = O.views(cfg, paper_m)        # Section 2.2.1: K/N on sliced, K otherwise
+    assert np.all(Vp["l1.W_in"] == K // N) and np.all(Vp["E"] == K) and np.all(Vp["lnf_g"] == K)
+
+
+def test_loss_at_init_is_log_vocab():
+    cfg, th, tok = tiny()
+    loss, _ = O.forward(cfg, th, tok, keep=False)
+    assert abs(loss - math.log(cfg.vocab)) < 0.01 * math.log(cfg.vocab)
