@@ -1,0 +1,338 @@
+// Bandwidth-bound kernels of the local step: embedding gather, LayerNorm forward and
+// input-gradient backward, rotary positions, fused cross-entropy, loss reduction.
+// All accesses are 16-byte vectors on rows that are multiples of 8 elements.
+#include "common.cuh"
+
+namespace {
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Block-wide sum with a fixed combination order (deterministic).
+template <int NW>
+__device__ __forceinline__ float block_sum(float v, float* red) {
+  v = warp_sum(v);
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  __syncthreads();
+  if (l == 0) red[w] = v;
+  __syncthreads();
+  float t = 0.f;
+#pragma unroll
+  for (int i = 0; i < NW; ++i) t += red[i];
+  return t;
+}
+template <int NW>
+__device__ __forceinline__ float block_max(float v, float* red) {
+  v = warp_max(v);
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  __syncthreads();
+  if (l == 0) red[w] = v;
+  __syncthreads();
+  float t = red[0];
+#pragma unroll
+  for (int i = 1; i < NW; ++i) t = fmaxf(t, red[i]);
+  return t;
+}
+
+__device__ __forceinline__ void unpack8(const uint4& u, float* f) {
+  const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 t = __bfloat1622float2(p[i]);
+    f[2 * i] = t.x;
+    f[2 * i + 1] = t.y;
+  }
+}
+__device__ __forceinline__ uint4 pack8(const float* f) {
+  uint4 u;
+  __nv_bfloat162* p = reinterpret_cast<__nv_bfloat162*>(&u);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) p[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+  return u;
+}
+
+// ---- embedding gather: x[t,:] = E[tok[t],:] (bf16 working copy -> fp32 stream) ----
+__global__ void embed_kernel(const int32_t* __restrict__ tok, const bf16* __restrict__ E,
+                             float* __restrict__ x, int T, int d, int V, int* flags) {
+  const int t = blockIdx.x;
+  int id = tok[t];
+  if (id < 0 || id >= V) {
+    if (threadIdx.x == 0) atomicExch(flags + PPU_FLAG_TOKEN, 1);
+    id = id < 0 ? 0 : V - 1;
+  }
+  const uint4* src = reinterpret_cast<const uint4*>(E + (int64_t)id * d);
+  float4* dst = reinterpret_cast<float4*>(x + (int64_t)t * d);
+  for (int i = threadIdx.x; i < d / 8; i += blockDim.x) {
+    float f[8];
+    unpack8(src[i], f);
+    dst[2 * i] = make_float4(f[0], f[1], f[2], f[3]);
+    dst[2 * i + 1] = make_float4(f[4], f[5], f[6], f[7]);
+  }
+}
+
+// ---- LayerNorm forward: one block per row, row staged in shared memory ----
+constexpr int LN_THREADS = 256;
+__global__ void __launch_bounds__(LN_THREADS)
+ln_fwd_kernel(const float* __restrict__ x, const float* __restrict__ g, const float* __restrict__ b,
+              bf16* __restrict__ y, float2* __restrict__ stats, int d, float eps) {
+  extern __shared__ float row[];
+  __shared__ float red[LN_THREADS / 32];
+  const int64_t t = blockIdx.x;
+  const float4* src = reinterpret_cast<const float4*>(x + t * d);
+  float s = 0.f;
+  for (int i = threadIdx.x; i < d / 4; i += LN_THREADS) {
+    float4 v = src[i];
+    reinterpret_cast<float4*>(row)[i] = v;
+    s += (v.x + v.y) + (v.z + v.w);
+  }
+  const float mean = block_sum<LN_THREADS / 32>(s, red) / d;
+  float q = 0.f;
+  for (int i = threadIdx.x; i < d / 4; i += LN_THREADS) {
+    float4 v = reinterpret_cast<float4*>(row)[i];
+    float a = v.x - mean, bb = v.y - mean, c = v.z - mean, e = v.w - mean;
+    q += (a * a + bb * bb) + (c * c + e * e);
+  }
+  const float var = block_sum<LN_THREADS / 32>(q, red) / d;
+  const float rstd = rsqrtf(var + eps);
+  if (threadIdx.x == 0) stats[t] = make_float2(mean, rstd);
+  uint4* dst = reinterpret_cast<uint4*>(y + t * d);
+  for (int i = threadIdx.x; i < d / 8; i += LN_THREADS) {
+    float f[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int c = 8 * i + j;
+      f[j] = (row[c] - mean) * rstd * g[c] + b[c];
+    }
+    dst[i] = pack8(f);
+  }
+}
+
+// ---- LayerNorm backward, input gradient only (gamma/beta are frozen) ----
+// gout = gin + rstd * (dy*gamma - mean(dy*gamma) - xhat * mean(dy*gamma*xhat))
+__global__ void __launch_bounds__(LN_THREADS)
+ln_bwd_kernel(const bf16* __restrict__ dy, const float* __restrict__ x,
+              const float2* __restrict__ stats, const float* __restrict__ gamma,
+              const float* gin, float* gout, bf16* __restrict__ gout16, int d) {
+  extern __shared__ float sm[];
+  float* dyg = sm;
+  float* xh = sm + d;
+  __shared__ float red[LN_THREADS / 32];
+  const int64_t t = blockIdx.x;
+  const float2 st = stats[t];
+  const uint4* dsrc = reinterpret_cast<const uint4*>(dy + t * d);
+  const float4* xsrc = reinterpret_cast<const float4*>(x + t * d);
+  float s1 = 0.f, s2 = 0.f;
+  for (int i = threadIdx.x; i < d / 8; i += LN_THREADS) {
+    float f[8];
+    unpack8(dsrc[i], f);
+    float4 xa = xsrc[2 * i], xb = xsrc[2 * i + 1];
+    float xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int c = 8 * i + j;
+      const float a = f[j] * gamma[c];
+      const float h = (xv[j] - st.x) * st.y;
+      dyg[c] = a;
+      xh[c] = h;
+      s1 += a;
+      s2 += a * h;
+    }
+  }
+  const float m1 = block_sum<LN_THREADS / 32>(s1, red) / d;
+  const float m2 = block_sum<LN_THREADS / 32>(s2, red) / d;
+  const float4* gsrc = gin ? reinterpret_cast<const float4*>(gin + t * d) : nullptr;
+  float4* gdst = reinterpret_cast<float4*>(gout + t * d);
+  uint4* g16 = reinterpret_cast<uint4*>(gout16 + t * d);
+  for (int i = threadIdx.x; i < d / 8; i += LN_THREADS) {
+    float f[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int c = 8 * i + j;
+      f[j] = st.y * (dyg[c] - m1 - xh[c] * m2);
+    }
+    if (gsrc) {
+      float4 a = gsrc[2 * i], bq = gsrc[2 * i + 1];
+      f[0] += a.x; f[1] += a.y; f[2] += a.z; f[3] += a.w;
+      f[4] += bq.x; f[5] += bq.y; f[6] += bq.z; f[7] += bq.w;
+    }
+    gdst[2 * i] = make_float4(f[0], f[1], f[2], f[3]);
+    gdst[2 * i + 1] = make_float4(f[4], f[5], f[6], f[7]);
+    g16[i] = pack8(f);
+  }
+}
+
+// ---- rotary positions on the q and k parts of qkv[T,3d], in place ----
+// cs: [S, dh/2] (cos, sin) pairs computed on the host in double precision.
+__global__ void rope_kernel(bf16* __restrict__ qkv, const float2* __restrict__ cs, int S, int d,
+                            int dh, int64_t n_vec, int inverse) {
+  // one thread per 8 consecutive elements (4 pairs) of q or k
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i >= n_vec) return;
+  const int per_row = 2 * d / 8;
+  const int64_t t = i / per_row;
+  const int c = (int)(i % per_row) * 8;       // column in [0, 2d)
+  const int pos = (int)(t % S);
+  const int pair0 = (c % dh) / 2;
+  uint4* p = reinterpret_cast<uint4*>(qkv + t * (int64_t)(3 * d) + c);
+  float f[8];
+  unpack8(*p, f);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    float2 w = cs[(int64_t)pos * (dh / 2) + pair0 + j];
+    if (inverse) w.y = -w.y;
+    const float a = f[2 * j], b = f[2 * j + 1];
+    f[2 * j] = a * w.x - b * w.y;
+    f[2 * j + 1] = a * w.y + b * w.x;
+  }
+  *p = pack8(f);
+}
+
+// ---- fused cross-entropy: one block per token row, row held in registers ----
+// Reads the logits once; writes dlogits = (softmax - onehot) / count in place.
+constexpr int XE_THREADS = 1024;
+template <int NCH>
+__global__ void __launch_bounds__(XE_THREADS)
+xent_kernel(bf16* __restrict__ logits, const int32_t* __restrict__ tok,
+            float* __restrict__ row_loss, int S, int V, float inv_count, int write_grad) {
+  __shared__ float red[XE_THREADS / 32];
+  const int64_t t = blockIdx.x;
+  const int s = (int)(t % S);
+  uint4* rowp = reinterpret_cast<uint4*>(logits + t * V);
+  const int nvec = V / 8;
+  if (s == S - 1) {  // no next token: no loss, zero gradient
+    if (write_grad)
+      for (int i = threadIdx.x; i < nvec; i += XE_THREADS) rowp[i] = make_uint4(0, 0, 0, 0);
+    if (threadIdx.x == 0) row_loss[t] = 0.f;
+    return;
+  }
+  int target = tok[t + 1];
+  target = target < 0 ? 0 : (target >= V ? V - 1 : target);
+  float v[NCH][8];
+  float mx = -INFINITY;
+#pragma unroll
+  for (int c = 0; c < NCH; ++c) {
+    const int i = threadIdx.x + c * XE_THREADS;
+    if (i < nvec) {
+      unpack8(rowp[i], v[c]);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) mx = fmaxf(mx, v[c][j]);
+    }
+  }
+  mx = block_max<XE_THREADS / 32>(mx, red);
+  float sum = 0.f;
+#pragma unroll
+  for (int c = 0; c < NCH; ++c) {
+    const int i = threadIdx.x + c * XE_THREADS;
+    if (i < nvec) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        v[c][j] = __expf(v[c][j] - mx);
+        sum += v[c][j];
+      }
+    }
+  }
+  sum = block_sum<XE_THREADS / 32>(sum, red);
+  const float inv = 1.f / sum;
+  if (threadIdx.x == 0) {
+    const float zt = __bfloat162float(logits[t * V + target]);
+    row_loss[t] = logf(sum) + mx - zt;
+  }
+  if (!write_grad) return;
+  __syncthreads();  // the target logit is read before anyone overwrites the row
+#pragma unroll
+  for (int c = 0; c < NCH; ++c) {
+    const int i = threadIdx.x + c * XE_THREADS;
+    if (i < nvec) {
+      float f[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float p = v[c][j] * inv;
+        if (8 * i + j == target) p -= 1.f;
+        f[j] = p * inv_count;
+      }
+      rowp[i] = pack8(f);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(1024)
+loss_reduce_kernel(const float* __restrict__ row_loss, int T, float inv_count, float* out) {
+  __shared__ float red[32];
+  float s = 0.f;
+  for (int i = threadIdx.x; i < T; i += 1024) s += row_loss[i];
+  s = block_sum<32>(s, red);
+  if (threadIdx.x == 0) *out = s * inv_count;
+}
+
+__global__ void cast_bf16_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int64_t n8) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n8;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    float4 a = reinterpret_cast<const float4*>(src)[2 * i];
+    float4 b = reinterpret_cast<const float4*>(src)[2 * i + 1];
+    float f[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    reinterpret_cast<uint4*>(dst)[i] = pack8(f);
+  }
+}
+
+}  // namespace
+
+void launch_embed(const int32_t* tok, const bf16* E16, float* x, int T, int d, int V, int* flags,
+                  cudaStream_t st) {
+  embed_kernel<<<T, 128, 0, st>>>(tok, E16, x, T, d, V, flags);
+}
+
+void launch_ln_fwd(const float* x, const float* g, const float* b, bf16* y, float2* stats, int T,
+                   int d, float eps, cudaStream_t st) {
+  ln_fwd_kernel<<<T, LN_THREADS, d * sizeof(float), st>>>(x, g, b, y, stats, d, eps);
+}
+
+void launch_ln_bwd(const bf16* dy, const float* x, const float2* stats, const float* gamma,
+                   const float* gin, float* gout, bf16* gout16, int T, int d, cudaStream_t st) {
+  ln_bwd_kernel<<<T, LN_THREADS, 2 * d * sizeof(float), st>>>(dy, x, stats, gamma, gin, gout,
+                                                              gout16, d);
+}
+
+void launch_rope(bf16* qkv, const float2* cs, int B, int S, int h, int dh, int inverse,
+                 cudaStream_t st) {
+  const int d = h * dh;
+  const int64_t n_vec = (int64_t)B * S * (2 * d / 8);
+  const int threads = 256;
+  rope_kernel<<<(unsigned)((n_vec + threads - 1) / threads), threads, 0, st>>>(
+      qkv, cs, S, d, dh, n_vec, inverse);
+}
+
+void launch_xent(bf16* logits, const int32_t* tok, float* row_loss, int B, int S, int V,
+                 int write_grad, cudaStream_t st) {
+  const int T = B * S;
+  const float inv_count = 1.f / (float)((int64_t)B * (S - 1));
+  const int nch = (V / 8 + XE_THREADS - 1) / XE_THREADS;
+  if (nch <= 1)
+    xent_kernel<1><<<T, XE_THREADS, 0, st>>>(logits, tok, row_loss, S, V, inv_count, write_grad);
+  else if (nch <= 2)
+    xent_kernel<2><<<T, XE_THREADS, 0, st>>>(logits, tok, row_loss, S, V, inv_count, write_grad);
+  else if (nch <= 4)
+    xent_kernel<4><<<T, XE_THREADS, 0, st>>>(logits, tok, row_loss, S, V, inv_count, write_grad);
+  else
+    xent_kernel<8><<<T, XE_THREADS, 0, st>>>(logits, tok, row_loss, S, V, inv_count, write_grad);
+}
+
+void launch_loss_reduce(const float* row_loss, int T, float inv_count, float* out, cudaStream_t st) {
+  loss_reduce_kernel<<<1, 1024, 0, st>>>(row_loss, T, inv_count, out);
+}
+
+void launch_cast_bf16(const float* src, bf16* dst, int64_t n, cudaStream_t st) {
+  const int64_t n8 = n / 8;
+  const int threads = 256;
+  int64_t blocks = (n8 + threads - 1) / threads;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  cast_bf16_kernel<<<(unsigned)blocks, threads, 0, st>>>(src, dst, n8);
+}

@@ -1,0 +1,73 @@
+// Host-side context of the ppu library: validated configuration, per-replica subset tables
+// and the carve-up of the caller's device arena.
+#pragma once
+#include <string>
+#include <vector>
+#include "../../include/ppu.h"
+#include "common.cuh"
+
+struct TensorRec { std::string name; int64_t offset; int ndim; int64_t shape[2]; };
+
+struct ReplicaState {
+  std::vector<int32_t> lo, hi;     // per layer trained hidden-unit range (lo == hi: none)
+  std::vector<SliceSeg> segs;      // one per trained layer, ascending layer
+  std::vector<int> seg_layer;      // layer of segs[i]
+  int64_t n_sub = 0;               // |I_k^train|
+  int lowest = -1;                 // lowest trained layer (-1: trains nothing)
+  int step = 0;                    // AdamW step count
+  bool stepped = false;
+  float *master = nullptr, *m = nullptr, *v = nullptr;  // device, packed
+  SliceSeg* d_segs = nullptr;      // device copy of segs
+};
+
+struct LayerActs {
+  float* x;        // block input (LayerNorm-1 input), fp32 [T,d]
+  float* x1;       // after the attention residual (LayerNorm-2 input), fp32 [T,d]
+  float2 *st1, *st2;
+  bf16* qkv;       // rotated q,k and v, [T,3d]
+  bf16* U;         // attention output before W_o, [T,d]
+  float* lse;      // [B,h,S]
+  bf16* b;         // LayerNorm-2 output (input of W_in), [T,d]
+  bf16* Hd;        // FFN pre-activation, [T,F]
+  bf16* A;         // gelu(Hd), [T,F]
+};
+
+struct ppu_ctx {
+  ppu_model_cfg cfg;
+  int K = 0;
+  cudaStream_t stream = nullptr;
+  int gemm_backend = 0;   // 0 tcgen05, 1 SIMT
+  int attn_backend = 0;   // 0 tensor-core tiles when the shape allows, 1 SIMT
+  // canonical geometry
+  int64_t P = 0, e_size = 0, layer_size = 0;
+  int64_t rel_ln1g, rel_ln1b, rel_wq, rel_wo, rel_ln2g, rel_ln2b, rel_win, rel_wout;
+  int64_t off_lnfg, off_lnfb;
+  std::vector<TensorRec> tensors;
+  std::vector<ReplicaState> reps;
+  int64_t max_sub = 0;
+  int resident = -1;      // replica whose subset is overlaid on the bf16 working copy
+  int last_stepped = -1;
+  float adam_lr;
+  // arena
+  uint8_t* arena = nullptr;
+  size_t arena_bytes = 0, state_bytes = 0, act_bytes = 0;
+  float *theta = nullptr, *buf = nullptr;
+  bf16* w16 = nullptr;
+  float* grad = nullptr;
+  std::vector<LayerActs> acts;
+  float* x_last = nullptr;      // input of the final LayerNorm
+  float2* stf = nullptr;
+  bf16 *a16 = nullptr, *f16 = nullptr, *logits = nullptr;
+  float* g = nullptr;
+  bf16 *g16 = nullptr, *dHd = nullptr, *t16 = nullptr, *dqkv = nullptr;
+  float *attn_scratch = nullptr, *row_loss = nullptr, *loss = nullptr;
+  int* flags = nullptr;
+  float2* rope_cs = nullptr;
+  int32_t* tok_stage = nullptr;
+  OuterOwner* d_owners = nullptr;
+  int32_t *d_unit_begin = nullptr, *d_unit_owner = nullptr;
+  std::vector<int32_t> cached_sync_list;
+  // stats
+  int64_t launches = 0, launches_last_step = 0, launches_last_sync = 0;
+  double flops_fwd = 0, flops_dgrad = 0, flops_wgrad = 0, outer_bytes = 0;
+};

@@ -1,0 +1,313 @@
+// Step scheduler: enqueues the kernels of one local step (Algorithm 1 lines 8-10) and of the
+// outer synchronisation (lines 12-15) on the context's stream.  No host synchronisation
+// happens inside a local step.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include "ppu_ctx.cuh"
+
+int ppu_fail(int code, const char* fmt, ...);
+#define CUDA_OK(call)                                                                    \
+  do {                                                                                   \
+    cudaError_t e_ = (call);                                                             \
+    if (e_ != cudaSuccess)                                                               \
+      return ppu_fail(PPU_ECUDA, "%s failed: %s", #call, cudaGetErrorString(e_));        \
+  } while (0)
+
+int ppu_check_flags(ppu_ctx* c) {
+  int h[PPU_FLAG_COUNT];
+  CUDA_OK(cudaMemcpy(h, c->flags, sizeof(h), cudaMemcpyDeviceToHost));
+  if (h[PPU_FLAG_TOKEN] || h[PPU_FLAG_TIMEOUT]) {
+    CUDA_OK(cudaMemset(c->flags, 0, sizeof(h)));
+    if (h[PPU_FLAG_TIMEOUT]) return ppu_fail(PPU_ETIMEOUT, "a bounded wait inside a kernel expired");
+    return ppu_fail(PPU_ETOKEN, "token id outside [0, vocab) was clamped");
+  }
+  return PPU_OK;
+}
+
+// Puts replica k's subset (or, for k = -1, the global values) into the bf16 working copy.
+int ppu_make_resident(ppu_ctx* c, int k) {
+  if (c->resident == k) return PPU_OK;
+  const int d = c->cfg.d_model, F = c->cfg.d_ff;
+  if (c->resident >= 0) {
+    ReplicaState& r = c->reps[c->resident];
+    launch_slices_to_w16(r.d_segs, (int)r.segs.size(), nullptr, c->theta, c->w16, 0, d, F, r.n_sub,
+                         c->stream);
+    c->launches++;
+  }
+  if (k >= 0) {
+    ReplicaState& r = c->reps[k];
+    launch_slices_to_w16(r.d_segs, (int)r.segs.size(), r.master, nullptr, c->w16, 1, d, F, r.n_sub,
+                         c->stream);
+    c->launches++;
+  }
+  c->resident = k;
+  return PPU_OK;
+}
+
+namespace {
+
+struct Sched {
+  ppu_ctx* c;
+  int B, S, T, d, F, V, h, dh, L;
+  int rc = 0;
+
+  explicit Sched(ppu_ctx* ctx, int B_, int S_) : c(ctx), B(B_), S(S_) {
+    T = B * S; d = c->cfg.d_model; F = c->cfg.d_ff; V = c->cfg.vocab; h = c->cfg.n_head;
+    dh = d / h; L = c->cfg.n_layer;
+  }
+  const bf16* W(int l, int64_t rel) const { return c->w16 + c->e_size + (int64_t)l * c->layer_size + rel; }
+  const float* Pf(int l, int64_t rel) const { return c->theta + c->e_size + (int64_t)l * c->layer_size + rel; }
+
+  void gemm(const bf16* A, int64_t lda, int ak, const bf16* Bm, int64_t ldb, int bk, int M, int N,
+            int K, int epi, void* C, int64_t ldc, void* C2, const void* aux, int64_t ldaux,
+            double* flop_counter) {
+    if (rc || M <= 0 || N <= 0) return;
+    GemmArgs g;
+    g.A = A; g.lda = lda; g.a_kmajor = ak; g.B = Bm; g.ldb = ldb; g.b_kmajor = bk;
+    g.M = M; g.N = N; g.K = K; g.epilogue = epi; g.C = C; g.ldc = ldc; g.C2 = C2; g.aux = aux;
+    g.ldaux = ldaux; g.flags = c->flags;
+    rc = c->gemm_backend == 1 ? launch_gemm_simt(g, c->stream) : launch_gemm_tc(g, c->stream);
+    c->launches++;
+    if (flop_counter) *flop_counter += 2.0 * M * N * (double)K;
+  }
+  bool use_mma_attn() const { return c->attn_backend == 0 && attn_mma_supported(S, dh); }
+
+  // Forward pass over all parameters (Appendix C.1 forward equations), saving what the
+  // restricted backward needs.
+  void forward(const int32_t* tok) {
+    cudaStream_t st = c->stream;
+    launch_embed(tok, c->w16, c->acts[0].x, T, d, V, c->flags, st); c->launches++;
+    for (int l = 0; l < L && !rc; ++l) {
+      LayerActs& a = c->acts[l];
+      float* x_next = (l + 1 < L) ? c->acts[l + 1].x : c->x_last;
+      launch_ln_fwd(a.x, Pf(l, c->rel_ln1g), Pf(l, c->rel_ln1b), c->a16, a.st1, T, d, c->cfg.ln_eps, st);
+      c->launches++;
+      gemm(c->a16, d, 1, W(l, c->rel_wq), d, 1, T, 3 * d, d, EPI_STORE_BF16, a.qkv, 3 * d, nullptr,
+           nullptr, 0, &c->flops_fwd);
+      launch_rope(a.qkv, c->rope_cs, B, S, h, dh, 0, st); c->launches++;
+      if (use_mma_attn()) rc |= launch_attn_fwd_mma(a.qkv, a.U, a.lse, B, S, h, dh, st);
+      else rc |= launch_attn_fwd_simt(a.qkv, a.U, a.lse, B, S, h, dh, st);
+      c->launches++;
+      c->flops_fwd += 4.0 * B * h * dh * 0.5 * S * (double)(S + 1);
+      gemm(a.U, d, 1, W(l, c->rel_wo), d, 1, T, d, d, EPI_RESID_F32, a.x1, d, nullptr, a.x, d,
+           &c->flops_fwd);
+      launch_ln_fwd(a.x1, Pf(l, c->rel_ln2g), Pf(l, c->rel_ln2b), a.b, a.st2, T, d, c->cfg.ln_eps, st);
+      c->launches++;
+      gemm(a.b, d, 1, W(l, c->rel_win), d, 1, T, F, d, EPI_GELU_DUAL, a.Hd, F, a.A, nullptr, 0,
+           &c->flops_fwd);
+      gemm(a.A, F, 1, W(l, c->rel_wout), F, 1, T, d, F, EPI_RESID_F32, x_next, d, nullptr, a.x1, d,
+           &c->flops_fwd);
+    }
+    launch_ln_fwd(c->x_last, c->theta + c->off_lnfg, c->theta + c->off_lnfb, c->f16, c->stf, T, d,
+                  c->cfg.ln_eps, st);
+    c->launches++;
+    gemm(c->f16, d, 1, c->w16, d, 1, T, V, d, EPI_STORE_BF16, c->logits, V, nullptr, nullptr, 0,
+         &c->flops_fwd);
+  }
+
+  void loss(const int32_t* tok, int write_grad, float* out) {
+    cudaStream_t st = c->stream;
+    launch_xent(c->logits, tok, c->row_loss, B, S, V, write_grad, st); c->launches++;
+    launch_loss_reduce(c->row_loss, T, 1.f / (float)((int64_t)B * (S - 1)), out, st); c->launches++;
+  }
+
+  // Restricted backward (Appendix C.1): input gradients through every slice and head down to
+  // the lowest trained layer, weight gradients only for the replica's own hidden-unit range.
+  void backward(const ReplicaState& r) {
+    if (r.lowest < 0) return;
+    cudaStream_t st = c->stream;
+    // output head (tied embedding is frozen: no weight gradient)
+    gemm(c->logits, V, 1, c->w16, d, 0, T, d, V, EPI_STORE_BF16, c->t16, d, nullptr, nullptr, 0,
+         &c->flops_dgrad);
+    launch_ln_bwd(c->t16, c->x_last, c->stf, c->theta + c->off_lnfg, nullptr, c->g, c->g16, T, d, st);
+    c->launches++;
+    int seg = (int)r.segs.size() - 1;
+    for (int l = L - 1; l >= r.lowest && !rc; --l) {
+      LayerActs& a = c->acts[l];
+      const bool trained = seg >= 0 && r.seg_layer[seg] == l;
+      const SliceSeg* s = trained ? &r.segs[seg] : nullptr;
+      const int w = trained ? s->hi - s->lo : 0;
+      if (l == r.lowest) {
+        // only this replica's slice: dA_n = G V_n, through the activation, then both products
+        gemm(c->g16, d, 1, W(l, c->rel_wout) + s->lo, F, 0, T, w, d, EPI_DGELU, c->dHd + s->lo, F,
+             nullptr, a.Hd + s->lo, F, &c->flops_dgrad);
+      } else {
+        gemm(c->g16, d, 1, W(l, c->rel_wout), F, 0, T, F, d, EPI_DGELU, c->dHd, F, nullptr, a.Hd, F,
+             &c->flops_dgrad);
+      }
+      if (trained) {
+        // dW_in[lo:hi,:] = dHd[:,lo:hi]^T b      dW_out[:,lo:hi] = g^T A[:,lo:hi]
+        gemm(c->dHd + s->lo, F, 0, a.b, d, 0, w, d, T, EPI_STORE_F32, c->grad + s->packed_off, d,
+             nullptr, nullptr, 0, &c->flops_wgrad);
+        gemm(c->g16, d, 0, a.A + s->lo, F, 0, d, w, T, EPI_STORE_F32,
+             c->grad + s->packed_off + (int64_t)w * d, w, nullptr, nullptr, 0, &c->flops_wgrad);
+        --seg;
+      }
+      if (l == r.lowest) break;
+      gemm(c->dHd, F, 1, W(l, c->rel_win), d, 0, T, d, F, EPI_STORE_BF16, c->t16, d, nullptr,
+           nullptr, 0, &c->flops_dgrad);
+      launch_ln_bwd(c->t16, a.x1, a.st2, Pf(l, c->rel_ln2g), c->g, c->g, c->g16, T, d, st);
+      c->launches++;
+      gemm(c->g16, d, 1, W(l, c->rel_wo), d, 0, T, d, d, EPI_STORE_BF16, c->t16, d, nullptr, nullptr,
+           0, &c->flops_dgrad);
+      if (use_mma_attn())
+        rc |= launch_attn_bwd_mma(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, st);
+      else
+        rc |= launch_attn_bwd_simt(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, st);
+      c->launches += 2;
+      c->flops_dgrad += 10.0 * B * h * dh * 0.5 * S * (double)(S + 1);
+      launch_rope(c->dqkv, c->rope_cs, B, S, h, dh, 1, st); c->launches++;
+      gemm(c->dqkv, 3 * d, 1, W(l, c->rel_wq), d, 0, T, d, 3 * d, EPI_STORE_BF16, c->t16, d, nullptr,
+           nullptr, 0, &c->flops_dgrad);
+      launch_ln_bwd(c->t16, a.x, a.st1, Pf(l, c->rel_ln1g), c->g, c->g, c->g16, T, d, st);
+      c->launches++;
+    }
+  }
+};
+
+int check_step_args(ppu_ctx* c, int replica, const void* tokens, int batch, int seq) {
+  if (!c) return ppu_fail(PPU_EINVAL, "ctx is null");
+  if (replica < 0 || replica >= c->K) return ppu_fail(PPU_EINVAL, "replica %d out of range", replica);
+  if (!tokens) return ppu_fail(PPU_EINVAL, "tokens is null");
+  if (batch < 1 || batch > c->cfg.max_batch || seq < 2 || seq > c->cfg.max_seq)
+    return ppu_fail(PPU_EINVAL, "batch/seq outside [1,%d] x [2,%d]", c->cfg.max_batch, c->cfg.max_seq);
+  if ((int64_t)batch * seq > (int64_t)c->cfg.max_batch * c->cfg.max_seq)
+    return ppu_fail(PPU_EINVAL, "batch*seq too large");
+  return PPU_OK;
+}
+
+}  // namespace
+
+extern "C" int ppu_local_step(ppu_ctx* c, int replica, const int32_t* tokens, int batch, int seq) {
+  int rc = check_step_args(c, replica, tokens, batch, seq);
+  if (rc) return rc;
+  ReplicaState& r = c->reps[replica];
+  const int64_t launches0 = c->launches;
+  c->flops_fwd = c->flops_dgrad = c->flops_wgrad = 0;
+  ppu_make_resident(c, replica);
+  Sched s(c, batch, seq);
+  s.forward(tokens);
+  s.loss(tokens, 1, c->loss + replica);
+  s.backward(r);
+  if (s.rc) return ppu_fail(PPU_ECUDA, "kernel launch failed in local step (%d)", s.rc);
+  r.step += 1;
+  if (r.n_sub > 0) {
+    AdamHyper hp;
+    hp.lr = c->adam_lr; hp.beta1 = c->cfg.adam_beta1; hp.beta2 = c->cfg.adam_beta2;
+    hp.eps = c->cfg.adam_eps; hp.wd = c->cfg.adam_wd;
+    hp.bc1 = (float)(1.0 - std::pow((double)hp.beta1, (double)r.step));
+    hp.bc2 = (float)(1.0 - std::pow((double)hp.beta2, (double)r.step));
+    launch_adamw(r.d_segs, (int)r.segs.size(), r.master, r.m, r.v, c->grad, 1, 0, c->w16,
+                 c->cfg.d_model, c->cfg.d_ff, r.n_sub, hp, c->stream);
+    c->launches++;
+  }
+  r.stepped = true;
+  c->last_stepped = replica;
+  c->launches_last_step = c->launches - launches0;
+  CUDA_OK(cudaGetLastError());
+  return PPU_OK;
+}
+
+extern "C" int ppu_local_step_host(ppu_ctx* c, int replica, const int32_t* tokens_host, int batch,
+                                   int seq, double* loss_out) {
+  int rc = check_step_args(c, replica, tokens_host, batch, seq);
+  if (rc) return rc;
+  if (!loss_out) return ppu_fail(PPU_EINVAL, "loss_out is null");
+  CUDA_OK(cudaMemcpyAsync(c->tok_stage, tokens_host, sizeof(int32_t) * batch * seq,
+                          cudaMemcpyHostToDevice, c->stream));
+  rc = ppu_local_step(c, replica, c->tok_stage, batch, seq);
+  if (rc) return rc;
+  return ppu_loss(c, replica, loss_out);
+}
+
+extern "C" int ppu_loss(ppu_ctx* c, int replica, double* loss_out) {
+  if (!c) return ppu_fail(PPU_EINVAL, "ctx is null");
+  if (replica < 0 || replica >= c->K) return ppu_fail(PPU_EINVAL, "replica %d out of range", replica);
+  if (!loss_out) return ppu_fail(PPU_EINVAL, "loss_out is null");
+  if (!c->reps[replica].stepped) return ppu_fail(PPU_ESTATE, "replica %d has not run a local step", replica);
+  float v = 0.f;
+  CUDA_OK(cudaMemcpyAsync(&v, c->loss + replica, 4, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  *loss_out = (double)v;
+  return ppu_check_flags(c);
+}
+
+extern "C" int ppu_eval_loss(ppu_ctx* c, int replica, const int32_t* tokens, int batch, int seq,
+                             double* loss_out) {
+  int rc = check_step_args(c, replica < 0 ? 0 : replica, tokens, batch, seq);
+  if (rc) return rc;
+  if (replica < -1) return ppu_fail(PPU_EINVAL, "replica out of range");
+  if (!loss_out) return ppu_fail(PPU_EINVAL, "loss_out is null");
+  ppu_make_resident(c, replica);
+  Sched s(c, batch, seq);
+  s.forward(tokens);
+  s.loss(tokens, 0, c->loss + c->K);
+  if (s.rc) return ppu_fail(PPU_ECUDA, "kernel launch failed in evaluation (%d)", s.rc);
+  float v = 0.f;
+  CUDA_OK(cudaMemcpyAsync(&v, c->loss + c->K, 4, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  CUDA_OK(cudaGetLastError());
+  *loss_out = (double)v;
+  return ppu_check_flags(c);
+}
+
+extern "C" int ppu_outer_sync(ppu_ctx* c, const int32_t* replicas, int n) {
+  if (!c) return ppu_fail(PPU_EINVAL, "ctx is null");
+  if (n < 0 || (n > 0 && !replicas)) return ppu_fail(PPU_EINVAL, "bad replica list");
+  std::vector<int32_t> list(replicas, replicas + n);
+  {
+    std::vector<int32_t> sorted = list;
+    std::sort(sorted.begin(), sorted.end());
+    for (int i = 0; i < n; ++i) {
+      if (sorted[i] < 0 || sorted[i] >= c->K) return ppu_fail(PPU_EINVAL, "replica %d out of range", sorted[i]);
+      if (i && sorted[i] == sorted[i - 1]) return ppu_fail(PPU_EINVAL, "replica %d listed twice", sorted[i]);
+    }
+  }
+  const int L = c->cfg.n_layer, F = c->cfg.d_ff, d = c->cfg.d_model;
+  const int64_t launches0 = c->launches;
+  double owned = 0;
+  for (int k : list) owned += (double)c->reps[k].n_sub;
+  if (list != c->cached_sync_list || list.empty()) {
+    std::vector<OuterOwner> owners;
+    std::vector<std::vector<int32_t>> per_group((size_t)L * (F / 8));
+    for (int k : list) {
+      const ReplicaState& r = c->reps[k];
+      for (size_t i = 0; i < r.segs.size(); ++i) {
+        const SliceSeg& s = r.segs[i];
+        OuterOwner o;
+        o.master = r.master; o.in_off = s.packed_off;
+        o.out_off = s.packed_off + (int64_t)(s.hi - s.lo) * d; o.lo = s.lo; o.hi = s.hi;
+        const int32_t id = (int32_t)owners.size();
+        owners.push_back(o);
+        const int l = r.seg_layer[i];
+        for (int u8 = s.lo / 8; u8 < s.hi / 8; ++u8) per_group[(size_t)l * (F / 8) + u8].push_back(id);
+      }
+    }
+    std::vector<int32_t> begin(per_group.size() + 1, 0), flat;
+    for (size_t gi = 0; gi < per_group.size(); ++gi) {
+      begin[gi] = (int32_t)flat.size();
+      flat.insert(flat.end(), per_group[gi].begin(), per_group[gi].end());
+    }
+    begin[per_group.size()] = (int32_t)flat.size();
+    // the previous sync's kernel may still be reading the tables
+    CUDA_OK(cudaStreamSynchronize(c->stream));
+    if (!owners.empty())
+      CUDA_OK(cudaMemcpy(c->d_owners, owners.data(), owners.size() * sizeof(OuterOwner), cudaMemcpyHostToDevice));
+    CUDA_OK(cudaMemcpy(c->d_unit_begin, begin.data(), begin.size() * 4, cudaMemcpyHostToDevice));
+    if (!flat.empty())
+      CUDA_OK(cudaMemcpy(c->d_unit_owner, flat.data(), flat.size() * 4, cudaMemcpyHostToDevice));
+    c->cached_sync_list = list;
+  }
+  OuterTables t;
+  t.owners = c->d_owners; t.unit_begin = c->d_unit_begin; t.unit_owner = c->d_unit_owner;
+  t.P = c->P; t.e_size = c->e_size; t.layer_size = c->layer_size; t.win_rel = c->rel_win;
+  t.wout_rel = c->rel_wout; t.L = L; t.d = d; t.F = F;
+  launch_outer(t, c->theta, c->buf, c->w16, c->cfg.outer_lr, c->cfg.outer_momentum, c->stream);
+  c->launches++;
+  c->resident = -1;   // the working copy now holds the new global parameters everywhere
+  c->launches_last_sync = c->launches - launches0;
+  c->outer_bytes = 18.0 * (double)c->P + 8.0 * owned;
+  CUDA_OK(cudaGetLastError());
+  return PPU_OK;
+}

@@ -1,0 +1,107 @@
+"""Kernel-level parity through the C ABI: GEMM (all operand orders, both backends) against
+the oracle's matmul, and fused causal attention against the oracle's attention equations."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import ppu_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+
+def _bf16_tensor(rng, shape, scale=1.0):
+    import torch
+    x = torch.from_numpy((rng.standard_normal(shape) * scale).astype(np.float32)).cuda().bfloat16()
+    return x, x.float().cpu().numpy().astype(np.float64)
+
+
+GEMM_SHAPES = [
+    (128, 256, 64),      # exactly one wide tile
+    (256, 512, 256),     # several tiles
+    (200, 328, 136),     # ragged in every dimension
+    (8, 8, 8),           # smaller than any tile
+    (1000, 96, 4096),    # long reduction, narrow output
+    (384, 768, 520),
+]
+
+
+@pytest.mark.parametrize("backend", [0, 1])
+@pytest.mark.parametrize("a_k,b_k", [(1, 1), (1, 0), (0, 1), (0, 0)])
+@pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
+def test_gemm_against_oracle_matmul(backend, a_k, b_k, M, N, K):
+    import torch
+    from paper_2509_22418_b200 import ppu
+    rng = np.random.default_rng(M * 7 + N * 3 + K + 2 * a_k + b_k)
+    A, A64 = _bf16_tensor(rng, (M, K) if a_k else (K, M))
+    B, B64 = _bf16_tensor(rng, (N, K) if b_k else (K, N))
+    ref = (A64 if a_k else A64.T) @ (B64.T if b_k else B64)
+    for out_f32 in (True, False):
+        Cd = ppu.ppu_gemm(A, a_k, B, b_k, M, N, K, out_f32=out_f32, backend=backend)
+        torch.cuda.synchronize()
+        got = Cd.float().cpu().numpy().astype(np.float64)
+        rms = math.sqrt(float((ref ** 2).mean()))
+        tol = (2e-5 if out_f32 else 2 ** -8)
+        err = np.abs(got - ref)
+        assert np.all(err <= tol * np.abs(ref) + tol * rms), (float(err.max()), rms)
+
+
+def test_gemm_strided_operands_and_column_offset():
+    """Operands that are column windows of wider matrices (how the subset products are issued)."""
+    import torch
+    from paper_2509_22418_b200 import ppu
+    rng = np.random.default_rng(5)
+    T, F, d, lo, hi = 300, 512, 192, 64, 256
+    dH, dH64 = _bf16_tensor(rng, (T, F))
+    b, b64 = _bf16_tensor(rng, (T, d))
+    ref = dH64[:, lo:hi].T @ b64                       # dW_in[lo:hi, :]
+    for backend in (0, 1):
+        got = ppu.ppu_gemm(dH[:, lo:hi], 0, b, 0, hi - lo, d, T, out_f32=True, backend=backend)
+        torch.cuda.synchronize()
+        err = np.abs(got.cpu().numpy() - ref)
+        assert err.max() <= 2e-5 * (np.abs(ref).max() + math.sqrt((ref ** 2).mean()))
+
+
+def _attention_case(B, S, h, dh, seed):
+    rng = np.random.default_rng(seed)
+    d = h * dh
+    qkv, qkv64 = _bf16_tensor(rng, (B * S, 3 * d))
+    dU, dU64 = _bf16_tensor(rng, (B * S, d))
+    q = qkv64[:, :d].reshape(B, S, h, dh)
+    k = qkv64[:, d:2 * d].reshape(B, S, h, dh)
+    v = qkv64[:, 2 * d:].reshape(B, S, h, dh)
+    A = O.attention_probs(q, k)
+    U = np.einsum("bhst,bthd->bshd", A, v).reshape(B * S, d)
+    sc = np.einsum("bshd,bthd->bhst", q, k) / math.sqrt(dh)
+    sc = np.where(np.tril(np.ones((S, S), bool))[None, None], sc, -np.inf)
+    mx = sc.max(-1)
+    lse = mx + np.log(np.exp(sc - mx[..., None]).sum(-1))
+    return qkv, dU, dict(q=q, k=k, v=v, A=A), U, lse, dU64
+
+
+@pytest.mark.parametrize("backend", [1, 0])
+@pytest.mark.parametrize("B,S,h,dh", [(2, 64, 4, 16), (1, 200, 2, 64), (2, 256, 2, 128), (1, 130, 3, 32)])
+def test_attention_forward_backward(backend, B, S, h, dh):
+    import torch
+    from paper_2509_22418_b200 import ppu
+    qkv, dU, L, U_ref, lse_ref, dU64 = _attention_case(B, S, h, dh, seed=S + dh)
+    try:
+        U, lse = ppu.ppu_attention_fwd(qkv, B, S, h, dh, backend=backend)
+    except ppu.PpuError as e:
+        if backend == 0 and e.code == -2:
+            pytest.skip("shape not covered by the tensor-core kernel")
+        raise
+    torch.cuda.synchronize()
+    Ug = U.float().cpu().numpy()
+    assert np.abs(Ug - U_ref).max() <= 2 ** -7 * max(1.0, np.abs(U_ref).max())
+    assert np.abs(lse.cpu().numpy() - lse_ref).max() <= 1e-3
+    dq, dk, dv = O._attention_bwd(O.Model(1, h * dh, h, 8, 8), L, dU64.reshape(B, S, h * dh), None)
+    # the kernel takes delta = rowsum(dU * U) from the bf16 U it is given: use its own forward output
+    dqkv = ppu.ppu_attention_bwd(qkv, U, lse, dU, B, S, h, dh, backend=backend)
+    torch.cuda.synchronize()
+    g = dqkv.float().cpu().numpy()
+    d = h * dh
+    for name, got, ref in (("dq", g[:, :d], dq), ("dk", g[:, d:2 * d], dk), ("dv", g[:, 2 * d:], dv)):
+        ref = ref.reshape(B * S, d)
+        err = np.abs(got - ref).max()
+        assert err <= 2e-2 * np.abs(ref).max(), (name, float(err), float(np.abs(ref).max()))

@@ -1,0 +1,196 @@
+"""End-to-end parity of the CUDA path with the CPU oracle through the C ABI.
+
+Tolerances: losses 1e-3 relative; subset gradients and updated weights 2e-2 in
+max-abs over l2-norm (bf16 products, fp32 accumulation); frozen parameters, the trained
+index set and positions no replica trains are bit-exact.
+"""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import ppu_oracle as O
+from tests._harness import (LOSS_RTOL, TENSOR_TOL, Pair, bf16_bits, max_abs_over_norm, rel_l2)
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_round(P: Pair, B, S, H, rnd=0, order=None, check=True):
+    """H local steps on every replica, then an outer sync; compares after every step."""
+    K = P.K
+    report = []
+    theta0_gpu = P.ctx.ppu_get_params(-1)
+    order = order or [(k, h) for k in range(K) for h in range(H)]
+    for k, h in order:
+        tok = P.tokens(k, rnd, h, B, S)
+        loss_gpu, _ = P.gpu_step(k, tok)
+        loss_ref = P.reps[k].local_step(P.theta, tok, P.adam)
+        g_gpu = P.ctx.ppu_get_subset_grads(k)
+        g_ref = P.reps[k].last_grad
+        th_gpu = P.ctx.ppu_get_params(k)
+        idx = P.reps[k].idx
+        rec = dict(k=k, h=h, loss_gpu=loss_gpu, loss_ref=loss_ref,
+                   grad_err=max_abs_over_norm(g_gpu, g_ref), grad_l2=rel_l2(g_gpu, g_ref),
+                   w_err=max_abs_over_norm(th_gpu[idx], P.reps[k].theta_sub))
+        report.append(rec)
+        if check:
+            assert abs(loss_gpu - loss_ref) <= LOSS_RTOL * abs(loss_ref), rec
+            assert rec["grad_err"] <= TENSOR_TOL, rec
+            assert rec["w_err"] <= TENSOR_TOL, rec
+            # frozen parameters: exactly the bits that were loaded
+            mask = np.ones(len(th_gpu), bool)
+            mask[idx] = False
+            assert np.array_equal(th_gpu[mask], theta0_gpu[mask])
+            # every trained position moved (weight decay alone moves it), nothing else did
+            assert np.all(th_gpu[idx] != theta0_gpu[idx]) or h > 0
+    return report
+
+
+def _check_outer(P: Pair, replicas):
+    theta_before = P.ctx.ppu_get_params(-1)
+    P.ctx.ppu_outer_sync(replicas)
+    P.ctx.ppu_sync()
+    th_gpu = P.ctx.ppu_get_params(-1)
+    buf_gpu = P.ctx.ppu_get_outer_momentum()
+    P.theta, P.buf, m = O.outer_sync(P.theta, P.buf, [P.reps[k] for k in replicas], P.outer)
+    assert np.array_equal(th_gpu[m == 0], theta_before[m == 0])       # untouched bits
+    assert np.all(buf_gpu[m == 0] == 0)
+    tr = m > 0
+    assert max_abs_over_norm(th_gpu[tr], P.theta[tr]) <= TENSOR_TOL
+    assert max_abs_over_norm(buf_gpu[tr], P.buf[tr]) <= TENSOR_TOL
+    # working copy is the bf16 rounding of the new parameters; replicas restart from them
+    assert np.array_equal(P.ctx.ppu_get_working_bf16(), bf16_bits(th_gpu))
+    for k in replicas:
+        assert np.array_equal(P.ctx.ppu_get_params(k), th_gpu)
+    return th_gpu
+
+
+@pytest.mark.parametrize("gemm", ["tc", "simt"])
+def test_tiny_config_full_protocol(gemm, monkeypatch):
+    """Configuration 1: 2 layers, d 64, 4 heads, FFN 256, vocab 512, batch 4 x 64, N = K = 4
+    slices of 64 hidden units, 3 AdamW steps (1e-3, 0.9/0.95, wd 0.1), outer 0.7 / 0.9."""
+    monkeypatch.setenv("PPU_GEMM", gemm)
+    dims = (2, 64, 4, 256, 512)
+    ranges = [O.slice_ranges(O.Model(*dims), 4, k) for k in range(4)]
+    P = Pair(dims, ranges, 4, 64, seed=1, adam=O.AdamW(1e-3, 0.9, 0.95, 1e-8, 0.1),
+             outer=O.Outer(0.7, 0.9))
+    try:
+        for k in range(4):      # the trained index set is exact
+            assert np.array_equal(P.ctx.ppu_subset_index(k), P.reps[k].idx)
+        rep = _run_round(P, 4, 64, 3)
+        print("\n".join(str(r) for r in rep))
+        _check_outer(P, [0, 1, 2, 3])
+        # second round continues from the merged parameters with the kept AdamW state
+        rep = _run_round(P, 4, 64, 1, rnd=1)
+        _check_outer(P, [0, 1, 2, 3])
+    finally:
+        P.close()
+
+
+@pytest.mark.parametrize("gemm", ["tc", "simt"])
+def test_ragged_model_mixed_subsets(gemm, monkeypatch):
+    """Shapes that are not multiples of any tile, different ranges per layer, one replica whose
+    lowest trained layer is 1 (nothing is back-propagated below it), overlapping owners."""
+    monkeypatch.setenv("PPU_GEMM", gemm)
+    dims = (3, 192, 3, 640, 1000)
+    ranges = [
+        [(64, 192), (0, 0), (0, 640)],
+        [(0, 0), (128, 640), (8, 16)],
+        [(0, 0), (0, 0), (320, 640)],
+        [(64, 128), (128, 256), (0, 0)],
+    ]
+    P = Pair(dims, ranges, 3, 80, seed=2, adam=O.AdamW(3e-4, 0.9, 0.99, 1e-8, 0.1),
+             outer=O.Outer(0.4, 0.9))
+    try:
+        for k in range(4):
+            assert np.array_equal(P.ctx.ppu_subset_index(k), P.reps[k].idx)
+        order = [(k, h) for h in range(2) for k in range(4)]     # interleaved replicas
+        rep = _run_round(P, 3, 80, 2, order=order)
+        print("\n".join(str(r) for r in rep))
+        _check_outer(P, [0, 1, 3])          # replica 2 sits this round out
+        # replica 2 was not listed: it keeps its own values of its subset
+        th2 = P.ctx.ppu_get_params(2)
+        assert max_abs_over_norm(th2[P.reps[2].idx], P.reps[2].theta_sub) <= TENSOR_TOL
+        # shorter batch than the maximum, then everyone joins
+        _run_round(P, 2, 48, 1, rnd=1)
+        _check_outer(P, [0, 1, 2, 3])
+    finally:
+        P.close()
+
+
+def test_run_to_run_and_interleaving_determinism():
+    dims = (2, 64, 4, 256, 512)
+    ranges = [O.slice_ranges(O.Model(*dims), 4, k) for k in range(4)]
+    outs = []
+    for order in ([(k, h) for k in range(4) for h in range(2)],
+                  [(k, h) for k in range(4) for h in range(2)],
+                  [(k, h) for h in range(2) for k in (3, 1, 0, 2)]):
+        P = Pair(dims, ranges, 4, 64, seed=3)
+        try:
+            _run_round(P, 4, 64, 2, order=order, check=False)
+            P.ctx.ppu_outer_sync([0, 1, 2, 3])
+            outs.append((P.ctx.ppu_get_params(-1), P.ctx.ppu_get_outer_momentum()))
+        finally:
+            P.close()
+    for th, bf in outs[1:]:
+        assert np.array_equal(th, outs[0][0]) and np.array_equal(bf, outs[0][1])
+
+
+def test_whole_layer_subsets_and_eval_loss():
+    import torch
+    from paper_2509_22418_b200 import ppu
+    dims = (4, 64, 4, 256, 512)
+    ranges = [O.layer_ranges(O.Model(*dims), 2, k) for k in range(2)]
+    P = Pair(dims, ranges, 2, 32, seed=4, mode=ppu.SUBSET_FFN_LAYERS, layer_stride=2)
+    try:
+        for k in range(2):
+            assert np.array_equal(P.ctx.ppu_subset_index(k), P.reps[k].idx)
+        _run_round(P, 2, 32, 2)
+        tok = P.tokens(0, 9, 9, 2, 32)
+        t = torch.from_numpy(tok).cuda()
+        for k in (-1, 0, 1):
+            th = P.theta if k < 0 else P.reps[k].materialise(P.theta)
+            ref, _ = O.forward(P.ocfg, th, tok, keep=False)
+            got = P.ctx.ppu_eval_loss(k, t)
+            assert abs(got - ref) <= LOSS_RTOL * ref
+        _check_outer(P, [0, 1])
+    finally:
+        P.close()
+
+
+def test_host_entry_point_and_argument_errors():
+    from paper_2509_22418_b200 import ppu
+    dims = (2, 64, 4, 256, 512)
+    ranges = [O.slice_ranges(O.Model(*dims), 4, k) for k in range(4)]
+    P = Pair(dims, ranges, 4, 64, seed=5)
+    try:
+        tok = P.tokens(0, 0, 0, 4, 64)
+        loss = P.ctx.ppu_local_step_host(0, tok)
+        ref = P.reps[0].local_step(P.theta, tok, P.adam)
+        assert abs(loss - ref) <= LOSS_RTOL * ref
+        with pytest.raises(ppu.PpuError):
+            P.ctx.ppu_outer_sync([0, 0])
+        with pytest.raises(ppu.PpuError):
+            P.ctx.ppu_outer_sync([7])
+        with pytest.raises(ppu.PpuError):
+            P.ctx.ppu_local_step_host(9, tok)
+        with pytest.raises(ppu.PpuError):
+            P.ctx.ppu_local_step_host(0, np.zeros((5, 64), np.int32))       # batch > max_batch
+        with pytest.raises(ppu.PpuError):
+            P.ctx.ppu_loss(3)                                                # never stepped
+        bad = tok.copy()
+        bad[1, 7] = 600                                                      # id >= vocab: clamped + reported
+        with pytest.raises(ppu.PpuError) as ei:
+            P.ctx.ppu_local_step_host(1, bad)
+        assert ei.value.code == -8
+        P.ctx.ppu_sync()                                                     # flag was cleared
+    finally:
+        P.close()
+    cfg = ppu.make_cfg(2, 60, 4, 256, 512, 4, 64)                            # d_head 15
+    spec, _ = ppu.make_spec(4, n_slices=4)
+    with pytest.raises(ppu.PpuError):
+        ppu.ppu_query_bytes(cfg, spec)
+    cfg = ppu.make_cfg(2, 64, 4, 256, 512, 4, 64)
+    spec, _ = ppu.make_spec(6, n_slices=4)                                   # K not a multiple of N
+    with pytest.raises(ppu.PpuError):
+        ppu.ppu_query_bytes(cfg, spec)
