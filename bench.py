@@ -1,0 +1,260 @@
+#!/usr/bin/env python
+"""Benchmark of the partial-parameter-update hot path on B200.
+
+A step is one local step (forward on all parameters, restricted backward, AdamW on the
+replica's subset) of one simulated replica on a fresh synthetic batch; the timed region runs
+`--steps` of them, cycling through the replicas, and ends with one outer sync over the replicas
+that stepped, so every stage of the path is inside the region.  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3|c2|c1] [--impl reference]
+
+With N > 1 (launched by torch.distributed.run) every rank runs its own replicas on its own GPU:
+the path has no cross-GPU exchange step here, so ranks are independent and scaling is weak.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+WORKLOADS = {
+    # name: (L, d, heads, F, V, batch, seq, K replicas, N slices, adam(lr,b1,b2,wd), outer(lr,mu))
+    "c1": dict(dims=(2, 64, 4, 256, 512), batch=4, seq=64, K=4, N=4,
+               desc="tiny 2-layer decoder, 4 replicas x 1/4 FFN slices"),
+    "c2": dict(dims=(12, 768, 12, 3072, 32768), batch=8, seq=1024, K=8, N=8,
+               desc="125M-class decoder, 8 replicas x 1/8 FFN slices, batch 8 x 1024"),
+    "c3": dict(dims=(24, 2048, 16, 8192, 32768), batch=4, seq=2048, K=32, N=32,
+               desc="1.3B-class decoder, 32 replicas x 1/32 FFN slices, microbatch 4 x 2048"),
+}
+ADAM = dict(lr=3e-4, beta1=0.9, beta2=0.99, eps=1e-8, wd=0.1)     # Section 3.1
+OUTER = dict(lr=0.7, momentum=0.9)
+SEED = 1234
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return dict(hbm=j["hbm_gbs"], tensor_burst=j["bf16_tflops"],
+                    tensor=j.get("bf16_tflops_sustained", j["bf16_tflops"]), src="measured")
+    return dict(hbm=6650.0, tensor_burst=1590.0, tensor=1400.0, src="fallback")
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.stop_flag = index, [], False
+        self.proc = None
+
+    def run(self):
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            for line in self.proc.stdout:
+                if self.stop_flag:
+                    break
+                self.samples.append([x.strip() for x in line.split(",")])
+        except Exception:
+            pass
+
+    def finish(self):
+        self.stop_flag = True
+        if self.proc:
+            self.proc.terminate()
+        sm, mx, reasons = [], 0, set()
+        for s in self.samples:
+            try:
+                sm.append(float(s[0])); mx = max(mx, float(s[1]))
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                    "sw_power_cap"), s[2:6]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                continue
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=mx or None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def oracle_sample(w, steps, rank0_print=True):
+    """The CPU oracle on a bounded sample of the workload: one replica, a short batch."""
+    from oracle import ppu_oracle as O
+    from paper_2509_22418_b200 import synth
+    L, d, h, F, V = w["dims"]
+    cfg = O.Model(L, d, h, F, V)
+    big = O.n_params(cfg) > 5e7
+    dtype = np.float32 if big else np.float64
+    B, S = (1, 256) if O.n_params(cfg) > 5e8 else ((1, 512) if big else (w["batch"], w["seq"]))
+    theta = synth.init_params(SEED, O.layout(cfg)).astype(dtype)
+    rep = O.Replica(cfg, theta, O.slice_ranges(cfg, w["N"], 0))
+    hp = O.AdamW(**{k: ADAM[k] for k in ("lr", "beta1", "beta2", "eps", "wd")})
+    times = []
+    for s in range(steps):
+        tok = synth.tokens(SEED, 0, 0, s, B, S, V)
+        t0 = time.perf_counter()
+        rep.local_step(theta, tok, hp)
+        times.append(time.perf_counter() - t0)
+    try:
+        import threadpoolctl
+        cores = max((p.get("num_threads", 1) for p in threadpoolctl.threadpool_info()), default=1)
+    except Exception:
+        cores = os.cpu_count()
+    t = float(np.mean(times))
+    return dict(value=B * S / t, unit="tokens/s", cores=int(cores), kind="oracle",
+                sample=f"{steps} local step(s) of replica 0 on a batch of {B} x {S} tokens, "
+                       f"{np.dtype(dtype).name}, {t:.2f} s each"), t, B * S
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cb, t, ntok = oracle_sample(w, max(1, min(args.steps, 2)))
+    out = dict(metric="local-step tokens/s", value=cb["value"], unit="tokens/s", n_gpus=args.gpus,
+               steps=args.steps, warmup=args.warmup, ms_per_step=t * 1e3, higher_is_better=True,
+               scaling="weak", vs_baseline=None, dtype=cb["sample"].split(", ")[1], data="synthetic",
+               impl="reference", config=dict(workload=f"{args.workload}: {w['desc']}"),
+               cpu_baseline=cb,
+               e2e=dict(value=cb["value"], unit="tokens/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c3", choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="ppu", choices=["ppu", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        return run_reference(args, w)
+
+    import torch
+    from paper_2509_22418_b200 import build, ppu, synth
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    build.build()
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    L, d, h, F, V = w["dims"]
+    B, S, K = w["batch"], w["seq"], w["K"]
+    cfg = ppu.make_cfg(L, d, h, F, V, B, S, adam_lr=ADAM["lr"], adam_beta1=ADAM["beta1"],
+                       adam_beta2=ADAM["beta2"], adam_eps=ADAM["eps"], adam_wd=ADAM["wd"],
+                       outer_lr=OUTER["lr"], outer_momentum=OUTER["momentum"])
+    spec, keep = ppu.make_spec(K, ppu.SUBSET_FFN_SLICE, n_slices=w["N"])
+    ctx = ppu.Context(cfg, spec, keep, device=f"cuda:{local}")
+    ctx.ppu_set_params(synth.init_params(SEED + rank, ctx.tensors()))
+    n_tok = args.warmup + args.steps
+    host_tok = [synth.tokens(SEED, rank * K + (i % K), 0, i, B, S, V) for i in range(n_tok)]
+    pinned = [torch.from_numpy(t).pin_memory() for t in host_tok]
+    dev_tok = [t.to(ctx.device) for t in pinned]
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def region(use_host, profile):
+        """warm-up, then `steps` local steps and one outer sync between two events."""
+        for i in range(args.warmup):
+            ctx.ppu_local_step(i % K, dev_tok[i])
+        ctx.ppu_outer_sync(sorted({i % K for i in range(args.warmup)}))
+        ctx.ppu_sync()
+        if profile:
+            ctx.ppu_profile_enable(True)
+            ctx.ppu_profile_read()
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        barrier()
+        e0.record()
+        for j in range(args.steps):
+            i = args.warmup + j
+            if use_host:
+                ctx.ppu_local_step_host(i % K, host_tok[i])
+            else:
+                ctx.ppu_local_step(i % K, dev_tok[i])
+        e1.record()
+        ctx.ppu_outer_sync(sorted({(args.warmup + j) % K for j in range(args.steps)}))
+        e2.record()
+        barrier()
+        prof = ctx.ppu_profile_read() if profile else None
+        ctx.ppu_profile_enable(False)
+        return e0.elapsed_time(e2), e0.elapsed_time(e1), e1.elapsed_time(e2), prof
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    total_ms, steps_ms, outer_ms, prof = region(False, True)
+    clocks = sampler.finish() if rank == 0 else None
+    e2e_ms, _, _, _ = region(True, False)
+    st = ctx.ppu_stats()
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([total_ms, e2e_ms, steps_ms, outer_ms], device=ctx.device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms, steps_ms, outer_ms = t.tolist()
+    if rank != 0:
+        return
+    pk = peaks()
+    tokens = args.steps * B * S * world
+    gemm_tflops = prof.gemm_flops / (prof.gemm_ms * 1e-3) / 1e12 if prof.gemm_ms > 0 else 0.0
+    attn_tflops = prof.attn_flops / (prof.attn_ms * 1e-3) / 1e12 if prof.attn_ms > 0 else 0.0
+    out = dict(
+        metric="local-step tokens/s", value=tokens / (total_ms * 1e-3), unit="tokens/s",
+        n_gpus=world, steps=args.steps, warmup=args.warmup, ms_per_step=total_ms / args.steps,
+        higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
+        config=dict(workload=f"{args.workload}: {w['desc']}", layers=L, d_model=d, heads=h, d_ff=F,
+                    vocab=V, batch=B, seq=S, replicas=K, slices=w["N"],
+                    l2="working set per step (bf16 weights + activations) is far larger than L2; "
+                       "fresh token batch every step"),
+        local_step_ms=steps_ms / args.steps,
+        outer_sync=dict(ms=outer_ms, algorithmic_bytes=st.outer_bytes,
+                        gbs=st.outer_bytes / (outer_ms * 1e-3) / 1e9, peak_gbs=pk["hbm"],
+                        frac=st.outer_bytes / (outer_ms * 1e-3) / 1e9 / pk["hbm"], of=pk["src"]),
+        step_flops=dict(fwd=st.flops_fwd, dgrad=st.flops_dgrad, wgrad=st.flops_wgrad),
+        roofline=dict(bound="tensor", kernel="gemm_tc_kernel (tcgen05 bf16 GEMM, all products of the step)",
+                      achieved=gemm_tflops, peak=pk["tensor"], unit="TFLOP/s",
+                      frac=gemm_tflops / pk["tensor"], peak_kind=f"sustained bf16, {pk['src']}",
+                      frac_of_burst=gemm_tflops / pk["tensor_burst"], frac_of_nominal=gemm_tflops / 2250.0,
+                      launches=int(prof.gemm_launches), avg_launch_ms=prof.gemm_ms / max(1, prof.gemm_launches),
+                      gemm_share_of_step=prof.gemm_ms / steps_ms, traffic=None),
+        attention=dict(tflops=attn_tflops, ms_per_step=prof.attn_ms / args.steps,
+                       share_of_step=prof.attn_ms / steps_ms),
+        e2e=dict(value=tokens / (e2e_ms * 1e-3), unit="tokens/s", h2d_bytes_per_step=B * S * 4,
+                 d2h_bytes_per_step=4),
+        gpu_launches=int(st.launches_last_step * args.steps + st.launches_last_sync),
+        clocks=clocks, hbm_bytes=dict(arena=st.arena_bytes, state=st.state_bytes,
+                                       activations=st.activation_bytes),
+    )
+    if not args.no_cpu_baseline and world == 1:
+        out["cpu_baseline"] = oracle_sample(w, 1)[0]
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()

@@ -167,6 +167,18 @@ int ppu_sync(ppu_ctx* ctx);   /* waits for the stream; reports PPU_ETOKEN / PPU_
 int ppu_stats(ppu_ctx* ctx, ppu_stats_t* out);
 const char* ppu_last_error(void);
 
+/* Per-kernel-class device timing.  While enabled, every GEMM and attention launch of a local
+ * step is bracketed by CUDA events on the context's stream (up to a fixed pool; launches
+ * beyond it are not recorded).  ppu_profile_read waits for the stream, sums the recorded
+ * intervals and their executed FLOPs since the last read, and empties the pool. */
+typedef struct {
+  double gemm_ms, gemm_flops;   /* tcgen05 (or SIMT) GEMM launches              */
+  double attn_ms, attn_flops;   /* attention forward + backward launches        */
+  int64_t gemm_launches, attn_launches, dropped;
+} ppu_profile_t;
+int ppu_profile_enable(ppu_ctx* ctx, int enable);
+int ppu_profile_read(ppu_ctx* ctx, ppu_profile_t* out);
+
 /* ---- single-operator entry points (kernel-level parity tests) -------------- */
 
 /* C[M,N] = A . B^T on bf16 operands with fp32 accumulation (the contraction of

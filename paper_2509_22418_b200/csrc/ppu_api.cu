@@ -303,6 +303,7 @@ extern "C" int ppu_create(const ppu_model_cfg* cfg, const ppu_subset_spec* spec,
 extern "C" int ppu_destroy(ppu_ctx* ctx) {
   if (!ctx) return PPU_OK;
   cudaStreamSynchronize(ctx->stream);
+  for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
   delete ctx;
   return PPU_OK;
 }
@@ -364,7 +365,7 @@ extern "C" int ppu_get_params(ppu_ctx* c, int replica, float* theta, int64_t n) 
     CUDA_OK(cudaStreamSynchronize(c->stream));
     return PPU_OK;
   }
-  // overlay the replica's subset on a scratch copy: the gradient stream buffer is free between calls
+  // global vector first, then the replica's packed subset is laid over it on the host
   ReplicaState& r = c->reps[replica];
   CUDA_OK(cudaMemcpyAsync(theta, c->theta, n * 4, cudaMemcpyDeviceToHost, c->stream));
   CUDA_OK(cudaStreamSynchronize(c->stream));

@@ -67,6 +67,12 @@ struct ppu_ctx {
   OuterOwner* d_owners = nullptr;
   int32_t *d_unit_begin = nullptr, *d_unit_owner = nullptr;
   std::vector<int32_t> cached_sync_list;
+  // per-class event timing
+  bool profiling = false;
+  std::vector<cudaEvent_t> ev_pool;           // pairs: [2i] start, [2i+1] stop
+  struct EvRec { int cls; double flops; };
+  std::vector<EvRec> ev_recs;
+  int64_t ev_dropped = 0;
   // stats
   int64_t launches = 0, launches_last_step = 0, launches_last_sync = 0;
   double flops_fwd = 0, flops_dgrad = 0, flops_wgrad = 0, outer_bytes = 0;

@@ -47,6 +47,26 @@ int ppu_make_resident(ppu_ctx* c, int k) {
 
 namespace {
 
+constexpr size_t EV_POOL_PAIRS = 16384;
+
+// Brackets one launch with events when profiling is on.
+struct EvScope {
+  ppu_ctx* c; int slot = -1;
+  EvScope(ppu_ctx* ctx, int cls, double flops) : c(ctx) {
+    if (!c->profiling) return;
+    if (c->ev_recs.size() >= EV_POOL_PAIRS) { c->ev_dropped++; return; }
+    slot = (int)c->ev_recs.size();
+    if (c->ev_pool.size() < 2 * (size_t)(slot + 1)) {
+      cudaEvent_t a, b;
+      if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { slot = -1; return; }
+      c->ev_pool.push_back(a); c->ev_pool.push_back(b);
+    }
+    c->ev_recs.push_back({cls, flops});
+    cudaEventRecord(c->ev_pool[2 * slot], c->stream);
+  }
+  ~EvScope() { if (slot >= 0) cudaEventRecord(c->ev_pool[2 * slot + 1], c->stream); }
+};
+
 struct Sched {
   ppu_ctx* c;
   int B, S, T, d, F, V, h, dh, L;
@@ -67,6 +87,7 @@ struct Sched {
     g.A = A; g.lda = lda; g.a_kmajor = ak; g.B = Bm; g.ldb = ldb; g.b_kmajor = bk;
     g.M = M; g.N = N; g.K = K; g.epilogue = epi; g.C = C; g.ldc = ldc; g.C2 = C2; g.aux = aux;
     g.ldaux = ldaux; g.flags = c->flags;
+    EvScope ev(c, 0, 2.0 * M * N * (double)K);
     rc = c->gemm_backend == 1 ? launch_gemm_simt(g, c->stream) : launch_gemm_tc(g, c->stream);
     c->launches++;
     if (flop_counter) *flop_counter += 2.0 * M * N * (double)K;
@@ -86,10 +107,14 @@ struct Sched {
       gemm(c->a16, d, 1, W(l, c->rel_wq), d, 1, T, 3 * d, d, EPI_STORE_BF16, a.qkv, 3 * d, nullptr,
            nullptr, 0, &c->flops_fwd);
       launch_rope(a.qkv, c->rope_cs, B, S, h, dh, 0, st); c->launches++;
-      if (use_mma_attn()) rc |= launch_attn_fwd_mma(a.qkv, a.U, a.lse, B, S, h, dh, st);
-      else rc |= launch_attn_fwd_simt(a.qkv, a.U, a.lse, B, S, h, dh, st);
-      c->launches++;
-      c->flops_fwd += 4.0 * B * h * dh * 0.5 * S * (double)(S + 1);
+      {
+        const double fl = 4.0 * B * h * dh * 0.5 * S * (double)(S + 1);
+        EvScope ev(c, 1, fl);
+        if (use_mma_attn()) rc |= launch_attn_fwd_mma(a.qkv, a.U, a.lse, B, S, h, dh, st);
+        else rc |= launch_attn_fwd_simt(a.qkv, a.U, a.lse, B, S, h, dh, st);
+        c->launches++;
+        c->flops_fwd += fl;
+      }
       gemm(a.U, d, 1, W(l, c->rel_wo), d, 1, T, d, d, EPI_RESID_F32, a.x1, d, nullptr, a.x, d,
            &c->flops_fwd);
       launch_ln_fwd(a.x1, Pf(l, c->rel_ln2g), Pf(l, c->rel_ln2b), a.b, a.st2, T, d, c->cfg.ln_eps, st);
@@ -151,12 +176,16 @@ struct Sched {
       c->launches++;
       gemm(c->g16, d, 1, W(l, c->rel_wo), d, 0, T, d, d, EPI_STORE_BF16, c->t16, d, nullptr, nullptr,
            0, &c->flops_dgrad);
-      if (use_mma_attn())
-        rc |= launch_attn_bwd_mma(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, st);
-      else
-        rc |= launch_attn_bwd_simt(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, st);
-      c->launches += 2;
-      c->flops_dgrad += 10.0 * B * h * dh * 0.5 * S * (double)(S + 1);
+      {
+        const double fl = 10.0 * B * h * dh * 0.5 * S * (double)(S + 1);
+        EvScope ev(c, 1, fl);
+        if (use_mma_attn())
+          rc |= launch_attn_bwd_mma(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, st);
+        else
+          rc |= launch_attn_bwd_simt(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, st);
+        c->launches += 2;
+        c->flops_dgrad += fl;
+      }
       launch_rope(c->dqkv, c->rope_cs, B, S, h, dh, 1, st); c->launches++;
       gemm(c->dqkv, 3 * d, 1, W(l, c->rel_wq), d, 0, T, d, 3 * d, EPI_STORE_BF16, c->t16, d, nullptr,
            nullptr, 0, &c->flops_dgrad);
@@ -309,5 +338,27 @@ extern "C" int ppu_outer_sync(ppu_ctx* c, const int32_t* replicas, int n) {
   c->launches_last_sync = c->launches - launches0;
   c->outer_bytes = 18.0 * (double)c->P + 8.0 * owned;
   CUDA_OK(cudaGetLastError());
+  return PPU_OK;
+}
+
+extern "C" int ppu_profile_enable(ppu_ctx* c, int enable) {
+  if (!c) return ppu_fail(PPU_EINVAL, "ctx is null");
+  c->profiling = enable != 0;
+  return PPU_OK;
+}
+
+extern "C" int ppu_profile_read(ppu_ctx* c, ppu_profile_t* out) {
+  if (!c || !out) return ppu_fail(PPU_EINVAL, "null argument");
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  memset(out, 0, sizeof(*out));
+  for (size_t i = 0; i < c->ev_recs.size(); ++i) {
+    float ms = 0.f;
+    CUDA_OK(cudaEventElapsedTime(&ms, c->ev_pool[2 * i], c->ev_pool[2 * i + 1]));
+    if (c->ev_recs[i].cls == 0) { out->gemm_ms += ms; out->gemm_flops += c->ev_recs[i].flops; out->gemm_launches++; }
+    else { out->attn_ms += ms; out->attn_flops += c->ev_recs[i].flops; out->attn_launches++; }
+  }
+  out->dropped = c->ev_dropped;
+  c->ev_recs.clear();
+  c->ev_dropped = 0;
   return PPU_OK;
 }

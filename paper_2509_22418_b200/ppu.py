@@ -48,6 +48,12 @@ class Stats(C.Structure):
                 ("flops_dgrad", C.c_double), ("flops_wgrad", C.c_double), ("outer_bytes", C.c_double)]
 
 
+class Profile(C.Structure):
+    _fields_ = [("gemm_ms", C.c_double), ("gemm_flops", C.c_double), ("attn_ms", C.c_double),
+                ("attn_flops", C.c_double), ("gemm_launches", C.c_int64),
+                ("attn_launches", C.c_int64), ("dropped", C.c_int64)]
+
+
 _lib = None
 
 
@@ -221,6 +227,14 @@ class Context:
 
     def ppu_sync(self) -> None:
         _check(lib().ppu_sync(self._h))
+
+    def ppu_profile_enable(self, enable: bool) -> None:
+        _check(lib().ppu_profile_enable(self._h, int(enable)))
+
+    def ppu_profile_read(self) -> Profile:
+        p = Profile()
+        _check(lib().ppu_profile_read(self._h, C.byref(p)))
+        return p
 
     def ppu_stats(self) -> Stats:
         s = Stats()

@@ -41,8 +41,8 @@ def _run_round(P: Pair, B, S, H, rnd=0, order=None, check=True):
             mask = np.ones(len(th_gpu), bool)
             mask[idx] = False
             assert np.array_equal(th_gpu[mask], theta0_gpu[mask])
-            # every trained position moved (weight decay alone moves it), nothing else did
-            assert np.all(th_gpu[idx] != theta0_gpu[idx]) or h > 0
+            # the trained positions moved (an update that rounds to nothing is a rare accident)
+            assert (th_gpu[idx] != theta0_gpu[idx]).mean() > 0.999
     return report
 
 
