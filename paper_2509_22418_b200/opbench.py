@@ -1,0 +1,70 @@
+"""Single-kernel timing driver: python -m paper_2509_22418_b200.opbench <op> [options]
+
+  gemm  --m M --n N --k K [--a-mn] [--b-mn] [--f32]   one GEMM through ppu_gemm
+  attn  --batch B --seq S --heads H --dh D             attention forward + backward
+Times with CUDA events on the launching stream after warm-up; operands are sized by the caller
+(keep them above the 126 MB L2 if DRAM behaviour matters).  Also the target of profiler runs.
+"""
+import argparse
+import sys
+
+import torch
+
+from . import build, ppu
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("op", choices=["gemm", "attn"])
+    ap.add_argument("--m", type=int, default=8192)
+    ap.add_argument("--n", type=int, default=8192)
+    ap.add_argument("--k", type=int, default=2048)
+    ap.add_argument("--a-mn", action="store_true")
+    ap.add_argument("--b-mn", action="store_true")
+    ap.add_argument("--f32", action="store_true")
+    ap.add_argument("--batch", type=int, default=4)
+    ap.add_argument("--seq", type=int, default=2048)
+    ap.add_argument("--heads", type=int, default=16)
+    ap.add_argument("--dh", type=int, default=128)
+    ap.add_argument("--iters", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    a = ap.parse_args()
+    build.build()
+    dev = torch.device("cuda:0")
+    g = torch.Generator(device="cpu").manual_seed(0)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def timed(fn):
+        for _ in range(a.warmup):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = ev(), ev()
+        e0.record()
+        for _ in range(a.iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / a.iters
+
+    if a.op == "gemm":
+        A = torch.randn((a.k, a.m) if a.a_mn else (a.m, a.k), generator=g).to(dev).bfloat16()
+        B = torch.randn((a.k, a.n) if a.b_mn else (a.n, a.k), generator=g).to(dev).bfloat16()
+        ms = timed(lambda: ppu.ppu_gemm(A, not a.a_mn, B, not a.b_mn, a.m, a.n, a.k, out_f32=a.f32))
+        fl = 2.0 * a.m * a.n * a.k
+        print(f"gemm M={a.m} N={a.n} K={a.k} a_mn={a.a_mn} b_mn={a.b_mn}: {ms:.4f} ms "
+              f"{fl / ms / 1e9:.1f} TFLOP/s")
+    else:
+        B_, S, h, dh = a.batch, a.seq, a.heads, a.dh
+        d = h * dh
+        qkv = torch.randn((B_ * S, 3 * d), generator=g).to(dev).bfloat16()
+        dU = torch.randn((B_ * S, d), generator=g).to(dev).bfloat16()
+        U, lse = ppu.ppu_attention_fwd(qkv, B_, S, h, dh)
+        fl = 4.0 * B_ * h * dh * 0.5 * S * (S + 1)
+        ms = timed(lambda: ppu.ppu_attention_fwd(qkv, B_, S, h, dh))
+        print(f"attn fwd B={B_} S={S} h={h} dh={dh}: {ms:.4f} ms {fl / ms / 1e9:.1f} TFLOP/s (causal)")
+        ms = timed(lambda: ppu.ppu_attention_bwd(qkv, U, lse, dU, B_, S, h, dh))
+        print(f"attn bwd: {ms:.4f} ms {2.5 * fl / ms / 1e9:.1f} TFLOP/s (causal, 2.5 x forward)")
+
+
+if __name__ == "__main__":
+    sys.exit(main())
