@@ -203,6 +203,23 @@ int ppu_attention_bwd(const void* qkv, const void* U, const float* lse, const vo
                       void* dqkv, float* scratch, int batch, int seq, int n_head, int d_head,
                       int backend, void* cuda_stream);
 
+/* No counterpart in the paper: a convenience for callers that cannot allocate device memory
+ * (code running while a stream is being captured, hosts whose framework owns the allocator,
+ * processes that are handed fixed buffers only).  Same computation and arguments as
+ * ppu_attention_bwd, but the per-row scratch lives in a fixed array inside the library image
+ * instead of being passed in; the call itself allocates nothing.
+ *  - Limit: batch * n_head * seq <= PPU_STATIC_SCRATCH_FLOATS, else PPU_ESHAPE.  Each GPU that
+ *    loads the library holds the array (4 MiB) until the process exits.
+ *  - The first call on a device looks up the array's device address (with that device current);
+ *    make that first call before starting any stream capture.
+ *  - All calls share the one array.  It needs no clearing (each call writes every row it later
+ *    reads), but two calls that overlap on the GPU - different streams, or different threads -
+ *    race on it: keep calls to this entry point on one stream, or order them yourself. */
+#define PPU_STATIC_SCRATCH_FLOATS (1 << 20)
+int ppu_attention_bwd_static(const void* qkv, const void* U, const float* lse, const void* dU,
+                             void* dqkv, int batch, int seq, int n_head, int d_head, int backend,
+                             void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

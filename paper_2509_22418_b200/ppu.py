@@ -277,3 +277,19 @@ def ppu_attention_bwd(qkv, U, lse, dU, batch, seq, n_head, d_head, backend=0):
                                    C.c_void_p(dqkv.data_ptr()), C.c_void_p(scratch.data_ptr()),
                                    batch, seq, n_head, d_head, backend, C.c_void_p(st)))
     return dqkv
+
+
+STATIC_SCRATCH_FLOATS = 1 << 20
+
+
+def ppu_attention_bwd_static(qkv, U, lse, dU, batch, seq, n_head, d_head, backend=0):
+    """Attention backward without caller scratch: for users who cannot allocate device memory
+    at the point of the call.  Limited to batch * n_head * seq <= STATIC_SCRATCH_FLOATS."""
+    import torch
+    dqkv = torch.empty_like(qkv)
+    st = torch.cuda.current_stream(qkv.device).cuda_stream
+    _check(lib().ppu_attention_bwd_static(C.c_void_p(qkv.data_ptr()), C.c_void_p(U.data_ptr()),
+                                          C.c_void_p(lse.data_ptr()), C.c_void_p(dU.data_ptr()),
+                                          C.c_void_p(dqkv.data_ptr()), batch, seq, n_head, d_head,
+                                          backend, C.c_void_p(st)))
+    return dqkv
