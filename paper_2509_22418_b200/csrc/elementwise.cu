@@ -169,6 +169,104 @@ ln_bwd_kernel(const bf16* __restrict__ dy, const float* __restrict__ x,
   }
 }
 
+// ---- warp-per-row LayerNorm (d a multiple of 256): the row lives in registers, lane l owns
+// the 8-element chunks l, l+32, ...; no shared memory, no block barrier ----
+template <int NV>
+__global__ void __launch_bounds__(128)
+ln_fwd_warp_kernel(const float* __restrict__ x, const float* __restrict__ g,
+                   const float* __restrict__ b, bf16* __restrict__ y, float2* __restrict__ stats,
+                   int T, float eps) {
+  constexpr int d = NV * 256;
+  const int64_t t = blockIdx.x * 4 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (t >= T) return;
+  const float4* src = reinterpret_cast<const float4*>(x + t * d);
+  float v[NV][8];
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int c = lane + 32 * i;
+    const float4 a = src[2 * c], bq = src[2 * c + 1];
+    v[i][0] = a.x; v[i][1] = a.y; v[i][2] = a.z; v[i][3] = a.w;
+    v[i][4] = bq.x; v[i][5] = bq.y; v[i][6] = bq.z; v[i][7] = bq.w;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) s += v[i][j];
+  }
+  const float mean = warp_sum(s) * (1.f / d);
+  float q = 0.f;
+#pragma unroll
+  for (int i = 0; i < NV; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { const float e = v[i][j] - mean; q += e * e; }
+  const float rstd = rsqrtf(warp_sum(q) * (1.f / d) + eps);
+  if (lane == 0) stats[t] = make_float2(mean, rstd);
+  uint4* dst = reinterpret_cast<uint4*>(y + t * d);
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int c = lane + 32 * i;
+    const float4 g0 = reinterpret_cast<const float4*>(g)[2 * c], g1 = reinterpret_cast<const float4*>(g)[2 * c + 1];
+    const float4 b0 = reinterpret_cast<const float4*>(b)[2 * c], b1 = reinterpret_cast<const float4*>(b)[2 * c + 1];
+    const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+    const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+    float f[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) f[j] = (v[i][j] - mean) * rstd * gg[j] + bb[j];
+    dst[c] = pack8(f);
+  }
+}
+
+template <int NV>
+__global__ void __launch_bounds__(128)
+ln_bwd_warp_kernel(const bf16* __restrict__ dy, const float* __restrict__ x,
+                   const float2* __restrict__ stats, const float* __restrict__ gamma,
+                   const float* gin, float* gout, bf16* __restrict__ gout16, int T) {
+  constexpr int d = NV * 256;
+  const int64_t t = blockIdx.x * 4 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (t >= T) return;
+  const float2 st = stats[t];
+  const uint4* dsrc = reinterpret_cast<const uint4*>(dy + t * d);
+  const float4* xsrc = reinterpret_cast<const float4*>(x + t * d);
+  float a[NV][8], hh[NV][8];
+  float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int c = lane + 32 * i;
+    float f[8];
+    unpack8(dsrc[c], f);
+    const float4 xa = xsrc[2 * c], xb = xsrc[2 * c + 1];
+    const float4 g0 = reinterpret_cast<const float4*>(gamma)[2 * c], g1 = reinterpret_cast<const float4*>(gamma)[2 * c + 1];
+    const float xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+    const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      a[i][j] = f[j] * gg[j];
+      hh[i][j] = (xv[j] - st.x) * st.y;
+      s1 += a[i][j];
+      s2 += a[i][j] * hh[i][j];
+    }
+  }
+  const float m1 = warp_sum(s1) * (1.f / d), m2 = warp_sum(s2) * (1.f / d);
+  const float4* gsrc = gin ? reinterpret_cast<const float4*>(gin + t * d) : nullptr;
+  float4* gdst = reinterpret_cast<float4*>(gout + t * d);
+  uint4* g16 = reinterpret_cast<uint4*>(gout16 + t * d);
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int c = lane + 32 * i;
+    float f[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) f[j] = st.y * (a[i][j] - m1 - hh[i][j] * m2);
+    if (gsrc) {
+      const float4 p0 = gsrc[2 * c], p1 = gsrc[2 * c + 1];
+      f[0] += p0.x; f[1] += p0.y; f[2] += p0.z; f[3] += p0.w;
+      f[4] += p1.x; f[5] += p1.y; f[6] += p1.z; f[7] += p1.w;
+    }
+    gdst[2 * c] = make_float4(f[0], f[1], f[2], f[3]);
+    gdst[2 * c + 1] = make_float4(f[4], f[5], f[6], f[7]);
+    g16[c] = pack8(f);
+  }
+}
+
 // ---- rotary positions on the q and k parts of qkv[T,3d], in place ----
 // cs: [S, dh/2] (cos, sin) pairs computed on the host in double precision.
 __global__ void rope_kernel(bf16* __restrict__ qkv, const float2* __restrict__ cs, int S, int d,
@@ -291,11 +389,25 @@ void launch_embed(const int32_t* tok, const bf16* E16, float* x, int T, int d, i
 
 void launch_ln_fwd(const float* x, const float* g, const float* b, bf16* y, float2* stats, int T,
                    int d, float eps, cudaStream_t st) {
+  const unsigned wb = (unsigned)((T + 3) / 4);
+  switch (d % 256 == 0 ? d / 256 : 0) {
+#define LNF(NV) case NV: ln_fwd_warp_kernel<NV><<<wb, 128, 0, st>>>(x, g, b, y, stats, T, eps); return;
+    LNF(1) LNF(2) LNF(3) LNF(4) LNF(6) LNF(8) LNF(12) LNF(16)
+#undef LNF
+    default: break;
+  }
   ln_fwd_kernel<<<T, LN_THREADS, d * sizeof(float), st>>>(x, g, b, y, stats, d, eps);
 }
 
 void launch_ln_bwd(const bf16* dy, const float* x, const float2* stats, const float* gamma,
                    const float* gin, float* gout, bf16* gout16, int T, int d, cudaStream_t st) {
+  const unsigned wb = (unsigned)((T + 3) / 4);
+  switch (d % 256 == 0 ? d / 256 : 0) {
+#define LNB(NV) case NV: ln_bwd_warp_kernel<NV><<<wb, 128, 0, st>>>(dy, x, stats, gamma, gin, gout, gout16, T); return;
+    LNB(1) LNB(2) LNB(3) LNB(4) LNB(6) LNB(8) LNB(12) LNB(16)
+#undef LNB
+    default: break;
+  }
   ln_bwd_kernel<<<T, LN_THREADS, 2 * d * sizeof(float), st>>>(dy, x, stats, gamma, gin, gout,
                                                               gout16, d);
 }

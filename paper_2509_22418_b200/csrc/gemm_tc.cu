@@ -17,7 +17,8 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;            // 64 bf16 = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
-constexpr int GEMM_THREADS = 192; // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr int EPI_WARPS = 8;      // two per TMEM lane quarter, each draining half the columns
+constexpr int GEMM_THREADS = 64 + 32 * EPI_WARPS;  // warp 0: TMA, warp 1: MMA + TMEM owner, then epilogue
 constexpr uint32_t WAIT_LIMIT = 1u << 20;
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
@@ -118,14 +119,20 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint
   return d;
 }
 
+// hardware tanh (relative error about 2^-11, below the bf16 rounding of the stored result)
+__device__ __forceinline__ float tanh_fast(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ float gelu_dev(float x) {
   const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
-  const float t = 1.f - 2.f / (1.f + __expf(2.f * u));
+  const float t = tanh_fast(u);
   return 0.5f * x * (1.f + t);
 }
 __device__ __forceinline__ float gelu_grad_dev(float x) {
   const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
-  const float t = 1.f - 2.f / (1.f + __expf(2.f * u));
+  const float t = tanh_fast(u);
   const float du = 0.7978845608028654f * (1.f + 3.f * 0.044715f * x * x);
   return 0.5f * (1.f + t) + 0.5f * x * (1.f - t * t) * du;
 }
@@ -178,7 +185,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), EPI_WARPS); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -269,65 +276,82 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
   } else {
     // ---------------- epilogue warps ----------------
     const int quarter = warp & 3;              // TMEM lanes [32 q, 32 q + 32) belong to this warp
+    const int half = (warp - 2) >> 2;          // which half of the tile's columns
     int acc = 0; uint32_t acc_ph = 0;
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
       const int m0 = (tile % p.tiles_m) * BM, n0 = (tile / p.tiles_m) * BN;
       if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.flags)) break;
       tc_fence_after();
       const int m = m0 + quarter * 32 + lane;
+      const bool row_ok = m < p.M;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        if (n0 + c0 >= p.N) break;             // warp-uniform
+      for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
+        const int nb = n0 + c0;
+        if (nb >= p.N) break;                  // warp-uniform
         uint32_t r[32];
-        tmem_ld32(t_row + c0, r);
-        tmem_ld_wait();
-        if (m < p.M) {
+        tmem_ld32(t_row + c0, r);              // asynchronous until tmem_ld_wait
+        const long long ci = (long long)m * p.ldc + nb;
+        const bool full = nb + 32 <= p.N;
+        if (p.epilogue == EPI_RESID_F32) {
+          float4 x[8];
+          const float4* rs = reinterpret_cast<const float4*>((const float*)p.aux + (long long)m * p.ldaux + nb);
 #pragma unroll
-          for (int g8 = 0; g8 < 4; ++g8) {
-            const int n = n0 + c0 + 8 * g8;
-            if (n >= p.N) break;
-            float f[8];
+          for (int j = 0; j < 8; ++j)
+            x[j] = (row_ok && (full || nb + 4 * j < p.N)) ? rs[j] : make_float4(0.f, 0.f, 0.f, 0.f);
+          tmem_ld_wait();
+          if (row_ok) {
+            float4* o = reinterpret_cast<float4*>((float*)p.C + ci);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(r[8 * g8 + j]);
-            const long long ci = (long long)m * p.ldc + n;
-            switch (p.epilogue) {
-              case EPI_STORE_BF16:
-                *reinterpret_cast<uint4*>((bf16*)p.C + ci) = pack8_bf16(f);
-                break;
-              case EPI_STORE_F32: {
-                float4* o = reinterpret_cast<float4*>((float*)p.C + ci);
+            for (int j = 0; j < 8; ++j)
+              if (full || nb + 4 * j < p.N)
+                o[j] = make_float4(x[j].x + __uint_as_float(r[4 * j]), x[j].y + __uint_as_float(r[4 * j + 1]),
+                                   x[j].z + __uint_as_float(r[4 * j + 2]), x[j].w + __uint_as_float(r[4 * j + 3]));
+          }
+        } else if (p.epilogue == EPI_DGELU) {
+          uint4 hv[4];
+          const uint4* hs = reinterpret_cast<const uint4*>((const bf16*)p.aux + (long long)m * p.ldaux + nb);
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            hv[j] = (row_ok && (full || nb + 8 * j < p.N)) ? hs[j] : make_uint4(0, 0, 0, 0);
+          tmem_ld_wait();
+          if (row_ok) {
+            uint4* o = reinterpret_cast<uint4*>((bf16*)p.C + ci);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              if (!(full || nb + 8 * j < p.N)) break;
+              const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hv[j]);
+              float a[8];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const float2 h2 = __bfloat1622float2(hp[q]);
+                a[2 * q] = __uint_as_float(r[8 * j + 2 * q]) * gelu_grad_dev(h2.x);
+                a[2 * q + 1] = __uint_as_float(r[8 * j + 2 * q + 1]) * gelu_grad_dev(h2.y);
+              }
+              o[j] = pack8_bf16(a);
+            }
+          }
+        } else {
+          tmem_ld_wait();
+          if (row_ok) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              if (!(full || nb + 8 * j < p.N)) break;
+              float f[8];
+#pragma unroll
+              for (int q = 0; q < 8; ++q) f[q] = __uint_as_float(r[8 * j + q]);
+              if (p.epilogue == EPI_STORE_F32) {
+                float4* o = reinterpret_cast<float4*>((float*)p.C + ci + 8 * j);
                 o[0] = make_float4(f[0], f[1], f[2], f[3]);
                 o[1] = make_float4(f[4], f[5], f[6], f[7]);
-              } break;
-              case EPI_GELU_DUAL: {
-                *reinterpret_cast<uint4*>((bf16*)p.C + ci) = pack8_bf16(f);
-                float a[8];
+              } else {
+                *reinterpret_cast<uint4*>((bf16*)p.C + ci + 8 * j) = pack8_bf16(f);
+                if (p.epilogue == EPI_GELU_DUAL) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) a[j] = gelu_dev(f[j]);
-                *reinterpret_cast<uint4*>((bf16*)p.C2 + ci) = pack8_bf16(a);
-              } break;
-              case EPI_RESID_F32: {
-                const float4* rs =
-                    reinterpret_cast<const float4*>((const float*)p.aux + (long long)m * p.ldaux + n);
-                const float4 r0 = rs[0], r1 = rs[1];
-                float4* o = reinterpret_cast<float4*>((float*)p.C + ci);
-                o[0] = make_float4(r0.x + f[0], r0.y + f[1], r0.z + f[2], r0.w + f[3]);
-                o[1] = make_float4(r1.x + f[4], r1.y + f[5], r1.z + f[6], r1.w + f[7]);
-              } break;
-              case EPI_DGELU: {
-                const uint4 hv = *reinterpret_cast<const uint4*>((const bf16*)p.aux +
-                                                                 (long long)m * p.ldaux + n);
-                const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hv);
-                float a[8];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  const float2 h2 = __bfloat1622float2(hp[j]);
-                  a[2 * j] = f[2 * j] * gelu_grad_dev(h2.x);
-                  a[2 * j + 1] = f[2 * j + 1] * gelu_grad_dev(h2.y);
+                  for (int q = 0; q < 8; ++q) f[q] = gelu_dev(f[q]);
+                  *reinterpret_cast<uint4*>((bf16*)p.C2 + ci + 8 * j) = pack8_bf16(f);
                 }
-                *reinterpret_cast<uint4*>((bf16*)p.C + ci) = pack8_bf16(a);
-              } break;
+              }
             }
           }
         }

@@ -118,6 +118,18 @@ def test_ragged_model_mixed_subsets(gemm, monkeypatch):
         P.close()
 
 
+def test_wide_rows_use_the_register_layernorm():
+    """d_model 256 / 768: rows that take the warp-per-row LayerNorm kernels; d_head 64 and 128."""
+    for dims, B, S in (((2, 256, 2, 512, 1024), 2, 96), ((2, 768, 12, 1024, 2048), 1, 160)):
+        ranges = [O.slice_ranges(O.Model(*dims), 2, k) for k in range(2)]
+        P = Pair(dims, ranges, B, S, seed=6)
+        try:
+            _run_round(P, B, S, 2)
+            _check_outer(P, [0, 1])
+        finally:
+            P.close()
+
+
 def test_run_to_run_and_interleaving_determinism():
     dims = (2, 64, 4, 256, 512)
     ranges = [O.slice_ranges(O.Model(*dims), 4, k) for k in range(4)]
