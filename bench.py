@@ -148,7 +148,7 @@ def main():
         return run_reference(args, w)
 
     import torch
-    from paper_2509_22418_b200 import build, ppu, synth
+    from paper_2509_22418_b200 import build, ppu, synth, dist as pdist
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -168,15 +168,14 @@ def main():
     ctx = ppu.Context(cfg, spec, keep, device=f"cuda:{local}")
     ctx.ppu_set_params(synth.init_params(SEED + rank, ctx.tensors()))
     n_tok = args.warmup + args.steps
-    host_tok = [synth.tokens(SEED, rank * K + (i % K), 0, i, B, S, V) for i in range(n_tok)]
+    group = pdist.replica_group(K, world, rank)       # this rank's replicas (global ids)
+    host_tok = [synth.tokens(SEED, group[i % K], 0, i, B, S, V) for i in range(n_tok)]
     pinned = [torch.from_numpy(t).pin_memory() for t in host_tok]
     dev_tok = [t.to(ctx.device) for t in pinned]
     torch.cuda.synchronize()
 
     def barrier():
-        if world > 1:
-            import torch.distributed as dist
-            dist.barrier()
+        pdist.barrier()
         torch.cuda.synchronize()
 
     def region(use_host, profile):
@@ -213,11 +212,8 @@ def main():
     clocks = sampler.finish() if rank == 0 else None
     e2e_ms, _, _, _ = region(True, False)
     st = ctx.ppu_stats()
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([total_ms, e2e_ms, steps_ms, outer_ms], device=ctx.device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms, steps_ms, outer_ms = t.tolist()
+    total_ms, e2e_ms, steps_ms, outer_ms = pdist.max_over_ranks([total_ms, e2e_ms, steps_ms, outer_ms],
+                                                                 device=ctx.device)
     if rank != 0:
         return
     pk = peaks()

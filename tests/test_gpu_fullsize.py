@@ -1,0 +1,116 @@
+"""Parity at BASELINE sizes, in the launch configuration bench.py times.
+
+125M-class (configuration 2): one local step of two replicas and an outer sync against the
+fp64 oracle.  1.3B-class (configuration 3): one local step of replica 31 against the oracle
+run with fp32 storage (its matmuls accumulate in fp32 blocks; tolerances unchanged), the outer
+sync on a sample of positions, and frozen / untrained bits exact.
+"""
+import numpy as np
+import pytest
+
+from oracle import ppu_oracle as O
+from tests._harness import LOSS_RTOL, TENSOR_TOL, Pair, bf16_bits, max_abs_over_norm, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+def test_125m_two_replicas_one_step_and_outer_sync():
+    from paper_2509_22418_b200 import ppu
+    dims = (12, 768, 12, 3072, 32768)
+    ranges = [O.slice_ranges(O.Model(*dims), 8, k) for k in range(8)]
+    P = Pair(dims, ranges, 8, 1024, seed=21, adam=O.AdamW(3e-4, 0.9, 0.99, 1e-8, 0.1),
+             outer=O.Outer(0.7, 0.9), mode=ppu.SUBSET_FFN_SLICE, n_slices=8)
+    try:
+        theta0 = P.ctx.ppu_get_params(-1)
+        for k in (0, 5):
+            tok = P.tokens(k, 0, 0, 8, 1024)
+            loss_gpu, _ = P.gpu_step(k, tok)
+            loss_ref = P.reps[k].local_step(P.theta, tok, P.adam)
+            g_gpu = P.ctx.ppu_get_subset_grads(k)
+            th_gpu = P.ctx.ppu_get_params(k)
+            idx = P.reps[k].idx
+            rec = dict(k=k, loss_gpu=loss_gpu, loss_ref=loss_ref,
+                       grad_err=max_abs_over_norm(g_gpu, P.reps[k].last_grad),
+                       grad_l2=rel_l2(g_gpu, P.reps[k].last_grad),
+                       w_err=max_abs_over_norm(th_gpu[idx], P.reps[k].theta_sub))
+            print(rec)
+            assert abs(loss_gpu - loss_ref) <= LOSS_RTOL * loss_ref, rec
+            assert rec["grad_err"] <= TENSOR_TOL and rec["w_err"] <= TENSOR_TOL, rec
+            mask = np.ones(len(th_gpu), bool)
+            mask[idx] = False
+            assert np.array_equal(th_gpu[mask], theta0[mask])
+        P.ctx.ppu_outer_sync([0, 5])
+        P.ctx.ppu_sync()
+        th_gpu = P.ctx.ppu_get_params(-1)
+        P.theta, P.buf, m = O.outer_sync(P.theta, P.buf, [P.reps[0], P.reps[5]], P.outer)
+        assert np.array_equal(th_gpu[m == 0], theta0[m == 0])
+        assert max_abs_over_norm(th_gpu[m > 0], P.theta[m > 0]) <= TENSOR_TOL
+        assert np.array_equal(P.ctx.ppu_get_working_bf16(), bf16_bits(th_gpu))
+    finally:
+        P.close()
+
+
+def test_1p3b_one_step_replica_31_and_sampled_outer_sync():
+    from paper_2509_22418_b200 import ppu
+    dims = (24, 2048, 16, 8192, 32768)
+    ocfg = O.Model(*dims)
+    K = 32
+    ranges = [O.slice_ranges(ocfg, 32, k) for k in range(K)]
+    adam, outer = O.AdamW(3e-4, 0.9, 0.99, 1e-8, 0.1), O.Outer(0.7, 0.9)
+    cfg = ppu.make_cfg(*dims, 4, 2048, adam_lr=adam.lr, adam_beta1=adam.beta1,
+                       adam_beta2=adam.beta2, adam_eps=adam.eps, adam_wd=adam.wd,
+                       outer_lr=outer.lr, outer_momentum=outer.momentum)
+    spec, keep = ppu.make_spec(K, ppu.SUBSET_FFN_SLICE, n_slices=32)
+    ctx = ppu.Context(cfg, spec, keep)
+    try:
+        from paper_2509_22418_b200 import synth
+        import torch
+        theta32 = synth.init_params(31, ctx.tensors())
+        ctx.ppu_set_params(theta32)
+        w16_before = ctx.ppu_get_working_bf16()
+        k = 31
+        tok = synth.tokens(31, k, 0, 0, 4, 2048, ocfg.vocab)
+        ctx.ppu_local_step(k, torch.from_numpy(tok).cuda())
+        loss_gpu = ctx.ppu_loss(k)
+        rep = O.Replica(ocfg, theta32, ranges[k])              # fp32 storage for the oracle
+        assert np.array_equal(ctx.ppu_subset_index(k), rep.idx)
+        loss_ref = rep.local_step(theta32, tok, adam)
+        g_gpu = ctx.ppu_get_subset_grads(k)
+        th_gpu = ctx.ppu_get_params(k)
+        rec = dict(loss_gpu=loss_gpu, loss_ref=loss_ref,
+                   grad_err=max_abs_over_norm(g_gpu, rep.last_grad), grad_l2=rel_l2(g_gpu, rep.last_grad),
+                   w_err=max_abs_over_norm(th_gpu[rep.idx], rep.theta_sub))
+        print(rec)
+        assert abs(loss_gpu - loss_ref) <= LOSS_RTOL * loss_ref, rec
+        assert rec["grad_err"] <= TENSOR_TOL and rec["w_err"] <= TENSOR_TOL, rec
+        mask = np.ones(len(th_gpu), bool)
+        mask[rep.idx] = False
+        assert np.array_equal(th_gpu[mask], theta32[mask])                    # frozen fp32 bits
+        w16_after = ctx.ppu_get_working_bf16()
+        assert np.array_equal(w16_after[mask], w16_before[mask])              # frozen working copy
+        assert np.array_equal(w16_after[rep.idx], bf16_bits(th_gpu[rep.idx]))
+        # outer sync over replicas 31 and 3 (3 never stepped: delta 0), checked on sampled positions
+        end31 = th_gpu
+        ctx.ppu_outer_sync([31, 3])
+        ctx.ppu_sync()
+        th_new = ctx.ppu_get_params(-1)
+        buf_new = ctx.ppu_get_outer_momentum()
+        rng = np.random.default_rng(0)
+        idx3 = O.train_index(ocfg, ranges[3])
+        sample = np.concatenate([rng.choice(rep.idx, 200000, replace=False),
+                                 rng.choice(idx3, 100000, replace=False),
+                                 rng.integers(0, len(th_new), 200000)])
+        own31 = np.zeros(len(th_new), bool); own31[rep.idx] = True
+        own3 = np.zeros(len(th_new), bool); own3[idx3] = True
+        t0 = theta32[sample].astype(np.float64)
+        e31 = np.where(own31[sample], end31[sample].astype(np.float64), np.nan)
+        e3 = np.where(own3[sample], t0, np.nan)
+        ts, bs = O.outer_elementwise(t0, np.zeros_like(t0), [e31, e3], outer)
+        assert max_abs_over_norm(th_new[sample], ts) <= TENSOR_TOL
+        assert np.abs(th_new[sample] - ts).max() <= 1e-6
+        assert np.abs(buf_new[sample] - bs).max() <= 1e-6
+        untouched = ~(own31 | own3)
+        assert np.array_equal(th_new[untouched], theta32[untouched])
+        assert np.all(buf_new[untouched] == 0)
+    finally:
+        ctx.close()
