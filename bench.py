@@ -134,8 +134,63 @@ def run_reference(args, w):
     print(json.dumps(out))
 
 
+def run_sweep(args):
+    """Subset-fraction sweep at the 1.3B shapes: FFN slice fractions 1, 1/2, 1/4, 1/8, 1/32 and the
+    whole-layer variant (every 4th block), one replica timed per variant.  Prints one JSON line."""
+    import torch
+    from paper_2509_22418_b200 import build, ppu, synth
+    build.build()
+    w = WORKLOADS["c3"]
+    L, d, h, F, V = w["dims"]
+    B, S = w["batch"], w["seq"]
+    theta = None
+    rows = []
+    variants = [("slice 1/1", ppu.SUBSET_FFN_SLICE, 1, 1, 0), ("slice 1/2", ppu.SUBSET_FFN_SLICE, 2, 1, 0),
+                ("slice 1/4", ppu.SUBSET_FFN_SLICE, 4, 1, 0), ("slice 1/8", ppu.SUBSET_FFN_SLICE, 8, 1, 0),
+                ("slice 1/32", ppu.SUBSET_FFN_SLICE, 32, 1, 0),
+                ("every 4th block, replica 0 (lowest trained layer 0)", ppu.SUBSET_FFN_LAYERS, 1, 4, 0),
+                ("every 4th block, replica 3 (lowest trained layer 3)", ppu.SUBSET_FFN_LAYERS, 1, 4, 3)]
+    for name, mode, N, stride, rep in variants:
+        K = N if mode == ppu.SUBSET_FFN_SLICE else 4
+        cfg = ppu.make_cfg(L, d, h, F, V, B, S, adam_lr=ADAM["lr"], adam_beta1=ADAM["beta1"],
+                           adam_beta2=ADAM["beta2"], adam_eps=ADAM["eps"], adam_wd=ADAM["wd"],
+                           outer_lr=OUTER["lr"], outer_momentum=OUTER["momentum"])
+        spec, keep = ppu.make_spec(K, mode, n_slices=N, layer_stride=stride)
+        ctx = ppu.Context(cfg, spec, keep)
+        if theta is None:
+            theta = synth.init_params(SEED, ctx.tensors())
+        ctx.ppu_set_params(theta)
+        toks = [torch.from_numpy(synth.tokens(SEED, rep, 0, i, B, S, V)).cuda()
+                for i in range(args.warmup + args.steps)]
+        for i in range(args.warmup):
+            ctx.ppu_local_step(rep, toks[i])
+        ctx.ppu_sync()
+        ctx.ppu_profile_enable(True)
+        ctx.ppu_profile_read()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(args.steps):
+            ctx.ppu_local_step(rep, toks[args.warmup + i])
+        e1.record()
+        torch.cuda.synchronize()
+        prof = ctx.ppu_profile_read()
+        st = ctx.ppu_stats()
+        ms = e0.elapsed_time(e1) / args.steps
+        rows.append(dict(variant=name, trainable_params=ctx.ppu_subset_count(rep), ms_per_step=ms,
+                         tokens_per_s=B * S / (ms * 1e-3), wgrad_tflop=st.flops_wgrad / 1e12,
+                         dgrad_tflop=st.flops_dgrad / 1e12, fwd_tflop=st.flops_fwd / 1e12,
+                         gemm_tflops=prof.gemm_flops / (prof.gemm_ms * 1e-3) / 1e12,
+                         hbm_bytes=st.arena_bytes, state_bytes=st.state_bytes, replicas_held=K))
+        ctx.close()
+        del ctx
+        torch.cuda.empty_cache()
+    print(json.dumps(dict(metric="subset-fraction sweep, 1.3B local step", unit="tokens/s",
+                          steps=args.steps, warmup=args.warmup, data="synthetic", rows=rows)))
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--sweep", action="store_true", help="subset-fraction sweep at the 1.3B shapes")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
@@ -144,6 +199,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     w = WORKLOADS[args.workload]
+    if args.sweep:
+        return run_sweep(args)
     if args.impl == "reference":
         return run_reference(args, w)
 

@@ -195,8 +195,9 @@ int ppu_gemm(const void* A, int64_t lda, int a_kmajor, const void* B, int64_t ld
  * batch*seq; q at column 0, k at d, v at 2d; head j at columns j*d_h).  Forward
  * writes U[T,d] bf16 and lse[batch, n_head, seq] fp32 (log-sum-exp of the scaled
  * scores).  Backward reads them plus dU[T,d] bf16 and writes dqkv[T,3d] bf16;
- * scratch is fp32 [batch*n_head*seq].  backend: 0 = tensor-core tiles,
- * 1 = plain SIMT check kernel.  All pointers DEVICE. */
+ * scratch is fp32 [batch*n_head*seq].  backend: 0 = tcgen05 / TMEM kernels,
+ * 1 = plain SIMT check kernel, 2 = mma.sync kernels (0 and 2 need d_head 64 or 128).
+ * All pointers DEVICE. */
 int ppu_attention_fwd(const void* qkv, void* U, float* lse, int batch, int seq, int n_head,
                       int d_head, int backend, void* cuda_stream);
 int ppu_attention_bwd(const void* qkv, const void* U, const float* lse, const void* dU,

@@ -170,12 +170,27 @@ def rope(x, cos, sin, inverse=False):
     return out
 
 
+def _heads(x):
+    """[B,S,h,dh] -> contiguous [B,h,S,dh], so that per-head products are batched matmuls."""
+    return np.ascontiguousarray(x.transpose(0, 2, 1, 3))
+
+
+def _mm(x, W):
+    """x[..., k] @ W[k, n] through a 2-D product (numpy hands 2-D operands to BLAS)."""
+    return (x.reshape(-1, x.shape[-1]) @ W).reshape(x.shape[:-1] + (W.shape[1],))
+
+
+def _unheads(x):
+    """[B,h,S,dh] -> [B,S,h,dh]."""
+    return x.transpose(0, 2, 1, 3)
+
+
 def attention_probs(q, k):
     """A = softmax_row(q k^T / sqrt(d_h)) with the causal mask s' <= s.
     q, k [B,S,h,dh] (already rotated) -> [B,h,S,S]."""
     S, dh = q.shape[1], q.shape[3]
     causal = np.tril(np.ones((S, S), dtype=bool))
-    sc = np.einsum("bshd,bthd->bhst", q, k) / math.sqrt(dh)
+    sc = _heads(q) @ _heads(k).transpose(0, 1, 3, 2) / math.sqrt(dh)
     sc = np.where(causal[None, None], sc, -np.inf)
     sc = sc - sc.max(axis=-1, keepdims=True)
     A = np.exp(sc)
@@ -199,22 +214,22 @@ def forward(cfg: Model, theta: np.ndarray, tokens: np.ndarray, keep=True):
     for l in range(cfg.n_layer):
         p = f"l{l}."
         a, ln1 = layernorm(x, P[p + "ln1_g"], P[p + "ln1_b"], cfg.ln_eps)
-        q = rope((a @ P[p + "W_q"].T).reshape(B, S, h, dh), cos, sin)
-        k = rope((a @ P[p + "W_k"].T).reshape(B, S, h, dh), cos, sin)
-        v = (a @ P[p + "W_v"].T).reshape(B, S, h, dh)
+        q = rope(_mm(a, P[p + "W_q"].T).reshape(B, S, h, dh), cos, sin)
+        k = rope(_mm(a, P[p + "W_k"].T).reshape(B, S, h, dh), cos, sin)
+        v = _mm(a, P[p + "W_v"].T).reshape(B, S, h, dh)
         A = attention_probs(q, k)                         # [B,h,S,S]
-        U = np.einsum("bhst,bthd->bshd", A, v).reshape(B, S, d)
-        x1 = x + U @ P[p + "W_o"].T
+        U = _unheads(A @ _heads(v)).reshape(B, S, d)
+        x1 = x + _mm(U, P[p + "W_o"].T)
         bb, ln2 = layernorm(x1, P[p + "ln2_g"], P[p + "ln2_b"], cfg.ln_eps)
-        Hd = bb @ P[p + "W_in"].T                         # [B,S,F]
+        Hd = _mm(bb, P[p + "W_in"].T)                        # [B,S,F]
         Ac = gelu(Hd)
-        x2 = x1 + Ac @ P[p + "W_out"].T
+        x2 = x1 + _mm(Ac, P[p + "W_out"].T)
         if keep:
             layers.append(dict(a=a, ln1=ln1, q=q, k=k, v=v, U=U, b=bb, ln2=ln2,
                                Hd=Hd, Ac=Ac, A=A if keep_probs else None))
         x = x2
     f, lnf = layernorm(x, P["lnf_g"], P["lnf_b"], cfg.ln_eps)
-    logits = f @ P["E"].T                                 # [B,S,V]
+    logits = _mm(f, P["E"].T)                                # [B,S,V]
     z = logits[:, :-1, :]
     zmax = z.max(axis=-1, keepdims=True)
     lse = zmax[..., 0] + np.log(np.exp(z - zmax).sum(axis=-1))
@@ -247,12 +262,12 @@ def _attention_bwd(cfg, L, dU, cache):
     B, S, h, dh = L["q"].shape
     dUh = dU.reshape(B, S, h, dh)
     A = L["A"] if L["A"] is not None else attention_probs(L["q"], L["k"])
-    dv = np.einsum("bhst,bshd->bthd", A, dUh)
-    dA = np.einsum("bshd,bthd->bhst", dUh, L["v"])
+    dv = _unheads(A.transpose(0, 1, 3, 2) @ _heads(dUh))
+    dA = _heads(dUh) @ _heads(L["v"]).transpose(0, 1, 3, 2)
     dS = A * (dA - (dA * A).sum(axis=-1, keepdims=True))
     dS = dS / math.sqrt(dh)
-    dq = np.einsum("bhst,bthd->bshd", dS, L["k"])
-    dk = np.einsum("bhst,bshd->bthd", dS, L["q"])
+    dq = _unheads(dS @ _heads(L["k"]))
+    dk = _unheads(dS.transpose(0, 1, 3, 2) @ _heads(L["q"]))
     return dq, dk, dv
 
 
@@ -269,7 +284,7 @@ def grad_full(cfg: Model, theta: np.ndarray, tokens: np.ndarray):
     d = cfg.d_model
     dl = _dlogits(cfg, c)
     G["E"] += dl.reshape(B * S, -1).T @ c["f"].reshape(B * S, d)
-    df = dl @ P["E"]
+    df = _mm(dl, P["E"])
     gx, dgam, dbet = layernorm_bwd(df, P["lnf_g"], c["lnf"])
     G["lnf_g"] += dgam; G["lnf_b"] += dbet
     for l in reversed(range(cfg.n_layer)):
@@ -278,16 +293,16 @@ def grad_full(cfg: Model, theta: np.ndarray, tokens: np.ndarray):
         T2 = lambda t: t.reshape(B * S, -1)
         # FFN (Appendix C.1, MLP steps 1-5 with every slice)
         G[p + "W_out"] += T2(gx).T @ T2(L["Ac"])
-        dA = gx @ P[p + "W_out"]
+        dA = _mm(gx, P[p + "W_out"])
         dH = dA * gelu_grad(L["Hd"])
         G[p + "W_in"] += T2(dH).T @ T2(L["b"])
-        db = dH @ P[p + "W_in"]
+        db = _mm(dH, P[p + "W_in"])
         dx1, dgam, dbet = layernorm_bwd(db, P[p + "ln2_g"], L["ln2"])
         G[p + "ln2_g"] += dgam; G[p + "ln2_b"] += dbet
         g1 = gx + dx1
         # attention
         G[p + "W_o"] += T2(g1).T @ T2(L["U"])
-        dU = g1 @ P[p + "W_o"]
+        dU = _mm(g1, P[p + "W_o"])
         dq, dk, dv = _attention_bwd(cfg, L, dU, c)
         dq = rope(dq, c["cos"], c["sin"], inverse=True)
         dk = rope(dk, c["cos"], c["sin"], inverse=True)
@@ -295,8 +310,8 @@ def grad_full(cfg: Model, theta: np.ndarray, tokens: np.ndarray):
         G[p + "W_q"] += T2(dq).T @ a2
         G[p + "W_k"] += T2(dk).T @ a2
         G[p + "W_v"] += T2(dv).T @ a2
-        da = (dq.reshape(B, S, d) @ P[p + "W_q"] + dk.reshape(B, S, d) @ P[p + "W_k"]
-              + dv.reshape(B, S, d) @ P[p + "W_v"])
+        da = (_mm(dq.reshape(B, S, d), P[p + "W_q"]) + _mm(dk.reshape(B, S, d), P[p + "W_k"])
+              + _mm(dv.reshape(B, S, d), P[p + "W_v"]))
         dx0, dgam, dbet = layernorm_bwd(da, P[p + "ln1_g"], L["ln1"])
         G[p + "ln1_g"] += dgam; G[p + "ln1_b"] += dbet
         gx = g1 + dx0
@@ -322,7 +337,7 @@ def grad_restricted(cfg: Model, theta: np.ndarray, tokens: np.ndarray, ranges):
         return loss, out
     l0 = min(trained)
     dl = _dlogits(cfg, c)
-    df = dl @ P["E"]
+    df = _mm(dl, P["E"])
     gx, _, _ = layernorm_bwd(df, P["lnf_g"], c["lnf"])
     T2 = lambda t: t.reshape(B * S, -1)
     for l in reversed(range(l0, cfg.n_layer)):
@@ -330,25 +345,25 @@ def grad_restricted(cfg: Model, theta: np.ndarray, tokens: np.ndarray, ranges):
         L = c["layers"][l]
         lo, hi = ranges[l]
         if l == l0:
-            dA_n = gx @ P[p + "W_out"][:, lo:hi]
+            dA_n = _mm(gx, P[p + "W_out"][:, lo:hi])
             dH_n = dA_n * gelu_grad(L["Hd"][..., lo:hi])
             out[l] = (T2(dH_n).T @ T2(L["b"]), T2(gx).T @ T2(L["Ac"][..., lo:hi]))
             break
-        dA = gx @ P[p + "W_out"]
+        dA = _mm(gx, P[p + "W_out"])
         dH = dA * gelu_grad(L["Hd"])
         if hi > lo:
             out[l] = (T2(dH[..., lo:hi]).T @ T2(L["b"]),
                       T2(gx).T @ T2(L["Ac"][..., lo:hi]))
-        db = dH @ P[p + "W_in"]
+        db = _mm(dH, P[p + "W_in"])
         dx1, _, _ = layernorm_bwd(db, P[p + "ln2_g"], L["ln2"])
         g1 = gx + dx1
-        dU = g1 @ P[p + "W_o"]
+        dU = _mm(g1, P[p + "W_o"])
         dq, dk, dv = _attention_bwd(cfg, L, dU, c)
         dq = rope(dq, c["cos"], c["sin"], inverse=True)
         dk = rope(dk, c["cos"], c["sin"], inverse=True)
         d = cfg.d_model
-        da = (dq.reshape(B, S, d) @ P[p + "W_q"] + dk.reshape(B, S, d) @ P[p + "W_k"]
-              + dv.reshape(B, S, d) @ P[p + "W_v"])
+        da = (_mm(dq.reshape(B, S, d), P[p + "W_q"]) + _mm(dk.reshape(B, S, d), P[p + "W_k"])
+              + _mm(dv.reshape(B, S, d), P[p + "W_v"]))
         dx0, _, _ = layernorm_bwd(da, P[p + "ln1_g"], L["ln1"])
         gx = g1 + dx0
     return loss, out

@@ -448,6 +448,13 @@ bool set_smem(K kernel, int bytes) {
 
 }  // namespace
 
+void launch_attn_delta(const bf16* U, const bf16* dU, float* delta, int B, int S, int h, int dh,
+                       cudaStream_t st) {
+  const int64_t rows = (int64_t)B * S;
+  const int64_t warps = rows * h;
+  attn_delta_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, st>>>(U, dU, delta, S, h, dh, rows);
+}
+
 bool attn_mma_supported(int S, int dh) { return (dh == 64 || dh == 128) && S >= 1; }
 
 int launch_attn_fwd_mma(const bf16* qkv, bf16* U, float* lse, int B, int S, int h, int dh,
@@ -471,9 +478,7 @@ int launch_attn_fwd_mma(const bf16* qkv, bf16* U, float* lse, int B, int S, int 
 
 int launch_attn_bwd_mma(const bf16* qkv, const bf16* U, const float* lse, const bf16* dU,
                         bf16* dqkv, float* scratch, int B, int S, int h, int dh, cudaStream_t st) {
-  const int64_t rows = (int64_t)B * S;
-  const int64_t warps = rows * h;
-  attn_delta_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, st>>>(U, dU, scratch, S, h, dh, rows);
+  launch_attn_delta(U, dU, scratch, B, S, h, dh, st);
   dim3 grid((S + BT - 1) / BT, h, B);
   if (dh == 64) {
     constexpr int SM = 6 * BT * 64 * 2 + 4 * BT * 4;

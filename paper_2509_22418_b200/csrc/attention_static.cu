@@ -55,11 +55,13 @@ extern "C" int ppu_attention_bwd_static(const void* qkv, const void* U, const fl
   cudaStream_t st = (cudaStream_t)cuda_stream;
   // Every row the kernels read from the scratch is written first by the same call, so nothing
   // left over from an earlier call is ever used and no clearing is needed.
-  if (backend == 0) {
+  if (backend == 0 || backend == 2) {
     if (!attn_mma_supported(seq, d_head))
       return ppu_fail(PPU_ESHAPE, "shape not covered by the tensor-core attention");
-    rc = launch_attn_bwd_mma((const bf16*)qkv, (const bf16*)U, lse, (const bf16*)dU, (bf16*)dqkv,
-                             scratch, batch, seq, n_head, d_head, st);
+    rc = backend == 0 ? launch_attn_bwd_tc((const bf16*)qkv, (const bf16*)U, lse, (const bf16*)dU,
+                                           (bf16*)dqkv, scratch, batch, seq, n_head, d_head, nullptr, st)
+                      : launch_attn_bwd_mma((const bf16*)qkv, (const bf16*)U, lse, (const bf16*)dU,
+                                            (bf16*)dqkv, scratch, batch, seq, n_head, d_head, st);
   } else {
     rc = launch_attn_bwd_simt((const bf16*)qkv, (const bf16*)U, lse, (const bf16*)dU, (bf16*)dqkv,
                               scratch, batch, seq, n_head, d_head, st);

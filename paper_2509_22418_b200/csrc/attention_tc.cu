@@ -1,0 +1,619 @@
+// Fused causal attention on the 5th-generation tensor cores (tcgen05.mma, accumulators in
+// tensor memory, operands brought in by TMA), head sizes 64 and 128.
+//
+//   forward   one CTA per 128 queries; per 128-key block S = Q K^T lands in TMEM, 128 softmax
+//             threads (one query row each, so row maxima and sums need no shuffles) turn it into
+//             bf16 probabilities in swizzled shared memory, and P V is a second MMA whose result
+//             is folded into a register accumulator with the online-softmax correction.
+//   dq        one CTA per 128 queries; S = Q K^T and dP = dU V^T in TMEM, the threads form
+//             dS = P (dP - delta) in shared memory, dQ += dS K accumulates in TMEM over all key
+//             blocks (no rescaling is needed in the backward).
+//   dk, dv    one CTA per 128 keys, query blocks of 64; the transposed products S^T = K Q^T,
+//             dP^T = V dU^T; dV += P^T dU and dK += dS^T Q accumulate in TMEM.
+// The two backward kernels recompute P from q, k and the saved log-sum-exp; nothing is
+// accumulated with atomics, so results are bitwise reproducible.  (Appendix C.1, MHA.)
+//
+// Warp roles: warp 0 issues TMA, warp 1 issues MMAs and owns the TMEM allocation, warps 2-5 are
+// the 128 row threads.  Every mbarrier wait is bounded; on expiry the CTA raises an abort flag,
+// all roles fall through to the common exit, TMEM is released and an error word is set.
+#include "tc_common.cuh"
+
+namespace {
+using namespace tc;
+
+constexpr int ATT_THREADS = 192;
+constexpr float LOG2E = 1.4426950408889634f;
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+// 16-byte chunk `idx` (8 bf16) of row `row` in a K-major operand made of [rows x 64] swizzled
+// half-tiles that are `half_bytes` apart
+__device__ __forceinline__ uint32_t op_chunk(uint32_t base, uint32_t half_bytes, int row, int idx) {
+  return base + (uint32_t)(idx >> 3) * half_bytes + (uint32_t)row * 128u + (uint32_t)(((idx & 7) ^ (row & 7)) << 4);
+}
+// 32 fp32 values -> 32 bf16 -> four 16-byte chunks starting at chunk index idx0
+__device__ __forceinline__ void store_row32(uint32_t base, uint32_t half_bytes, int row, int idx0, const float* v) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    st_shared_v4(op_chunk(base, half_bytes, row, idx0 + q), pack2(v[8 * q], v[8 * q + 1]),
+                 pack2(v[8 * q + 2], v[8 * q + 3]), pack2(v[8 * q + 4], v[8 * q + 5]),
+                 pack2(v[8 * q + 6], v[8 * q + 7]));
+}
+
+struct AttnParams {
+  const float* lse; const float* delta;
+  bf16* U; float* lse_out; bf16* dqkv;
+  int S, h; int* flags;
+};
+
+// A [ROWS x DH] K-major operand tile: DH/64 half-tiles of ROWS*128 bytes.  K-step ks (16 columns).
+template <int ROWS>
+__device__ __forceinline__ uint64_t kmajor_desc(uint32_t tile, int ks) {
+  return make_desc(tile + (uint32_t)(ks >> 2) * (ROWS * 128u) + (uint32_t)(ks & 3) * 32u, 16, 1024);
+}
+// The same tile read as an MN-major B operand (rows are the reduction index): step ks = 16 rows.
+template <int ROWS>
+__device__ __forceinline__ uint64_t mnmajor_desc(uint32_t tile, int ks) {
+  return make_desc(tile + (uint32_t)ks * 2048u, ROWS * 128u, 1024);
+}
+__device__ __forceinline__ uint8_t* align1k(uint8_t* p) {
+  return reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(p) + 1023) & ~(uintptr_t)1023);
+}
+
+// ------------------------------------------------------------------ forward
+template <int DH>
+__global__ void __launch_bounds__(ATT_THREADS, 1)
+attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams p) {
+  constexpr int NH = DH / 64, QT = 128 * DH * 2, PT = 128 * 128 * 2;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = align1k(smem_raw);
+  const uint32_t Qs = smem_u32(smem), Ks = Qs + QT, Vs = Ks + 2 * QT, Ps = Vs + 2 * QT;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 5 * QT + PT);
+  enum { Q_FULL = 0, K_FULL = 1, K_EMPTY = 3, V_FULL = 5, V_EMPTY = 7, S_FULL = 9, S_EMPTY = 11,
+         P_FULL = 13, P_EMPTY = 14, O_FULL = 15, O_EMPTY = 16, NBAR = 17 };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t bar0 = smem_u32(bars);
+  auto B = [&](int i) { return bar0 + 8u * i; };
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int qb = gridDim.x - 1 - blockIdx.x, head = blockIdx.y, b = blockIdx.z;
+  const int d = p.h * DH, S = p.S;
+  const int n = qb + 1;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
+    mbar_init(B(S_EMPTY), 128); mbar_init(B(S_EMPTY + 1), 128);
+    mbar_init(B(P_FULL), 128); mbar_init(B(O_EMPTY), 128);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tS = tmem, tO = tmem + 256;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      mbar_expect_tx(B(Q_FULL), QT);
+      for (int hf = 0; hf < NH; ++hf)
+        tma_load_3d(Qs + hf * 16384, &mapQKV, B(Q_FULL), head * DH + hf * 64, qb * 128, b);
+      for (int j = 0; j < n; ++j) {
+        const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
+        if (!mbar_wait(B(K_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) break;
+        mbar_expect_tx(B(K_FULL + st), QT);
+        for (int hf = 0; hf < NH; ++hf)
+          tma_load_3d(Ks + st * QT + hf * 16384, &mapQKV, B(K_FULL + st), d + head * DH + hf * 64, j * 128, b);
+        if (!mbar_wait(B(V_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) break;
+        mbar_expect_tx(B(V_FULL + st), QT);
+        for (int hf = 0; hf < NH; ++hf)
+          tma_load_3d(Vs + st * QT + hf * 16384, &mapQKV, B(V_FULL + st), 2 * d + head * DH + hf * 64, j * 128, b);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
+      constexpr uint32_t idesc_o = make_idesc(128, DH, false, true);
+      bool ok = mbar_wait(B(Q_FULL), 0, abort_flag, p.flags);
+      auto issue_s = [&](int j) -> bool {
+        const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
+        if (!mbar_wait(B(K_FULL + st), ph, abort_flag, p.flags)) return false;
+        if (!mbar_wait(B(S_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks)
+          umma_bf16(tS + st * 128, kmajor_desc<128>(Qs, ks), kmajor_desc<128>(Ks + st * QT, ks), idesc_s, ks > 0);
+        umma_commit(B(S_FULL + st));
+        umma_commit(B(K_EMPTY + st));
+        return true;
+      };
+      if (ok) ok = issue_s(0);
+      for (int j = 0; j < n && ok; ++j) {
+        if (j + 1 < n) { ok = issue_s(j + 1); if (!ok) break; }
+        const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
+        if (!mbar_wait(B(P_FULL), j & 1, abort_flag, p.flags)) break;
+        if (!mbar_wait(B(V_FULL + st), ph, abort_flag, p.flags)) break;
+        if (!mbar_wait(B(O_EMPTY), (j & 1) ^ 1u, abort_flag, p.flags)) break;
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          umma_bf16(tO, kmajor_desc<128>(Ps, ks), mnmajor_desc<128>(Vs + st * QT, ks), idesc_o, ks > 0);
+        umma_commit(B(O_FULL));
+        umma_commit(B(P_EMPTY));
+        umma_commit(B(V_EMPTY + st));
+      }
+    }
+  } else {
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const int grow = qb * 128 + row;
+    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+    const float c = rsqrtf((float)DH) * LOG2E;
+    float o[DH];
+#pragma unroll
+    for (int e = 0; e < DH; ++e) o[e] = 0.f;
+    float m = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int j = 0; j < n && ok; ++j) {
+      const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
+      if (!mbar_wait(B(S_FULL + st), ph, abort_flag, p.flags)) { ok = false; break; }
+      tc_fence_after();
+      const bool diag = (j == qb) || ((j + 1) * 128 > S);
+      float mx = -INFINITY;
+#pragma unroll 1
+      for (int cc = 0; cc < 4; ++cc) {
+        uint32_t r[32];
+        tmem_ld32(tS + lane_off + st * 128 + cc * 32, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const int col = j * 128 + cc * 32 + e;
+          const float v = __uint_as_float(r[e]);
+          if (!diag || (col <= grow && col < S)) mx = fmaxf(mx, v);
+        }
+      }
+      const float m_new = fmaxf(m, mx * c);
+      const float corr = ex2(m - m_new);
+      float sum = 0.f;
+#pragma unroll 1
+      for (int cc = 0; cc < 4; ++cc) {
+        uint32_t r[32];
+        tmem_ld32(tS + lane_off + st * 128 + cc * 32, r);
+        tmem_ld_wait();
+        float pv[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const int col = j * 128 + cc * 32 + e;
+          float pe = ex2(__uint_as_float(r[e]) * c - m_new);
+          if (diag && (col > grow || col >= S)) pe = 0.f;
+          pv[e] = pe;
+          sum += pe;
+        }
+        if (cc == 0 && !mbar_wait(B(P_EMPTY), (j & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+        store_row32(Ps, 16384, row, cc * 4, pv);
+      }
+      if (!ok) break;
+      tc_fence_before();
+      fence_async_smem();
+      mbar_arrive(B(P_FULL));
+      mbar_arrive(B(S_EMPTY + st));
+      l = l * corr + sum;
+      m = m_new;
+#pragma unroll
+      for (int e = 0; e < DH; ++e) o[e] *= corr;
+      if (!mbar_wait(B(O_FULL), j & 1, abort_flag, p.flags)) { ok = false; break; }
+      tc_fence_after();
+#pragma unroll
+      for (int cc = 0; cc < DH / 32; ++cc) {
+        uint32_t r[32];
+        tmem_ld32(tO + lane_off + cc * 32, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) o[cc * 32 + e] += __uint_as_float(r[e]);
+      }
+      tc_fence_before();
+      mbar_arrive(B(O_EMPTY));
+    }
+    if (ok && grow < S) {
+      const float inv = 1.f / l;
+      bf16* out = p.U + ((int64_t)b * S + grow) * d + head * DH;
+#pragma unroll
+      for (int e = 0; e < DH; e += 8) {
+        uint4 u;
+        u.x = pack2(o[e] * inv, o[e + 1] * inv); u.y = pack2(o[e + 2] * inv, o[e + 3] * inv);
+        u.z = pack2(o[e + 4] * inv, o[e + 5] * inv); u.w = pack2(o[e + 6] * inv, o[e + 7] * inv);
+        *reinterpret_cast<uint4*>(out + e) = u;
+      }
+      p.lse_out[((int64_t)b * p.h + head) * S + grow] = (m + log2f(l)) * (1.f / LOG2E);
+    }
+  }
+  if (*abort_flag) for (int i = 0; i < 64; ++i) __nanosleep(2000);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, 512); }
+}
+
+// ------------------------------------------------------------------ backward: dq
+template <int DH>
+__global__ void __launch_bounds__(ATT_THREADS, 1)
+attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapG,
+                  const AttnParams p) {
+  constexpr int NH = DH / 64, QT = 128 * DH * 2, PT = 128 * 128 * 2;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = align1k(smem_raw);
+  const uint32_t Qs = smem_u32(smem), Gs = Qs + QT, Ks = Gs + QT, Vs = Ks + 2 * QT, Ds = Vs + 2 * QT;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 6 * QT + PT);
+  enum { Q_FULL = 0, K_FULL = 1, K_EMPTY = 3, V_FULL = 5, V_EMPTY = 7, SDP_FULL = 9, SDP_EMPTY = 10,
+         DS_FULL = 11, DS_EMPTY = 12, DQ_FULL = 13, NBAR = 14 };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t bar0 = smem_u32(bars);
+  auto B = [&](int i) { return bar0 + 8u * i; };
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int qb = gridDim.x - 1 - blockIdx.x, head = blockIdx.y, b = blockIdx.z;
+  const int d = p.h * DH, S = p.S;
+  const int n = qb + 1;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
+    mbar_init(B(SDP_EMPTY), 128); mbar_init(B(DS_FULL), 128);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tS = tmem, tP = tmem + 128, tQ = tmem + 256;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      mbar_expect_tx(B(Q_FULL), 2 * QT);
+      for (int hf = 0; hf < NH; ++hf) {
+        tma_load_3d(Qs + hf * 16384, &mapQKV, B(Q_FULL), head * DH + hf * 64, qb * 128, b);
+        tma_load_3d(Gs + hf * 16384, &mapG, B(Q_FULL), head * DH + hf * 64, qb * 128, b);
+      }
+      for (int j = 0; j < n; ++j) {
+        const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
+        if (!mbar_wait(B(K_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) break;
+        mbar_expect_tx(B(K_FULL + st), QT);
+        for (int hf = 0; hf < NH; ++hf)
+          tma_load_3d(Ks + st * QT + hf * 16384, &mapQKV, B(K_FULL + st), d + head * DH + hf * 64, j * 128, b);
+        if (!mbar_wait(B(V_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) break;
+        mbar_expect_tx(B(V_FULL + st), QT);
+        for (int hf = 0; hf < NH; ++hf)
+          tma_load_3d(Vs + st * QT + hf * 16384, &mapQKV, B(V_FULL + st), 2 * d + head * DH + hf * 64, j * 128, b);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
+      constexpr uint32_t idesc_q = make_idesc(128, DH, false, true);
+      bool ok = mbar_wait(B(Q_FULL), 0, abort_flag, p.flags);
+      for (int j = 0; j < n && ok; ++j) {
+        const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
+        if (!mbar_wait(B(K_FULL + st), ph, abort_flag, p.flags)) break;
+        if (!mbar_wait(B(V_FULL + st), ph, abort_flag, p.flags)) break;
+        if (!mbar_wait(B(SDP_EMPTY), (j & 1) ^ 1u, abort_flag, p.flags)) break;
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks)
+          umma_bf16(tS, kmajor_desc<128>(Qs, ks), kmajor_desc<128>(Ks + st * QT, ks), idesc_s, ks > 0);
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks)
+          umma_bf16(tP, kmajor_desc<128>(Gs, ks), kmajor_desc<128>(Vs + st * QT, ks), idesc_s, ks > 0);
+        umma_commit(B(SDP_FULL));
+        umma_commit(B(V_EMPTY + st));
+        if (!mbar_wait(B(DS_FULL), j & 1, abort_flag, p.flags)) break;
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          umma_bf16(tQ, kmajor_desc<128>(Ds, ks), mnmajor_desc<128>(Ks + st * QT, ks), idesc_q, (j > 0 || ks > 0));
+        umma_commit(B(DS_EMPTY));
+        umma_commit(B(K_EMPTY + st));
+        if (j == n - 1) umma_commit(B(DQ_FULL));
+      }
+    }
+  } else {
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const int grow = qb * 128 + row;
+    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+    const float scale = rsqrtf((float)DH), c = scale * LOG2E;
+    const int64_t si = ((int64_t)b * p.h + head) * S + (grow < S ? grow : S - 1);
+    const float l2 = p.lse[si] * LOG2E, dl = p.delta[si];
+    bool ok = true;
+    for (int j = 0; j < n && ok; ++j) {
+      if (!mbar_wait(B(SDP_FULL), j & 1, abort_flag, p.flags)) { ok = false; break; }
+      tc_fence_after();
+      const bool diag = (j == qb) || ((j + 1) * 128 > S);
+#pragma unroll 1
+      for (int cc = 0; cc < 4; ++cc) {
+        uint32_t rs[32], rd[32];
+        tmem_ld32(tS + lane_off + cc * 32, rs);
+        tmem_ld32(tP + lane_off + cc * 32, rd);
+        tmem_ld_wait();
+        float ds[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const int col = j * 128 + cc * 32 + e;
+          float pe = ex2(__uint_as_float(rs[e]) * c - l2);
+          if (diag && (col > grow || col >= S)) pe = 0.f;
+          ds[e] = pe * (__uint_as_float(rd[e]) - dl);
+        }
+        if (cc == 0 && !mbar_wait(B(DS_EMPTY), (j & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+        store_row32(Ds, 16384, row, cc * 4, ds);
+      }
+      if (!ok) break;
+      tc_fence_before();
+      fence_async_smem();
+      mbar_arrive(B(DS_FULL));
+      mbar_arrive(B(SDP_EMPTY));
+    }
+    if (ok && mbar_wait(B(DQ_FULL), 0, abort_flag, p.flags)) {
+      tc_fence_after();
+      bf16* out = p.dqkv + ((int64_t)b * S + grow) * (3 * d) + head * DH;
+#pragma unroll 1
+      for (int cc = 0; cc < DH / 32; ++cc) {
+        uint32_t r[32];
+        tmem_ld32(tQ + lane_off + cc * 32, r);
+        tmem_ld_wait();
+        if (grow < S) {
+#pragma unroll
+          for (int e = 0; e < 32; e += 8) {
+            uint4 u;
+            u.x = pack2(__uint_as_float(r[e]) * scale, __uint_as_float(r[e + 1]) * scale);
+            u.y = pack2(__uint_as_float(r[e + 2]) * scale, __uint_as_float(r[e + 3]) * scale);
+            u.z = pack2(__uint_as_float(r[e + 4]) * scale, __uint_as_float(r[e + 5]) * scale);
+            u.w = pack2(__uint_as_float(r[e + 6]) * scale, __uint_as_float(r[e + 7]) * scale);
+            *reinterpret_cast<uint4*>(out + cc * 32 + e) = u;
+          }
+        }
+      }
+    }
+  }
+  if (*abort_flag) for (int i = 0; i < 64; ++i) __nanosleep(2000);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, 512); }
+}
+
+// ------------------------------------------------------------------ backward: dk, dv
+template <int DH>
+__global__ void __launch_bounds__(ATT_THREADS, 1)
+attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_constant__ CUtensorMap mapQ64,
+                   const __grid_constant__ CUtensorMap mapG64, const AttnParams p) {
+  constexpr int NH = DH / 64, QT = 128 * DH * 2, HT = 64 * DH * 2, PT = 128 * 64 * 2;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = align1k(smem_raw);
+  const uint32_t Ks = smem_u32(smem), Vs = Ks + QT, Qs = Vs + QT, Gs = Qs + 2 * HT, Ps = Gs + 2 * HT,
+                 Ds = Ps + PT;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * QT + 4 * HT + 2 * PT);
+  enum { KV_FULL = 0, QG_FULL = 1, QG_EMPTY = 3, SDP_FULL = 5, SDP_EMPTY = 6, PDS_FULL = 7,
+         PDS_EMPTY = 8, OUT_FULL = 9, NBAR = 10 };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t bar0 = smem_u32(bars);
+  auto B = [&](int i) { return bar0 + 8u * i; };
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kb = blockIdx.x, head = blockIdx.y, b = blockIdx.z;
+  const int d = p.h * DH, S = p.S;
+  const int i0 = 2 * kb, n = (S + 63) / 64 - i0;      // query blocks of 64 from the diagonal down
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
+    mbar_init(B(SDP_EMPTY), 128); mbar_init(B(PDS_FULL), 128);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tS = tmem, tP = tmem + 64, tV = tmem + 128, tK = tmem + 128 + DH;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      mbar_expect_tx(B(KV_FULL), 2 * QT);
+      for (int hf = 0; hf < NH; ++hf) {
+        tma_load_3d(Ks + hf * 16384, &mapKV, B(KV_FULL), d + head * DH + hf * 64, kb * 128, b);
+        tma_load_3d(Vs + hf * 16384, &mapKV, B(KV_FULL), 2 * d + head * DH + hf * 64, kb * 128, b);
+      }
+      for (int it = 0; it < n; ++it) {
+        const int st = it & 1; const uint32_t ph = (it >> 1) & 1;
+        if (!mbar_wait(B(QG_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) break;
+        mbar_expect_tx(B(QG_FULL + st), 2 * HT);
+        for (int hf = 0; hf < NH; ++hf) {
+          tma_load_3d(Qs + st * HT + hf * 8192, &mapQ64, B(QG_FULL + st), head * DH + hf * 64, (i0 + it) * 64, b);
+          tma_load_3d(Gs + st * HT + hf * 8192, &mapG64, B(QG_FULL + st), head * DH + hf * 64, (i0 + it) * 64, b);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc(128, 64, false, false);
+      constexpr uint32_t idesc_o = make_idesc(128, DH, false, true);
+      bool ok = mbar_wait(B(KV_FULL), 0, abort_flag, p.flags);
+      for (int it = 0; it < n && ok; ++it) {
+        const int st = it & 1; const uint32_t ph = (it >> 1) & 1;
+        if (!mbar_wait(B(QG_FULL + st), ph, abort_flag, p.flags)) break;
+        if (!mbar_wait(B(SDP_EMPTY), (it & 1) ^ 1u, abort_flag, p.flags)) break;
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks)
+          umma_bf16(tS, kmajor_desc<128>(Ks, ks), kmajor_desc<64>(Qs + st * HT, ks), idesc_s, ks > 0);
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks)
+          umma_bf16(tP, kmajor_desc<128>(Vs, ks), kmajor_desc<64>(Gs + st * HT, ks), idesc_s, ks > 0);
+        umma_commit(B(SDP_FULL));
+        if (!mbar_wait(B(PDS_FULL), it & 1, abort_flag, p.flags)) break;
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          umma_bf16(tV, kmajor_desc<128>(Ps, ks), mnmajor_desc<64>(Gs + st * HT, ks), idesc_o, (it > 0 || ks > 0));
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          umma_bf16(tK, kmajor_desc<128>(Ds, ks), mnmajor_desc<64>(Qs + st * HT, ks), idesc_o, (it > 0 || ks > 0));
+        umma_commit(B(PDS_EMPTY));
+        umma_commit(B(QG_EMPTY + st));
+        if (it == n - 1) umma_commit(B(OUT_FULL));
+      }
+    }
+  } else {
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const int key = kb * 128 + row;
+    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+    const float scale = rsqrtf((float)DH), c = scale * LOG2E;
+    const float* lrow = p.lse + ((int64_t)b * p.h + head) * S;
+    const float* drow = p.delta + ((int64_t)b * p.h + head) * S;
+    bool ok = true;
+    for (int it = 0; it < n && ok; ++it) {
+      const int q0 = (i0 + it) * 64;
+      if (!mbar_wait(B(SDP_FULL), it & 1, abort_flag, p.flags)) { ok = false; break; }
+      tc_fence_after();
+#pragma unroll 1
+      for (int cc = 0; cc < 2; ++cc) {
+        uint32_t rs[32], rd[32];
+        tmem_ld32(tS + lane_off + cc * 32, rs);
+        tmem_ld32(tP + lane_off + cc * 32, rd);
+        tmem_ld_wait();
+        float pv[32], ds[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const int q = q0 + cc * 32 + e;
+          const int qc = q < S ? q : S - 1;
+          float pe = ex2(__uint_as_float(rs[e]) * c - __ldg(lrow + qc) * LOG2E);
+          if (key > q || q >= S) pe = 0.f;
+          pv[e] = pe;
+          ds[e] = pe * (__uint_as_float(rd[e]) - __ldg(drow + qc));
+        }
+        if (cc == 0 && !mbar_wait(B(PDS_EMPTY), (it & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+        store_row32(Ps, 0, row, cc * 4, pv);
+        store_row32(Ds, 0, row, cc * 4, ds);
+      }
+      if (!ok) break;
+      tc_fence_before();
+      fence_async_smem();
+      mbar_arrive(B(PDS_FULL));
+      mbar_arrive(B(SDP_EMPTY));
+    }
+    if (ok && mbar_wait(B(OUT_FULL), 0, abort_flag, p.flags)) {
+      tc_fence_after();
+      bf16* out = p.dqkv + ((int64_t)b * S + key) * (3 * d) + head * DH;
+#pragma unroll 1
+      for (int cc = 0; cc < 2 * DH / 32; ++cc) {
+        const bool is_k = cc >= DH / 32;
+        const int c0 = (is_k ? cc - DH / 32 : cc) * 32;
+        uint32_t r[32];
+        tmem_ld32((is_k ? tK : tV) + lane_off + c0, r);
+        tmem_ld_wait();
+        const float f = is_k ? scale : 1.f;
+        if (key < S) {
+          bf16* o = out + (is_k ? d : 2 * d) + c0;
+#pragma unroll
+          for (int e = 0; e < 32; e += 8) {
+            uint4 u;
+            u.x = pack2(__uint_as_float(r[e]) * f, __uint_as_float(r[e + 1]) * f);
+            u.y = pack2(__uint_as_float(r[e + 2]) * f, __uint_as_float(r[e + 3]) * f);
+            u.z = pack2(__uint_as_float(r[e + 4]) * f, __uint_as_float(r[e + 5]) * f);
+            u.w = pack2(__uint_as_float(r[e + 6]) * f, __uint_as_float(r[e + 7]) * f);
+            *reinterpret_cast<uint4*>(o + e) = u;
+          }
+        }
+      }
+    }
+  }
+  if (*abort_flag) for (int i = 0; i < 64; ++i) __nanosleep(2000);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, 512); }
+}
+
+// 3-D tensor map over a [B, S, cols] bf16 array (row stride ld elements), boxes of 64 columns
+bool encode3d(CUtensorMap* map, const bf16* base, int cols, int S, int B, int64_t ld, int box_rows) {
+  EncodeTiledFn enc = get_encoder();
+  if (!enc) return false;
+  cuuint64_t gdim[3] = {(cuuint64_t)cols, (cuuint64_t)S, (cuuint64_t)B};
+  cuuint64_t gstride[2] = {(cuuint64_t)ld * 2, (cuuint64_t)S * ld * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)base, gdim, gstride, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <typename K>
+bool set_smem(K kernel, int bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+}
+constexpr int EXTRA = 1024 + 256;   // alignment slack + barriers
+
+template <int DH>
+int fwd_t(const bf16* qkv, bf16* U, float* lse, int B, int S, int h, int* flags, cudaStream_t st) {
+  constexpr int SM = 5 * 128 * DH * 2 + 128 * 128 * 2 + EXTRA;
+  static bool ok = set_smem(attn_fwd_tc_kernel<DH>, SM);
+  if (!ok) return -2;
+  CUtensorMap m;
+  if (!encode3d(&m, qkv, 3 * h * DH, S, B, 3 * (int64_t)h * DH, 128)) return -3;
+  AttnParams p{}; p.U = U; p.lse_out = lse; p.S = S; p.h = h; p.flags = flags;
+  dim3 grid((S + 127) / 128, h, B);
+  attn_fwd_tc_kernel<DH><<<grid, ATT_THREADS, SM, st>>>(m, p);
+  return 0;
+}
+
+template <int DH>
+int bwd_t(const bf16* qkv, const float* lse, const bf16* dU, bf16* dqkv, const float* delta, int B,
+          int S, int h, int* flags, cudaStream_t st) {
+  constexpr int SM_DQ = 6 * 128 * DH * 2 + 128 * 128 * 2 + EXTRA;
+  constexpr int SM_KV = 2 * 128 * DH * 2 + 4 * 64 * DH * 2 + 2 * 128 * 64 * 2 + EXTRA;
+  static bool ok = set_smem(attn_dq_tc_kernel<DH>, SM_DQ) && set_smem(attn_dkv_tc_kernel<DH>, SM_KV);
+  if (!ok) return -2;
+  const int d = h * DH;
+  CUtensorMap mQKV, mG, mQ64, mG64;
+  if (!encode3d(&mQKV, qkv, 3 * d, S, B, 3 * (int64_t)d, 128) || !encode3d(&mG, dU, d, S, B, d, 128) ||
+      !encode3d(&mQ64, qkv, 3 * d, S, B, 3 * (int64_t)d, 64) || !encode3d(&mG64, dU, d, S, B, d, 64))
+    return -3;
+  AttnParams p{}; p.lse = lse; p.delta = delta; p.dqkv = dqkv; p.S = S; p.h = h; p.flags = flags;
+  dim3 grid((S + 127) / 128, h, B);
+  attn_dq_tc_kernel<DH><<<grid, ATT_THREADS, SM_DQ, st>>>(mQKV, mG, p);
+  attn_dkv_tc_kernel<DH><<<grid, ATT_THREADS, SM_KV, st>>>(mQKV, mQ64, mG64, p);
+  return 0;
+}
+
+}  // namespace
+
+bool attn_tc_supported(int S, int dh) { return (dh == 64 || dh == 128) && S >= 1; }
+
+int launch_attn_fwd_tc(const bf16* qkv, bf16* U, float* lse, int B, int S, int h, int dh, int* flags,
+                       cudaStream_t st) {
+  if (gemm_tc_init() != 0) return -1;
+  if (dh == 64) return fwd_t<64>(qkv, U, lse, B, S, h, flags, st);
+  if (dh == 128) return fwd_t<128>(qkv, U, lse, B, S, h, flags, st);
+  return -1;
+}
+
+int launch_attn_bwd_tc(const bf16* qkv, const bf16* U, const float* lse, const bf16* dU, bf16* dqkv,
+                       float* scratch, int B, int S, int h, int dh, int* flags, cudaStream_t st) {
+  if (gemm_tc_init() != 0) return -1;
+  launch_attn_delta(U, dU, scratch, B, S, h, dh, st);
+  if (dh == 64) return bwd_t<64>(qkv, lse, dU, dqkv, scratch, B, S, h, flags, st);
+  if (dh == 128) return bwd_t<128>(qkv, lse, dU, dqkv, scratch, B, S, h, flags, st);
+  return -1;
+}

@@ -43,6 +43,15 @@ int launch_attn_fwd_mma(const bf16* qkv, bf16* U, float* lse, int B, int S, int 
 int launch_attn_bwd_mma(const bf16* qkv, const bf16* U, const float* lse, const bf16* dU,
                         bf16* dqkv, float* scratch, int B, int S, int h, int dh, cudaStream_t st);
 bool attn_mma_supported(int S, int dh);
+// tcgen05 attention (TMEM accumulators, TMA operands); flags: device error words or null
+bool attn_tc_supported(int S, int dh);
+int launch_attn_fwd_tc(const bf16* qkv, bf16* U, float* lse, int B, int S, int h, int dh, int* flags,
+                       cudaStream_t st);
+int launch_attn_bwd_tc(const bf16* qkv, const bf16* U, const float* lse, const bf16* dU, bf16* dqkv,
+                       float* scratch, int B, int S, int h, int dh, int* flags, cudaStream_t st);
+// delta[b,h,s] = sum_e dU * U of the head's slice
+void launch_attn_delta(const bf16* U, const bf16* dU, float* delta, int B, int S, int h, int dh,
+                       cudaStream_t st);
 
 // ---- bandwidth-bound kernels -------------------------------------------------
 void launch_embed(const int32_t* tok, const bf16* E16, float* x, int T, int d, int V, int* flags,

@@ -248,7 +248,7 @@ extern "C" int ppu_create(const ppu_model_cfg* cfg, const ppu_subset_spec* spec,
   const char* e = getenv("PPU_GEMM");
   c->gemm_backend = (e && !strcmp(e, "simt")) ? 1 : 0;
   e = getenv("PPU_ATTN");
-  c->attn_backend = (e && !strcmp(e, "simt")) ? 1 : 0;
+  c->attn_backend = (e && !strcmp(e, "simt")) ? 1 : (e && !strcmp(e, "mma")) ? 2 : 0;
   if (c->gemm_backend == 0 && gemm_tc_init() != 0) {
     delete c;
     return ppu_fail(PPU_ECUDA, "cuTensorMapEncodeTiled not available from the driver");
@@ -501,9 +501,10 @@ extern "C" int ppu_attention_fwd(const void* qkv, void* U, float* lse, int batch
                                  int n_head, int d_head, int backend, void* cuda_stream) {
   if (!qkv || !U || !lse) return ppu_fail(PPU_EINVAL, "null operand");
   int rc;
-  if (backend == 0) {
+  if (backend == 0 || backend == 2) {
     if (!attn_mma_supported(seq, d_head)) return ppu_fail(PPU_ESHAPE, "shape not covered by the tensor-core attention");
-    rc = launch_attn_fwd_mma((const bf16*)qkv, (bf16*)U, lse, batch, seq, n_head, d_head, (cudaStream_t)cuda_stream);
+    rc = backend == 0 ? launch_attn_fwd_tc((const bf16*)qkv, (bf16*)U, lse, batch, seq, n_head, d_head, nullptr, (cudaStream_t)cuda_stream)
+                      : launch_attn_fwd_mma((const bf16*)qkv, (bf16*)U, lse, batch, seq, n_head, d_head, (cudaStream_t)cuda_stream);
   } else {
     rc = launch_attn_fwd_simt((const bf16*)qkv, (bf16*)U, lse, batch, seq, n_head, d_head, (cudaStream_t)cuda_stream);
   }
@@ -516,9 +517,10 @@ extern "C" int ppu_attention_bwd(const void* qkv, const void* U, const float* ls
                                  int d_head, int backend, void* cuda_stream) {
   if (!qkv || !U || !lse || !dU || !dqkv || !scratch) return ppu_fail(PPU_EINVAL, "null operand");
   int rc;
-  if (backend == 0) {
+  if (backend == 0 || backend == 2) {
     if (!attn_mma_supported(seq, d_head)) return ppu_fail(PPU_ESHAPE, "shape not covered by the tensor-core attention");
-    rc = launch_attn_bwd_mma((const bf16*)qkv, (const bf16*)U, lse, (const bf16*)dU, (bf16*)dqkv, scratch, batch, seq, n_head, d_head, (cudaStream_t)cuda_stream);
+    rc = backend == 0 ? launch_attn_bwd_tc((const bf16*)qkv, (const bf16*)U, lse, (const bf16*)dU, (bf16*)dqkv, scratch, batch, seq, n_head, d_head, nullptr, (cudaStream_t)cuda_stream)
+                      : launch_attn_bwd_mma((const bf16*)qkv, (const bf16*)U, lse, (const bf16*)dU, (bf16*)dqkv, scratch, batch, seq, n_head, d_head, (cudaStream_t)cuda_stream);
   } else {
     rc = launch_attn_bwd_simt((const bf16*)qkv, (const bf16*)U, lse, (const bf16*)dU, (bf16*)dqkv, scratch, batch, seq, n_head, d_head, (cudaStream_t)cuda_stream);
   }

@@ -92,7 +92,12 @@ struct Sched {
     c->launches++;
     if (flop_counter) *flop_counter += 2.0 * M * N * (double)K;
   }
-  bool use_mma_attn() const { return c->attn_backend == 0 && attn_mma_supported(S, dh); }
+  // 0: tcgen05 kernels, 2: mma.sync kernels (both need d_h 64 or 128), 1: SIMT
+  int attn_kind() const {
+    if (c->attn_backend == 0 && attn_tc_supported(S, dh)) return 0;
+    if (c->attn_backend != 1 && attn_mma_supported(S, dh)) return 2;
+    return 1;
+  }
 
   // Forward pass over all parameters (Appendix C.1 forward equations), saving what the
   // restricted backward needs.
@@ -110,7 +115,9 @@ struct Sched {
       {
         const double fl = 4.0 * B * h * dh * 0.5 * S * (double)(S + 1);
         EvScope ev(c, 1, fl);
-        if (use_mma_attn()) rc |= launch_attn_fwd_mma(a.qkv, a.U, a.lse, B, S, h, dh, st);
+        const int kind = attn_kind();
+        if (kind == 0) rc |= launch_attn_fwd_tc(a.qkv, a.U, a.lse, B, S, h, dh, c->flags, st);
+        else if (kind == 2) rc |= launch_attn_fwd_mma(a.qkv, a.U, a.lse, B, S, h, dh, st);
         else rc |= launch_attn_fwd_simt(a.qkv, a.U, a.lse, B, S, h, dh, st);
         c->launches++;
         c->flops_fwd += fl;
@@ -179,11 +186,14 @@ struct Sched {
       {
         const double fl = 10.0 * B * h * dh * 0.5 * S * (double)(S + 1);
         EvScope ev(c, 1, fl);
-        if (use_mma_attn())
+        const int kind = attn_kind();
+        if (kind == 0)
+          rc |= launch_attn_bwd_tc(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, c->flags, st);
+        else if (kind == 2)
           rc |= launch_attn_bwd_mma(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, st);
         else
           rc |= launch_attn_bwd_simt(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, st);
-        c->launches += 2;
+        c->launches += kind == 1 ? 2 : 3;
         c->flops_dgrad += fl;
       }
       launch_rope(c->dqkv, c->rope_cs, B, S, h, dh, 1, st); c->launches++;

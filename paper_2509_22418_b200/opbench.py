@@ -26,6 +26,7 @@ def main():
     ap.add_argument("--seq", type=int, default=2048)
     ap.add_argument("--heads", type=int, default=16)
     ap.add_argument("--dh", type=int, default=128)
+    ap.add_argument("--backend", type=int, default=0, help="attention: 0 tcgen05, 1 SIMT, 2 mma.sync")
     ap.add_argument("--iters", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     a = ap.parse_args()
@@ -58,11 +59,11 @@ def main():
         d = h * dh
         qkv = torch.randn((B_ * S, 3 * d), generator=g).to(dev).bfloat16()
         dU = torch.randn((B_ * S, d), generator=g).to(dev).bfloat16()
-        U, lse = ppu.ppu_attention_fwd(qkv, B_, S, h, dh)
+        U, lse = ppu.ppu_attention_fwd(qkv, B_, S, h, dh, backend=a.backend)
         fl = 4.0 * B_ * h * dh * 0.5 * S * (S + 1)
-        ms = timed(lambda: ppu.ppu_attention_fwd(qkv, B_, S, h, dh))
+        ms = timed(lambda: ppu.ppu_attention_fwd(qkv, B_, S, h, dh, backend=a.backend))
         print(f"attn fwd B={B_} S={S} h={h} dh={dh}: {ms:.4f} ms {fl / ms / 1e9:.1f} TFLOP/s (causal)")
-        ms = timed(lambda: ppu.ppu_attention_bwd(qkv, U, lse, dU, B_, S, h, dh))
+        ms = timed(lambda: ppu.ppu_attention_bwd(qkv, U, lse, dU, B_, S, h, dh, backend=a.backend))
         print(f"attn bwd: {ms:.4f} ms {2.5 * fl / ms / 1e9:.1f} TFLOP/s (causal, 2.5 x forward)")
 
 
