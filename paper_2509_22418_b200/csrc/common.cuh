@@ -27,6 +27,9 @@ struct GemmArgs {
   void* C2;                     // EPI_GELU_DUAL second output (ld = ldc)
   const void* aux; int64_t ldaux;
   int* flags;                   // device error words (may be null for the test entry)
+  // split-K: the reduction is cut into `splits` ranges; range s writes its partial product to
+  // C + s * split_stride (elements).  The consumer adds the partials in index order.
+  int splits = 1; int64_t split_stride = 0;
 };
 
 int launch_gemm_simt(const GemmArgs& g, cudaStream_t st);

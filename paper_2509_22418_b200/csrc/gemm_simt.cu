@@ -81,6 +81,19 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
 int launch_gemm_simt(const GemmArgs& g, cudaStream_t st) {
   if (g.M <= 0 || g.N <= 0) return 0;
   dim3 grid((g.N + TS - 1) / TS, (g.M + TS - 1) / TS);
-  gemm_simt_kernel<<<grid, 256, 0, st>>>(g);
+  const int k_blocks = (g.K + 63) / 64;      // same reduction ranges as the tcgen05 kernel
+  const int splits = g.splits < 1 ? 1 : (g.splits > k_blocks ? k_blocks : g.splits);
+  for (int sp = 0; sp < splits; ++sp) {
+    const int k0 = (int)((long long)sp * k_blocks / splits) * 64;
+    int k1 = (int)((long long)(sp + 1) * k_blocks / splits) * 64;
+    if (k1 > g.K) k1 = g.K;
+    GemmArgs s = g;
+    s.K = k1 - k0;
+    s.A = g.A + (g.a_kmajor ? (int64_t)k0 : (int64_t)k0 * g.lda);
+    s.B = g.B + (g.b_kmajor ? (int64_t)k0 : (int64_t)k0 * g.ldb);
+    if (g.epilogue == EPI_STORE_F32) s.C = (float*)g.C + (int64_t)sp * g.split_stride;
+    else s.C = (bf16*)g.C + (int64_t)sp * g.split_stride;
+    gemm_simt_kernel<<<grid, 256, 0, st>>>(s);
+  }
   return 0;
 }

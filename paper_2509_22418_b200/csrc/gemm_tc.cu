@@ -58,6 +58,7 @@ struct TcParams {
   const void* aux; long long ldaux;
   int* flags;
   int tiles_m, tiles_n;
+  int splits; long long split_stride;
 };
 
 template <int BN> struct Cfg {
@@ -104,7 +105,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int num_tiles = p.tiles_m * p.tiles_n;
+  const int tiles_mn = p.tiles_m * p.tiles_n;
+  const int num_tiles = tiles_mn * p.splits;
   const int k_blocks = (p.K + BK - 1) / BK;
 
   if (warp == 0) {
@@ -112,9 +114,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
       // ---------------- TMA producer ----------------
       int s = 0; uint32_t ph = 0;
       for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
-        const int m0 = (tile % p.tiles_m) * BM, n0 = (tile / p.tiles_m) * BN;
+        const int sp = tile / tiles_mn, t2 = tile - sp * tiles_mn;
+        const int m0 = (t2 % p.tiles_m) * BM, n0 = (t2 / p.tiles_m) * BN;
+        const int kb0 = (int)((long long)sp * k_blocks / p.splits);
+        const int kb1 = (int)((long long)(sp + 1) * k_blocks / p.splits);
         bool ok = true;
-        for (int kb = 0; kb < k_blocks && ok; ++kb) {
+        for (int kb = kb0; kb < kb1 && ok; ++kb) {
           ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.flags);
           if (!ok) break;
           const uint32_t a_dst = smem_u32(smem + s * C::STAGE_BYTES);
@@ -149,11 +154,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
       int s = 0; uint32_t ph = 0;
       int acc = 0; uint32_t acc_ph = 0;
       for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
+        const int sp = tile / tiles_mn;
+        const int kb0 = (int)((long long)sp * k_blocks / p.splits);
+        const int kb1 = (int)((long long)(sp + 1) * k_blocks / p.splits);
         if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.flags)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
         bool ok = true;
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           ok = mbar_wait(full_bar(s), ph, abort_flag, p.flags);
           if (!ok) break;
           tc_fence_after();
@@ -165,7 +173,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
                                        : make_desc(a_addr + k * 2048, 8192, 1024);
             const uint64_t bdesc = B_K ? make_desc(b_addr + k * 32, 16, 1024)
                                        : make_desc(b_addr + k * 2048, 8192, 1024);
-            umma_bf16(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            umma_bf16(d_tmem, adesc, bdesc, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
           }
           umma_commit(empty_bar(s));           // slot is free once these MMAs have read it
           if (++s == C::STAGES) { s = 0; ph ^= 1u; }
@@ -181,7 +189,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     const int half = (warp - 2) >> 2;          // which half of the tile's columns
     int acc = 0; uint32_t acc_ph = 0;
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
-      const int m0 = (tile % p.tiles_m) * BM, n0 = (tile / p.tiles_m) * BN;
+      const int sp = tile / tiles_mn, t2 = tile - sp * tiles_mn;
+      const int m0 = (t2 % p.tiles_m) * BM, n0 = (t2 / p.tiles_m) * BN;
       if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.flags)) break;
       tc_fence_after();
       const int m = m0 + quarter * 32 + lane;
@@ -193,7 +202,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         if (nb >= p.N) break;                  // warp-uniform
         uint32_t r[32];
         tmem_ld32(t_row + c0, r);              // asynchronous until tmem_ld_wait
-        const long long ci = (long long)m * p.ldc + nb;
+        const long long ci = (long long)m * p.ldc + nb + (long long)sp * p.split_stride;
         const bool full = nb + 32 <= p.N;
         if (p.epilogue == EPI_RESID_F32) {
           float4 x[8];
@@ -316,7 +325,10 @@ int launch_t(const GemmArgs& g, cudaStream_t st) {
   p.C = g.C; p.ldc = g.ldc; p.C2 = g.C2; p.aux = g.aux; p.ldaux = g.ldaux; p.flags = g.flags;
   p.tiles_m = (g.M + BM - 1) / BM;
   p.tiles_n = (g.N + BN - 1) / BN;
-  const int tiles = p.tiles_m * p.tiles_n;
+  const int k_blocks = (g.K + BK - 1) / BK;
+  p.splits = g.splits < 1 ? 1 : (g.splits > k_blocks ? k_blocks : g.splits);
+  p.split_stride = g.split_stride;
+  const int tiles = p.tiles_m * p.tiles_n * p.splits;
   static int n_sm = 0;
   if (n_sm == 0) {
     int dev = 0;
@@ -358,7 +370,7 @@ int launch_gemm_tc(const GemmArgs& g, cudaStream_t st) {
       (reinterpret_cast<uintptr_t>(g.C) & 15))
     return -4;
   // Wide tiles when the grid still fills the machine; narrow ones for small outputs.
-  const long long tiles256 = (long long)((g.M + BM - 1) / BM) * ((g.N + 255) / 256);
+  const long long tiles256 = (long long)((g.M + BM - 1) / BM) * ((g.N + 255) / 256) * (g.splits > 1 ? g.splits : 1);
   if (g.N > 128 && tiles256 >= 148) return launch_bn<256>(g, st);
   return launch_bn<128>(g, st);
 }

@@ -143,6 +143,16 @@ static void build_geometry(ppu_ctx* c) {
     }
     if (r2.n_sub > c->max_sub) c->max_sub = r2.n_sub;
   }
+  // The subset products have few output tiles when slices are narrow: cut their reduction over
+  // tokens so that about one wave of CTAs works on them.  One factor for the whole context.
+  int64_t min_tiles = 1 << 30;
+  for (auto& r2 : c->reps)
+    for (auto& s : r2.segs) {
+      const int64_t t = (int64_t)((s.hi - s.lo + 127) / 128) * ((d + 127) / 128);
+      if (t < min_tiles) min_tiles = t;
+    }
+  c->wgrad_splits = 1;
+  while (min_tiles * c->wgrad_splits * 2 <= 148 && c->wgrad_splits < 8) c->wgrad_splits *= 2;
 }
 
 // Carves the arena.  With base == nullptr only the sizes are computed.
@@ -165,7 +175,8 @@ static size_t carve(ppu_ctx* c, uint8_t* base) {
     r.v = (float*)take(r.n_sub * 4);
     r.d_segs = (SliceSeg*)take(sizeof(SliceSeg) * (r.segs.size() + 1));
   }
-  c->grad = (float*)take(c->max_sub * 4);
+  c->max_sub = (c->max_sub + 63) & ~(int64_t)63;
+  c->grad = (float*)take(c->max_sub * 4 * c->wgrad_splits);
   c->loss = (float*)take(sizeof(float) * (c->K + 1));
   c->flags = (int*)take(sizeof(int) * PPU_FLAG_COUNT);
   c->rope_cs = (float2*)take(sizeof(float2) * c->cfg.max_seq * (d / h / 2));
@@ -435,6 +446,13 @@ extern "C" int ppu_get_subset_grads(ppu_ctx* c, int replica, float* grads, int64
   if (!grads || n != c->reps[replica].n_sub) return ppu_fail(PPU_EINVAL, "grads null or wrong length");
   CUDA_OK(cudaMemcpyAsync(grads, c->grad, n * 4, cudaMemcpyDeviceToHost, c->stream));
   CUDA_OK(cudaStreamSynchronize(c->stream));
+  if (c->last_partials > 1) {   // add the split-K partials in the order the optimizer kernel uses
+    std::vector<float> part(n);
+    for (int q = 1; q < c->last_partials; ++q) {
+      CUDA_OK(cudaMemcpy(part.data(), c->grad + (int64_t)q * c->max_sub, n * 4, cudaMemcpyDeviceToHost));
+      for (int64_t i = 0; i < n; ++i) grads[i] += part[i];
+    }
+  }
   return PPU_OK;
 }
 extern "C" int ppu_get_subset_state(ppu_ctx* c, int replica, float* m, float* v, int32_t* step,

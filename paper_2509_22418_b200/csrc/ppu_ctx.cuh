@@ -45,6 +45,8 @@ struct ppu_ctx {
   std::vector<TensorRec> tensors;
   std::vector<ReplicaState> reps;
   int64_t max_sub = 0;
+  int wgrad_splits = 1;   // split-K factor of the subset weight-gradient products
+  int last_partials = 1;  // partial gradient buffers written by the most recent step
   int resident = -1;      // replica whose subset is overlaid on the bf16 working copy
   int last_stepped = -1;
   float adam_lr;

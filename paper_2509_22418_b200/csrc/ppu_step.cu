@@ -81,17 +81,19 @@ struct Sched {
 
   void gemm(const bf16* A, int64_t lda, int ak, const bf16* Bm, int64_t ldb, int bk, int M, int N,
             int K, int epi, void* C, int64_t ldc, void* C2, const void* aux, int64_t ldaux,
-            double* flop_counter) {
+            double* flop_counter, int splits = 1, int64_t split_stride = 0) {
     if (rc || M <= 0 || N <= 0) return;
     GemmArgs g;
     g.A = A; g.lda = lda; g.a_kmajor = ak; g.B = Bm; g.ldb = ldb; g.b_kmajor = bk;
     g.M = M; g.N = N; g.K = K; g.epilogue = epi; g.C = C; g.ldc = ldc; g.C2 = C2; g.aux = aux;
-    g.ldaux = ldaux; g.flags = c->flags;
+    g.ldaux = ldaux; g.flags = c->flags; g.splits = splits; g.split_stride = split_stride;
     EvScope ev(c, 0, 2.0 * M * N * (double)K);
     rc = c->gemm_backend == 1 ? launch_gemm_simt(g, c->stream) : launch_gemm_tc(g, c->stream);
     c->launches++;
     if (flop_counter) *flop_counter += 2.0 * M * N * (double)K;
   }
+  // split-K partial buffers the subset weight-gradient products of this step write
+  int partials() const { const int kb = (T + 63) / 64; return c->wgrad_splits < kb ? c->wgrad_splits : kb; }
   // 0: tcgen05 kernels, 2: mma.sync kernels (both need d_h 64 or 128), 1: SIMT
   int attn_kind() const {
     if (c->attn_backend == 0 && attn_tc_supported(S, dh)) return 0;
@@ -171,9 +173,10 @@ struct Sched {
       if (trained) {
         // dW_in[lo:hi,:] = dHd[:,lo:hi]^T b      dW_out[:,lo:hi] = g^T A[:,lo:hi]
         gemm(c->dHd + s->lo, F, 0, a.b, d, 0, w, d, T, EPI_STORE_F32, c->grad + s->packed_off, d,
-             nullptr, nullptr, 0, &c->flops_wgrad);
+             nullptr, nullptr, 0, &c->flops_wgrad, partials(), c->max_sub);
         gemm(c->g16, d, 0, a.A + s->lo, F, 0, d, w, T, EPI_STORE_F32,
-             c->grad + s->packed_off + (int64_t)w * d, w, nullptr, nullptr, 0, &c->flops_wgrad);
+             c->grad + s->packed_off + (int64_t)w * d, w, nullptr, nullptr, 0, &c->flops_wgrad,
+             partials(), c->max_sub);
         --seg;
       }
       if (l == r.lowest) break;
@@ -237,7 +240,8 @@ extern "C" int ppu_local_step(ppu_ctx* c, int replica, const int32_t* tokens, in
     hp.eps = c->cfg.adam_eps; hp.wd = c->cfg.adam_wd;
     hp.bc1 = (float)(1.0 - std::pow((double)hp.beta1, (double)r.step));
     hp.bc2 = (float)(1.0 - std::pow((double)hp.beta2, (double)r.step));
-    launch_adamw(r.d_segs, (int)r.segs.size(), r.master, r.m, r.v, c->grad, 1, 0, c->w16,
+    c->last_partials = s.partials();
+    launch_adamw(r.d_segs, (int)r.segs.size(), r.master, r.m, r.v, c->grad, c->last_partials, c->max_sub, c->w16,
                  c->cfg.d_model, c->cfg.d_ff, r.n_sub, hp, c->stream);
     c->launches++;
   }
