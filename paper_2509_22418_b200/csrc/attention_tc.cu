@@ -50,6 +50,14 @@ __device__ __forceinline__ void store_row32(uint32_t base, uint32_t half_bytes, 
                  pack2(v[8 * q + 6], v[8 * q + 7]));
 }
 
+// One arrival per warp: 128 single-thread arrivals on one mbarrier serialise in shared memory
+// and cost more than the arithmetic between them.  __syncwarp orders the lanes' earlier
+// accesses before lane 0's releasing arrive.
+__device__ __forceinline__ void warp_arrive(uint32_t bar) {
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+}
+
 struct AttnParams {
   const float* lse; const float* delta;
   bf16* U; float* lse_out; bf16* dqkv;
@@ -65,6 +73,24 @@ __device__ __forceinline__ uint64_t kmajor_desc(uint32_t tile, int ks) {
 template <int ROWS>
 __device__ __forceinline__ uint64_t mnmajor_desc(uint32_t tile, int ks) {
   return make_desc(tile + (uint32_t)ks * 2048u, ROWS * 128u, 1024);
+}
+// Lean MMA issue: the issuing thread is the critical resource here (each K=16 step of a
+// 64-column product is only 32 tensor cycles), so descriptors are kept as a precomputed low word
+// plus compile-time step offsets, and the constant high word (SBO 1024 B, version 1, 128-byte
+// swizzle) is shared.
+constexpr uint32_t DESC_HI = 64u | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t klo(uint32_t tile) { return ((tile >> 4) & 0x3FFFu) | (1u << 16); }
+template <int ROWS>
+__device__ __forceinline__ uint32_t mlo(uint32_t tile) { return ((tile >> 4) & 0x3FFFu) | ((uint32_t)(ROWS * 8) << 16); }
+template <int ROWS> __host__ __device__ constexpr uint32_t kstep(int ks) { return (uint32_t)((ks >> 2) * ROWS * 8 + (ks & 3) * 2); }
+__host__ __device__ constexpr uint32_t mstep(int ks) { return (uint32_t)(ks * 128); }
+__device__ __forceinline__ void umma_lo(uint32_t tmem_d, uint32_t alo, uint32_t blo, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n.reg .pred p;\n.reg .b64 da, db;\nsetp.ne.b32 p, %4, 0;\n"
+      "mov.b64 da, {%1, %5};\nmov.b64 db, {%2, %5};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n}" ::"r"(tmem_d),
+      "r"(alo), "r"(blo), "r"(idesc), "r"(acc), "r"(DESC_HI)
+      : "memory");
 }
 __device__ __forceinline__ uint8_t* align1k(uint8_t* p) {
   return reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(p) + 1023) & ~(uintptr_t)1023);
@@ -92,8 +118,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
-    mbar_init(B(S_EMPTY), 128); mbar_init(B(S_EMPTY + 1), 128);
-    mbar_init(B(P_FULL), 128); mbar_init(B(O_EMPTY), 128);
+    mbar_init(B(S_EMPTY), 4); mbar_init(B(S_EMPTY + 1), 4);
+    mbar_init(B(P_FULL), 4); mbar_init(B(O_EMPTY), 4);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -134,7 +160,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks)
-          umma_bf16(tS + st * 128, kmajor_desc<128>(Qs, ks), kmajor_desc<128>(Ks + st * QT, ks), idesc_s, ks > 0);
+          umma_lo(tS + st * 128, klo(Qs) + kstep<128>(ks), klo(Ks + st * QT) + kstep<128>(ks), idesc_s, ks > 0);
         umma_commit(B(S_FULL + st));
         umma_commit(B(K_EMPTY + st));
         return true;
@@ -149,7 +175,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
-          umma_bf16(tO, kmajor_desc<128>(Ps, ks), mnmajor_desc<128>(Vs + st * QT, ks), idesc_o, ks > 0);
+          umma_lo(tO, klo(Ps) + kstep<128>(ks), mlo<128>(Vs + st * QT) + mstep(ks), idesc_o, ks > 0);
         umma_commit(B(O_FULL));
         umma_commit(B(P_EMPTY));
         umma_commit(B(V_EMPTY + st));
@@ -207,8 +233,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
       if (!ok) break;
       tc_fence_before();
       fence_async_smem();
-      mbar_arrive(B(P_FULL));
-      mbar_arrive(B(S_EMPTY + st));
+      warp_arrive(B(P_FULL));
+      warp_arrive(B(S_EMPTY + st));
       l = l * corr + sum;
       m = m_new;
 #pragma unroll
@@ -224,7 +250,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
         for (int e = 0; e < 32; ++e) o[cc * 32 + e] += __uint_as_float(r[e]);
       }
       tc_fence_before();
-      mbar_arrive(B(O_EMPTY));
+      warp_arrive(B(O_EMPTY));
     }
     if (ok && grow < S) {
       const float inv = 1.f / l;
@@ -246,17 +272,21 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
 }
 
 // ------------------------------------------------------------------ backward: dq
+// One CTA owns 128 queries (Q and dU tiles resident) and streams 64-key slabs of K and V
+// through a 4-deep TMA ring.  S = Q K^T and dP = dU V^T of slab i+1 are issued into a second
+// pair of TMEM buffers while the 128 row threads turn slab i into dS = P (dP - delta);
+// dQ += dS K accumulates in TMEM over all slabs.
 template <int DH>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapG,
-                  const AttnParams p) {
-  constexpr int NH = DH / 64, QT = 128 * DH * 2, PT = 128 * 128 * 2;
+                  const __grid_constant__ CUtensorMap mapKV64, const AttnParams p) {
+  constexpr int NH = DH / 64, QT = 128 * DH * 2, HT = 64 * DH * 2, PT = 128 * 64 * 2, NS = 4;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align1k(smem_raw);
-  const uint32_t Qs = smem_u32(smem), Gs = Qs + QT, Ks = Gs + QT, Vs = Ks + 2 * QT, Ds = Vs + 2 * QT;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 6 * QT + PT);
-  enum { Q_FULL = 0, K_FULL = 1, K_EMPTY = 3, V_FULL = 5, V_EMPTY = 7, SDP_FULL = 9, SDP_EMPTY = 10,
-         DS_FULL = 11, DS_EMPTY = 12, DQ_FULL = 13, NBAR = 14 };
+  const uint32_t Qs = smem_u32(smem), Gs = Qs + QT, Ds = Gs + QT, Rs = Ds + 2 * PT;   // two dS tiles; ring: K then V per stage
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * QT + 2 * PT + NS * 2 * HT);
+  enum { Q_FULL = 0, KV_FULL = 1, KV_EMPTY = 1 + NS, SDP_FULL = 1 + 2 * NS, SDP_EMPTY = 3 + 2 * NS,
+         DS_FULL = 5 + 2 * NS, DS_EMPTY = 7 + 2 * NS, DQ_FULL = 9 + 2 * NS, NBAR = 10 + 2 * NS };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar0 = smem_u32(bars);
@@ -264,11 +294,11 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qb = gridDim.x - 1 - blockIdx.x, head = blockIdx.y, b = blockIdx.z;
   const int d = p.h * DH, S = p.S;
-  const int n = qb + 1;
+  const int n = min(2 * (qb + 1), (S + 63) / 64);      // 64-key slabs up to the diagonal
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
-    mbar_init(B(SDP_EMPTY), 128); mbar_init(B(DS_FULL), 128);
+    mbar_init(B(SDP_EMPTY), 4); mbar_init(B(SDP_EMPTY + 1), 4); mbar_init(B(DS_FULL), 4); mbar_init(B(DS_FULL + 1), 4);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -278,7 +308,7 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tS = tmem, tP = tmem + 128, tQ = tmem + 256;
+  const uint32_t tQ = tmem + 256;      // S of buffer bf at tmem + 128 bf, dP at tmem + 128 bf + 64
 
   if (warp == 0) {
     if (lane == 0) {
@@ -287,45 +317,55 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
         tma_load_3d(Qs + hf * 16384, &mapQKV, B(Q_FULL), head * DH + hf * 64, qb * 128, b);
         tma_load_3d(Gs + hf * 16384, &mapG, B(Q_FULL), head * DH + hf * 64, qb * 128, b);
       }
-      for (int j = 0; j < n; ++j) {
-        const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
-        if (!mbar_wait(B(K_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) break;
-        mbar_expect_tx(B(K_FULL + st), QT);
-        for (int hf = 0; hf < NH; ++hf)
-          tma_load_3d(Ks + st * QT + hf * 16384, &mapQKV, B(K_FULL + st), d + head * DH + hf * 64, j * 128, b);
-        if (!mbar_wait(B(V_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) break;
-        mbar_expect_tx(B(V_FULL + st), QT);
-        for (int hf = 0; hf < NH; ++hf)
-          tma_load_3d(Vs + st * QT + hf * 16384, &mapQKV, B(V_FULL + st), 2 * d + head * DH + hf * 64, j * 128, b);
+      for (int it = 0; it < n; ++it) {
+        const int st = it % NS; const uint32_t ph = (it / NS) & 1;
+        if (!mbar_wait(B(KV_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) break;
+        mbar_expect_tx(B(KV_FULL + st), 2 * HT);
+        for (int hf = 0; hf < NH; ++hf) {
+          tma_load_3d(Rs + st * 2 * HT + hf * 8192, &mapKV64, B(KV_FULL + st), d + head * DH + hf * 64, it * 64, b);
+          tma_load_3d(Rs + st * 2 * HT + HT + hf * 8192, &mapKV64, B(KV_FULL + st), 2 * d + head * DH + hf * 64, it * 64, b);
+        }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
+      constexpr uint32_t idesc_s = make_idesc(128, 64, false, false);
       constexpr uint32_t idesc_q = make_idesc(128, DH, false, true);
+      auto issue_sdp = [&](int it) -> bool {
+        const int st = it % NS, bf = it & 1;
+        if (!mbar_wait(B(KV_FULL + st), (it / NS) & 1, abort_flag, p.flags)) return false;
+        if (!mbar_wait(B(SDP_EMPTY + bf), ((it >> 1) & 1) ^ 1u, abort_flag, p.flags)) return false;
+        tc_fence_after();
+        const uint32_t tS = tmem + 128 * bf, tP = tS + 64, Kst = Rs + st * 2 * HT, Vst = Kst + HT;
+        const uint32_t q_lo = klo(Qs), g_lo = klo(Gs), k_lo = klo(Kst), v_lo = klo(Vst);
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks)
+          umma_lo(tS, q_lo + kstep<128>(ks), k_lo + kstep<64>(ks), idesc_s, ks > 0);
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks)
+          umma_lo(tP, g_lo + kstep<128>(ks), v_lo + kstep<64>(ks), idesc_s, ks > 0);
+        umma_commit(B(SDP_FULL + bf));
+        return true;
+      };
+      auto issue_dq = [&](int it) -> bool {
+        const int st = it % NS, db = it & 1;
+        if (!mbar_wait(B(DS_FULL + db), (it >> 1) & 1, abort_flag, p.flags)) return false;
+        tc_fence_after();
+        const uint32_t ds_lo = klo(Ds + db * PT), kmn_lo = mlo<64>(Rs + st * 2 * HT);
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          umma_lo(tQ, ds_lo + kstep<128>(ks), kmn_lo + mstep(ks), idesc_q, (it > 0 || ks > 0));
+        umma_commit(B(DS_EMPTY + db));
+        umma_commit(B(KV_EMPTY + st));
+        if (it == n - 1) umma_commit(B(DQ_FULL));
+        return true;
+      };
       bool ok = mbar_wait(B(Q_FULL), 0, abort_flag, p.flags);
-      for (int j = 0; j < n && ok; ++j) {
-        const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
-        if (!mbar_wait(B(K_FULL + st), ph, abort_flag, p.flags)) break;
-        if (!mbar_wait(B(V_FULL + st), ph, abort_flag, p.flags)) break;
-        if (!mbar_wait(B(SDP_EMPTY), (j & 1) ^ 1u, abort_flag, p.flags)) break;
-        tc_fence_after();
-#pragma unroll
-        for (int ks = 0; ks < DH / 16; ++ks)
-          umma_bf16(tS, kmajor_desc<128>(Qs, ks), kmajor_desc<128>(Ks + st * QT, ks), idesc_s, ks > 0);
-#pragma unroll
-        for (int ks = 0; ks < DH / 16; ++ks)
-          umma_bf16(tP, kmajor_desc<128>(Gs, ks), kmajor_desc<128>(Vs + st * QT, ks), idesc_s, ks > 0);
-        umma_commit(B(SDP_FULL));
-        umma_commit(B(V_EMPTY + st));
-        if (!mbar_wait(B(DS_FULL), j & 1, abort_flag, p.flags)) break;
-        tc_fence_after();
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          umma_bf16(tQ, kmajor_desc<128>(Ds, ks), mnmajor_desc<128>(Ks + st * QT, ks), idesc_q, (j > 0 || ks > 0));
-        umma_commit(B(DS_EMPTY));
-        umma_commit(B(K_EMPTY + st));
-        if (j == n - 1) umma_commit(B(DQ_FULL));
+      ok = ok && issue_sdp(0);
+      if (ok && n > 1) ok = issue_sdp(1);
+      for (int it = 0; it < n && ok; ++it) {
+        ok = issue_dq(it);
+        if (ok && it + 2 < n) ok = issue_sdp(it + 2);
       }
     }
   } else {
@@ -337,32 +377,31 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
     const int64_t si = ((int64_t)b * p.h + head) * S + (grow < S ? grow : S - 1);
     const float l2 = p.lse[si] * LOG2E, dl = p.delta[si];
     bool ok = true;
-    for (int j = 0; j < n && ok; ++j) {
-      if (!mbar_wait(B(SDP_FULL), j & 1, abort_flag, p.flags)) { ok = false; break; }
+    for (int it = 0; it < n && ok; ++it) {
+      const int bf = it & 1;
+      const uint32_t tS = tmem + 128 * bf + lane_off, tP = tS + 64;
+      if (!mbar_wait(B(SDP_FULL + bf), (it >> 1) & 1, abort_flag, p.flags)) { ok = false; break; }
       tc_fence_after();
-      const bool diag = (j == qb) || ((j + 1) * 128 > S);
-#pragma unroll 1
-      for (int cc = 0; cc < 4; ++cc) {
-        uint32_t rs[32], rd[32];
-        tmem_ld32(tS + lane_off + cc * 32, rs);
-        tmem_ld32(tP + lane_off + cc * 32, rd);
-        tmem_ld_wait();
-        float ds[32];
-#pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const int col = j * 128 + cc * 32 + e;
-          float pe = ex2(__uint_as_float(rs[e]) * c - l2);
-          if (diag && (col > grow || col >= S)) pe = 0.f;
-          ds[e] = pe * (__uint_as_float(rd[e]) - dl);
-        }
-        if (cc == 0 && !mbar_wait(B(DS_EMPTY), (j & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
-        store_row32(Ds, 16384, row, cc * 4, ds);
-      }
-      if (!ok) break;
+      uint32_t rs[64], rd[64];
+      tmem_ld32(tS, rs); tmem_ld32(tS + 32, rs + 32);
+      tmem_ld32(tP, rd); tmem_ld32(tP + 32, rd + 32);
+      tmem_ld_wait();
       tc_fence_before();
+      warp_arrive(B(SDP_EMPTY + bf));          // the accumulators are in registers: free them early
+      const bool diag = ((it + 1) * 64 > qb * 128) || ((it + 1) * 64 > S);
+      float ds[64];
+#pragma unroll
+      for (int e = 0; e < 64; ++e) {
+        const int col = it * 64 + e;
+        float pe = ex2(__uint_as_float(rs[e]) * c - l2);
+        if (diag && (col > grow || col >= S)) pe = 0.f;
+        ds[e] = pe * (__uint_as_float(rd[e]) - dl);
+      }
+      if (!mbar_wait(B(DS_EMPTY + bf), ((it >> 1) & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+      store_row32(Ds + bf * PT, 0, row, 0, ds);
+      store_row32(Ds + bf * PT, 0, row, 4, ds + 32);
       fence_async_smem();
-      mbar_arrive(B(DS_FULL));
-      mbar_arrive(B(SDP_EMPTY));
+      warp_arrive(B(DS_FULL + bf));
     }
     if (ok && mbar_wait(B(DQ_FULL), 0, abort_flag, p.flags)) {
       tc_fence_after();
@@ -393,18 +432,21 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
 }
 
 // ------------------------------------------------------------------ backward: dk, dv
+// One CTA owns 128 keys (K and V tiles resident) and streams 64-query slabs of Q and dU through
+// a 4-deep TMA ring.  The transposed products S^T = K Q^T and dP^T = V dU^T of slab i+1 are
+// issued into a second pair of TMEM buffers while the 128 row threads (one key each) form
+// P^T and dS^T of slab i; dV += P^T dU and dK += dS^T Q accumulate in TMEM.
 template <int DH>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_constant__ CUtensorMap mapQ64,
                    const __grid_constant__ CUtensorMap mapG64, const AttnParams p) {
-  constexpr int NH = DH / 64, QT = 128 * DH * 2, HT = 64 * DH * 2, PT = 128 * 64 * 2;
+  constexpr int NH = DH / 64, QT = 128 * DH * 2, HT = 64 * DH * 2, PT = 128 * 64 * 2, NS = 3;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align1k(smem_raw);
-  const uint32_t Ks = smem_u32(smem), Vs = Ks + QT, Qs = Vs + QT, Gs = Qs + 2 * HT, Ps = Gs + 2 * HT,
-                 Ds = Ps + PT;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * QT + 4 * HT + 2 * PT);
-  enum { KV_FULL = 0, QG_FULL = 1, QG_EMPTY = 3, SDP_FULL = 5, SDP_EMPTY = 6, PDS_FULL = 7,
-         PDS_EMPTY = 8, OUT_FULL = 9, NBAR = 10 };
+  const uint32_t Ks = smem_u32(smem), Vs = Ks + QT, Ps = Vs + QT, Ds = Ps + 2 * PT, Rs = Ds + 2 * PT;  // two P^T / dS^T tiles; ring: Q then dU
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * QT + 4 * PT + NS * 2 * HT);
+  enum { KV_FULL = 0, QG_FULL = 1, QG_EMPTY = 1 + NS, SDP_FULL = 1 + 2 * NS, SDP_EMPTY = 3 + 2 * NS,
+         PDS_FULL = 5 + 2 * NS, PDS_EMPTY = 7 + 2 * NS, OUT_FULL = 9 + 2 * NS, NBAR = 10 + 2 * NS };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar0 = smem_u32(bars);
@@ -412,11 +454,11 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_const
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kb = blockIdx.x, head = blockIdx.y, b = blockIdx.z;
   const int d = p.h * DH, S = p.S;
-  const int i0 = 2 * kb, n = (S + 63) / 64 - i0;      // query blocks of 64 from the diagonal down
+  const int i0 = 2 * kb, n = (S + 63) / 64 - i0;      // 64-query slabs from the diagonal down
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
-    mbar_init(B(SDP_EMPTY), 128); mbar_init(B(PDS_FULL), 128);
+    mbar_init(B(SDP_EMPTY), 4); mbar_init(B(SDP_EMPTY + 1), 4); mbar_init(B(PDS_FULL), 4); mbar_init(B(PDS_FULL + 1), 4);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -426,7 +468,7 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tS = tmem, tP = tmem + 64, tV = tmem + 128, tK = tmem + 128 + DH;
+  const uint32_t tV = tmem + 256, tK = tmem + 256 + DH;   // S^T of buffer bf at tmem + 128 bf, dP^T at + 64
 
   if (warp == 0) {
     if (lane == 0) {
@@ -436,12 +478,12 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_const
         tma_load_3d(Vs + hf * 16384, &mapKV, B(KV_FULL), 2 * d + head * DH + hf * 64, kb * 128, b);
       }
       for (int it = 0; it < n; ++it) {
-        const int st = it & 1; const uint32_t ph = (it >> 1) & 1;
+        const int st = it % NS; const uint32_t ph = (it / NS) & 1;
         if (!mbar_wait(B(QG_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) break;
         mbar_expect_tx(B(QG_FULL + st), 2 * HT);
         for (int hf = 0; hf < NH; ++hf) {
-          tma_load_3d(Qs + st * HT + hf * 8192, &mapQ64, B(QG_FULL + st), head * DH + hf * 64, (i0 + it) * 64, b);
-          tma_load_3d(Gs + st * HT + hf * 8192, &mapG64, B(QG_FULL + st), head * DH + hf * 64, (i0 + it) * 64, b);
+          tma_load_3d(Rs + st * 2 * HT + hf * 8192, &mapQ64, B(QG_FULL + st), head * DH + hf * 64, (i0 + it) * 64, b);
+          tma_load_3d(Rs + st * 2 * HT + HT + hf * 8192, &mapG64, B(QG_FULL + st), head * DH + hf * 64, (i0 + it) * 64, b);
         }
       }
     }
@@ -449,30 +491,45 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_const
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc(128, 64, false, false);
       constexpr uint32_t idesc_o = make_idesc(128, DH, false, true);
-      bool ok = mbar_wait(B(KV_FULL), 0, abort_flag, p.flags);
-      for (int it = 0; it < n && ok; ++it) {
-        const int st = it & 1; const uint32_t ph = (it >> 1) & 1;
-        if (!mbar_wait(B(QG_FULL + st), ph, abort_flag, p.flags)) break;
-        if (!mbar_wait(B(SDP_EMPTY), (it & 1) ^ 1u, abort_flag, p.flags)) break;
+      auto issue_sdp = [&](int it) -> bool {
+        const int st = it % NS, bf = it & 1;
+        if (!mbar_wait(B(QG_FULL + st), (it / NS) & 1, abort_flag, p.flags)) return false;
+        if (!mbar_wait(B(SDP_EMPTY + bf), ((it >> 1) & 1) ^ 1u, abort_flag, p.flags)) return false;
         tc_fence_after();
+        const uint32_t tS = tmem + 128 * bf, tP = tS + 64, Qst = Rs + st * 2 * HT, Gst = Qst + HT;
+        const uint32_t k_lo = klo(Ks), v_lo = klo(Vs), q_lo = klo(Qst), g_lo = klo(Gst);
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks)
-          umma_bf16(tS, kmajor_desc<128>(Ks, ks), kmajor_desc<64>(Qs + st * HT, ks), idesc_s, ks > 0);
+          umma_lo(tS, k_lo + kstep<128>(ks), q_lo + kstep<64>(ks), idesc_s, ks > 0);
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks)
-          umma_bf16(tP, kmajor_desc<128>(Vs, ks), kmajor_desc<64>(Gs + st * HT, ks), idesc_s, ks > 0);
-        umma_commit(B(SDP_FULL));
-        if (!mbar_wait(B(PDS_FULL), it & 1, abort_flag, p.flags)) break;
+          umma_lo(tP, v_lo + kstep<128>(ks), g_lo + kstep<64>(ks), idesc_s, ks > 0);
+        umma_commit(B(SDP_FULL + bf));
+        return true;
+      };
+      auto issue_out = [&](int it) -> bool {
+        const int st = it % NS, db = it & 1;
+        const uint32_t Qst = Rs + st * 2 * HT, Gst = Qst + HT;
+        if (!mbar_wait(B(PDS_FULL + db), (it >> 1) & 1, abort_flag, p.flags)) return false;
         tc_fence_after();
+        const uint32_t p_lo = klo(Ps + db * PT), ds_lo = klo(Ds + db * PT), gmn_lo = mlo<64>(Gst), qmn_lo = mlo<64>(Qst);
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
-          umma_bf16(tV, kmajor_desc<128>(Ps, ks), mnmajor_desc<64>(Gs + st * HT, ks), idesc_o, (it > 0 || ks > 0));
+          umma_lo(tV, p_lo + kstep<128>(ks), gmn_lo + mstep(ks), idesc_o, (it > 0 || ks > 0));
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
-          umma_bf16(tK, kmajor_desc<128>(Ds, ks), mnmajor_desc<64>(Qs + st * HT, ks), idesc_o, (it > 0 || ks > 0));
-        umma_commit(B(PDS_EMPTY));
+          umma_lo(tK, ds_lo + kstep<128>(ks), qmn_lo + mstep(ks), idesc_o, (it > 0 || ks > 0));
+        umma_commit(B(PDS_EMPTY + db));
         umma_commit(B(QG_EMPTY + st));
         if (it == n - 1) umma_commit(B(OUT_FULL));
+        return true;
+      };
+      bool ok = mbar_wait(B(KV_FULL), 0, abort_flag, p.flags);
+      ok = ok && issue_sdp(0);
+      if (ok && n > 1) ok = issue_sdp(1);
+      for (int it = 0; it < n && ok; ++it) {
+        ok = issue_out(it);
+        if (ok && it + 2 < n) ok = issue_sdp(it + 2);
       }
     }
   } else {
@@ -485,14 +542,17 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_const
     const float* drow = p.delta + ((int64_t)b * p.h + head) * S;
     bool ok = true;
     for (int it = 0; it < n && ok; ++it) {
+      const int bf = it & 1;
+      const uint32_t tS = tmem + 128 * bf + lane_off, tP = tS + 64;
       const int q0 = (i0 + it) * 64;
-      if (!mbar_wait(B(SDP_FULL), it & 1, abort_flag, p.flags)) { ok = false; break; }
+      if (!mbar_wait(B(SDP_FULL + bf), (it >> 1) & 1, abort_flag, p.flags)) { ok = false; break; }
       tc_fence_after();
+      if (!mbar_wait(B(PDS_EMPTY + bf), ((it >> 1) & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
 #pragma unroll 1
       for (int cc = 0; cc < 2; ++cc) {
         uint32_t rs[32], rd[32];
-        tmem_ld32(tS + lane_off + cc * 32, rs);
-        tmem_ld32(tP + lane_off + cc * 32, rd);
+        tmem_ld32(tS + cc * 32, rs);
+        tmem_ld32(tP + cc * 32, rd);
         tmem_ld_wait();
         float pv[32], ds[32];
 #pragma unroll
@@ -504,15 +564,13 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_const
           pv[e] = pe;
           ds[e] = pe * (__uint_as_float(rd[e]) - __ldg(drow + qc));
         }
-        if (cc == 0 && !mbar_wait(B(PDS_EMPTY), (it & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
-        store_row32(Ps, 0, row, cc * 4, pv);
-        store_row32(Ds, 0, row, cc * 4, ds);
+        store_row32(Ps + bf * PT, 0, row, cc * 4, pv);
+        store_row32(Ds + bf * PT, 0, row, cc * 4, ds);
       }
-      if (!ok) break;
       tc_fence_before();
+      warp_arrive(B(SDP_EMPTY + bf));
       fence_async_smem();
-      mbar_arrive(B(PDS_FULL));
-      mbar_arrive(B(SDP_EMPTY));
+      warp_arrive(B(PDS_FULL + bf));
     }
     if (ok && mbar_wait(B(OUT_FULL), 0, abort_flag, p.flags)) {
       tc_fence_after();
@@ -581,8 +639,8 @@ int fwd_t(const bf16* qkv, bf16* U, float* lse, int B, int S, int h, int* flags,
 template <int DH>
 int bwd_t(const bf16* qkv, const float* lse, const bf16* dU, bf16* dqkv, const float* delta, int B,
           int S, int h, int* flags, cudaStream_t st) {
-  constexpr int SM_DQ = 6 * 128 * DH * 2 + 128 * 128 * 2 + EXTRA;
-  constexpr int SM_KV = 2 * 128 * DH * 2 + 4 * 64 * DH * 2 + 2 * 128 * 64 * 2 + EXTRA;
+  constexpr int SM_DQ = 2 * 128 * DH * 2 + 2 * 128 * 64 * 2 + 4 * 2 * 64 * DH * 2 + EXTRA;
+  constexpr int SM_KV = 2 * 128 * DH * 2 + 4 * 128 * 64 * 2 + 3 * 2 * 64 * DH * 2 + EXTRA;
   static bool ok = set_smem(attn_dq_tc_kernel<DH>, SM_DQ) && set_smem(attn_dkv_tc_kernel<DH>, SM_KV);
   if (!ok) return -2;
   const int d = h * DH;
@@ -592,7 +650,7 @@ int bwd_t(const bf16* qkv, const float* lse, const bf16* dU, bf16* dqkv, const f
     return -3;
   AttnParams p{}; p.lse = lse; p.delta = delta; p.dqkv = dqkv; p.S = S; p.h = h; p.flags = flags;
   dim3 grid((S + 127) / 128, h, B);
-  attn_dq_tc_kernel<DH><<<grid, ATT_THREADS, SM_DQ, st>>>(mQKV, mG, p);
+  attn_dq_tc_kernel<DH><<<grid, ATT_THREADS, SM_DQ, st>>>(mQKV, mG, mQ64, p);
   attn_dkv_tc_kernel<DH><<<grid, ATT_THREADS, SM_KV, st>>>(mQKV, mQ64, mG64, p);
   return 0;
 }
