@@ -50,6 +50,23 @@ __device__ __forceinline__ uint4 pack8_bf16(const float* f) {
   return u;
 }
 
+// 32-byte global accesses (one full sector per lane and instruction)
+__device__ __forceinline__ void st_v8(void* p, const uint32_t* v) {
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(v[0]), "r"(v[1]),
+               "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
+}
+__device__ __forceinline__ void ld_v8(uint32_t* v, const void* p) {
+  asm volatile("ld.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+                 "=r"(v[7])
+               : "l"(p));
+}
+__device__ __forceinline__ uint32_t pack2_bf16(float a, float b) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
 struct TcParams {
   int M, N, K;
   int epilogue;
@@ -59,6 +76,7 @@ struct TcParams {
   int* flags;
   int tiles_m, tiles_n;
   int splits; long long split_stride;
+  int wide;   // every output / auxiliary row start is 32-byte aligned: use 32-byte accesses
 };
 
 template <int BN> struct Cfg {
@@ -204,6 +222,63 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         tmem_ld32(t_row + c0, r);              // asynchronous until tmem_ld_wait
         const long long ci = (long long)m * p.ldc + nb + (long long)sp * p.split_stride;
         const bool full = nb + 32 <= p.N;
+        if (p.wide && full) {
+          // whole 32-column chunk with 32-byte accesses
+          if (p.epilogue == EPI_RESID_F32) {
+            uint32_t x[32];
+            const float* rs = (const float*)p.aux + (long long)m * p.ldaux + nb;
+            if (row_ok) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j) ld_v8(x + 8 * j, rs + 8 * j);
+            }
+            tmem_ld_wait();
+            if (row_ok) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) x[j] = __float_as_uint(__uint_as_float(x[j]) + __uint_as_float(r[j]));
+#pragma unroll
+              for (int j = 0; j < 4; ++j) st_v8((float*)p.C + ci + 8 * j, x + 8 * j);
+            }
+          } else if (p.epilogue == EPI_DGELU) {
+            uint32_t hv[16];
+            const bf16* hs = (const bf16*)p.aux + (long long)m * p.ldaux + nb;
+            if (row_ok) { ld_v8(hv, hs); ld_v8(hv + 8, hs + 16); }
+            tmem_ld_wait();
+            if (row_ok) {
+              uint32_t o[16];
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const float2 h2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&hv[j]));
+                o[j] = pack2_bf16(__uint_as_float(r[2 * j]) * gelu_grad_dev(h2.x),
+                                  __uint_as_float(r[2 * j + 1]) * gelu_grad_dev(h2.y));
+              }
+              st_v8((bf16*)p.C + ci, o);
+              st_v8((bf16*)p.C + ci + 16, o + 8);
+            }
+          } else if (p.epilogue == EPI_STORE_F32) {
+            tmem_ld_wait();
+            if (row_ok) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j) st_v8((float*)p.C + ci + 8 * j, r + 8 * j);
+            }
+          } else {
+            tmem_ld_wait();
+            if (row_ok) {
+              uint32_t o[16];
+#pragma unroll
+              for (int j = 0; j < 16; ++j) o[j] = pack2_bf16(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+              st_v8((bf16*)p.C + ci, o);
+              st_v8((bf16*)p.C + ci + 16, o + 8);
+              if (p.epilogue == EPI_GELU_DUAL) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                  o[j] = pack2_bf16(gelu_dev(__uint_as_float(r[2 * j])), gelu_dev(__uint_as_float(r[2 * j + 1])));
+                st_v8((bf16*)p.C2 + ci, o);
+                st_v8((bf16*)p.C2 + ci + 16, o + 8);
+              }
+            }
+          }
+          continue;
+        }
         if (p.epilogue == EPI_RESID_F32) {
           float4 x[8];
           const float4* rs = reinterpret_cast<const float4*>((const float*)p.aux + (long long)m * p.ldaux + nb);
@@ -328,6 +403,16 @@ int launch_t(const GemmArgs& g, cudaStream_t st) {
   const int k_blocks = (g.K + BK - 1) / BK;
   p.splits = g.splits < 1 ? 1 : (g.splits > k_blocks ? k_blocks : g.splits);
   p.split_stride = g.split_stride;
+  {
+    const bool f32 = g.epilogue == EPI_STORE_F32 || g.epilogue == EPI_RESID_F32;
+    const long long out_unit = f32 ? 8 : 16;   // elements per 32 bytes
+    bool w = (reinterpret_cast<uintptr_t>(g.C) % 32 == 0) && (g.ldc % out_unit == 0) &&
+             (g.split_stride % out_unit == 0);
+    if (g.epilogue == EPI_GELU_DUAL) w = w && (reinterpret_cast<uintptr_t>(g.C2) % 32 == 0);
+    if (g.epilogue == EPI_RESID_F32) w = w && (reinterpret_cast<uintptr_t>(g.aux) % 32 == 0) && (g.ldaux % 8 == 0);
+    if (g.epilogue == EPI_DGELU) w = w && (reinterpret_cast<uintptr_t>(g.aux) % 32 == 0) && (g.ldaux % 16 == 0);
+    p.wide = w ? 1 : 0;
+  }
   const int tiles = p.tiles_m * p.tiles_n * p.splits;
   static int n_sm = 0;
   if (n_sm == 0) {

@@ -84,78 +84,96 @@ slice_move_kernel(const SliceSeg* __restrict__ segs, float* packed, float* dense
   }
 }
 
-// Outer sweep over the whole canonical vector, one float4 per thread-iteration.
+// Outer sweep (Algorithm 1 lines 12-15).  blockIdx.y selects a segment of the canonical
+// vector - a quarter of E, a layer's non-FFN block, its W_in, its W_out, or the final
+// LayerNorm - so that the position decoding is block-uniform; within a segment every thread
+// keeps four independent float4 streams in flight.
+constexpr int OUTER_U = 4;
+
+__device__ __forceinline__ void outer_update(float4& th, float4& bu, const float4& total, int count,
+                                             float lr, float mu) {
+  const float m = count > 0 ? (float)count : 1.f;
+  float* pt = &th.x; float* pb = &bu.x; const float* pd = &total.x;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float g = -(pd[e] / m);
+    const float b = mu * pb[e] + g;
+    pt[e] = pt[e] - lr * (g + mu * b);
+    pb[e] = b;
+  }
+}
+
 __global__ void __launch_bounds__(256)
 outer_kernel(OuterTables t, float* __restrict__ theta, float* __restrict__ buf,
              bf16* __restrict__ w16, float lr, float mu) {
-  const int64_t n4 = t.P / 4;
-  const int64_t win_end = t.win_rel + (int64_t)t.F * t.d;
-  const int64_t wout_end = t.wout_rel + (int64_t)t.F * t.d;
-  for (int64_t i4 = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i4 < n4;
-       i4 += (int64_t)gridDim.x * blockDim.x) {
-    const int64_t i = 4 * i4;
-    float4 th = *reinterpret_cast<const float4*>(theta + i);
-    float4 bu = *reinterpret_cast<const float4*>(buf + i);
-    float4 total = make_float4(0.f, 0.f, 0.f, 0.f);
-    int count = 0;
-    float* slot[8];  // owners' packed positions to restart (at most 8 kept inline)
-    int ob = 0, oe = 0;
-    int64_t rel = i - t.e_size;
-    int layer = -1, unit = 0, which = 0;
-    int64_t inner = 0;  // W_in: column; W_out: row
-    if (rel >= 0) {
-      const int64_t l = rel / t.layer_size;
-      if (l < t.L) {
-        const int64_t r = rel - l * t.layer_size;
-        if (r >= t.win_rel && r < win_end) {
-          const int64_t q = r - t.win_rel;
-          unit = (int)(q / t.d); inner = q - (int64_t)unit * t.d; which = 1; layer = (int)l;
-        } else if (r >= t.wout_rel && r < wout_end) {
-          const int64_t q = r - t.wout_rel;
-          inner = q / t.F; unit = (int)(q - inner * t.F); which = 2; layer = (int)l;
-        }
-      }
-    }
-    if (which) {
-      const int64_t grp = (int64_t)layer * (t.F / 8) + unit / 8;
-      ob = t.unit_begin[grp];
-      oe = t.unit_begin[grp + 1];
-    }
-    for (int o = ob; o < oe; ++o) {
-      const OuterOwner ow = t.owners[t.unit_owner[o]];
-      float* p = which == 1
-                     ? ow.master + ow.in_off + (int64_t)(unit - ow.lo) * t.d + inner
-                     : ow.master + ow.out_off + inner * (ow.hi - ow.lo) + (unit - ow.lo);
-      const float4 e = *reinterpret_cast<const float4*>(p);
-      total.x += e.x - th.x; total.y += e.y - th.y; total.z += e.z - th.z; total.w += e.w - th.w;
-      if (count < 8) slot[count] = p;
-      ++count;
-    }
-    float4 nt;
-    {
-      const float inv_m = count > 0 ? (float)count : 1.f;
-      float* pt = &th.x; float* pb = &bu.x; float* pd = &total.x; float* pn = &nt.x;
+  // ---- segment decoding (uniform per block) ----
+  const int seg = blockIdx.y;
+  int64_t start; int64_t len; int kind = 0, layer = 0;
+  const int64_t fd = (int64_t)t.F * t.d;
+  if (seg < 4) {
+    const int64_t q = ((t.e_size / 4 + 3) / 4) * 4;          // quarter of E, whole float4s
+    start = seg * q;
+    len = seg < 3 ? q : t.e_size - 3 * q;
+    if (len < 0) len = 0;
+    if (start > t.e_size) { start = t.e_size; len = 0; }
+  } else if (seg == 4 + 3 * t.L) {
+    start = t.e_size + (int64_t)t.L * t.layer_size;
+    len = t.P - start;
+  } else {
+    layer = (seg - 4) / 3;
+    const int w = (seg - 4) - 3 * layer;
+    const int64_t base = t.e_size + (int64_t)layer * t.layer_size;
+    if (w == 0) { start = base; len = t.win_rel; }
+    else if (w == 1) { start = base + t.win_rel; len = fd; kind = 1; }
+    else { start = base + t.wout_rel; len = fd; kind = 2; }
+  }
+  const uint32_t n4 = (uint32_t)(len / 4);
+  const uint32_t stride = gridDim.x * blockDim.x;
+  float* th_p = theta + start;
+  float* bu_p = buf + start;
+  bf16* w_p = w16 + start;
+  const int32_t* ub = t.unit_begin + (int64_t)layer * (t.F / 8);
+
+  for (uint32_t e0 = blockIdx.x * blockDim.x + threadIdx.x; e0 < n4; e0 += OUTER_U * stride) {
+    float4 th[OUTER_U], bu[OUTER_U];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float g = -(pd[e] / inv_m);
-        const float b = mu * pb[e] + g;
-        pn[e] = pt[e] - lr * (g + mu * b);
-        pb[e] = b;
+    for (int k = 0; k < OUTER_U; ++k) {
+      const uint32_t e = e0 + k * stride;
+      if (e < n4) {
+        th[k] = reinterpret_cast<const float4*>(th_p)[e];
+        bu[k] = reinterpret_cast<const float4*>(bu_p)[e];
       }
     }
-    *reinterpret_cast<float4*>(theta + i) = nt;
-    *reinterpret_cast<float4*>(buf + i) = bu;
-    store_bf16x4(w16 + i, nt);
-    for (int c = 0; c < count && c < 8; ++c) *reinterpret_cast<float4*>(slot[c]) = nt;
-    if (count > 8) {  // rare: more than 8 replicas share this position
-      int c = 0;
-      for (int o = ob; o < oe; ++o, ++c) {
-        if (c < 8) continue;
+#pragma unroll
+    for (int k = 0; k < OUTER_U; ++k) {
+      const uint32_t e = e0 + k * stride;
+      if (e >= n4) break;
+      float4 total = make_float4(0.f, 0.f, 0.f, 0.f);
+      int count = 0, ob = 0, oe = 0;
+      uint32_t unit = 0, inner = 0;
+      if (kind == 1) { unit = (4u * e) / (uint32_t)t.d; inner = 4u * e - unit * (uint32_t)t.d; }
+      else if (kind == 2) { inner = (4u * e) / (uint32_t)t.F; unit = 4u * e - inner * (uint32_t)t.F; }
+      if (kind) { ob = ub[unit >> 3]; oe = ub[(unit >> 3) + 1]; }
+      const float4 old = th[k];
+      for (int o = ob; o < oe; ++o) {
         const OuterOwner ow = t.owners[t.unit_owner[o]];
-        float* p = which == 1
-                       ? ow.master + ow.in_off + (int64_t)(unit - ow.lo) * t.d + inner
-                       : ow.master + ow.out_off + inner * (ow.hi - ow.lo) + (unit - ow.lo);
-        *reinterpret_cast<float4*>(p) = nt;
+        const float* p = kind == 1
+                             ? ow.master + ow.in_off + (int64_t)((int)unit - ow.lo) * t.d + inner
+                             : ow.master + ow.out_off + (int64_t)inner * (ow.hi - ow.lo) + ((int)unit - ow.lo);
+        const float4 v = *reinterpret_cast<const float4*>(p);
+        total.x += v.x - old.x; total.y += v.y - old.y; total.z += v.z - old.z; total.w += v.w - old.w;
+        ++count;
+      }
+      outer_update(th[k], bu[k], total, count, lr, mu);
+      reinterpret_cast<float4*>(th_p)[e] = th[k];
+      reinterpret_cast<float4*>(bu_p)[e] = bu[k];
+      store_bf16x4(w_p + 4 * (int64_t)e, th[k]);
+      for (int o = ob; o < oe; ++o) {       // the owners restart from the new parameters
+        const OuterOwner ow = t.owners[t.unit_owner[o]];
+        float* p = kind == 1
+                       ? ow.master + ow.in_off + (int64_t)((int)unit - ow.lo) * t.d + inner
+                       : ow.master + ow.out_off + (int64_t)inner * (ow.hi - ow.lo) + ((int)unit - ow.lo);
+        *reinterpret_cast<float4*>(p) = th[k];
       }
     }
   }
@@ -209,5 +227,7 @@ void launch_slices_scatter_f32(const SliceSeg* segs, int n_seg, const float* pac
 
 void launch_outer(const OuterTables& t, float* theta, float* buf, bf16* w16, float lr, float mu,
                   cudaStream_t st) {
-  outer_kernel<<<grid_for(t.P / 4, 256, 8), 256, 0, st>>>(t, theta, buf, w16, lr, mu);
+  // 4 segments for E, 3 per layer, 1 for the final LayerNorm; ~2 waves of 256-thread blocks
+  dim3 grid(32, 4 + 3 * t.L + 1);
+  outer_kernel<<<grid, 256, 0, st>>>(t, theta, buf, w16, lr, mu);
 }
