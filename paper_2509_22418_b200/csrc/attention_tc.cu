@@ -33,6 +33,29 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
   __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&v);
 }
+// 32 consecutive head columns starting at c0, scaled by f and (optionally) rotated back by the
+// position's angle, packed to bf16 and stored
+__device__ __forceinline__ void drain32(bf16* out, const uint32_t* r, float f, const float2* cs_row, int c0) {
+  float v[32];
+#pragma unroll
+  for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]) * f;
+  if (cs_row) {
+#pragma unroll
+    for (int q = 0; q < 16; ++q) {
+      const float2 w = __ldg(cs_row + c0 / 2 + q);
+      const float a = v[2 * q], b = v[2 * q + 1];
+      v[2 * q] = a * w.x + b * w.y;
+      v[2 * q + 1] = b * w.x - a * w.y;
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 32; e += 8) {
+    uint4 u;
+    u.x = pack2(v[e], v[e + 1]); u.y = pack2(v[e + 2], v[e + 3]);
+    u.z = pack2(v[e + 4], v[e + 5]); u.w = pack2(v[e + 6], v[e + 7]);
+    *reinterpret_cast<uint4*>(out + e) = u;
+  }
+}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -62,6 +85,7 @@ struct AttnParams {
   const float* lse; const float* delta;
   bf16* U; float* lse_out; bf16* dqkv;
   int S, h; int* flags;
+  const float2* inv_rope;   // (cos, sin) table [S][d_h/2]: rotate dq, dk by -angle on the way out (or null)
 };
 
 // A [ROWS x DH] K-major operand tile: DH/64 half-tiles of ROWS*128 bytes.  K-step ks (16 columns).
@@ -411,17 +435,8 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
         uint32_t r[32];
         tmem_ld32(tQ + lane_off + cc * 32, r);
         tmem_ld_wait();
-        if (grow < S) {
-#pragma unroll
-          for (int e = 0; e < 32; e += 8) {
-            uint4 u;
-            u.x = pack2(__uint_as_float(r[e]) * scale, __uint_as_float(r[e + 1]) * scale);
-            u.y = pack2(__uint_as_float(r[e + 2]) * scale, __uint_as_float(r[e + 3]) * scale);
-            u.z = pack2(__uint_as_float(r[e + 4]) * scale, __uint_as_float(r[e + 5]) * scale);
-            u.w = pack2(__uint_as_float(r[e + 6]) * scale, __uint_as_float(r[e + 7]) * scale);
-            *reinterpret_cast<uint4*>(out + cc * 32 + e) = u;
-          }
-        }
+        if (grow < S)
+          drain32(out + cc * 32, r, scale, p.inv_rope ? p.inv_rope + (int64_t)grow * (DH / 2) : nullptr, cc * 32);
       }
     }
   }
@@ -582,19 +597,9 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_const
         uint32_t r[32];
         tmem_ld32((is_k ? tK : tV) + lane_off + c0, r);
         tmem_ld_wait();
-        const float f = is_k ? scale : 1.f;
-        if (key < S) {
-          bf16* o = out + (is_k ? d : 2 * d) + c0;
-#pragma unroll
-          for (int e = 0; e < 32; e += 8) {
-            uint4 u;
-            u.x = pack2(__uint_as_float(r[e]) * f, __uint_as_float(r[e + 1]) * f);
-            u.y = pack2(__uint_as_float(r[e + 2]) * f, __uint_as_float(r[e + 3]) * f);
-            u.z = pack2(__uint_as_float(r[e + 4]) * f, __uint_as_float(r[e + 5]) * f);
-            u.w = pack2(__uint_as_float(r[e + 6]) * f, __uint_as_float(r[e + 7]) * f);
-            *reinterpret_cast<uint4*>(o + e) = u;
-          }
-        }
+        if (key < S)
+          drain32(out + (is_k ? d : 2 * d) + c0, r, is_k ? scale : 1.f,
+                  (is_k && p.inv_rope) ? p.inv_rope + (int64_t)key * (DH / 2) : nullptr, c0);
       }
     }
   }
@@ -638,7 +643,7 @@ int fwd_t(const bf16* qkv, bf16* U, float* lse, int B, int S, int h, int* flags,
 
 template <int DH>
 int bwd_t(const bf16* qkv, const float* lse, const bf16* dU, bf16* dqkv, const float* delta, int B,
-          int S, int h, int* flags, cudaStream_t st) {
+          int S, int h, int* flags, cudaStream_t st, const float2* inv_rope) {
   constexpr int SM_DQ = 2 * 128 * DH * 2 + 2 * 128 * 64 * 2 + 4 * 2 * 64 * DH * 2 + EXTRA;
   constexpr int SM_KV = 2 * 128 * DH * 2 + 4 * 128 * 64 * 2 + 3 * 2 * 64 * DH * 2 + EXTRA;
   static bool ok = set_smem(attn_dq_tc_kernel<DH>, SM_DQ) && set_smem(attn_dkv_tc_kernel<DH>, SM_KV);
@@ -649,6 +654,7 @@ int bwd_t(const bf16* qkv, const float* lse, const bf16* dU, bf16* dqkv, const f
       !encode3d(&mQ64, qkv, 3 * d, S, B, 3 * (int64_t)d, 64) || !encode3d(&mG64, dU, d, S, B, d, 64))
     return -3;
   AttnParams p{}; p.lse = lse; p.delta = delta; p.dqkv = dqkv; p.S = S; p.h = h; p.flags = flags;
+  p.inv_rope = inv_rope;
   dim3 grid((S + 127) / 128, h, B);
   attn_dq_tc_kernel<DH><<<grid, ATT_THREADS, SM_DQ, st>>>(mQKV, mG, mQ64, p);
   attn_dkv_tc_kernel<DH><<<grid, ATT_THREADS, SM_KV, st>>>(mQKV, mQ64, mG64, p);
@@ -668,10 +674,11 @@ int launch_attn_fwd_tc(const bf16* qkv, bf16* U, float* lse, int B, int S, int h
 }
 
 int launch_attn_bwd_tc(const bf16* qkv, const bf16* U, const float* lse, const bf16* dU, bf16* dqkv,
-                       float* scratch, int B, int S, int h, int dh, int* flags, cudaStream_t st) {
+                       float* scratch, int B, int S, int h, int dh, int* flags, cudaStream_t st,
+                       const float2* inv_rope_cs) {
   if (gemm_tc_init() != 0) return -1;
   launch_attn_delta(U, dU, scratch, B, S, h, dh, st);
-  if (dh == 64) return bwd_t<64>(qkv, lse, dU, dqkv, scratch, B, S, h, flags, st);
-  if (dh == 128) return bwd_t<128>(qkv, lse, dU, dqkv, scratch, B, S, h, flags, st);
+  if (dh == 64) return bwd_t<64>(qkv, lse, dU, dqkv, scratch, B, S, h, flags, st, inv_rope_cs);
+  if (dh == 128) return bwd_t<128>(qkv, lse, dU, dqkv, scratch, B, S, h, flags, st, inv_rope_cs);
   return -1;
 }

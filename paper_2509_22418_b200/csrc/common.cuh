@@ -15,7 +15,8 @@ enum GemmEpilogue {
   EPI_STORE_F32 = 1,   // C fp32
   EPI_GELU_DUAL = 2,   // C bf16 = acc (pre-activation), C2 bf16 = gelu(acc)
   EPI_RESID_F32 = 3,   // C fp32 = aux fp32 + acc (residual stream)
-  EPI_DGELU = 4        // C bf16 = acc * gelu'(aux bf16)
+  EPI_DGELU = 4,       // C bf16 = acc * gelu'(aux bf16)
+  EPI_ROPE_BF16 = 5    // C bf16 = acc with rotary positions applied to the columns < rope_cols
 };
 
 struct GemmArgs {
@@ -30,6 +31,8 @@ struct GemmArgs {
   // split-K: the reduction is cut into `splits` ranges; range s writes its partial product to
   // C + s * split_stride (elements).  The consumer adds the partials in index order.
   int splits = 1; int64_t split_stride = 0;
+  // EPI_ROPE_BF16: aux is the (cos, sin) table [rope_S][rope_dh / 2]; row m is position m % rope_S
+  int rope_S = 0, rope_dh = 0, rope_cols = 0;
 };
 
 int launch_gemm_simt(const GemmArgs& g, cudaStream_t st);
@@ -51,7 +54,8 @@ bool attn_tc_supported(int S, int dh);
 int launch_attn_fwd_tc(const bf16* qkv, bf16* U, float* lse, int B, int S, int h, int dh, int* flags,
                        cudaStream_t st);
 int launch_attn_bwd_tc(const bf16* qkv, const bf16* U, const float* lse, const bf16* dU, bf16* dqkv,
-                       float* scratch, int B, int S, int h, int dh, int* flags, cudaStream_t st);
+                       float* scratch, int B, int S, int h, int dh, int* flags, cudaStream_t st,
+                       const float2* inv_rope_cs = nullptr);   // non-null: rotate dq, dk back by -angle
 // delta[b,h,s] = sum_e dU * U of the head's slice
 void launch_attn_delta(const bf16* U, const bf16* dU, float* delta, int B, int S, int h, int dh,
                        cudaStream_t st);

@@ -67,6 +67,18 @@ __device__ __forceinline__ uint32_t pack2_bf16(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// rotary positions on `pairs` adjacent pairs of f starting at column n0 of a [.., heads x dh] row
+__device__ __forceinline__ void rope_pairs(float* f, int pairs, const float2* cs_row, int n0, int dh) {
+#pragma unroll
+  for (int q = 0; q < 16; ++q) {
+    if (q >= pairs) break;
+    const float2 w = __ldg(cs_row + ((n0 + 2 * q) % dh) / 2);
+    const float a = f[2 * q], b = f[2 * q + 1];
+    f[2 * q] = a * w.x - b * w.y;
+    f[2 * q + 1] = a * w.y + b * w.x;
+  }
+}
+
 struct TcParams {
   int M, N, K;
   int epilogue;
@@ -77,6 +89,7 @@ struct TcParams {
   int tiles_m, tiles_n;
   int splits; long long split_stride;
   int wide;   // every output / auxiliary row start is 32-byte aligned: use 32-byte accesses
+  int rope_S, rope_dh, rope_cols;
 };
 
 template <int BN> struct Cfg {
@@ -263,6 +276,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
           } else {
             tmem_ld_wait();
             if (row_ok) {
+              if (p.epilogue == EPI_ROPE_BF16 && nb < p.rope_cols)
+                rope_pairs(reinterpret_cast<float*>(r), 16,
+                           (const float2*)p.aux + (long long)(m % p.rope_S) * (p.rope_dh / 2), nb, p.rope_dh);
               uint32_t o[16];
 #pragma unroll
               for (int j = 0; j < 16; ++j) o[j] = pack2_bf16(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
@@ -326,6 +342,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
               float f[8];
 #pragma unroll
               for (int q = 0; q < 8; ++q) f[q] = __uint_as_float(r[8 * j + q]);
+              if (p.epilogue == EPI_ROPE_BF16 && nb + 8 * j < p.rope_cols)
+                rope_pairs(f, 4, (const float2*)p.aux + (long long)(m % p.rope_S) * (p.rope_dh / 2), nb + 8 * j,
+                           p.rope_dh);
               if (p.epilogue == EPI_STORE_F32) {
                 float4* o = reinterpret_cast<float4*>((float*)p.C + ci + 8 * j);
                 o[0] = make_float4(f[0], f[1], f[2], f[3]);
@@ -403,6 +422,7 @@ int launch_t(const GemmArgs& g, cudaStream_t st) {
   const int k_blocks = (g.K + BK - 1) / BK;
   p.splits = g.splits < 1 ? 1 : (g.splits > k_blocks ? k_blocks : g.splits);
   p.split_stride = g.split_stride;
+  p.rope_S = g.rope_S > 0 ? g.rope_S : 1; p.rope_dh = g.rope_dh > 0 ? g.rope_dh : 2; p.rope_cols = g.rope_cols;
   {
     const bool f32 = g.epilogue == EPI_STORE_F32 || g.epilogue == EPI_RESID_F32;
     const long long out_unit = f32 ? 8 : 16;   // elements per 32 bytes

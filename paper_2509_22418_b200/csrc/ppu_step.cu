@@ -81,12 +81,13 @@ struct Sched {
 
   void gemm(const bf16* A, int64_t lda, int ak, const bf16* Bm, int64_t ldb, int bk, int M, int N,
             int K, int epi, void* C, int64_t ldc, void* C2, const void* aux, int64_t ldaux,
-            double* flop_counter, int splits = 1, int64_t split_stride = 0) {
+            double* flop_counter, int splits = 1, int64_t split_stride = 0, int rope_cols = 0) {
     if (rc || M <= 0 || N <= 0) return;
     GemmArgs g;
     g.A = A; g.lda = lda; g.a_kmajor = ak; g.B = Bm; g.ldb = ldb; g.b_kmajor = bk;
     g.M = M; g.N = N; g.K = K; g.epilogue = epi; g.C = C; g.ldc = ldc; g.C2 = C2; g.aux = aux;
     g.ldaux = ldaux; g.flags = c->flags; g.splits = splits; g.split_stride = split_stride;
+    g.rope_S = S; g.rope_dh = dh; g.rope_cols = rope_cols;
     EvScope ev(c, 0, 2.0 * M * N * (double)K);
     rc = c->gemm_backend == 1 ? launch_gemm_simt(g, c->stream) : launch_gemm_tc(g, c->stream);
     c->launches++;
@@ -111,9 +112,14 @@ struct Sched {
       float* x_next = (l + 1 < L) ? c->acts[l + 1].x : c->x_last;
       launch_ln_fwd(a.x, Pf(l, c->rel_ln1g), Pf(l, c->rel_ln1b), c->a16, a.st1, T, d, c->cfg.ln_eps, st);
       c->launches++;
-      gemm(c->a16, d, 1, W(l, c->rel_wq), d, 1, T, 3 * d, d, EPI_STORE_BF16, a.qkv, 3 * d, nullptr,
-           nullptr, 0, &c->flops_fwd);
-      launch_rope(a.qkv, c->rope_cs, B, S, h, dh, 0, st); c->launches++;
+      if (c->gemm_backend == 0) {   // rotary positions applied in the projection's epilogue
+        gemm(c->a16, d, 1, W(l, c->rel_wq), d, 1, T, 3 * d, d, EPI_ROPE_BF16, a.qkv, 3 * d, nullptr,
+             c->rope_cs, 0, &c->flops_fwd, 1, 0, 2 * d);
+      } else {
+        gemm(c->a16, d, 1, W(l, c->rel_wq), d, 1, T, 3 * d, d, EPI_STORE_BF16, a.qkv, 3 * d, nullptr,
+             nullptr, 0, &c->flops_fwd);
+        launch_rope(a.qkv, c->rope_cs, B, S, h, dh, 0, st); c->launches++;
+      }
       {
         const double fl = 4.0 * B * h * dh * 0.5 * S * (double)(S + 1);
         EvScope ev(c, 1, fl);
@@ -191,7 +197,8 @@ struct Sched {
         EvScope ev(c, 1, fl);
         const int kind = attn_kind();
         if (kind == 0)
-          rc |= launch_attn_bwd_tc(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, c->flags, st);
+          rc |= launch_attn_bwd_tc(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, c->flags, st,
+                                   c->rope_cs);   // dq, dk leave the kernel already rotated back
         else if (kind == 2)
           rc |= launch_attn_bwd_mma(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, st);
         else
@@ -199,7 +206,7 @@ struct Sched {
         c->launches += kind == 1 ? 2 : 3;
         c->flops_dgrad += fl;
       }
-      launch_rope(c->dqkv, c->rope_cs, B, S, h, dh, 1, st); c->launches++;
+      if (attn_kind() != 0) { launch_rope(c->dqkv, c->rope_cs, B, S, h, dh, 1, st); c->launches++; }
       gemm(c->dqkv, 3 * d, 1, W(l, c->rel_wq), d, 0, T, d, 3 * d, EPI_STORE_BF16, c->t16, d, nullptr,
            nullptr, 0, &c->flops_dgrad);
       launch_ln_bwd(c->t16, a.x, a.st1, Pf(l, c->rel_ln1g), c->g, c->g, c->g16, T, d, st);
