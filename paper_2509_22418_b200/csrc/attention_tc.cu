@@ -22,6 +22,7 @@ namespace {
 using namespace tc;
 
 constexpr int ATT_THREADS = 192;
+constexpr int BWD_THREADS = 320;  // warp 0 TMA, warp 1 MMA, warps 2-5 and 6-9: two row groups, half the slab columns each
 constexpr float LOG2E = 1.4426950408889634f;
 
 __device__ __forceinline__ float ex2(float x) {
@@ -121,6 +122,14 @@ __device__ __forceinline__ uint8_t* align1k(uint8_t* p) {
 }
 
 // ------------------------------------------------------------------ forward
+// One CTA per 128 queries, 128-key blocks.  S = Q K^T of block j+1 is issued into the second TMEM
+// buffer while the 128 row threads (one query row each) turn block j into bf16 probabilities in
+// one of two shared-memory tiles; O += P V accumulates in TMEM.  The softmax reference maximum is
+// only raised when a row's block maximum exceeds it by more than 2^8 (the stored probabilities
+// then stay below 256); raising it rescales the row of O in TMEM.  Sums, O and the final
+// normalisation all use the same reference, so the result is the exact softmax.
+constexpr float RESCALE_LOG2 = 8.f;
+
 template <int DH>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams p) {
@@ -128,9 +137,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align1k(smem_raw);
   const uint32_t Qs = smem_u32(smem), Ks = Qs + QT, Vs = Ks + 2 * QT, Ps = Vs + 2 * QT;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 5 * QT + PT);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 5 * QT + 2 * PT);
   enum { Q_FULL = 0, K_FULL = 1, K_EMPTY = 3, V_FULL = 5, V_EMPTY = 7, S_FULL = 9, S_EMPTY = 11,
-         P_FULL = 13, P_EMPTY = 14, O_FULL = 15, O_EMPTY = 16, NBAR = 17 };
+         P_FULL = 13, P_EMPTY = 15, PV_DONE = 17, NBAR = 18 };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar0 = smem_u32(bars);
@@ -142,8 +151,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
-    mbar_init(B(S_EMPTY), 4); mbar_init(B(S_EMPTY + 1), 4);
-    mbar_init(B(P_FULL), 4); mbar_init(B(O_EMPTY), 4);
+    for (int i = 0; i < 2; ++i) { mbar_init(B(S_EMPTY + i), 4); mbar_init(B(P_FULL + i), 4); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -176,15 +184,17 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
       constexpr uint32_t idesc_o = make_idesc(128, DH, false, true);
+      const uint32_t q_lo = klo(Qs);
       bool ok = mbar_wait(B(Q_FULL), 0, abort_flag, p.flags);
       auto issue_s = [&](int j) -> bool {
         const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
         if (!mbar_wait(B(K_FULL + st), ph, abort_flag, p.flags)) return false;
         if (!mbar_wait(B(S_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) return false;
         tc_fence_after();
+        const uint32_t k_lo = klo(Ks + st * QT);
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks)
-          umma_lo(tS + st * 128, klo(Qs) + kstep<128>(ks), klo(Ks + st * QT) + kstep<128>(ks), idesc_s, ks > 0);
+          umma_lo(tS + st * 128, q_lo + kstep<128>(ks), k_lo + kstep<128>(ks), idesc_s, ks > 0);
         umma_commit(B(S_FULL + st));
         umma_commit(B(K_EMPTY + st));
         return true;
@@ -193,15 +203,15 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
       for (int j = 0; j < n && ok; ++j) {
         if (j + 1 < n) { ok = issue_s(j + 1); if (!ok) break; }
         const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
-        if (!mbar_wait(B(P_FULL), j & 1, abort_flag, p.flags)) break;
+        if (!mbar_wait(B(P_FULL + st), ph, abort_flag, p.flags)) break;
         if (!mbar_wait(B(V_FULL + st), ph, abort_flag, p.flags)) break;
-        if (!mbar_wait(B(O_EMPTY), (j & 1) ^ 1u, abort_flag, p.flags)) break;
         tc_fence_after();
+        const uint32_t p_lo = klo(Ps + st * PT), v_lo = mlo<128>(Vs + st * QT);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
-          umma_lo(tO, klo(Ps) + kstep<128>(ks), mlo<128>(Vs + st * QT) + mstep(ks), idesc_o, ks > 0);
-        umma_commit(B(O_FULL));
-        umma_commit(B(P_EMPTY));
+          umma_lo(tO, p_lo + kstep<128>(ks), v_lo + mstep(ks), idesc_o, (j > 0 || ks > 0));
+        umma_commit(B(PV_DONE));
+        umma_commit(B(P_EMPTY + st));
         umma_commit(B(V_EMPTY + st));
       }
     }
@@ -211,82 +221,101 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
     const int grow = qb * 128 + row;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     const float c = rsqrtf((float)DH) * LOG2E;
-    float o[DH];
-#pragma unroll
-    for (int e = 0; e < DH; ++e) o[e] = 0.f;
-    float m = -INFINITY, l = 0.f;
+    float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     for (int j = 0; j < n && ok; ++j) {
       const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
       if (!mbar_wait(B(S_FULL + st), ph, abort_flag, p.flags)) { ok = false; break; }
       tc_fence_after();
+      uint32_t r[128];
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) tmem_ld32(tS + lane_off + st * 128 + cc * 32, r + 32 * cc);
+      tmem_ld_wait();
+      tc_fence_before();
+      warp_arrive(B(S_EMPTY + st));               // the scores are in registers: free the buffer
       const bool diag = (j == qb) || ((j + 1) * 128 > S);
-      float mx = -INFINITY;
-#pragma unroll 1
-      for (int cc = 0; cc < 4; ++cc) {
-        uint32_t r[32];
-        tmem_ld32(tS + lane_off + st * 128 + cc * 32, r);
-        tmem_ld_wait();
+      // eight independent partial maxima / sums: a single warp per scheduler cannot hide the
+      // latency of one 128-long dependent chain
+      float mx8[8];
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const int col = j * 128 + cc * 32 + e;
-          const float v = __uint_as_float(r[e]);
-          if (!diag || (col <= grow && col < S)) mx = fmaxf(mx, v);
+      for (int q = 0; q < 8; ++q) mx8[q] = -INFINITY;
+      if (!diag) {
+#pragma unroll
+        for (int e = 0; e < 128; ++e) mx8[e & 7] = fmaxf(mx8[e & 7], __uint_as_float(r[e]));
+      } else {
+#pragma unroll
+        for (int e = 0; e < 128; ++e) {
+          const int col = j * 128 + e;
+          if (col <= grow && col < S) mx8[e & 7] = fmaxf(mx8[e & 7], __uint_as_float(r[e]));
         }
       }
-      const float m_new = fmaxf(m, mx * c);
-      const float corr = ex2(m - m_new);
-      float sum = 0.f;
+      const float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
+                             fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
+      const float m_blk = mx * c;
+      const bool need = m_blk > m_ref + RESCALE_LOG2;
+      if (__any_sync(0xffffffffu, need)) {
+        const float new_ref = need ? m_blk : m_ref;
+        const float factor = need ? ex2(m_ref - new_ref) : 1.f;
+        if (j > 0) {
+          // O must be complete up to block j-1 before its rows are rescaled in place
+          if (!mbar_wait(B(PV_DONE), (j - 1) & 1, abort_flag, p.flags)) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll 1
+          for (int cc = 0; cc < DH / 32; ++cc) {
+            uint32_t o[32];
+            tmem_ld32(tO + lane_off + cc * 32, o);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
+            tmem_st32(tO + lane_off + cc * 32, o);
+          }
+          tmem_st_wait();
+        }
+        l *= factor;
+        m_ref = new_ref;
+      }
+      float sum8[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) sum8[q] = 0.f;
+      if (!mbar_wait(B(P_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+#pragma unroll
       for (int cc = 0; cc < 4; ++cc) {
-        uint32_t r[32];
-        tmem_ld32(tS + lane_off + st * 128 + cc * 32, r);
-        tmem_ld_wait();
         float pv[32];
+        if (!diag) {
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const int col = j * 128 + cc * 32 + e;
-          float pe = ex2(__uint_as_float(r[e]) * c - m_new);
-          if (diag && (col > grow || col >= S)) pe = 0.f;
-          pv[e] = pe;
-          sum += pe;
+          for (int e = 0; e < 32; ++e) {
+            pv[e] = ex2(fmaf(__uint_as_float(r[cc * 32 + e]), c, -m_ref));
+            sum8[e & 7] += pv[e];
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            const int col = j * 128 + cc * 32 + e;
+            float pe = ex2(fmaf(__uint_as_float(r[cc * 32 + e]), c, -m_ref));
+            if (col > grow || col >= S) pe = 0.f;
+            pv[e] = pe;
+            sum8[e & 7] += pe;
+          }
         }
-        if (cc == 0 && !mbar_wait(B(P_EMPTY), (j & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
-        store_row32(Ps, 16384, row, cc * 4, pv);
+        store_row32(Ps + st * PT, 16384, row, cc * 4, pv);
       }
-      if (!ok) break;
+      l += ((sum8[0] + sum8[1]) + (sum8[2] + sum8[3])) + ((sum8[4] + sum8[5]) + (sum8[6] + sum8[7]));
       tc_fence_before();
       fence_async_smem();
-      warp_arrive(B(P_FULL));
-      warp_arrive(B(S_EMPTY + st));
-      l = l * corr + sum;
-      m = m_new;
-#pragma unroll
-      for (int e = 0; e < DH; ++e) o[e] *= corr;
-      if (!mbar_wait(B(O_FULL), j & 1, abort_flag, p.flags)) { ok = false; break; }
-      tc_fence_after();
-#pragma unroll
-      for (int cc = 0; cc < DH / 32; ++cc) {
-        uint32_t r[32];
-        tmem_ld32(tO + lane_off + cc * 32, r);
-        tmem_ld_wait();
-#pragma unroll
-        for (int e = 0; e < 32; ++e) o[cc * 32 + e] += __uint_as_float(r[e]);
-      }
-      tc_fence_before();
-      warp_arrive(B(O_EMPTY));
+      warp_arrive(B(P_FULL + st));
     }
-    if (ok && grow < S) {
+    if (ok && mbar_wait(B(PV_DONE), (n - 1) & 1, abort_flag, p.flags)) {
+      tc_fence_after();
       const float inv = 1.f / l;
       bf16* out = p.U + ((int64_t)b * S + grow) * d + head * DH;
-#pragma unroll
-      for (int e = 0; e < DH; e += 8) {
-        uint4 u;
-        u.x = pack2(o[e] * inv, o[e + 1] * inv); u.y = pack2(o[e + 2] * inv, o[e + 3] * inv);
-        u.z = pack2(o[e + 4] * inv, o[e + 5] * inv); u.w = pack2(o[e + 6] * inv, o[e + 7] * inv);
-        *reinterpret_cast<uint4*>(out + e) = u;
+#pragma unroll 1
+      for (int cc = 0; cc < DH / 32; ++cc) {
+        uint32_t o[32];
+        tmem_ld32(tO + lane_off + cc * 32, o);
+        tmem_ld_wait();
+        if (grow < S) drain32(out + cc * 32, o, inv, nullptr, 0);
       }
-      p.lse_out[((int64_t)b * p.h + head) * S + grow] = (m + log2f(l)) * (1.f / LOG2E);
+      if (grow < S) p.lse_out[((int64_t)b * p.h + head) * S + grow] = (m_ref + log2f(l)) * (1.f / LOG2E);
     }
   }
   if (*abort_flag) for (int i = 0; i < 64; ++i) __nanosleep(2000);
@@ -301,7 +330,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
 // pair of TMEM buffers while the 128 row threads turn slab i into dS = P (dP - delta);
 // dQ += dS K accumulates in TMEM over all slabs.
 template <int DH>
-__global__ void __launch_bounds__(ATT_THREADS, 1)
+__global__ void __launch_bounds__(BWD_THREADS, 1)
 attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapG,
                   const __grid_constant__ CUtensorMap mapKV64, const AttnParams p) {
   constexpr int NH = DH / 64, QT = 128 * DH * 2, HT = 64 * DH * 2, PT = 128 * 64 * 2, NS = 4;
@@ -322,7 +351,7 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
-    mbar_init(B(SDP_EMPTY), 4); mbar_init(B(SDP_EMPTY + 1), 4); mbar_init(B(DS_FULL), 4); mbar_init(B(DS_FULL + 1), 4);
+    mbar_init(B(SDP_EMPTY), 8); mbar_init(B(SDP_EMPTY + 1), 8); mbar_init(B(DS_FULL), 8); mbar_init(B(DS_FULL + 1), 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -393,6 +422,7 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
       }
     }
   } else {
+    const int grp = (warp - 2) >> 2;               // column half of every slab this thread handles
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const int grow = qb * 128 + row;
@@ -406,24 +436,23 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
       const uint32_t tS = tmem + 128 * bf + lane_off, tP = tS + 64;
       if (!mbar_wait(B(SDP_FULL + bf), (it >> 1) & 1, abort_flag, p.flags)) { ok = false; break; }
       tc_fence_after();
-      uint32_t rs[64], rd[64];
-      tmem_ld32(tS, rs); tmem_ld32(tS + 32, rs + 32);
-      tmem_ld32(tP, rd); tmem_ld32(tP + 32, rd + 32);
+      uint32_t rs[32], rd[32];
+      tmem_ld32(tS + 32 * grp, rs);
+      tmem_ld32(tP + 32 * grp, rd);
       tmem_ld_wait();
       tc_fence_before();
       warp_arrive(B(SDP_EMPTY + bf));          // the accumulators are in registers: free them early
       const bool diag = ((it + 1) * 64 > qb * 128) || ((it + 1) * 64 > S);
-      float ds[64];
+      float ds[32];
 #pragma unroll
-      for (int e = 0; e < 64; ++e) {
-        const int col = it * 64 + e;
+      for (int e = 0; e < 32; ++e) {
+        const int col = it * 64 + 32 * grp + e;
         float pe = ex2(__uint_as_float(rs[e]) * c - l2);
         if (diag && (col > grow || col >= S)) pe = 0.f;
         ds[e] = pe * (__uint_as_float(rd[e]) - dl);
       }
       if (!mbar_wait(B(DS_EMPTY + bf), ((it >> 1) & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
-      store_row32(Ds + bf * PT, 0, row, 0, ds);
-      store_row32(Ds + bf * PT, 0, row, 4, ds + 32);
+      store_row32(Ds + bf * PT, 0, row, 4 * grp, ds);
       fence_async_smem();
       warp_arrive(B(DS_FULL + bf));
     }
@@ -431,7 +460,7 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
       tc_fence_after();
       bf16* out = p.dqkv + ((int64_t)b * S + grow) * (3 * d) + head * DH;
 #pragma unroll 1
-      for (int cc = 0; cc < DH / 32; ++cc) {
+      for (int cc = grp; cc < DH / 32; cc += 2) {       // the two groups drain alternate column chunks
         uint32_t r[32];
         tmem_ld32(tQ + lane_off + cc * 32, r);
         tmem_ld_wait();
@@ -452,7 +481,7 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
 // issued into a second pair of TMEM buffers while the 128 row threads (one key each) form
 // P^T and dS^T of slab i; dV += P^T dU and dK += dS^T Q accumulate in TMEM.
 template <int DH>
-__global__ void __launch_bounds__(ATT_THREADS, 1)
+__global__ void __launch_bounds__(BWD_THREADS, 1)
 attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_constant__ CUtensorMap mapQ64,
                    const __grid_constant__ CUtensorMap mapG64, const AttnParams p) {
   constexpr int NH = DH / 64, QT = 128 * DH * 2, HT = 64 * DH * 2, PT = 128 * 64 * 2, NS = 3;
@@ -473,7 +502,7 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_const
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
-    mbar_init(B(SDP_EMPTY), 4); mbar_init(B(SDP_EMPTY + 1), 4); mbar_init(B(PDS_FULL), 4); mbar_init(B(PDS_FULL + 1), 4);
+    mbar_init(B(SDP_EMPTY), 8); mbar_init(B(SDP_EMPTY + 1), 8); mbar_init(B(PDS_FULL), 8); mbar_init(B(PDS_FULL + 1), 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -548,6 +577,7 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_const
       }
     }
   } else {
+    const int grp = (warp - 2) >> 2;               // column half of every slab this thread handles
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const int key = kb * 128 + row;
@@ -563,8 +593,8 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_const
       if (!mbar_wait(B(SDP_FULL + bf), (it >> 1) & 1, abort_flag, p.flags)) { ok = false; break; }
       tc_fence_after();
       if (!mbar_wait(B(PDS_EMPTY + bf), ((it >> 1) & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
-#pragma unroll 1
-      for (int cc = 0; cc < 2; ++cc) {
+      {
+        const int cc = grp;
         uint32_t rs[32], rd[32];
         tmem_ld32(tS + cc * 32, rs);
         tmem_ld32(tP + cc * 32, rd);
@@ -591,7 +621,7 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_const
       tc_fence_after();
       bf16* out = p.dqkv + ((int64_t)b * S + key) * (3 * d) + head * DH;
 #pragma unroll 1
-      for (int cc = 0; cc < 2 * DH / 32; ++cc) {
+      for (int cc = grp; cc < 2 * DH / 32; cc += 2) {
         const bool is_k = cc >= DH / 32;
         const int c0 = (is_k ? cc - DH / 32 : cc) * 32;
         uint32_t r[32];
@@ -630,7 +660,7 @@ constexpr int EXTRA = 1024 + 256;   // alignment slack + barriers
 
 template <int DH>
 int fwd_t(const bf16* qkv, bf16* U, float* lse, int B, int S, int h, int* flags, cudaStream_t st) {
-  constexpr int SM = 5 * 128 * DH * 2 + 128 * 128 * 2 + EXTRA;
+  constexpr int SM = 5 * 128 * DH * 2 + 2 * 128 * 128 * 2 + EXTRA;
   static bool ok = set_smem(attn_fwd_tc_kernel<DH>, SM);
   if (!ok) return -2;
   CUtensorMap m;
@@ -656,8 +686,8 @@ int bwd_t(const bf16* qkv, const float* lse, const bf16* dU, bf16* dqkv, const f
   AttnParams p{}; p.lse = lse; p.delta = delta; p.dqkv = dqkv; p.S = S; p.h = h; p.flags = flags;
   p.inv_rope = inv_rope;
   dim3 grid((S + 127) / 128, h, B);
-  attn_dq_tc_kernel<DH><<<grid, ATT_THREADS, SM_DQ, st>>>(mQKV, mG, mQ64, p);
-  attn_dkv_tc_kernel<DH><<<grid, ATT_THREADS, SM_KV, st>>>(mQKV, mQ64, mG64, p);
+  attn_dq_tc_kernel<DH><<<grid, BWD_THREADS, SM_DQ, st>>>(mQKV, mG, mQ64, p);
+  attn_dkv_tc_kernel<DH><<<grid, BWD_THREADS, SM_KV, st>>>(mQKV, mQ64, mG64, p);
   return 0;
 }
 
