@@ -91,6 +91,14 @@ class ClockSampler(threading.Thread):
                     reasons=sorted(reasons), samples=len(sm))
 
 
+def workload_config(name, w):
+    L, d, h, F, V = w["dims"]
+    return dict(workload=f"{name}: {w['desc']}", layers=L, d_model=d, heads=h, d_ff=F, vocab=V,
+                batch=w["batch"], seq=w["seq"], replicas=w["K"], slices=w["N"],
+                l2="working set per step (bf16 weights + activations) is far larger than L2; "
+                   "fresh token batch every step")
+
+
 def oracle_sample(w, steps, rank0_print=True):
     """The CPU oracle on a bounded sample of the workload: one replica, a short batch."""
     from oracle import ppu_oracle as O
@@ -99,7 +107,7 @@ def oracle_sample(w, steps, rank0_print=True):
     cfg = O.Model(L, d, h, F, V)
     big = O.n_params(cfg) > 5e7
     dtype = np.float32 if big else np.float64
-    B, S = (1, 256) if O.n_params(cfg) > 5e8 else ((1, 512) if big else (w["batch"], w["seq"]))
+    B, S = (1, 1024) if O.n_params(cfg) > 5e8 else ((2, 1024) if big else (w["batch"], w["seq"]))
     theta = synth.init_params(SEED, O.layout(cfg)).astype(dtype)
     rep = O.Replica(cfg, theta, O.slice_ranges(cfg, w["N"], 0))
     hp = O.AdamW(**{k: ADAM[k] for k in ("lr", "beta1", "beta2", "eps", "wd")})
@@ -128,7 +136,7 @@ def run_reference(args, w):
     out = dict(metric="local-step tokens/s", value=cb["value"], unit="tokens/s", n_gpus=args.gpus,
                steps=args.steps, warmup=args.warmup, ms_per_step=t * 1e3, higher_is_better=True,
                scaling="weak", vs_baseline=None, dtype=cb["sample"].split(", ")[1], data="synthetic",
-               impl="reference", config=dict(workload=f"{args.workload}: {w['desc']}"),
+               impl="reference", config=workload_config(args.workload, w),
                cpu_baseline=cb,
                e2e=dict(value=cb["value"], unit="tokens/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0))
     print(json.dumps(out))
@@ -188,8 +196,53 @@ def run_sweep(args):
                           steps=args.steps, warmup=args.warmup, data="synthetic", rows=rows)))
 
 
+def run_round(args):
+    """One full outer round at the 1.3B shapes: 8 replicas (1/8 FFN slices) x 50 inner steps each,
+    then the pseudo-gradient average and the outer Nesterov step.  Prints one JSON line."""
+    import torch
+    from paper_2509_22418_b200 import build, ppu, synth
+    build.build()
+    w = WORKLOADS["c3"]
+    L, d, h, F, V = w["dims"]
+    B, S, K, H = w["batch"], w["seq"], 8, args.inner_steps
+    cfg = ppu.make_cfg(L, d, h, F, V, B, S, adam_lr=ADAM["lr"], adam_beta1=ADAM["beta1"],
+                       adam_beta2=ADAM["beta2"], adam_eps=ADAM["eps"], adam_wd=ADAM["wd"],
+                       outer_lr=OUTER["lr"], outer_momentum=OUTER["momentum"])
+    spec, keep = ppu.make_spec(K, ppu.SUBSET_FFN_SLICE, n_slices=K)
+    ctx = ppu.Context(cfg, spec, keep)
+    ctx.ppu_set_params(synth.init_params(SEED, ctx.tensors()))
+    toks = {(k, hh): torch.from_numpy(synth.tokens(SEED, k, 0, hh, B, S, V)).cuda()
+            for k in range(K) for hh in range(H)}
+    for k in range(min(K, 3)):                       # warm-up outside the round
+        ctx.ppu_local_step(k, toks[(k, 0)])
+    ctx.ppu_outer_sync(list(range(K)))
+    ctx.ppu_sync()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    ev[0].record()
+    for k in range(K):
+        for hh in range(H):
+            ctx.ppu_local_step(k, toks[(k, hh)])
+    ev[1].record()
+    ctx.ppu_outer_sync(list(range(K)))
+    ev[2].record()
+    torch.cuda.synchronize()
+    losses = [ctx.ppu_loss(k) for k in range(K)]
+    st = ctx.ppu_stats()
+    steps_ms, outer_ms = ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2])
+    pk = peaks()
+    print(json.dumps(dict(
+        metric="full outer round, 1.3B", replicas=K, inner_steps=H, round_s=(steps_ms + outer_ms) * 1e-3,
+        tokens_per_s=K * H * B * S / ((steps_ms + outer_ms) * 1e-3), local_step_ms=steps_ms / (K * H),
+        outer_sync=dict(ms=outer_ms, algorithmic_bytes=st.outer_bytes,
+                        gbs=st.outer_bytes / (outer_ms * 1e-3) / 1e9, peak_gbs=pk["hbm"],
+                        frac=st.outer_bytes / (outer_ms * 1e-3) / 1e9 / pk["hbm"], of=pk["src"]),
+        last_losses=losses, data="synthetic", hbm_bytes=st.arena_bytes)))
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--round", action="store_true", help="one full outer round at the 1.3B shapes")
+    ap.add_argument("--inner-steps", type=int, default=50)
     ap.add_argument("--sweep", action="store_true", help="subset-fraction sweep at the 1.3B shapes")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
@@ -201,6 +254,8 @@ def main():
     w = WORKLOADS[args.workload]
     if args.sweep:
         return run_sweep(args)
+    if args.round:
+        return run_round(args)
     if args.impl == "reference":
         return run_reference(args, w)
 
@@ -281,10 +336,7 @@ def main():
         metric="local-step tokens/s", value=tokens / (total_ms * 1e-3), unit="tokens/s",
         n_gpus=world, steps=args.steps, warmup=args.warmup, ms_per_step=total_ms / args.steps,
         higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
-        config=dict(workload=f"{args.workload}: {w['desc']}", layers=L, d_model=d, heads=h, d_ff=F,
-                    vocab=V, batch=B, seq=S, replicas=K, slices=w["N"],
-                    l2="working set per step (bf16 weights + activations) is far larger than L2; "
-                       "fresh token batch every step"),
+        config=workload_config(args.workload, w),
         local_step_ms=steps_ms / args.steps,
         outer_sync=dict(ms=outer_ms, algorithmic_bytes=st.outer_bytes,
                         gbs=st.outer_bytes / (outer_ms * 1e-3) / 1e9, peak_gbs=pk["hbm"],

@@ -179,6 +179,15 @@ typedef struct {
 int ppu_profile_enable(ppu_ctx* ctx, int enable);
 int ppu_profile_read(ppu_ctx* ctx, ppu_profile_t* out);
 
+/* Failure-detection self-test.  Every wait inside the tcgen05 kernels is bounded: when a
+ * barrier is not signalled within the limit the kernel sets an error word, releases what it
+ * holds and returns, and the next synchronising call reports PPU_ETIMEOUT.  This call exercises
+ * that path without any fault: one CTA waits `limit` polls (1..65536) on a barrier nothing
+ * arrives at.  Returns PPU_ETIMEOUT when the kernel gave up as designed (the expected outcome),
+ * PPU_OK if the wait was somehow satisfied, PPU_ECUDA on a runtime error.  The context stays
+ * usable afterwards.  Synchronises the stream. */
+int ppu_wait_probe(int limit, void* cuda_stream);
+
 /* ---- single-operator entry points (kernel-level parity tests) -------------- */
 
 /* C[M,N] = A . B^T on bf16 operands with fp32 accumulation (the contraction of

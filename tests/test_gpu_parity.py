@@ -170,6 +170,22 @@ def test_whole_layer_subsets_and_eval_loss():
         P.close()
 
 
+def test_bounded_wait_reports_timeout_and_context_survives():
+    """A wait that nothing satisfies runs out, the kernel reports it and returns; afterwards the
+    library still computes (no fault, trap or hang is involved)."""
+    import ctypes
+    import torch
+    from paper_2509_22418_b200 import ppu
+    st = torch.cuda.current_stream().cuda_stream
+    rc = ppu.lib().ppu_wait_probe(2000, ctypes.c_void_p(st))
+    assert rc == -7 and b"expired" in ppu.lib().ppu_last_error()
+    assert ppu.lib().ppu_wait_probe(0, ctypes.c_void_p(st)) == -1
+    a = torch.ones((128, 64), device="cuda", dtype=torch.bfloat16)
+    c = ppu.ppu_gemm(a, 1, a, 1, 128, 128, 64, out_f32=True)
+    torch.cuda.synchronize()
+    assert torch.all(c == 64)
+
+
 def test_host_entry_point_and_argument_errors():
     from paper_2509_22418_b200 import ppu
     dims = (2, 64, 4, 256, 512)
