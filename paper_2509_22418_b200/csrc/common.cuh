@@ -31,6 +31,9 @@ struct GemmArgs {
   // split-K: the reduction is cut into `splits` ranges; range s writes its partial product to
   // C + s * split_stride (elements).  The consumer adds the partials in index order.
   int splits = 1; int64_t split_stride = 0;
+  // EPI_GELU_DUAL: columns [c3_lo, c3_hi) of gelu(acc) are also stored, packed, to C3[m, n - c3_lo]
+  // (the slice of the activation that a subset weight gradient will read); C3 may be null
+  void* C3 = nullptr; int64_t ldc3 = 0; int c3_lo = 0, c3_hi = 0;
   // EPI_ROPE_BF16: aux is the (cos, sin) table [rope_S][rope_dh / 2]; row m is position m % rope_S
   int rope_S = 0, rope_dh = 0, rope_cols = 0;
 };

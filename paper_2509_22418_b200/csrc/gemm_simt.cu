@@ -63,6 +63,8 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
         case EPI_GELU_DUAL:
           ((bf16*)g.C)[ci] = __float2bfloat16_rn(a);
           ((bf16*)g.C2)[ci] = __float2bfloat16_rn(gelu_f(a));
+          if (g.C3 && n >= g.c3_lo && n < g.c3_hi)
+            ((bf16*)g.C3)[(int64_t)m * g.ldc3 + (n - g.c3_lo)] = __float2bfloat16_rn(gelu_f(a));
           break;
         case EPI_RESID_F32:
           ((float*)g.C)[ci] = ((const float*)g.aux)[(int64_t)m * g.ldaux + n] + a;

@@ -90,6 +90,7 @@ struct TcParams {
   int splits; long long split_stride;
   int wide;   // every output / auxiliary row start is 32-byte aligned: use 32-byte accesses
   int rope_S, rope_dh, rope_cols;
+  void* C3; long long ldc3; int c3_lo, c3_hi;
 };
 
 template <int BN> struct Cfg {
@@ -276,9 +277,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
           } else {
             tmem_ld_wait();
             if (row_ok) {
-              if (p.epilogue == EPI_ROPE_BF16 && nb < p.rope_cols)
-                rope_pairs(reinterpret_cast<float*>(r), 16,
-                           (const float2*)p.aux + (long long)(m % p.rope_S) * (p.rope_dh / 2), nb, p.rope_dh);
+              if (p.epilogue == EPI_ROPE_BF16 && nb < p.rope_cols) {
+                const float2* cs_row = (const float2*)p.aux + (long long)(m % p.rope_S) * (p.rope_dh / 2);
+                if (p.rope_dh % 32 == 0) {
+                  // the chunk lies inside one head: its 16 (cos, sin) pairs are 128 contiguous bytes
+                  uint32_t w[32];
+                  const float2* src = cs_row + (nb % p.rope_dh) / 2;
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) ld_v8(w + 8 * j, src + 4 * j);
+#pragma unroll
+                  for (int q = 0; q < 16; ++q) {
+                    const float cw = __uint_as_float(w[2 * q]), sw = __uint_as_float(w[2 * q + 1]);
+                    const float a = __uint_as_float(r[2 * q]), b = __uint_as_float(r[2 * q + 1]);
+                    r[2 * q] = __float_as_uint(a * cw - b * sw);
+                    r[2 * q + 1] = __float_as_uint(a * sw + b * cw);
+                  }
+                } else {
+                  rope_pairs(reinterpret_cast<float*>(r), 16, cs_row, nb, p.rope_dh);
+                }
+              }
               uint32_t o[16];
 #pragma unroll
               for (int j = 0; j < 16; ++j) o[j] = pack2_bf16(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
@@ -290,6 +307,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
                   o[j] = pack2_bf16(gelu_dev(__uint_as_float(r[2 * j])), gelu_dev(__uint_as_float(r[2 * j + 1])));
                 st_v8((bf16*)p.C2 + ci, o);
                 st_v8((bf16*)p.C2 + ci + 16, o + 8);
+                if (p.C3 && nb < p.c3_hi && nb + 32 > p.c3_lo) {
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    const int col = nb + 8 * j;
+                    if (col >= p.c3_lo && col + 8 <= p.c3_hi)
+                      *reinterpret_cast<uint4*>((bf16*)p.C3 + (long long)m * p.ldc3 + (col - p.c3_lo)) =
+                          make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                  }
+                }
               }
             }
           }
@@ -354,7 +380,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
                 if (p.epilogue == EPI_GELU_DUAL) {
 #pragma unroll
                   for (int q = 0; q < 8; ++q) f[q] = gelu_dev(f[q]);
-                  *reinterpret_cast<uint4*>((bf16*)p.C2 + ci + 8 * j) = pack8_bf16(f);
+                  const uint4 gv = pack8_bf16(f);
+                  *reinterpret_cast<uint4*>((bf16*)p.C2 + ci + 8 * j) = gv;
+                  const int col = nb + 8 * j;
+                  if (p.C3 && col >= p.c3_lo && col + 8 <= p.c3_hi)
+                    *reinterpret_cast<uint4*>((bf16*)p.C3 + (long long)m * p.ldc3 + (col - p.c3_lo)) = gv;
                 }
               }
             }
@@ -422,6 +452,7 @@ int launch_t(const GemmArgs& g, cudaStream_t st) {
   const int k_blocks = (g.K + BK - 1) / BK;
   p.splits = g.splits < 1 ? 1 : (g.splits > k_blocks ? k_blocks : g.splits);
   p.split_stride = g.split_stride;
+  p.C3 = g.C3; p.ldc3 = g.ldc3; p.c3_lo = g.c3_lo; p.c3_hi = g.c3_hi;
   p.rope_S = g.rope_S > 0 ? g.rope_S : 1; p.rope_dh = g.rope_dh > 0 ? g.rope_dh : 2; p.rope_cols = g.rope_cols;
   {
     const bool f32 = g.epilogue == EPI_STORE_F32 || g.epilogue == EPI_RESID_F32;

@@ -5,6 +5,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <algorithm>
 #include "ppu_ctx.cuh"
 
 static thread_local char g_err[512] = "";
@@ -143,6 +144,9 @@ static void build_geometry(ppu_ctx* c) {
     }
     if (r2.n_sub > c->max_sub) c->max_sub = r2.n_sub;
   }
+  c->wmax.assign(L, 0);
+  for (auto& r2 : c->reps)
+    for (int l = 0; l < L; ++l) c->wmax[l] = std::max(c->wmax[l], (int)(r2.hi[l] - r2.lo[l]));
   // The subset products have few output tiles when slices are narrow: cut their reduction over
   // tokens so that about one wave of CTAs works on them.  One factor for the whole context.
   int64_t min_tiles = 1 << 30;
@@ -197,11 +201,12 @@ static size_t carve(ppu_ctx* c, uint8_t* base) {
     a.lse = (float*)take(T * h * 4);
     a.b = (bf16*)take(T * d * 2);
     a.Hd = (bf16*)take(T * F * 2);
-    a.A = (bf16*)take(T * F * 2);
+    a.As = (bf16*)take(T * (int64_t)c->wmax[l] * 2);
   }
   c->x_last = (float*)take(T * d * 4);
   c->stf = (float2*)take(T * 8);
   c->a16 = (bf16*)take(T * d * 2);
+  c->A_tmp = (bf16*)take(T * F * 2);
   c->f16 = (bf16*)take(T * d * 2);
   c->logits = (bf16*)take(T * V * 2);
   c->g = (float*)take(T * d * 4);

@@ -29,7 +29,7 @@ struct LayerActs {
   float* lse;      // [B,h,S]
   bf16* b;         // LayerNorm-2 output (input of W_in), [T,d]
   bf16* Hd;        // FFN pre-activation, [T,F]
-  bf16* A;         // gelu(Hd), [T,F]
+  bf16* As;        // gelu(Hd) restricted to the widest trained slice of this layer, packed [T,w]
 };
 
 struct ppu_ctx {
@@ -60,6 +60,8 @@ struct ppu_ctx {
   float* x_last = nullptr;      // input of the final LayerNorm
   float2* stf = nullptr;
   bf16 *a16 = nullptr, *f16 = nullptr, *logits = nullptr;
+  bf16* A_tmp = nullptr;        // gelu(Hd) of the layer in flight, [T,F] (only its trained slice is kept)
+  std::vector<int> wmax;        // per layer: widest trained range over the replicas
   float* g = nullptr;
   bf16 *g16 = nullptr, *dHd = nullptr, *t16 = nullptr, *dqkv = nullptr;
   float *attn_scratch = nullptr, *row_loss = nullptr, *loss = nullptr;

@@ -81,13 +81,15 @@ struct Sched {
 
   void gemm(const bf16* A, int64_t lda, int ak, const bf16* Bm, int64_t ldb, int bk, int M, int N,
             int K, int epi, void* C, int64_t ldc, void* C2, const void* aux, int64_t ldaux,
-            double* flop_counter, int splits = 1, int64_t split_stride = 0, int rope_cols = 0) {
+            double* flop_counter, int splits = 1, int64_t split_stride = 0, int rope_cols = 0,
+            void* C3 = nullptr, int64_t ldc3 = 0, int c3_lo = 0, int c3_hi = 0) {
     if (rc || M <= 0 || N <= 0) return;
     GemmArgs g;
     g.A = A; g.lda = lda; g.a_kmajor = ak; g.B = Bm; g.ldb = ldb; g.b_kmajor = bk;
     g.M = M; g.N = N; g.K = K; g.epilogue = epi; g.C = C; g.ldc = ldc; g.C2 = C2; g.aux = aux;
     g.ldaux = ldaux; g.flags = c->flags; g.splits = splits; g.split_stride = split_stride;
     g.rope_S = S; g.rope_dh = dh; g.rope_cols = rope_cols;
+    g.C3 = C3; g.ldc3 = ldc3; g.c3_lo = c3_lo; g.c3_hi = c3_hi;
     EvScope ev(c, 0, 2.0 * M * N * (double)K);
     rc = c->gemm_backend == 1 ? launch_gemm_simt(g, c->stream) : launch_gemm_tc(g, c->stream);
     c->launches++;
@@ -104,7 +106,7 @@ struct Sched {
 
   // Forward pass over all parameters (Appendix C.1 forward equations), saving what the
   // restricted backward needs.
-  void forward(const int32_t* tok) {
+  void forward(const int32_t* tok, const ReplicaState* rep = nullptr) {
     cudaStream_t st = c->stream;
     launch_embed(tok, c->w16, c->acts[0].x, T, d, V, c->flags, st); c->launches++;
     for (int l = 0; l < L && !rc; ++l) {
@@ -134,9 +136,11 @@ struct Sched {
            &c->flops_fwd);
       launch_ln_fwd(a.x1, Pf(l, c->rel_ln2g), Pf(l, c->rel_ln2b), a.b, a.st2, T, d, c->cfg.ln_eps, st);
       c->launches++;
-      gemm(a.b, d, 1, W(l, c->rel_win), d, 1, T, F, d, EPI_GELU_DUAL, a.Hd, F, a.A, nullptr, 0,
-           &c->flops_fwd);
-      gemm(a.A, F, 1, W(l, c->rel_wout), F, 1, T, d, F, EPI_RESID_F32, x_next, d, nullptr, a.x1, d,
+      // gelu(Hd) goes to a buffer shared by all layers; only the replica's own columns are kept
+      const int lo = rep ? rep->lo[l] : 0, hi = rep ? rep->hi[l] : 0;
+      gemm(a.b, d, 1, W(l, c->rel_win), d, 1, T, F, d, EPI_GELU_DUAL, a.Hd, F, c->A_tmp, nullptr, 0,
+           &c->flops_fwd, 1, 0, 0, hi > lo ? a.As : nullptr, hi - lo, lo, hi);
+      gemm(c->A_tmp, F, 1, W(l, c->rel_wout), F, 1, T, d, F, EPI_RESID_F32, x_next, d, nullptr, a.x1, d,
            &c->flops_fwd);
     }
     launch_ln_fwd(c->x_last, c->theta + c->off_lnfg, c->theta + c->off_lnfb, c->f16, c->stf, T, d,
@@ -180,7 +184,7 @@ struct Sched {
         // dW_in[lo:hi,:] = dHd[:,lo:hi]^T b      dW_out[:,lo:hi] = g^T A[:,lo:hi]
         gemm(c->dHd + s->lo, F, 0, a.b, d, 0, w, d, T, EPI_STORE_F32, c->grad + s->packed_off, d,
              nullptr, nullptr, 0, &c->flops_wgrad, partials(), c->max_sub);
-        gemm(c->g16, d, 0, a.A + s->lo, F, 0, d, w, T, EPI_STORE_F32,
+        gemm(c->g16, d, 0, a.As, w, 0, d, w, T, EPI_STORE_F32,
              c->grad + s->packed_off + (int64_t)w * d, w, nullptr, nullptr, 0, &c->flops_wgrad,
              partials(), c->max_sub);
         --seg;
@@ -197,8 +201,7 @@ struct Sched {
         EvScope ev(c, 1, fl);
         const int kind = attn_kind();
         if (kind == 0)
-          rc |= launch_attn_bwd_tc(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, c->flags, st,
-                                   c->rope_cs);   // dq, dk leave the kernel already rotated back
+          rc |= launch_attn_bwd_tc(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, c->flags, st);
         else if (kind == 2)
           rc |= launch_attn_bwd_mma(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, st);
         else
@@ -206,7 +209,9 @@ struct Sched {
         c->launches += kind == 1 ? 2 : 3;
         c->flops_dgrad += fl;
       }
-      if (attn_kind() != 0) { launch_rope(c->dqkv, c->rope_cs, B, S, h, dh, 1, st); c->launches++; }
+      // (the tcgen05 kernels can rotate dq, dk on the way out, but the table lookups sit on each
+      // CTA's critical path and cost more than this separate pass)
+      launch_rope(c->dqkv, c->rope_cs, B, S, h, dh, 1, st); c->launches++;
       gemm(c->dqkv, 3 * d, 1, W(l, c->rel_wq), d, 0, T, d, 3 * d, EPI_STORE_BF16, c->t16, d, nullptr,
            nullptr, 0, &c->flops_dgrad);
       launch_ln_bwd(c->t16, a.x, a.st1, Pf(l, c->rel_ln1g), c->g, c->g, c->g16, T, d, st);
@@ -236,7 +241,7 @@ extern "C" int ppu_local_step(ppu_ctx* c, int replica, const int32_t* tokens, in
   c->flops_fwd = c->flops_dgrad = c->flops_wgrad = 0;
   ppu_make_resident(c, replica);
   Sched s(c, batch, seq);
-  s.forward(tokens);
+  s.forward(tokens, &r);
   s.loss(tokens, 1, c->loss + replica);
   s.backward(r);
   if (s.rc) return ppu_fail(PPU_ECUDA, "kernel launch failed in local step (%d)", s.rc);
