@@ -1,10 +1,11 @@
 // Fused causal attention on the 5th-generation tensor cores (tcgen05.mma, accumulators in
 // tensor memory, operands brought in by TMA), head sizes 64 and 128.
 //
-//   forward   one CTA per 128 queries; per 128-key block S = Q K^T lands in TMEM, 128 softmax
-//             threads (one query row each, so row maxima and sums need no shuffles) turn it into
-//             bf16 probabilities in swizzled shared memory, and P V is a second MMA whose result
-//             is folded into a register accumulator with the online-softmax correction.
+//   forward   one CTA per 128 queries; per 128-key block S = Q K^T lands in TMEM, two groups of
+//             128 softmax threads (one query row each, half of the block's key columns per
+//             group, so row maxima and sums need no shuffles) turn it into bf16 probabilities
+//             in swizzled shared memory, and P V accumulates in TMEM, one accumulator per group,
+//             with lazy online-softmax rescaling; the two partial softmaxes are merged at the end.
 //   dq        one CTA per 128 queries; S = Q K^T and dP = dU V^T in TMEM, the threads form
 //             dS = P (dP - delta) in shared memory, dQ += dS K accumulates in TMEM over all key
 //             blocks (no rescaling is needed in the backward).
@@ -13,15 +14,14 @@
 // The two backward kernels recompute P from q, k and the saved log-sum-exp; nothing is
 // accumulated with atomics, so results are bitwise reproducible.  (Appendix C.1, MHA.)
 //
-// Warp roles: warp 0 issues TMA, warp 1 issues MMAs and owns the TMEM allocation, warps 2-5 are
-// the 128 row threads.  Every mbarrier wait is bounded; on expiry the CTA raises an abort flag,
+// Warp roles: warp 0 issues TMA, warp 1 issues MMAs and owns the TMEM allocation, warps 2-5 and
+// 6-9 are two groups of 128 row threads.  Every mbarrier wait is bounded; on expiry the CTA raises an abort flag,
 // all roles fall through to the common exit, TMEM is released and an error word is set.
 #include "tc_common.cuh"
 
 namespace {
 using namespace tc;
 
-constexpr int ATT_THREADS = 192;
 constexpr int BWD_THREADS = 320;  // warp 0 TMA, warp 1 MMA, warps 2-5 and 6-9: two row groups, half the slab columns each
 constexpr float LOG2E = 1.4426950408889634f;
 
@@ -123,25 +123,34 @@ __device__ __forceinline__ uint8_t* align1k(uint8_t* p) {
 
 // ------------------------------------------------------------------ forward
 // One CTA per 128 queries, 128-key blocks.  S = Q K^T of block j+1 is issued into the second TMEM
-// buffer while the 128 row threads (one query row each) turn block j into bf16 probabilities in
-// one of two shared-memory tiles; O += P V accumulates in TMEM.  The softmax reference maximum is
-// only raised when a row's block maximum exceeds it by more than 2^8 (the stored probabilities
-// then stay below 256); raising it rescales the row of O in TMEM.  Sums, O and the final
-// normalisation all use the same reference, so the result is the exact softmax.
+// buffer while the row threads turn block j into bf16 probabilities in one of two shared-memory
+// tiles.  Two groups of 128 row threads share the work by key columns: group g owns columns
+// [64g, 64g+64) of every block, keeps its own softmax reference and row sum, and its half of
+// P V accumulates in its own TMEM accumulator O_g (two K=64 products per block).  The exponentials
+// (the MUFU unit) and the shared-memory stores of P are the row threads' cost, so halving the
+// columns per thread halves the time a block spends outside the tensor pipe.  At the end the two
+// partial softmaxes are merged exactly: with m = max(m_A, m_B),
+// O = (2^(m_A-m) O_A + 2^(m_B-m) O_B) / (2^(m_A-m) l_A + 2^(m_B-m) l_B).
+// A reference is only raised when a row's block maximum exceeds it by more than 2^8 (stored
+// probabilities then stay below 256); raising it rescales that group's rows of O_g in TMEM.
 constexpr float RESCALE_LOG2 = 8.f;
+constexpr int FWD_THREADS = 320;   // warp 0 TMA, warp 1 MMA, warps 2-5 group A, warps 6-9 group B
 
 template <int DH>
-__global__ void __launch_bounds__(ATT_THREADS, 1)
+__global__ void __launch_bounds__(FWD_THREADS, 1)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams p) {
   constexpr int NH = DH / 64, QT = 128 * DH * 2, PT = 128 * 128 * 2;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align1k(smem_raw);
   const uint32_t Qs = smem_u32(smem), Ks = Qs + QT, Vs = Ks + 2 * QT, Ps = Vs + 2 * QT;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 5 * QT + 2 * PT);
+  // P_FULL / P_EMPTY are indexed [group * 2 + stage], PV_DONE by group
   enum { Q_FULL = 0, K_FULL = 1, K_EMPTY = 3, V_FULL = 5, V_EMPTY = 7, S_FULL = 9, S_EMPTY = 11,
-         P_FULL = 13, P_EMPTY = 15, PV_DONE = 17, NBAR = 18 };
+         P_FULL = 13, P_EMPTY = 17, PV_DONE = 21, ALL_DONE = 23, MERGE = 24, NBAR = 25 };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  // (reference, sum) of each row and group; overlays the Q tile once every MMA has completed
+  float2* exch = reinterpret_cast<float2*>(smem);
   const uint32_t bar0 = smem_u32(bars);
   auto B = [&](int i) { return bar0 + 8u * i; };
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -151,7 +160,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
-    for (int i = 0; i < 2; ++i) { mbar_init(B(S_EMPTY + i), 4); mbar_init(B(P_FULL + i), 4); }
+    for (int i = 0; i < 2; ++i) mbar_init(B(S_EMPTY + i), 8);
+    for (int i = 0; i < 4; ++i) mbar_init(B(P_FULL + i), 4);
+    mbar_init(B(MERGE), 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -161,7 +172,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tS = tmem, tO = tmem + 256;
+  const uint32_t tS = tmem, tO = tmem + 256;   // O_g at tO + g * DH
 
   if (warp == 0) {
     if (lane == 0) {
@@ -203,23 +214,31 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
       for (int j = 0; j < n && ok; ++j) {
         if (j + 1 < n) { ok = issue_s(j + 1); if (!ok) break; }
         const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
-        if (!mbar_wait(B(P_FULL + st), ph, abort_flag, p.flags)) break;
-        if (!mbar_wait(B(V_FULL + st), ph, abort_flag, p.flags)) break;
-        tc_fence_after();
         const uint32_t p_lo = klo(Ps + st * PT), v_lo = mlo<128>(Vs + st * QT);
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          umma_lo(tO, p_lo + kstep<128>(ks), v_lo + mstep(ks), idesc_o, (j > 0 || ks > 0));
-        umma_commit(B(PV_DONE));
-        umma_commit(B(P_EMPTY + st));
+        for (int g = 0; g < 2; ++g) {
+          if (!mbar_wait(B(P_FULL + g * 2 + st), ph, abort_flag, p.flags)) { ok = false; break; }
+          if (g == 0 && !mbar_wait(B(V_FULL + st), ph, abort_flag, p.flags)) { ok = false; break; }
+          tc_fence_after();
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            umma_lo(tO + g * DH, p_lo + kstep<128>(4 * g + ks), v_lo + mstep(4 * g + ks), idesc_o,
+                    (j > 0 || ks > 0));
+          umma_commit(B(PV_DONE + g));
+          umma_commit(B(P_EMPTY + g * 2 + st));
+        }
+        if (!ok) break;
         umma_commit(B(V_EMPTY + st));
       }
+      if (ok) umma_commit(B(ALL_DONE));
     }
   } else {
-    const int quarter = warp & 3;
+    const int g = (warp - 2) >> 2;                // column group
+    const int quarter = warp & 3;                 // TMEM lane quarter this warp may access
     const int row = quarter * 32 + lane;
     const int grow = qb * 128 + row;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+    const uint32_t tOg = tO + g * DH + lane_off;
     const float c = rsqrtf((float)DH) * LOG2E;
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
@@ -227,25 +246,26 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
       const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
       if (!mbar_wait(B(S_FULL + st), ph, abort_flag, p.flags)) { ok = false; break; }
       tc_fence_after();
-      uint32_t r[128];
-#pragma unroll
-      for (int cc = 0; cc < 4; ++cc) tmem_ld32(tS + lane_off + st * 128 + cc * 32, r + 32 * cc);
+      uint32_t r[64];
+      tmem_ld32(tS + lane_off + st * 128 + g * 64, r);
+      tmem_ld32(tS + lane_off + st * 128 + g * 64 + 32, r + 32);
       tmem_ld_wait();
       tc_fence_before();
       warp_arrive(B(S_EMPTY + st));               // the scores are in registers: free the buffer
+      const int col0 = j * 128 + g * 64;
       const bool diag = (j == qb) || ((j + 1) * 128 > S);
       // eight independent partial maxima / sums: a single warp per scheduler cannot hide the
-      // latency of one 128-long dependent chain
+      // latency of one long dependent chain
       float mx8[8];
 #pragma unroll
       for (int q = 0; q < 8; ++q) mx8[q] = -INFINITY;
       if (!diag) {
 #pragma unroll
-        for (int e = 0; e < 128; ++e) mx8[e & 7] = fmaxf(mx8[e & 7], __uint_as_float(r[e]));
+        for (int e = 0; e < 64; ++e) mx8[e & 7] = fmaxf(mx8[e & 7], __uint_as_float(r[e]));
       } else {
 #pragma unroll
-        for (int e = 0; e < 128; ++e) {
-          const int col = j * 128 + e;
+        for (int e = 0; e < 64; ++e) {
+          const int col = col0 + e;
           if (col <= grow && col < S) mx8[e & 7] = fmaxf(mx8[e & 7], __uint_as_float(r[e]));
         }
       }
@@ -257,17 +277,19 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
         const float new_ref = need ? m_blk : m_ref;
         const float factor = need ? ex2(m_ref - new_ref) : 1.f;
         if (j > 0) {
-          // O must be complete up to block j-1 before its rows are rescaled in place
-          if (!mbar_wait(B(PV_DONE), (j - 1) & 1, abort_flag, p.flags)) { ok = false; break; }
+          // O_g must be complete up to block j-1 before its rows are rescaled in place.  S of
+          // block j was issued after both P V products of block j-2, so that phase has already
+          // completed and the parity test cannot alias an older one.
+          if (!mbar_wait(B(PV_DONE + g), (j - 1) & 1, abort_flag, p.flags)) { ok = false; break; }
           tc_fence_after();
 #pragma unroll 1
           for (int cc = 0; cc < DH / 32; ++cc) {
             uint32_t o[32];
-            tmem_ld32(tO + lane_off + cc * 32, o);
+            tmem_ld32(tOg + cc * 32, o);
             tmem_ld_wait();
 #pragma unroll
             for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
-            tmem_st32(tO + lane_off + cc * 32, o);
+            tmem_st32(tOg + cc * 32, o);
           }
           tmem_st_wait();
         }
@@ -277,9 +299,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
       float sum8[8];
 #pragma unroll
       for (int q = 0; q < 8; ++q) sum8[q] = 0.f;
-      if (!mbar_wait(B(P_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+      if (!mbar_wait(B(P_EMPTY + g * 2 + st), ph ^ 1u, abort_flag, p.flags)) { ok = false; break; }
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
+      for (int cc = 0; cc < 2; ++cc) {
         float pv[32];
         if (!diag) {
 #pragma unroll
@@ -288,34 +310,53 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
             sum8[e & 7] += pv[e];
           }
         } else {
+          // a group whose columns are all masked so far still has m_ref = -inf; the select
+          // below discards whatever the exponential made of that
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
-            const int col = j * 128 + cc * 32 + e;
+            const int col = col0 + cc * 32 + e;
             float pe = ex2(fmaf(__uint_as_float(r[cc * 32 + e]), c, -m_ref));
             if (col > grow || col >= S) pe = 0.f;
             pv[e] = pe;
             sum8[e & 7] += pe;
           }
         }
-        store_row32(Ps + st * PT, 16384, row, cc * 4, pv);
+        store_row32(Ps + st * PT + g * 16384, 16384, row, cc * 4, pv);
       }
       l += ((sum8[0] + sum8[1]) + (sum8[2] + sum8[3])) + ((sum8[4] + sum8[5]) + (sum8[6] + sum8[7]));
       tc_fence_before();
       fence_async_smem();
-      warp_arrive(B(P_FULL + st));
+      warp_arrive(B(P_FULL + g * 2 + st));
     }
-    if (ok && mbar_wait(B(PV_DONE), (n - 1) & 1, abort_flag, p.flags)) {
+    // every MMA has completed: the Q tile is free to carry the groups' (reference, sum) pairs
+    if (ok && mbar_wait(B(ALL_DONE), 0, abort_flag, p.flags)) {
       tc_fence_after();
-      const float inv = 1.f / l;
-      bf16* out = p.U + ((int64_t)b * S + grow) * d + head * DH;
+      exch[g * 128 + row] = make_float2(m_ref, l);
+      warp_arrive(B(MERGE));
+      if (mbar_wait(B(MERGE), 0, abort_flag, p.flags)) {
+        const float2 other = exch[(g ^ 1) * 128 + row];
+        const float m = fmaxf(m_ref, other.x);
+        // group A always has a finite reference (key 0 is visible to every query), so m is finite
+        const float w_own = ex2(m_ref - m), w_oth = ex2(other.x - m);
+        const float l_tot = w_own * l + w_oth * other.y;
+        const float inv = 1.f / l_tot;
+        const float fa = (g == 0 ? w_own : w_oth) * inv, fb = (g == 0 ? w_oth : w_own) * inv;
+        bf16* out = p.U + ((int64_t)b * S + grow) * d + head * DH;
+        // each group writes half of the head's columns
 #pragma unroll 1
-      for (int cc = 0; cc < DH / 32; ++cc) {
-        uint32_t o[32];
-        tmem_ld32(tO + lane_off + cc * 32, o);
-        tmem_ld_wait();
-        if (grow < S) drain32(out + cc * 32, o, inv, nullptr, 0);
+        for (int cc = g * (DH / 64); cc < (g + 1) * (DH / 64); ++cc) {
+          uint32_t oa[32], ob[32];
+          tmem_ld32(tO + lane_off + cc * 32, oa);
+          tmem_ld32(tO + DH + lane_off + cc * 32, ob);
+          tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            oa[e] = __float_as_uint(__uint_as_float(oa[e]) * fa + __uint_as_float(ob[e]) * fb);
+          if (grow < S) drain32(out + cc * 32, oa, 1.f, nullptr, 0);
+        }
+        if (g == 0 && grow < S)
+          p.lse_out[((int64_t)b * p.h + head) * S + grow] = (m + log2f(l_tot)) * (1.f / LOG2E);
       }
-      if (grow < S) p.lse_out[((int64_t)b * p.h + head) * S + grow] = (m_ref + log2f(l)) * (1.f / LOG2E);
     }
   }
   if (*abort_flag) for (int i = 0; i < 64; ++i) __nanosleep(2000);
@@ -667,7 +708,7 @@ int fwd_t(const bf16* qkv, bf16* U, float* lse, int B, int S, int h, int* flags,
   if (!encode3d(&m, qkv, 3 * h * DH, S, B, 3 * (int64_t)h * DH, 128)) return -3;
   AttnParams p{}; p.U = U; p.lse_out = lse; p.S = S; p.h = h; p.flags = flags;
   dim3 grid((S + 127) / 128, h, B);
-  attn_fwd_tc_kernel<DH><<<grid, ATT_THREADS, SM, st>>>(m, p);
+  attn_fwd_tc_kernel<DH><<<grid, FWD_THREADS, SM, st>>>(m, p);
   return 0;
 }
 

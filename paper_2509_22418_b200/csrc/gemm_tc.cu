@@ -9,7 +9,7 @@
 //
 // Every mbarrier wait is bounded: on expiry the CTA raises a shared abort flag and a device
 // error word, all roles leave their loops, tensor memory is released and the kernel returns.
-#include "tc_common.cuh"
+#include "gemm_epilogue.cuh"
 
 namespace tc {
 static EncodeTiledFn g_encode = nullptr;
@@ -18,80 +18,7 @@ EncodeTiledFn get_encoder() { return g_encode; }
 
 namespace {
 using namespace tc;
-
-constexpr int BM = 128;
-constexpr int BK = 64;            // 64 bf16 = 128 bytes = one swizzle row
-constexpr int UMMA_K = 16;
-constexpr int EPI_WARPS = 8;      // two per TMEM lane quarter, each draining half the columns
-constexpr int GEMM_THREADS = 64 + 32 * EPI_WARPS;  // warp 0: TMA, warp 1: MMA + TMEM owner, then epilogue
-
-// hardware tanh (relative error about 2^-11, below the bf16 rounding of the stored result)
-__device__ __forceinline__ float tanh_fast(float x) {
-  float y;
-  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ float gelu_dev(float x) {
-  const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
-  const float t = tanh_fast(u);
-  return 0.5f * x * (1.f + t);
-}
-__device__ __forceinline__ float gelu_grad_dev(float x) {
-  const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
-  const float t = tanh_fast(u);
-  const float du = 0.7978845608028654f * (1.f + 3.f * 0.044715f * x * x);
-  return 0.5f * (1.f + t) + 0.5f * x * (1.f - t * t) * du;
-}
-__device__ __forceinline__ uint4 pack8_bf16(const float* f) {
-  uint4 u;
-  __nv_bfloat162* p = reinterpret_cast<__nv_bfloat162*>(&u);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) p[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
-  return u;
-}
-
-// 32-byte global accesses (one full sector per lane and instruction)
-__device__ __forceinline__ void st_v8(void* p, const uint32_t* v) {
-  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(v[0]), "r"(v[1]),
-               "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
-               : "memory");
-}
-__device__ __forceinline__ void ld_v8(uint32_t* v, const void* p) {
-  asm volatile("ld.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
-                 "=r"(v[7])
-               : "l"(p));
-}
-__device__ __forceinline__ uint32_t pack2_bf16(float a, float b) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
-
-// rotary positions on `pairs` adjacent pairs of f starting at column n0 of a [.., heads x dh] row
-__device__ __forceinline__ void rope_pairs(float* f, int pairs, const float2* cs_row, int n0, int dh) {
-#pragma unroll
-  for (int q = 0; q < 16; ++q) {
-    if (q >= pairs) break;
-    const float2 w = __ldg(cs_row + ((n0 + 2 * q) % dh) / 2);
-    const float a = f[2 * q], b = f[2 * q + 1];
-    f[2 * q] = a * w.x - b * w.y;
-    f[2 * q + 1] = a * w.y + b * w.x;
-  }
-}
-
-struct TcParams {
-  int M, N, K;
-  int epilogue;
-  void* C; long long ldc;
-  void* C2;
-  const void* aux; long long ldaux;
-  int* flags;
-  int tiles_m, tiles_n;
-  int splits; long long split_stride;
-  int wide;   // every output / auxiliary row start is 32-byte aligned: use 32-byte accesses
-  int rope_S, rope_dh, rope_cols;
-  void* C3; long long ldc3; int c3_lo, c3_hi;
-};
+using namespace gemm_tc_detail;
 
 template <int BN> struct Cfg {
   static constexpr int STAGES = BN == 256 ? 4 : 6;
@@ -225,172 +152,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
       const int m0 = (t2 % p.tiles_m) * BM, n0 = (t2 / p.tiles_m) * BN;
       if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.flags)) break;
       tc_fence_after();
-      const int m = m0 + quarter * 32 + lane;
-      const bool row_ok = m < p.M;
-      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
-#pragma unroll 1
-      for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
-        const int nb = n0 + c0;
-        if (nb >= p.N) break;                  // warp-uniform
-        uint32_t r[32];
-        tmem_ld32(t_row + c0, r);              // asynchronous until tmem_ld_wait
-        const long long ci = (long long)m * p.ldc + nb + (long long)sp * p.split_stride;
-        const bool full = nb + 32 <= p.N;
-        if (p.wide && full) {
-          // whole 32-column chunk with 32-byte accesses
-          if (p.epilogue == EPI_RESID_F32) {
-            uint32_t x[32];
-            const float* rs = (const float*)p.aux + (long long)m * p.ldaux + nb;
-            if (row_ok) {
-#pragma unroll
-              for (int j = 0; j < 4; ++j) ld_v8(x + 8 * j, rs + 8 * j);
-            }
-            tmem_ld_wait();
-            if (row_ok) {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) x[j] = __float_as_uint(__uint_as_float(x[j]) + __uint_as_float(r[j]));
-#pragma unroll
-              for (int j = 0; j < 4; ++j) st_v8((float*)p.C + ci + 8 * j, x + 8 * j);
-            }
-          } else if (p.epilogue == EPI_DGELU) {
-            uint32_t hv[16];
-            const bf16* hs = (const bf16*)p.aux + (long long)m * p.ldaux + nb;
-            if (row_ok) { ld_v8(hv, hs); ld_v8(hv + 8, hs + 16); }
-            tmem_ld_wait();
-            if (row_ok) {
-              uint32_t o[16];
-#pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                const float2 h2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&hv[j]));
-                o[j] = pack2_bf16(__uint_as_float(r[2 * j]) * gelu_grad_dev(h2.x),
-                                  __uint_as_float(r[2 * j + 1]) * gelu_grad_dev(h2.y));
-              }
-              st_v8((bf16*)p.C + ci, o);
-              st_v8((bf16*)p.C + ci + 16, o + 8);
-            }
-          } else if (p.epilogue == EPI_STORE_F32) {
-            tmem_ld_wait();
-            if (row_ok) {
-#pragma unroll
-              for (int j = 0; j < 4; ++j) st_v8((float*)p.C + ci + 8 * j, r + 8 * j);
-            }
-          } else {
-            tmem_ld_wait();
-            if (row_ok) {
-              if (p.epilogue == EPI_ROPE_BF16 && nb < p.rope_cols) {
-                const float2* cs_row = (const float2*)p.aux + (long long)(m % p.rope_S) * (p.rope_dh / 2);
-                if (p.rope_dh % 32 == 0) {
-                  // the chunk lies inside one head: its 16 (cos, sin) pairs are 128 contiguous bytes
-                  uint32_t w[32];
-                  const float2* src = cs_row + (nb % p.rope_dh) / 2;
-#pragma unroll
-                  for (int j = 0; j < 4; ++j) ld_v8(w + 8 * j, src + 4 * j);
-#pragma unroll
-                  for (int q = 0; q < 16; ++q) {
-                    const float cw = __uint_as_float(w[2 * q]), sw = __uint_as_float(w[2 * q + 1]);
-                    const float a = __uint_as_float(r[2 * q]), b = __uint_as_float(r[2 * q + 1]);
-                    r[2 * q] = __float_as_uint(a * cw - b * sw);
-                    r[2 * q + 1] = __float_as_uint(a * sw + b * cw);
-                  }
-                } else {
-                  rope_pairs(reinterpret_cast<float*>(r), 16, cs_row, nb, p.rope_dh);
-                }
-              }
-              uint32_t o[16];
-#pragma unroll
-              for (int j = 0; j < 16; ++j) o[j] = pack2_bf16(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
-              st_v8((bf16*)p.C + ci, o);
-              st_v8((bf16*)p.C + ci + 16, o + 8);
-              if (p.epilogue == EPI_GELU_DUAL) {
-#pragma unroll
-                for (int j = 0; j < 16; ++j)
-                  o[j] = pack2_bf16(gelu_dev(__uint_as_float(r[2 * j])), gelu_dev(__uint_as_float(r[2 * j + 1])));
-                st_v8((bf16*)p.C2 + ci, o);
-                st_v8((bf16*)p.C2 + ci + 16, o + 8);
-                if (p.C3 && nb < p.c3_hi && nb + 32 > p.c3_lo) {
-#pragma unroll
-                  for (int j = 0; j < 4; ++j) {
-                    const int col = nb + 8 * j;
-                    if (col >= p.c3_lo && col + 8 <= p.c3_hi)
-                      *reinterpret_cast<uint4*>((bf16*)p.C3 + (long long)m * p.ldc3 + (col - p.c3_lo)) =
-                          make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
-                  }
-                }
-              }
-            }
-          }
-          continue;
-        }
-        if (p.epilogue == EPI_RESID_F32) {
-          float4 x[8];
-          const float4* rs = reinterpret_cast<const float4*>((const float*)p.aux + (long long)m * p.ldaux + nb);
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            x[j] = (row_ok && (full || nb + 4 * j < p.N)) ? rs[j] : make_float4(0.f, 0.f, 0.f, 0.f);
-          tmem_ld_wait();
-          if (row_ok) {
-            float4* o = reinterpret_cast<float4*>((float*)p.C + ci);
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-              if (full || nb + 4 * j < p.N)
-                o[j] = make_float4(x[j].x + __uint_as_float(r[4 * j]), x[j].y + __uint_as_float(r[4 * j + 1]),
-                                   x[j].z + __uint_as_float(r[4 * j + 2]), x[j].w + __uint_as_float(r[4 * j + 3]));
-          }
-        } else if (p.epilogue == EPI_DGELU) {
-          uint4 hv[4];
-          const uint4* hs = reinterpret_cast<const uint4*>((const bf16*)p.aux + (long long)m * p.ldaux + nb);
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            hv[j] = (row_ok && (full || nb + 8 * j < p.N)) ? hs[j] : make_uint4(0, 0, 0, 0);
-          tmem_ld_wait();
-          if (row_ok) {
-            uint4* o = reinterpret_cast<uint4*>((bf16*)p.C + ci);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              if (!(full || nb + 8 * j < p.N)) break;
-              const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hv[j]);
-              float a[8];
-#pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                const float2 h2 = __bfloat1622float2(hp[q]);
-                a[2 * q] = __uint_as_float(r[8 * j + 2 * q]) * gelu_grad_dev(h2.x);
-                a[2 * q + 1] = __uint_as_float(r[8 * j + 2 * q + 1]) * gelu_grad_dev(h2.y);
-              }
-              o[j] = pack8_bf16(a);
-            }
-          }
-        } else {
-          tmem_ld_wait();
-          if (row_ok) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              if (!(full || nb + 8 * j < p.N)) break;
-              float f[8];
-#pragma unroll
-              for (int q = 0; q < 8; ++q) f[q] = __uint_as_float(r[8 * j + q]);
-              if (p.epilogue == EPI_ROPE_BF16 && nb + 8 * j < p.rope_cols)
-                rope_pairs(f, 4, (const float2*)p.aux + (long long)(m % p.rope_S) * (p.rope_dh / 2), nb + 8 * j,
-                           p.rope_dh);
-              if (p.epilogue == EPI_STORE_F32) {
-                float4* o = reinterpret_cast<float4*>((float*)p.C + ci + 8 * j);
-                o[0] = make_float4(f[0], f[1], f[2], f[3]);
-                o[1] = make_float4(f[4], f[5], f[6], f[7]);
-              } else {
-                *reinterpret_cast<uint4*>((bf16*)p.C + ci + 8 * j) = pack8_bf16(f);
-                if (p.epilogue == EPI_GELU_DUAL) {
-#pragma unroll
-                  for (int q = 0; q < 8; ++q) f[q] = gelu_dev(f[q]);
-                  const uint4 gv = pack8_bf16(f);
-                  *reinterpret_cast<uint4*>((bf16*)p.C2 + ci + 8 * j) = gv;
-                  const int col = nb + 8 * j;
-                  if (p.C3 && col >= p.c3_lo && col + 8 <= p.c3_hi)
-                    *reinterpret_cast<uint4*>((bf16*)p.C3 + (long long)m * p.ldc3 + (col - p.c3_lo)) = gv;
-                }
-              }
-            }
-          }
-        }
-      }
+      drain_tile<BN>(p, m0, n0, sp, tmem_base + (uint32_t)(acc * BN), quarter, half, lane);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
@@ -411,6 +173,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
   }
 }
 
+}  // namespace
+
+namespace gemm_tc_detail {
 bool encode_map(CUtensorMap* map, const bf16* base, long long ld, bool kmajor, int rows, int K,
                 int box_rows) {
   // kmajor: memory is [rows, K] (inner = K).  else: memory is [K, rows] (inner = rows).
@@ -425,12 +190,33 @@ bool encode_map(CUtensorMap* map, const bf16* base, long long ld, bool kmajor, i
     gdim[0] = (cuuint64_t)rows; gdim[1] = (cuuint64_t)K;
     box[0] = 64; box[1] = BK;
   }
-  CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)base, gdim, gstride, box,
+  CUresult r = tc::g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)base, gdim, gstride, box,
                         estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 
+// launch parameters common to every tile shape (tile counts and split-K are set by the launcher)
+TcParams make_params(const GemmArgs& g) {
+  TcParams p;
+  p.M = g.M; p.N = g.N; p.K = g.K; p.epilogue = g.epilogue;
+  p.C = g.C; p.ldc = g.ldc; p.C2 = g.C2; p.aux = g.aux; p.ldaux = g.ldaux; p.flags = g.flags;
+  p.tiles_m = p.tiles_n = 0; p.splits = 1; p.split_stride = 0;
+  p.C3 = g.C3; p.ldc3 = g.ldc3; p.c3_lo = g.c3_lo; p.c3_hi = g.c3_hi;
+  p.rope_S = g.rope_S > 0 ? g.rope_S : 1; p.rope_dh = g.rope_dh > 0 ? g.rope_dh : 2; p.rope_cols = g.rope_cols;
+  const bool f32 = g.epilogue == EPI_STORE_F32 || g.epilogue == EPI_RESID_F32;
+  const long long out_unit = f32 ? 8 : 16;   // elements per 32 bytes
+  bool w = (reinterpret_cast<uintptr_t>(g.C) % 32 == 0) && (g.ldc % out_unit == 0) &&
+           (g.split_stride % out_unit == 0);
+  if (g.epilogue == EPI_GELU_DUAL) w = w && (reinterpret_cast<uintptr_t>(g.C2) % 32 == 0);
+  if (g.epilogue == EPI_RESID_F32) w = w && (reinterpret_cast<uintptr_t>(g.aux) % 32 == 0) && (g.ldaux % 8 == 0);
+  if (g.epilogue == EPI_DGELU) w = w && (reinterpret_cast<uintptr_t>(g.aux) % 32 == 0) && (g.ldaux % 16 == 0);
+  p.wide = w ? 1 : 0;
+  return p;
+}
+}  // namespace gemm_tc_detail
+
+namespace {
 template <int BN, bool A_K, bool B_K>
 int launch_t(const GemmArgs& g, cudaStream_t st) {
   using C = Cfg<BN>;
@@ -444,26 +230,12 @@ int launch_t(const GemmArgs& g, cudaStream_t st) {
   CUtensorMap mapA, mapB;
   if (!encode_map(&mapA, g.A, g.lda, A_K, g.M, g.K, BM)) return -2;
   if (!encode_map(&mapB, g.B, g.ldb, B_K, g.N, g.K, BN)) return -2;
-  TcParams p;
-  p.M = g.M; p.N = g.N; p.K = g.K; p.epilogue = g.epilogue;
-  p.C = g.C; p.ldc = g.ldc; p.C2 = g.C2; p.aux = g.aux; p.ldaux = g.ldaux; p.flags = g.flags;
+  TcParams p = make_params(g);
   p.tiles_m = (g.M + BM - 1) / BM;
   p.tiles_n = (g.N + BN - 1) / BN;
   const int k_blocks = (g.K + BK - 1) / BK;
   p.splits = g.splits < 1 ? 1 : (g.splits > k_blocks ? k_blocks : g.splits);
   p.split_stride = g.split_stride;
-  p.C3 = g.C3; p.ldc3 = g.ldc3; p.c3_lo = g.c3_lo; p.c3_hi = g.c3_hi;
-  p.rope_S = g.rope_S > 0 ? g.rope_S : 1; p.rope_dh = g.rope_dh > 0 ? g.rope_dh : 2; p.rope_cols = g.rope_cols;
-  {
-    const bool f32 = g.epilogue == EPI_STORE_F32 || g.epilogue == EPI_RESID_F32;
-    const long long out_unit = f32 ? 8 : 16;   // elements per 32 bytes
-    bool w = (reinterpret_cast<uintptr_t>(g.C) % 32 == 0) && (g.ldc % out_unit == 0) &&
-             (g.split_stride % out_unit == 0);
-    if (g.epilogue == EPI_GELU_DUAL) w = w && (reinterpret_cast<uintptr_t>(g.C2) % 32 == 0);
-    if (g.epilogue == EPI_RESID_F32) w = w && (reinterpret_cast<uintptr_t>(g.aux) % 32 == 0) && (g.ldaux % 8 == 0);
-    if (g.epilogue == EPI_DGELU) w = w && (reinterpret_cast<uintptr_t>(g.aux) % 32 == 0) && (g.ldaux % 16 == 0);
-    p.wide = w ? 1 : 0;
-  }
   const int tiles = p.tiles_m * p.tiles_n * p.splits;
   static int n_sm = 0;
   if (n_sm == 0) {
@@ -506,6 +278,11 @@ int launch_gemm_tc(const GemmArgs& g, cudaStream_t st) {
       (reinterpret_cast<uintptr_t>(g.C) & 15))
     return -4;
   // Wide tiles when the grid still fills the machine; narrow ones for small outputs.
+  // SM pairs on 256 x 256 tiles when those still fill the machine and the product is not split.
+  const long long tiles_pair = (long long)((g.M + 255) / 256) * ((g.N + 255) / 256);
+  if (g.tile_shape == 2 && g.splits > 1) return -4;
+  if (g.tile_shape == 2 || (g.tile_shape == 0 && g.splits <= 1 && g.M > 128 && g.N > 128 && tiles_pair >= 74))
+    return launch_gemm_tc_pair(g, make_params(g), st);
   const long long tiles256 = (long long)((g.M + BM - 1) / BM) * ((g.N + 255) / 256) * (g.splits > 1 ? g.splits : 1);
   if (g.N > 128 && tiles256 >= 148) return launch_bn<256>(g, st);
   return launch_bn<128>(g, st);

@@ -1,0 +1,253 @@
+// tcgen05 GEMM on SM pairs (cta_group::2): C[M,N] = A . B^T, bf16 operands, fp32 accumulation.
+//
+// A cluster of two CTAs (the two SMs of one TPC) owns a 256 x 256 output tile.  CTA r of the
+// pair loads rows [128 r, 128 r + 128) of the A tile and of the B tile; one thread of the
+// leader CTA (rank 0) issues tcgen05.mma.cta_group::2 with M = 256, N = 256, K = 16, for which
+// each SM reads its own A half and shares its B half with its peer, and each SM's tensor memory
+// receives its 128 rows of the 256-column accumulator.  Per SM and MMA that is 8 KB of operands
+// read from shared memory for 128 x 256 x 16 multiply-adds, against 12 KB for a single-CTA
+// 128 x 256 tile: the operand path, not the tensor pipe, limits the single-CTA kernel.
+//
+// Protocol.  Stage barriers live at the same shared-memory offsets in both CTAs.
+//   full[s]    only the leader's is used: its producer posts the expected bytes of BOTH CTAs'
+//              loads, and both CTAs' TMA loads complete on it (.cta_group::2 form of the copy).
+//   empty[s]   one per CTA, signalled in both by the MMA thread's multicast commit.
+//   tfull[a]   one per CTA (multicast commit): accumulator a is complete.
+//   tempty[a]  the leader's counts the epilogue warps of both CTAs (the peer's arrive remotely).
+// Every wait is bounded; on expiry the CTA raises its abort flag and an error word and all roles
+// fall through to the common exit, where both CTAs meet at a cluster barrier (reached
+// unconditionally by every thread) before tensor memory is released.
+#include "gemm_epilogue.cuh"
+
+namespace {
+using namespace tc;
+using namespace gemm_tc_detail;
+
+constexpr int PAIR_BN = 256;                 // accumulator columns (N of the pair's tile)
+constexpr int PAIR_STAGES = 6;
+constexpr int HALF_BYTES = 128 * BK * 2;     // one CTA's A (or B) slab: 128 rows x 64 k
+constexpr int PAIR_STAGE_BYTES = 2 * HALF_BYTES;
+constexpr int PAIR_SMEM = PAIR_STAGES * PAIR_STAGE_BYTES + 1024 + 256;
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA tile load of a CTA pair: the bytes land in this CTA's shared memory, the completion is
+// counted on the barrier at cluster address `bar` (the leader's)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+      "l"(map), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate) {
+  const uint32_t z = 0;
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n}" ::"r"(tmem_d),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(z)
+      : "memory");
+}
+// arrives, once the pair's earlier MMAs have completed, on the barrier at this offset in both CTAs
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+      "h"(mask)
+      : "memory");
+}
+
+template <bool A_K, bool B_K>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                    const TcParams p) {
+  constexpr int ST = PAIR_STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  // the dynamic window starts at the same offset in both CTAs, so aligned offsets match too
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + ST * PAIR_STAGE_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * ST + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();
+  const bool leader = rank == 0;
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (ST + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * ST + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * ST + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < ST; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 2 * EPI_WARPS); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();          // the peer's barriers are initialised before anything signals them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int n_pairs = gridDim.x >> 1, pair = blockIdx.x >> 1;
+  const int num_tiles = p.tiles_m * p.tiles_n;
+  const int k_blocks = (p.K + BK - 1) / BK;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---------------- TMA producer (both CTAs) ----------------
+      int s = 0; uint32_t ph = 0;
+      bool ok = true;
+      for (int tile = pair; tile < num_tiles && ok; tile += n_pairs) {
+        const int m0 = (tile % p.tiles_m) * 256 + (int)rank * 128;
+        const int n0 = (tile / p.tiles_m) * PAIR_BN + (int)rank * 128;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.flags);
+          if (!ok) break;
+          const uint32_t a_dst = smem_u32(smem + s * PAIR_STAGE_BYTES);
+          const uint32_t b_dst = a_dst + HALF_BYTES;
+          const uint32_t fb = map_to_rank(full_bar(s), 0);
+          if (leader) mbar_expect_tx(full_bar(s), 2 * PAIR_STAGE_BYTES);
+          if (A_K) {
+            tma_load_2d_pair(a_dst, &mapA, fb, kb * BK, m0);
+          } else {
+            tma_load_2d_pair(a_dst, &mapA, fb, m0, kb * BK);
+            tma_load_2d_pair(a_dst + 8192, &mapA, fb, m0 + 64, kb * BK);
+          }
+          if (B_K) {
+            tma_load_2d_pair(b_dst, &mapB, fb, kb * BK, n0);
+          } else {
+            tma_load_2d_pair(b_dst, &mapB, fb, n0, kb * BK);
+            tma_load_2d_pair(b_dst + 8192, &mapB, fb, n0 + 64, kb * BK);
+          }
+          if (++s == ST) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && leader) {
+      // ---------------- MMA issuer (leader CTA only) ----------------
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_K ? 0u : 1u) << 15) |
+                             ((B_K ? 0u : 1u) << 16) | ((uint32_t)(PAIR_BN >> 3) << 17) |
+                             ((uint32_t)(256 >> 4) << 24);
+      int s = 0; uint32_t ph = 0;
+      int acc = 0; uint32_t acc_ph = 0;
+      for (int tile = pair; tile < num_tiles; tile += n_pairs) {
+        if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.flags)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * PAIR_BN);
+        bool ok = true;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          ok = mbar_wait(full_bar(s), ph, abort_flag, p.flags);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(smem + s * PAIR_STAGE_BYTES);
+          const uint32_t b_addr = a_addr + HALF_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t adesc = A_K ? make_desc(a_addr + k * 32, 16, 1024) : make_desc(a_addr + k * 2048, 8192, 1024);
+            const uint64_t bdesc = B_K ? make_desc(b_addr + k * 32, 16, 1024) : make_desc(b_addr + k * 2048, 8192, 1024);
+            umma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit_pair(empty_bar(s));        // both CTAs' slots are free once these MMAs have read them
+          if (++s == ST) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit_pair(tfull_bar(acc));        // both halves of the accumulator are complete
+        if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+      }
+    }
+  } else {
+    // ---------------- epilogue warps (both CTAs, 128 rows each) ----------------
+    const int quarter = warp & 3;
+    const int half = (warp - 2) >> 2;
+    int acc = 0; uint32_t acc_ph = 0;
+    for (int tile = pair; tile < num_tiles; tile += n_pairs) {
+      const int m0 = (tile % p.tiles_m) * 256 + (int)rank * 128;
+      const int n0 = (tile / p.tiles_m) * PAIR_BN;
+      if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.flags)) break;
+      tc_fence_after();
+      drain_tile<PAIR_BN>(p, m0, n0, 0, tmem_base + (uint32_t)(acc * PAIR_BN), quarter, half, lane);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_rank(tempty_bar(acc), 0));
+      if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+    }
+  }
+
+  // ---------------- common exit ----------------
+  if (*abort_flag) {
+    for (int i = 0; i < 64; ++i) __nanosleep(2000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();          // neither CTA leaves (or frees tensor memory) while its peer may still signal it
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+template <bool A_K, bool B_K>
+int launch_pair_t(const GemmArgs& g, const TcParams& p0, cudaStream_t st) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(gemm_tc_pair_kernel<A_K, B_K>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             PAIR_SMEM) != cudaSuccess)
+      return -1;
+    attr_done = true;
+  }
+  CUtensorMap mapA, mapB;
+  if (!encode_map(&mapA, g.A, g.lda, A_K, g.M, g.K, 128)) return -2;
+  if (!encode_map(&mapB, g.B, g.ldb, B_K, g.N, g.K, 128)) return -2;
+  TcParams p = p0;
+  p.tiles_m = (g.M + 255) / 256;
+  p.tiles_n = (g.N + PAIR_BN - 1) / PAIR_BN;
+  p.splits = 1; p.split_stride = 0;
+  const int tiles = p.tiles_m * p.tiles_n;
+  static int n_sm = 0;
+  if (n_sm == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (n_sm <= 0) n_sm = 148;
+  }
+  const int pairs = tiles < n_sm / 2 ? tiles : n_sm / 2;
+  gemm_tc_pair_kernel<A_K, B_K><<<2 * pairs, GEMM_THREADS, PAIR_SMEM, st>>>(mapA, mapB, p);
+  return cudaGetLastError() == cudaSuccess ? 0 : -3;
+}
+
+}  // namespace
+
+namespace gemm_tc_detail {
+int launch_gemm_tc_pair(const GemmArgs& g, const TcParams& p, cudaStream_t st) {
+  if (g.a_kmajor && g.b_kmajor) return launch_pair_t<true, true>(g, p, st);
+  if (g.a_kmajor && !g.b_kmajor) return launch_pair_t<true, false>(g, p, st);
+  if (!g.a_kmajor && g.b_kmajor) return launch_pair_t<false, true>(g, p, st);
+  return launch_pair_t<false, false>(g, p, st);
+}
+}  // namespace gemm_tc_detail

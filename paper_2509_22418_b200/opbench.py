@@ -26,7 +26,8 @@ def main():
     ap.add_argument("--seq", type=int, default=2048)
     ap.add_argument("--heads", type=int, default=16)
     ap.add_argument("--dh", type=int, default=128)
-    ap.add_argument("--backend", type=int, default=0, help="attention: 0 tcgen05, 1 SIMT, 2 mma.sync")
+    ap.add_argument("--backend", type=int, default=0, help="attention: 0 tcgen05, 1 SIMT, 2 mma.sync; gemm: 0 tcgen05 (shape chosen), 1 SIMT, "
+                         "2 tcgen05 one CTA per tile, 3 tcgen05 SM pairs")
     ap.add_argument("--iters", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     a = ap.parse_args()
@@ -50,9 +51,10 @@ def main():
     if a.op == "gemm":
         A = torch.randn((a.k, a.m) if a.a_mn else (a.m, a.k), generator=g).to(dev).bfloat16()
         B = torch.randn((a.k, a.n) if a.b_mn else (a.n, a.k), generator=g).to(dev).bfloat16()
-        ms = timed(lambda: ppu.ppu_gemm(A, not a.a_mn, B, not a.b_mn, a.m, a.n, a.k, out_f32=a.f32))
+        ms = timed(lambda: ppu.ppu_gemm(A, not a.a_mn, B, not a.b_mn, a.m, a.n, a.k, out_f32=a.f32,
+                                         backend=a.backend))
         fl = 2.0 * a.m * a.n * a.k
-        print(f"gemm M={a.m} N={a.n} K={a.k} a_mn={a.a_mn} b_mn={a.b_mn}: {ms:.4f} ms "
+        print(f"gemm M={a.m} N={a.n} K={a.k} a_mn={a.a_mn} b_mn={a.b_mn} backend={a.backend}: {ms:.4f} ms "
               f"{fl / ms / 1e9:.1f} TFLOP/s")
     else:
         B_, S, h, dh = a.batch, a.seq, a.heads, a.dh

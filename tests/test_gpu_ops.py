@@ -23,10 +23,14 @@ GEMM_SHAPES = [
     (8, 8, 8),           # smaller than any tile
     (1000, 96, 4096),    # long reduction, narrow output
     (384, 768, 520),
+    (512, 768, 320),     # several 256 x 256 tiles of an SM pair
+    (1104, 520, 264),    # the same, ragged in every dimension
 ]
 
 
-@pytest.mark.parametrize("backend", [0, 1])
+# backends: 0 tcgen05 with the tile shape the step would choose, 1 SIMT, 2 tcgen05 one CTA per tile,
+# 3 tcgen05 SM pairs (cta_group::2)
+@pytest.mark.parametrize("backend", [0, 1, 2, 3])
 @pytest.mark.parametrize("a_k,b_k", [(1, 1), (1, 0), (0, 1), (0, 0)])
 @pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
 def test_gemm_against_oracle_matmul(backend, a_k, b_k, M, N, K):
@@ -55,7 +59,7 @@ def test_gemm_strided_operands_and_column_offset():
     dH, dH64 = _bf16_tensor(rng, (T, F))
     b, b64 = _bf16_tensor(rng, (T, d))
     ref = dH64[:, lo:hi].T @ b64                       # dW_in[lo:hi, :]
-    for backend in (0, 1):
+    for backend in (0, 1, 2, 3):
         got = ppu.ppu_gemm(dH[:, lo:hi], 0, b, 0, hi - lo, d, T, out_f32=True, backend=backend)
         torch.cuda.synchronize()
         err = np.abs(got.cpu().numpy() - ref)
