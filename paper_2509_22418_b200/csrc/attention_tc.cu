@@ -6,11 +6,13 @@
 //             group, so row maxima and sums need no shuffles) turn it into bf16 probabilities
 //             in swizzled shared memory, and P V accumulates in TMEM, one accumulator per group,
 //             with lazy online-softmax rescaling; the two partial softmaxes are merged at the end.
-//   dq        one CTA per 128 queries; S = Q K^T and dP = dU V^T in TMEM, the threads form
-//             dS = P (dP - delta) in shared memory, dQ += dS K accumulates in TMEM over all key
-//             blocks (no rescaling is needed in the backward).
-//   dk, dv    one CTA per 128 keys, query blocks of 64; the transposed products S^T = K Q^T,
-//             dP^T = V dU^T; dV += P^T dU and dK += dS^T Q accumulate in TMEM.
+//   dq        one CTA per 128 queries, 128-key slabs; S = Q K^T and dP = dU V^T in TMEM, the
+//             threads form dS = P (dP - delta) and write it back to TMEM as bf16, from where it is
+//             the A operand of dQ += dS K, which accumulates in TMEM over all slabs (no rescaling
+//             is needed in the backward).
+//   dk, dv    one CTA per 128 keys, 128-query slabs; the transposed products S^T = K Q^T,
+//             dP^T = V dU^T; P^T and dS^T overwrite them in TMEM as bf16 and feed dV += P^T dU and
+//             dK += dS^T Q, which accumulate in TMEM.
 // The two backward kernels recompute P from q, k and the saved log-sum-exp; nothing is
 // accumulated with atomics, so results are bitwise reproducible.  (Appendix C.1, MHA.)
 //
@@ -366,21 +368,34 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
 }
 
 // ------------------------------------------------------------------ backward: dq
-// One CTA owns 128 queries (Q and dU tiles resident) and streams 64-key slabs of K and V
-// through a 4-deep TMA ring.  S = Q K^T and dP = dU V^T of slab i+1 are issued into a second
-// pair of TMEM buffers while the 128 row threads turn slab i into dS = P (dP - delta);
-// dQ += dS K accumulates in TMEM over all slabs.
+// A operand from tensor memory (bf16 pairs, one row per lane), B from shared memory
+__device__ __forceinline__ void umma_ts_lo(uint32_t tmem_d, uint32_t tmem_a, uint32_t blo, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n.reg .pred p;\n.reg .b64 db;\nsetp.ne.b32 p, %4, 0;\n"
+      "mov.b64 db, {%2, %5};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n}" ::"r"(tmem_d),
+      "r"(tmem_a), "r"(blo), "r"(idesc), "r"(acc), "r"(DESC_HI)
+      : "memory");
+}
+
+// One CTA owns 128 queries (Q and dU tiles resident) and streams 128-key slabs of K and V through
+// a two-deep TMA ring.  S = Q K^T and dP = dU V^T of a slab land in tensor memory; the 256 row
+// threads (one query row each, half of the slab's key columns per group) pull them into
+// registers, which frees the two accumulators for the next slab, form dS = P (dP - delta) and
+// write it as bf16 into one of two tensor-memory buffers, from where it is the A operand of
+// dQ += dS K.  The MMA-issuing thread is the scarce resource of this kernel (its waits, commits
+// and instruction issue are latency-bound), hence few, wide instructions: 24 per 128 keys.
 template <int DH>
 __global__ void __launch_bounds__(BWD_THREADS, 1)
 attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapG,
-                  const __grid_constant__ CUtensorMap mapKV64, const AttnParams p) {
-  constexpr int NH = DH / 64, QT = 128 * DH * 2, HT = 64 * DH * 2, PT = 128 * 64 * 2, NS = 4;
+                  const AttnParams p) {
+  constexpr int NH = DH / 64, QT = 128 * DH * 2, NK = 3, NV = 2;   // K lives until its slab's dQ product, V only until dP
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align1k(smem_raw);
-  const uint32_t Qs = smem_u32(smem), Gs = Qs + QT, Ds = Gs + QT, Rs = Ds + 2 * PT;   // two dS tiles; ring: K then V per stage
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * QT + 2 * PT + NS * 2 * HT);
-  enum { Q_FULL = 0, KV_FULL = 1, KV_EMPTY = 1 + NS, SDP_FULL = 1 + 2 * NS, SDP_EMPTY = 3 + 2 * NS,
-         DS_FULL = 5 + 2 * NS, DS_EMPTY = 7 + 2 * NS, DQ_FULL = 9 + 2 * NS, NBAR = 10 + 2 * NS };
+  const uint32_t Qs = smem_u32(smem), Gs = Qs + QT, Kr = Gs + QT, Vr = Kr + NK * QT;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (2 + NK + NV) * QT);
+  enum { Q_FULL = 0, K_FULL = 1, V_FULL = K_FULL + NK, K_EMPTY = V_FULL + NV, V_EMPTY = K_EMPTY + NK,
+         SDP_FULL = V_EMPTY + NV, SDP_EMPTY, DS_FULL, DS_EMPTY = DS_FULL + 2, DQ_FULL = DS_EMPTY + 2, NBAR };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar0 = smem_u32(bars);
@@ -388,11 +403,11 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qb = gridDim.x - 1 - blockIdx.x, head = blockIdx.y, b = blockIdx.z;
   const int d = p.h * DH, S = p.S;
-  const int n = min(2 * (qb + 1), (S + 63) / 64);      // 64-key slabs up to the diagonal
+  const int n = min(qb + 1, (S + 127) / 128);      // 128-key slabs up to the diagonal
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
-    mbar_init(B(SDP_EMPTY), 8); mbar_init(B(SDP_EMPTY + 1), 8); mbar_init(B(DS_FULL), 8); mbar_init(B(DS_FULL + 1), 8);
+    mbar_init(B(SDP_EMPTY), 8); mbar_init(B(DS_FULL), 8); mbar_init(B(DS_FULL + 1), 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -402,7 +417,7 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tQ = tmem + 256;      // S of buffer bf at tmem + 128 bf, dP at tmem + 128 bf + 64
+  const uint32_t tS = tmem, tP = tmem + 128, tD = tmem + 256, tQ = tmem + 384;   // dS buffer b at tD + 64 b
 
   if (warp == 0) {
     if (lane == 0) {
@@ -412,54 +427,57 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
         tma_load_3d(Gs + hf * 16384, &mapG, B(Q_FULL), head * DH + hf * 64, qb * 128, b);
       }
       for (int it = 0; it < n; ++it) {
-        const int st = it % NS; const uint32_t ph = (it / NS) & 1;
-        if (!mbar_wait(B(KV_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) break;
-        mbar_expect_tx(B(KV_FULL + st), 2 * HT);
-        for (int hf = 0; hf < NH; ++hf) {
-          tma_load_3d(Rs + st * 2 * HT + hf * 8192, &mapKV64, B(KV_FULL + st), d + head * DH + hf * 64, it * 64, b);
-          tma_load_3d(Rs + st * 2 * HT + HT + hf * 8192, &mapKV64, B(KV_FULL + st), 2 * d + head * DH + hf * 64, it * 64, b);
-        }
+        const int sk = it % NK, sv = it % NV;
+        if (!mbar_wait(B(K_EMPTY + sk), ((it / NK) & 1) ^ 1u, abort_flag, p.flags)) break;
+        mbar_expect_tx(B(K_FULL + sk), QT);
+        for (int hf = 0; hf < NH; ++hf)
+          tma_load_3d(Kr + sk * QT + hf * 16384, &mapQKV, B(K_FULL + sk), d + head * DH + hf * 64, it * 128, b);
+        if (!mbar_wait(B(V_EMPTY + sv), ((it / NV) & 1) ^ 1u, abort_flag, p.flags)) break;
+        mbar_expect_tx(B(V_FULL + sv), QT);
+        for (int hf = 0; hf < NH; ++hf)
+          tma_load_3d(Vr + sv * QT + hf * 16384, &mapQKV, B(V_FULL + sv), 2 * d + head * DH + hf * 64, it * 128, b);
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc_s = make_idesc(128, 64, false, false);
+      constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
       constexpr uint32_t idesc_q = make_idesc(128, DH, false, true);
+      const uint32_t q_lo = klo(Qs), g_lo = klo(Gs);
       auto issue_sdp = [&](int it) -> bool {
-        const int st = it % NS, bf = it & 1;
-        if (!mbar_wait(B(KV_FULL + st), (it / NS) & 1, abort_flag, p.flags)) return false;
-        if (!mbar_wait(B(SDP_EMPTY + bf), ((it >> 1) & 1) ^ 1u, abort_flag, p.flags)) return false;
+        const int sk = it % NK, sv = it % NV;
+        if (!mbar_wait(B(K_FULL + sk), (it / NK) & 1, abort_flag, p.flags)) return false;
+        if (!mbar_wait(B(V_FULL + sv), (it / NV) & 1, abort_flag, p.flags)) return false;
+        if (it > 0 && !mbar_wait(B(SDP_EMPTY), (uint32_t)(it - 1) & 1u, abort_flag, p.flags)) return false;
         tc_fence_after();
-        const uint32_t tS = tmem + 128 * bf, tP = tS + 64, Kst = Rs + st * 2 * HT, Vst = Kst + HT;
-        const uint32_t q_lo = klo(Qs), g_lo = klo(Gs), k_lo = klo(Kst), v_lo = klo(Vst);
+        const uint32_t k_lo = klo(Kr + sk * QT), v_lo = klo(Vr + sv * QT);
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks)
-          umma_lo(tS, q_lo + kstep<128>(ks), k_lo + kstep<64>(ks), idesc_s, ks > 0);
+          umma_lo(tS, q_lo + kstep<128>(ks), k_lo + kstep<128>(ks), idesc_s, ks > 0);
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks)
-          umma_lo(tP, g_lo + kstep<128>(ks), v_lo + kstep<64>(ks), idesc_s, ks > 0);
-        umma_commit(B(SDP_FULL + bf));
+          umma_lo(tP, g_lo + kstep<128>(ks), v_lo + kstep<128>(ks), idesc_s, ks > 0);
+        umma_commit(B(SDP_FULL));
+        umma_commit(B(V_EMPTY + sv));
         return true;
       };
       auto issue_dq = [&](int it) -> bool {
-        const int st = it % NS, db = it & 1;
+        const int sk = it % NK, db = it & 1;
         if (!mbar_wait(B(DS_FULL + db), (it >> 1) & 1, abort_flag, p.flags)) return false;
         tc_fence_after();
-        const uint32_t ds_lo = klo(Ds + db * PT), kmn_lo = mlo<64>(Rs + st * 2 * HT);
+        const uint32_t kmn_lo = mlo<128>(Kr + sk * QT);
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-          umma_lo(tQ, ds_lo + kstep<128>(ks), kmn_lo + mstep(ks), idesc_q, (it > 0 || ks > 0));
+        for (int ks = 0; ks < 8; ++ks)
+          umma_ts_lo(tQ, tD + 64 * db + 8 * ks, kmn_lo + mstep(ks), idesc_q, (it > 0 || ks > 0));
         umma_commit(B(DS_EMPTY + db));
-        umma_commit(B(KV_EMPTY + st));
+        umma_commit(B(K_EMPTY + sk));
         if (it == n - 1) umma_commit(B(DQ_FULL));
         return true;
       };
       bool ok = mbar_wait(B(Q_FULL), 0, abort_flag, p.flags);
       ok = ok && issue_sdp(0);
-      if (ok && n > 1) ok = issue_sdp(1);
       for (int it = 0; it < n && ok; ++it) {
-        ok = issue_dq(it);
-        if (ok && it + 2 < n) ok = issue_sdp(it + 2);
+        if (it + 1 < n) ok = issue_sdp(it + 1);
+        ok = ok && issue_dq(it);
       }
     }
   } else {
@@ -473,29 +491,43 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
     const float l2 = p.lse[si] * LOG2E, dl = p.delta[si];
     bool ok = true;
     for (int it = 0; it < n && ok; ++it) {
-      const int bf = it & 1;
-      const uint32_t tS = tmem + 128 * bf + lane_off, tP = tS + 64;
-      if (!mbar_wait(B(SDP_FULL + bf), (it >> 1) & 1, abort_flag, p.flags)) { ok = false; break; }
+      const int db = it & 1;
+      if (!mbar_wait(B(SDP_FULL), (uint32_t)it & 1u, abort_flag, p.flags)) { ok = false; break; }
       tc_fence_after();
-      uint32_t rs[32], rd[32];
-      tmem_ld32(tS + 32 * grp, rs);
-      tmem_ld32(tP + 32 * grp, rd);
+      uint32_t rs[64], rd[64];
+      tmem_ld32(tS + lane_off + 64 * grp, rs);
+      tmem_ld32(tS + lane_off + 64 * grp + 32, rs + 32);
+      tmem_ld32(tP + lane_off + 64 * grp, rd);
+      tmem_ld32(tP + lane_off + 64 * grp + 32, rd + 32);
       tmem_ld_wait();
       tc_fence_before();
-      warp_arrive(B(SDP_EMPTY + bf));          // the accumulators are in registers: free them early
-      const bool diag = ((it + 1) * 64 > qb * 128) || ((it + 1) * 64 > S);
-      float ds[32];
+      warp_arrive(B(SDP_EMPTY));               // the accumulators are in registers: free them early
+      const bool diag = (it == qb) || ((it + 1) * 128 > S);
+      const int col0 = it * 128 + 64 * grp;
+      if (!diag) {
 #pragma unroll
-      for (int e = 0; e < 32; ++e) {
-        const int col = it * 64 + 32 * grp + e;
-        float pe = ex2(__uint_as_float(rs[e]) * c - l2);
-        if (diag && (col > grow || col >= S)) pe = 0.f;
-        ds[e] = pe * (__uint_as_float(rd[e]) - dl);
+        for (int e = 0; e < 64; e += 2) {
+          const float p0 = ex2(fmaf(__uint_as_float(rs[e]), c, -l2));
+          const float p1 = ex2(fmaf(__uint_as_float(rs[e + 1]), c, -l2));
+          rs[e >> 1] = pack2(p0 * (__uint_as_float(rd[e]) - dl), p1 * (__uint_as_float(rd[e + 1]) - dl));
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 64; e += 2) {
+          const int col = col0 + e;
+          float p0 = ex2(fmaf(__uint_as_float(rs[e]), c, -l2));
+          float p1 = ex2(fmaf(__uint_as_float(rs[e + 1]), c, -l2));
+          if (col > grow || col >= S) p0 = 0.f;
+          if (col + 1 > grow || col + 1 >= S) p1 = 0.f;
+          rs[e >> 1] = pack2(p0 * (__uint_as_float(rd[e]) - dl), p1 * (__uint_as_float(rd[e + 1]) - dl));
+        }
       }
-      if (!mbar_wait(B(DS_EMPTY + bf), ((it >> 1) & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
-      store_row32(Ds + bf * PT, 0, row, 4 * grp, ds);
-      fence_async_smem();
-      warp_arrive(B(DS_FULL + bf));
+      if (!mbar_wait(B(DS_EMPTY + db), ((it >> 1) & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+      tc_fence_after();
+      tmem_st32(tD + 64 * db + lane_off + 32 * grp, rs);
+      tmem_st_wait();
+      tc_fence_before();
+      warp_arrive(B(DS_FULL + db));
     }
     if (ok && mbar_wait(B(DQ_FULL), 0, abort_flag, p.flags)) {
       tc_fence_after();
@@ -517,21 +549,25 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
 }
 
 // ------------------------------------------------------------------ backward: dk, dv
-// One CTA owns 128 keys (K and V tiles resident) and streams 64-query slabs of Q and dU through
-// a 4-deep TMA ring.  The transposed products S^T = K Q^T and dP^T = V dU^T of slab i+1 are
-// issued into a second pair of TMEM buffers while the 128 row threads (one key each) form
-// P^T and dS^T of slab i; dV += P^T dU and dK += dS^T Q accumulate in TMEM.
+// One CTA owns 128 keys (K and V tiles resident) and streams 128-query slabs of Q and dU through
+// a two-deep TMA ring.  The transposed products S^T = K Q^T and dP^T = V dU^T of a slab land in
+// tensor memory; the 256 row threads (one key each, half of the slab's queries per group) turn
+// them into bf16 P^T and dS^T written back over the accumulators they came from (half their
+// columns), and dV += P^T dU, dK += dS^T Q take those as A operands straight from tensor memory.
+// The products of a slab are serial (the tensor-memory budget - two 128-column accumulators for
+// dV and dK plus the two score buffers - leaves no room to double-buffer the scores); the next
+// slab's Q and dU arrive meanwhile.
 template <int DH>
 __global__ void __launch_bounds__(BWD_THREADS, 1)
-attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_constant__ CUtensorMap mapQ64,
-                   const __grid_constant__ CUtensorMap mapG64, const AttnParams p) {
-  constexpr int NH = DH / 64, QT = 128 * DH * 2, HT = 64 * DH * 2, PT = 128 * 64 * 2, NS = 3;
+attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapG,
+                   const AttnParams p) {
+  constexpr int NH = DH / 64, QT = 128 * DH * 2, NS = 2;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align1k(smem_raw);
-  const uint32_t Ks = smem_u32(smem), Vs = Ks + QT, Ps = Vs + QT, Ds = Ps + 2 * PT, Rs = Ds + 2 * PT;  // two P^T / dS^T tiles; ring: Q then dU
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * QT + 4 * PT + NS * 2 * HT);
-  enum { KV_FULL = 0, QG_FULL = 1, QG_EMPTY = 1 + NS, SDP_FULL = 1 + 2 * NS, SDP_EMPTY = 3 + 2 * NS,
-         PDS_FULL = 5 + 2 * NS, PDS_EMPTY = 7 + 2 * NS, OUT_FULL = 9 + 2 * NS, NBAR = 10 + 2 * NS };
+  const uint32_t Ks = smem_u32(smem), Vs = Ks + QT, Rs = Vs + QT;   // ring: Q then dU per stage
+  float* row_stat = reinterpret_cast<float*>(smem + (2 + 2 * NS) * QT);   // [parity][lse * log2e | delta][128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (2 + 2 * NS) * QT + 2 * 2 * 128 * 4);
+  enum { KV_FULL = 0, QG_FULL = 1, QG_EMPTY = 1 + NS, SDP_FULL = 1 + 2 * NS, LOADED, PDS_FULL, OUT_FULL, NBAR };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar0 = smem_u32(bars);
@@ -539,11 +575,11 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_const
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kb = blockIdx.x, head = blockIdx.y, b = blockIdx.z;
   const int d = p.h * DH, S = p.S;
-  const int i0 = 2 * kb, n = (S + 63) / 64 - i0;      // 64-query slabs from the diagonal down
+  const int n = (S + 127) / 128 - kb;      // 128-query slabs from the diagonal down
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
-    mbar_init(B(SDP_EMPTY), 8); mbar_init(B(SDP_EMPTY + 1), 8); mbar_init(B(PDS_FULL), 8); mbar_init(B(PDS_FULL + 1), 8);
+    mbar_init(B(LOADED), 8); mbar_init(B(PDS_FULL), 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -553,72 +589,61 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tV = tmem + 256, tK = tmem + 256 + DH;   // S^T of buffer bf at tmem + 128 bf, dP^T at + 64
+  const uint32_t tS = tmem, tP = tmem + 128, tV = tmem + 256, tK = tmem + 384;   // P^T overlays S^T, dS^T overlays dP^T
 
   if (warp == 0) {
     if (lane == 0) {
       mbar_expect_tx(B(KV_FULL), 2 * QT);
       for (int hf = 0; hf < NH; ++hf) {
-        tma_load_3d(Ks + hf * 16384, &mapKV, B(KV_FULL), d + head * DH + hf * 64, kb * 128, b);
-        tma_load_3d(Vs + hf * 16384, &mapKV, B(KV_FULL), 2 * d + head * DH + hf * 64, kb * 128, b);
+        tma_load_3d(Ks + hf * 16384, &mapQKV, B(KV_FULL), d + head * DH + hf * 64, kb * 128, b);
+        tma_load_3d(Vs + hf * 16384, &mapQKV, B(KV_FULL), 2 * d + head * DH + hf * 64, kb * 128, b);
       }
       for (int it = 0; it < n; ++it) {
         const int st = it % NS; const uint32_t ph = (it / NS) & 1;
         if (!mbar_wait(B(QG_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) break;
-        mbar_expect_tx(B(QG_FULL + st), 2 * HT);
+        mbar_expect_tx(B(QG_FULL + st), 2 * QT);
         for (int hf = 0; hf < NH; ++hf) {
-          tma_load_3d(Rs + st * 2 * HT + hf * 8192, &mapQ64, B(QG_FULL + st), head * DH + hf * 64, (i0 + it) * 64, b);
-          tma_load_3d(Rs + st * 2 * HT + HT + hf * 8192, &mapG64, B(QG_FULL + st), head * DH + hf * 64, (i0 + it) * 64, b);
+          tma_load_3d(Rs + st * 2 * QT + hf * 16384, &mapQKV, B(QG_FULL + st), head * DH + hf * 64, (kb + it) * 128, b);
+          tma_load_3d(Rs + st * 2 * QT + QT + hf * 16384, &mapG, B(QG_FULL + st), head * DH + hf * 64, (kb + it) * 128, b);
         }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc_s = make_idesc(128, 64, false, false);
+      constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
       constexpr uint32_t idesc_o = make_idesc(128, DH, false, true);
-      auto issue_sdp = [&](int it) -> bool {
-        const int st = it % NS, bf = it & 1;
-        if (!mbar_wait(B(QG_FULL + st), (it / NS) & 1, abort_flag, p.flags)) return false;
-        if (!mbar_wait(B(SDP_EMPTY + bf), ((it >> 1) & 1) ^ 1u, abort_flag, p.flags)) return false;
+      const uint32_t k_lo = klo(Ks), v_lo = klo(Vs);
+      bool ok = mbar_wait(B(KV_FULL), 0, abort_flag, p.flags);
+      for (int it = 0; it < n && ok; ++it) {
+        const int st = it % NS;
+        const uint32_t Qst = Rs + st * 2 * QT, Gst = Qst + QT;
+        if (!mbar_wait(B(QG_FULL + st), (it / NS) & 1, abort_flag, p.flags)) break;
         tc_fence_after();
-        const uint32_t tS = tmem + 128 * bf, tP = tS + 64, Qst = Rs + st * 2 * HT, Gst = Qst + HT;
-        const uint32_t k_lo = klo(Ks), v_lo = klo(Vs), q_lo = klo(Qst), g_lo = klo(Gst);
+        // these overwrite P^T / dS^T of the previous slab: the products that read them were
+        // issued earlier by this thread and the tensor pipe runs its instructions in order
+        const uint32_t q_lo = klo(Qst), g_lo = klo(Gst);
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks)
-          umma_lo(tS, k_lo + kstep<128>(ks), q_lo + kstep<64>(ks), idesc_s, ks > 0);
+          umma_lo(tS, k_lo + kstep<128>(ks), q_lo + kstep<128>(ks), idesc_s, ks > 0);
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks)
-          umma_lo(tP, v_lo + kstep<128>(ks), g_lo + kstep<64>(ks), idesc_s, ks > 0);
-        umma_commit(B(SDP_FULL + bf));
-        return true;
-      };
-      auto issue_out = [&](int it) -> bool {
-        const int st = it % NS, db = it & 1;
-        const uint32_t Qst = Rs + st * 2 * HT, Gst = Qst + HT;
-        if (!mbar_wait(B(PDS_FULL + db), (it >> 1) & 1, abort_flag, p.flags)) return false;
+          umma_lo(tP, v_lo + kstep<128>(ks), g_lo + kstep<128>(ks), idesc_s, ks > 0);
+        umma_commit(B(SDP_FULL));
+        if (!mbar_wait(B(PDS_FULL), (uint32_t)it & 1u, abort_flag, p.flags)) break;
         tc_fence_after();
-        const uint32_t p_lo = klo(Ps + db * PT), ds_lo = klo(Ds + db * PT), gmn_lo = mlo<64>(Gst), qmn_lo = mlo<64>(Qst);
+        const uint32_t gmn_lo = mlo<128>(Gst), qmn_lo = mlo<128>(Qst);
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-          umma_lo(tV, p_lo + kstep<128>(ks), gmn_lo + mstep(ks), idesc_o, (it > 0 || ks > 0));
+        for (int ks = 0; ks < 8; ++ks)
+          umma_ts_lo(tV, tS + 8 * ks, gmn_lo + mstep(ks), idesc_o, (it > 0 || ks > 0));
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-          umma_lo(tK, ds_lo + kstep<128>(ks), qmn_lo + mstep(ks), idesc_o, (it > 0 || ks > 0));
-        umma_commit(B(PDS_EMPTY + db));
+        for (int ks = 0; ks < 8; ++ks)
+          umma_ts_lo(tK, tP + 8 * ks, qmn_lo + mstep(ks), idesc_o, (it > 0 || ks > 0));
         umma_commit(B(QG_EMPTY + st));
         if (it == n - 1) umma_commit(B(OUT_FULL));
-        return true;
-      };
-      bool ok = mbar_wait(B(KV_FULL), 0, abort_flag, p.flags);
-      ok = ok && issue_sdp(0);
-      if (ok && n > 1) ok = issue_sdp(1);
-      for (int it = 0; it < n && ok; ++it) {
-        ok = issue_out(it);
-        if (ok && it + 2 < n) ok = issue_sdp(it + 2);
       }
     }
   } else {
-    const int grp = (warp - 2) >> 2;               // column half of every slab this thread handles
+    const int grp = (warp - 2) >> 2;               // query half of every slab this thread handles
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const int key = kb * 128 + row;
@@ -628,35 +653,51 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapKV, const __grid_const
     const float* drow = p.delta + ((int64_t)b * p.h + head) * S;
     bool ok = true;
     for (int it = 0; it < n && ok; ++it) {
-      const int bf = it & 1;
-      const uint32_t tS = tmem + 128 * bf + lane_off, tP = tS + 64;
-      const int q0 = (i0 + it) * 64;
-      if (!mbar_wait(B(SDP_FULL + bf), (it >> 1) & 1, abort_flag, p.flags)) { ok = false; break; }
-      tc_fence_after();
-      if (!mbar_wait(B(PDS_EMPTY + bf), ((it >> 1) & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+      const uint32_t ph = (uint32_t)it & 1u;
+      // per-query log-sum-exp and delta of this slab, staged once for all row threads
       {
-        const int cc = grp;
-        uint32_t rs[32], rd[32];
-        tmem_ld32(tS + cc * 32, rs);
-        tmem_ld32(tP + cc * 32, rd);
-        tmem_ld_wait();
-        float pv[32], ds[32];
-#pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const int q = q0 + cc * 32 + e;
-          const int qc = q < S ? q : S - 1;
-          float pe = ex2(__uint_as_float(rs[e]) * c - __ldg(lrow + qc) * LOG2E);
-          if (key > q || q >= S) pe = 0.f;
-          pv[e] = pe;
-          ds[e] = pe * (__uint_as_float(rd[e]) - __ldg(drow + qc));
-        }
-        store_row32(Ps + bf * PT, 0, row, cc * 4, pv);
-        store_row32(Ds + bf * PT, 0, row, cc * 4, ds);
+        const int q = (kb + it) * 128 + row;
+        const int qc = q < S ? q : S - 1;
+        row_stat[(ph * 2 + grp) * 128 + row] = grp == 0 ? __ldg(lrow + qc) * LOG2E : __ldg(drow + qc);
       }
+      if (!mbar_wait(B(SDP_FULL), ph, abort_flag, p.flags)) { ok = false; break; }
+      tc_fence_after();
+      uint32_t rs[64], rd[64];
+      tmem_ld32(tS + lane_off + 64 * grp, rs);
+      tmem_ld32(tS + lane_off + 64 * grp + 32, rs + 32);
+      tmem_ld32(tP + lane_off + 64 * grp, rd);
+      tmem_ld32(tP + lane_off + 64 * grp + 32, rd + 32);
+      tmem_ld_wait();
       tc_fence_before();
-      warp_arrive(B(SDP_EMPTY + bf));
-      fence_async_smem();
-      warp_arrive(B(PDS_FULL + bf));
+      // every row thread has its scores in registers (they may now be overwritten in place) and
+      // has staged its share of the slab's row statistics
+      warp_arrive(B(LOADED));
+      if (!mbar_wait(B(LOADED), ph, abort_flag, p.flags)) { ok = false; break; }
+      const float4* sl = reinterpret_cast<const float4*>(row_stat + (ph * 2 + 0) * 128 + 64 * grp);
+      const float4* sd = reinterpret_cast<const float4*>(row_stat + (ph * 2 + 1) * 128 + 64 * grp);
+      const int q0 = (kb + it) * 128 + 64 * grp;
+      const bool diag = (it == 0) || ((kb + it + 1) * 128 > S);
+#pragma unroll
+      for (int e4 = 0; e4 < 16; ++e4) {
+        const float4 l4 = sl[e4], d4 = sd[e4];
+        const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dv[4] = {d4.x, d4.y, d4.z, d4.w};
+        float pe[4], de[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int e = 4 * e4 + u;
+          float x = ex2(fmaf(__uint_as_float(rs[e]), c, -lv[u]));
+          if (diag && (key > q0 + e || q0 + e >= S)) x = 0.f;
+          pe[u] = x;
+          de[u] = x * (__uint_as_float(rd[e]) - dv[u]);
+        }
+        rs[2 * e4] = pack2(pe[0], pe[1]); rs[2 * e4 + 1] = pack2(pe[2], pe[3]);
+        rd[2 * e4] = pack2(de[0], de[1]); rd[2 * e4 + 1] = pack2(de[2], de[3]);
+      }
+      tmem_st32(tS + lane_off + 32 * grp, rs);
+      tmem_st32(tP + lane_off + 32 * grp, rd);
+      tmem_st_wait();
+      tc_fence_before();
+      warp_arrive(B(PDS_FULL));
     }
     if (ok && mbar_wait(B(OUT_FULL), 0, abort_flag, p.flags)) {
       tc_fence_after();
@@ -715,20 +756,19 @@ int fwd_t(const bf16* qkv, bf16* U, float* lse, int B, int S, int h, int* flags,
 template <int DH>
 int bwd_t(const bf16* qkv, const float* lse, const bf16* dU, bf16* dqkv, const float* delta, int B,
           int S, int h, int* flags, cudaStream_t st, const float2* inv_rope) {
-  constexpr int SM_DQ = 2 * 128 * DH * 2 + 2 * 128 * 64 * 2 + 4 * 2 * 64 * DH * 2 + EXTRA;
-  constexpr int SM_KV = 2 * 128 * DH * 2 + 4 * 128 * 64 * 2 + 3 * 2 * 64 * DH * 2 + EXTRA;
+  constexpr int SM_DQ = 7 * 128 * DH * 2 + EXTRA;
+  constexpr int SM_KV = 6 * 128 * DH * 2 + 2 * 2 * 128 * 4 + EXTRA;
   static bool ok = set_smem(attn_dq_tc_kernel<DH>, SM_DQ) && set_smem(attn_dkv_tc_kernel<DH>, SM_KV);
   if (!ok) return -2;
   const int d = h * DH;
-  CUtensorMap mQKV, mG, mQ64, mG64;
-  if (!encode3d(&mQKV, qkv, 3 * d, S, B, 3 * (int64_t)d, 128) || !encode3d(&mG, dU, d, S, B, d, 128) ||
-      !encode3d(&mQ64, qkv, 3 * d, S, B, 3 * (int64_t)d, 64) || !encode3d(&mG64, dU, d, S, B, d, 64))
+  CUtensorMap mQKV, mG;
+  if (!encode3d(&mQKV, qkv, 3 * d, S, B, 3 * (int64_t)d, 128) || !encode3d(&mG, dU, d, S, B, d, 128))
     return -3;
   AttnParams p{}; p.lse = lse; p.delta = delta; p.dqkv = dqkv; p.S = S; p.h = h; p.flags = flags;
   p.inv_rope = inv_rope;
   dim3 grid((S + 127) / 128, h, B);
-  attn_dq_tc_kernel<DH><<<grid, BWD_THREADS, SM_DQ, st>>>(mQKV, mG, mQ64, p);
-  attn_dkv_tc_kernel<DH><<<grid, BWD_THREADS, SM_KV, st>>>(mQKV, mQ64, mG64, p);
+  attn_dq_tc_kernel<DH><<<grid, BWD_THREADS, SM_DQ, st>>>(mQKV, mG, p);
+  attn_dkv_tc_kernel<DH><<<grid, BWD_THREADS, SM_KV, st>>>(mQKV, mG, p);
   return 0;
 }
 
