@@ -4,8 +4,9 @@
 //   forward   one CTA per 128 queries; per 128-key block S = Q K^T lands in TMEM, two groups of
 //             128 softmax threads (one query row each, half of the block's key columns per
 //             group, so row maxima and sums need no shuffles) turn it into bf16 probabilities
-//             in swizzled shared memory, and P V accumulates in TMEM, one accumulator per group,
-//             with lazy online-softmax rescaling; the two partial softmaxes are merged at the end.
+//             written back to TMEM over the scores, and P V (A operand from TMEM) accumulates in
+//             TMEM, one accumulator per group, with lazy online-softmax rescaling; the two
+//             partial softmaxes are merged at the end.
 //   dq        one CTA per 128 queries, 128-key slabs; S = Q K^T and dP = dU V^T in TMEM, the
 //             threads form dS = P (dP - delta) and write it back to TMEM as bf16, from where it is
 //             the A operand of dQ += dS K, which accumulates in TMEM over all slabs (no rescaling
@@ -17,13 +18,17 @@
 // accumulated with atomics, so results are bitwise reproducible.  (Appendix C.1, MHA.)
 //
 // Warp roles: warp 0 issues TMA, warp 1 issues MMAs and owns the TMEM allocation, warps 2-5 and
-// 6-9 are two groups of 128 row threads.  Every mbarrier wait is bounded; on expiry the CTA raises an abort flag,
-// all roles fall through to the common exit, TMEM is released and an error word is set.
+// 6-9 are two groups of 128 row threads; the forward and dq kernels have a second MMA-issuing
+// thread in warp 10 (a thread that issues tcgen05.mma stalls while the tensor pipe is busy, so
+// one thread alone would serialise its barrier waits with the products).  Every mbarrier wait is
+// bounded; on expiry the CTA raises an abort flag, all roles fall through to the common exit,
+// TMEM is released and an error word is set.
 #include "tc_common.cuh"
 
 namespace {
 using namespace tc;
 
+constexpr int DQ_THREADS = 352;   // as BWD_THREADS plus warp 10: second MMA-issuing thread
 constexpr int BWD_THREADS = 320;  // warp 0 TMA, warp 1 MMA, warps 2-5 and 6-9: two row groups, half the slab columns each
 constexpr float LOG2E = 1.4426950408889634f;
 
@@ -125,30 +130,42 @@ __device__ __forceinline__ uint8_t* align1k(uint8_t* p) {
 
 // ------------------------------------------------------------------ forward
 // One CTA per 128 queries, 128-key blocks.  S = Q K^T of block j+1 is issued into the second TMEM
-// buffer while the row threads turn block j into bf16 probabilities in one of two shared-memory
-// tiles.  Two groups of 128 row threads share the work by key columns: group g owns columns
-// [64g, 64g+64) of every block, keeps its own softmax reference and row sum, and its half of
-// P V accumulates in its own TMEM accumulator O_g (two K=64 products per block).  The exponentials
-// (the MUFU unit) and the shared-memory stores of P are the row threads' cost, so halving the
-// columns per thread halves the time a block spends outside the tensor pipe.  At the end the two
+// buffer while the row threads work on block j.  Two groups of 128 row threads share a block by
+// key columns: group g owns columns [64g, 64g+64) of every block, keeps its own softmax
+// reference and row sum, writes its bf16 probabilities back into tensor memory over the first
+// half of the scores they came from, and its half of P V (A operand straight from tensor memory,
+// two K=64 products per block) accumulates in its own accumulator O_g.  At the end the two
 // partial softmaxes are merged exactly: with m = max(m_A, m_B),
 // O = (2^(m_A-m) O_A + 2^(m_B-m) O_B) / (2^(m_A-m) l_A + 2^(m_B-m) l_B).
 // A reference is only raised when a row's block maximum exceeds it by more than 2^8 (stored
 // probabilities then stay below 256); raising it rescales that group's rows of O_g in TMEM.
+// Two threads issue the products (one S, one P V): an issuing thread stalls while the tensor
+// pipe is busy, so with a single one every barrier wait would serialise with the products.
 constexpr float RESCALE_LOG2 = 8.f;
-constexpr int FWD_THREADS = 320;   // warp 0 TMA, warp 1 MMA, warps 2-5 group A, warps 6-9 group B
+constexpr int FWD_THREADS = 352;   // warp 0 TMA, warp 1 S products, warps 2-5 group A, warps 6-9 group B, warp 10 P V products
+
+// A operand from tensor memory (bf16 pairs, one row per lane), B from shared memory
+__device__ __forceinline__ void umma_ts_lo(uint32_t tmem_d, uint32_t tmem_a, uint32_t blo, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n.reg .pred p;\n.reg .b64 db;\nsetp.ne.b32 p, %4, 0;\n"
+      "mov.b64 db, {%2, %5};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n}" ::"r"(tmem_d),
+      "r"(tmem_a), "r"(blo), "r"(idesc), "r"(acc), "r"(DESC_HI)
+      : "memory");
+}
 
 template <int DH>
 __global__ void __launch_bounds__(FWD_THREADS, 1)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams p) {
-  constexpr int NH = DH / 64, QT = 128 * DH * 2, PT = 128 * 128 * 2;
+  constexpr int NH = DH / 64, QT = 128 * DH * 2, NS = 3;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align1k(smem_raw);
-  const uint32_t Qs = smem_u32(smem), Ks = Qs + QT, Vs = Ks + 2 * QT, Ps = Vs + 2 * QT;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 5 * QT + 2 * PT);
-  // P_FULL / P_EMPTY are indexed [group * 2 + stage], PV_DONE by group
-  enum { Q_FULL = 0, K_FULL = 1, K_EMPTY = 3, V_FULL = 5, V_EMPTY = 7, S_FULL = 9, S_EMPTY = 11,
-         P_FULL = 13, P_EMPTY = 17, PV_DONE = 21, ALL_DONE = 23, MERGE = 24, NBAR = 25 };
+  const uint32_t Qs = smem_u32(smem), Ks = Qs + QT, Vs = Ks + NS * QT;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (1 + 2 * NS) * QT);
+  // P_FULL is indexed [group * 2 + buffer], PV_DONE by group
+  enum { Q_FULL = 0, K_FULL = 1, K_EMPTY = K_FULL + NS, V_FULL = K_EMPTY + NS, V_EMPTY = V_FULL + NS,
+         S_FULL = V_EMPTY + NS, S_EMPTY = S_FULL + 2, P_FULL = S_EMPTY + 2, PV_DONE = P_FULL + 4,
+         ALL_DONE = PV_DONE + 2, MERGE, NBAR };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   // (reference, sum) of each row and group; overlays the Q tile once every MMA has completed
@@ -162,7 +179,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
-    for (int i = 0; i < 2; ++i) mbar_init(B(S_EMPTY + i), 8);
     for (int i = 0; i < 4; ++i) mbar_init(B(P_FULL + i), 4);
     mbar_init(B(MERGE), 8);
     *abort_flag = 0;
@@ -174,7 +190,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tS = tmem, tO = tmem + 256;   // O_g at tO + g * DH
+  const uint32_t tS = tmem, tO = tmem + 256;   // S buffer s at tS + 128 s; O_g at tO + g * DH
 
   if (warp == 0) {
     if (lane == 0) {
@@ -182,7 +198,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
       for (int hf = 0; hf < NH; ++hf)
         tma_load_3d(Qs + hf * 16384, &mapQKV, B(Q_FULL), head * DH + hf * 64, qb * 128, b);
       for (int j = 0; j < n; ++j) {
-        const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
+        const int st = j % NS; const uint32_t ph = (j / NS) & 1;
         if (!mbar_wait(B(K_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) break;
         mbar_expect_tx(B(K_FULL + st), QT);
         for (int hf = 0; hf < NH; ++hf)
@@ -196,40 +212,42 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
-      constexpr uint32_t idesc_o = make_idesc(128, DH, false, true);
       const uint32_t q_lo = klo(Qs);
       bool ok = mbar_wait(B(Q_FULL), 0, abort_flag, p.flags);
-      auto issue_s = [&](int j) -> bool {
-        const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
-        if (!mbar_wait(B(K_FULL + st), ph, abort_flag, p.flags)) return false;
-        if (!mbar_wait(B(S_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) return false;
+      for (int j = 0; j < n && ok; ++j) {
+        const int st = j % NS, sb = j & 1;
+        if (!mbar_wait(B(K_FULL + st), (j / NS) & 1, abort_flag, p.flags)) break;
+        // buffer sb still holds the probabilities of block j-2 until their P V products are done
+        if (!mbar_wait(B(S_EMPTY + sb), ((j >> 1) & 1) ^ 1u, abort_flag, p.flags)) break;
         tc_fence_after();
         const uint32_t k_lo = klo(Ks + st * QT);
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks)
-          umma_lo(tS + st * 128, q_lo + kstep<128>(ks), k_lo + kstep<128>(ks), idesc_s, ks > 0);
-        umma_commit(B(S_FULL + st));
+          umma_lo(tS + sb * 128, q_lo + kstep<128>(ks), k_lo + kstep<128>(ks), idesc_s, ks > 0);
+        umma_commit(B(S_FULL + sb));
         umma_commit(B(K_EMPTY + st));
-        return true;
-      };
-      if (ok) ok = issue_s(0);
+      }
+    }
+  } else if (warp == 10) {
+    if (lane == 0) {
+      constexpr uint32_t idesc_o = make_idesc(128, DH, false, true);
+      bool ok = true;
       for (int j = 0; j < n && ok; ++j) {
-        if (j + 1 < n) { ok = issue_s(j + 1); if (!ok) break; }
-        const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
-        const uint32_t p_lo = klo(Ps + st * PT), v_lo = mlo<128>(Vs + st * QT);
+        const int st = j % NS, sb = j & 1; const uint32_t ph = (j >> 1) & 1;
+        const uint32_t v_lo = mlo<128>(Vs + st * QT);
+        if (!mbar_wait(B(V_FULL + st), (j / NS) & 1, abort_flag, p.flags)) break;
 #pragma unroll
         for (int g = 0; g < 2; ++g) {
-          if (!mbar_wait(B(P_FULL + g * 2 + st), ph, abort_flag, p.flags)) { ok = false; break; }
-          if (g == 0 && !mbar_wait(B(V_FULL + st), ph, abort_flag, p.flags)) { ok = false; break; }
+          if (!mbar_wait(B(P_FULL + g * 2 + sb), ph, abort_flag, p.flags)) { ok = false; break; }
           tc_fence_after();
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)
-            umma_lo(tO + g * DH, p_lo + kstep<128>(4 * g + ks), v_lo + mstep(4 * g + ks), idesc_o,
-                    (j > 0 || ks > 0));
+            umma_ts_lo(tO + g * DH, tS + sb * 128 + 64 * g + 8 * ks, v_lo + mstep(4 * g + ks), idesc_o,
+                       (j > 0 || ks > 0));
           umma_commit(B(PV_DONE + g));
-          umma_commit(B(P_EMPTY + g * 2 + st));
         }
         if (!ok) break;
+        umma_commit(B(S_EMPTY + sb));
         umma_commit(B(V_EMPTY + st));
       }
       if (ok) umma_commit(B(ALL_DONE));
@@ -245,15 +263,14 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     for (int j = 0; j < n && ok; ++j) {
-      const int st = j & 1; const uint32_t ph = (j >> 1) & 1;
-      if (!mbar_wait(B(S_FULL + st), ph, abort_flag, p.flags)) { ok = false; break; }
+      const int sb = j & 1; const uint32_t ph = (j >> 1) & 1;
+      const uint32_t tSg = tS + lane_off + sb * 128 + g * 64;
+      if (!mbar_wait(B(S_FULL + sb), ph, abort_flag, p.flags)) { ok = false; break; }
       tc_fence_after();
       uint32_t r[64];
-      tmem_ld32(tS + lane_off + st * 128 + g * 64, r);
-      tmem_ld32(tS + lane_off + st * 128 + g * 64 + 32, r + 32);
+      tmem_ld32(tSg, r);
+      tmem_ld32(tSg + 32, r + 32);
       tmem_ld_wait();
-      tc_fence_before();
-      warp_arrive(B(S_EMPTY + st));               // the scores are in registers: free the buffer
       const int col0 = j * 128 + g * 64;
       const bool diag = (j == qb) || ((j + 1) * 128 > S);
       // eight independent partial maxima / sums: a single warp per scheduler cannot hide the
@@ -279,10 +296,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
         const float new_ref = need ? m_blk : m_ref;
         const float factor = need ? ex2(m_ref - new_ref) : 1.f;
         if (j > 0) {
-          // O_g must be complete up to block j-1 before its rows are rescaled in place.  S of
-          // block j was issued after both P V products of block j-2, so that phase has already
-          // completed and the parity test cannot alias an older one.
-          if (!mbar_wait(B(PV_DONE + g), (j - 1) & 1, abort_flag, p.flags)) { ok = false; break; }
+          // O_g must be complete up to block j-1 before its rows are rescaled in place
+          if (!mbar_wait(B(PV_DONE + g), (uint32_t)(j - 1) & 1u, abort_flag, p.flags)) { ok = false; break; }
           tc_fence_after();
 #pragma unroll 1
           for (int cc = 0; cc < DH / 32; ++cc) {
@@ -293,7 +308,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
             for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
             tmem_st32(tOg + cc * 32, o);
           }
-          tmem_st_wait();
         }
         l *= factor;
         m_ref = new_ref;
@@ -301,34 +315,34 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
       float sum8[8];
 #pragma unroll
       for (int q = 0; q < 8; ++q) sum8[q] = 0.f;
-      if (!mbar_wait(B(P_EMPTY + g * 2 + st), ph ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+      // a group whose columns are all masked so far still has m_ref = -inf; the selects below
+      // discard whatever the exponential made of that
+      if (!diag) {
 #pragma unroll
-      for (int cc = 0; cc < 2; ++cc) {
-        float pv[32];
-        if (!diag) {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            pv[e] = ex2(fmaf(__uint_as_float(r[cc * 32 + e]), c, -m_ref));
-            sum8[e & 7] += pv[e];
-          }
-        } else {
-          // a group whose columns are all masked so far still has m_ref = -inf; the select
-          // below discards whatever the exponential made of that
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            const int col = col0 + cc * 32 + e;
-            float pe = ex2(fmaf(__uint_as_float(r[cc * 32 + e]), c, -m_ref));
-            if (col > grow || col >= S) pe = 0.f;
-            pv[e] = pe;
-            sum8[e & 7] += pe;
-          }
+        for (int e = 0; e < 64; e += 2) {
+          const float p0 = ex2(fmaf(__uint_as_float(r[e]), c, -m_ref));
+          const float p1 = ex2(fmaf(__uint_as_float(r[e + 1]), c, -m_ref));
+          sum8[e & 7] += p0; sum8[(e + 1) & 7] += p1;
+          r[e >> 1] = pack2(p0, p1);
         }
-        store_row32(Ps + st * PT + g * 16384, 16384, row, cc * 4, pv);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 64; e += 2) {
+          const int col = col0 + e;
+          float p0 = ex2(fmaf(__uint_as_float(r[e]), c, -m_ref));
+          float p1 = ex2(fmaf(__uint_as_float(r[e + 1]), c, -m_ref));
+          if (col > grow || col >= S) p0 = 0.f;
+          if (col + 1 > grow || col + 1 >= S) p1 = 0.f;
+          sum8[e & 7] += p0; sum8[(e + 1) & 7] += p1;
+          r[e >> 1] = pack2(p0, p1);
+        }
       }
       l += ((sum8[0] + sum8[1]) + (sum8[2] + sum8[3])) + ((sum8[4] + sum8[5]) + (sum8[6] + sum8[7]));
+      // the probabilities replace the first half of this thread's own scores
+      tmem_st32(tSg, r);
+      tmem_st_wait();
       tc_fence_before();
-      fence_async_smem();
-      warp_arrive(B(P_FULL + g * 2 + st));
+      warp_arrive(B(P_FULL + g * 2 + sb));
     }
     // every MMA has completed: the Q tile is free to carry the groups' (reference, sum) pairs
     if (ok && mbar_wait(B(ALL_DONE), 0, abort_flag, p.flags)) {
@@ -368,16 +382,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
 }
 
 // ------------------------------------------------------------------ backward: dq
-// A operand from tensor memory (bf16 pairs, one row per lane), B from shared memory
-__device__ __forceinline__ void umma_ts_lo(uint32_t tmem_d, uint32_t tmem_a, uint32_t blo, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n.reg .pred p;\n.reg .b64 db;\nsetp.ne.b32 p, %4, 0;\n"
-      "mov.b64 db, {%2, %5};\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n}" ::"r"(tmem_d),
-      "r"(tmem_a), "r"(blo), "r"(idesc), "r"(acc), "r"(DESC_HI)
-      : "memory");
-}
-
 // One CTA owns 128 queries (Q and dU tiles resident) and streams 128-key slabs of K and V through
 // a two-deep TMA ring.  S = Q K^T and dP = dU V^T of a slab land in tensor memory; the 256 row
 // threads (one query row each, half of the slab's key columns per group) pull them into
@@ -386,7 +390,7 @@ __device__ __forceinline__ void umma_ts_lo(uint32_t tmem_d, uint32_t tmem_a, uin
 // dQ += dS K.  The MMA-issuing thread is the scarce resource of this kernel (its waits, commits
 // and instruction issue are latency-bound), hence few, wide instructions: 24 per 128 keys.
 template <int DH>
-__global__ void __launch_bounds__(BWD_THREADS, 1)
+__global__ void __launch_bounds__(DQ_THREADS, 1)
 attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapG,
                   const AttnParams p) {
   constexpr int NH = DH / 64, QT = 128 * DH * 2, NK = 3, NV = 2;   // K lives until its slab's dQ product, V only until dP
@@ -441,7 +445,6 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
-      constexpr uint32_t idesc_q = make_idesc(128, DH, false, true);
       const uint32_t q_lo = klo(Qs), g_lo = klo(Gs);
       auto issue_sdp = [&](int it) -> bool {
         const int sk = it % NK, sv = it % NV;
@@ -460,9 +463,20 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
         umma_commit(B(V_EMPTY + sv));
         return true;
       };
-      auto issue_dq = [&](int it) -> bool {
+      bool ok = mbar_wait(B(Q_FULL), 0, abort_flag, p.flags);
+      for (int it = 0; it < n && ok; ++it) ok = issue_sdp(it);
+    }
+  } else if (warp == 10) {
+    // second issuing thread: its waits overlap the first thread's instructions and vice versa
+    // (an issuing thread stalls while the tensor pipe is busy, so one thread alone would
+    // serialise every wait with the products)
+    if (lane == 0) {
+      constexpr uint32_t idesc_q = make_idesc(128, DH, false, true);
+      bool ok = true;
+      for (int it = 0; it < n && ok; ++it) {
         const int sk = it % NK, db = it & 1;
-        if (!mbar_wait(B(DS_FULL + db), (it >> 1) & 1, abort_flag, p.flags)) return false;
+        if (!mbar_wait(B(K_FULL + sk), (it / NK) & 1, abort_flag, p.flags)) break;
+        if (!mbar_wait(B(DS_FULL + db), (it >> 1) & 1, abort_flag, p.flags)) break;
         tc_fence_after();
         const uint32_t kmn_lo = mlo<128>(Kr + sk * QT);
 #pragma unroll
@@ -471,13 +485,6 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
         umma_commit(B(DS_EMPTY + db));
         umma_commit(B(K_EMPTY + sk));
         if (it == n - 1) umma_commit(B(DQ_FULL));
-        return true;
-      };
-      bool ok = mbar_wait(B(Q_FULL), 0, abort_flag, p.flags);
-      ok = ok && issue_sdp(0);
-      for (int it = 0; it < n && ok; ++it) {
-        if (it + 1 < n) ok = issue_sdp(it + 1);
-        ok = ok && issue_dq(it);
       }
     }
   } else {
@@ -742,7 +749,7 @@ constexpr int EXTRA = 1024 + 256;   // alignment slack + barriers
 
 template <int DH>
 int fwd_t(const bf16* qkv, bf16* U, float* lse, int B, int S, int h, int* flags, cudaStream_t st) {
-  constexpr int SM = 5 * 128 * DH * 2 + 2 * 128 * 128 * 2 + EXTRA;
+  constexpr int SM = 7 * 128 * DH * 2 + EXTRA;
   static bool ok = set_smem(attn_fwd_tc_kernel<DH>, SM);
   if (!ok) return -2;
   CUtensorMap m;
@@ -767,7 +774,7 @@ int bwd_t(const bf16* qkv, const float* lse, const bf16* dU, bf16* dqkv, const f
   AttnParams p{}; p.lse = lse; p.delta = delta; p.dqkv = dqkv; p.S = S; p.h = h; p.flags = flags;
   p.inv_rope = inv_rope;
   dim3 grid((S + 127) / 128, h, B);
-  attn_dq_tc_kernel<DH><<<grid, BWD_THREADS, SM_DQ, st>>>(mQKV, mG, p);
+  attn_dq_tc_kernel<DH><<<grid, DQ_THREADS, SM_DQ, st>>>(mQKV, mG, p);
   attn_dkv_tc_kernel<DH><<<grid, BWD_THREADS, SM_KV, st>>>(mQKV, mG, p);
   return 0;
 }
