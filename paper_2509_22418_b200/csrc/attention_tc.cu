@@ -1,7 +1,7 @@
 // Fused causal attention on the 5th-generation tensor cores (tcgen05.mma, accumulators in
 // tensor memory, operands brought in by TMA), head sizes 64 and 128.
 //
-//   forward   one CTA per 128 queries; per 128-key block S = Q K^T lands in TMEM, two groups of
+//   forward   128 queries per work item; per 128-key block S = Q K^T lands in TMEM, two groups of
 //             128 softmax threads (one query row each, half of the block's key columns per
 //             group, so row maxima and sums need no shuffles) turn it into bf16 probabilities
 //             written back to TMEM over the scores, and P V (A operand from TMEM) accumulates in
@@ -14,11 +14,14 @@
 //   dk, dv    one CTA per 128 keys, 128-query slabs; the transposed products S^T = K Q^T,
 //             dP^T = V dU^T; P^T and dS^T overwrite them in TMEM as bf16 and feed dV += P^T dU and
 //             dK += dS^T Q, which accumulate in TMEM.
+// The forward kernel is persistent: one CTA per SM walks a balanced list of (sequence, head,
+// query block) items, so set-up, the first loads and the output drain of an item overlap with
+// the products of its neighbours.
 // The two backward kernels recompute P from q, k and the saved log-sum-exp; nothing is
 // accumulated with atomics, so results are bitwise reproducible.  (Appendix C.1, MHA.)
 //
 // Warp roles: warp 0 issues TMA, warp 1 issues MMAs and owns the TMEM allocation, warps 2-5 and
-// 6-9 are two groups of 128 row threads; the forward and dq kernels have a second MMA-issuing
+// 6-9 are two groups of 128 row threads; every kernel has a second MMA-issuing
 // thread in warp 10 (a thread that issues tcgen05.mma stalls while the tensor pipe is busy, so
 // one thread alone would serialise its barrier waits with the products).  Every mbarrier wait is
 // bounded; on expiry the CTA raises an abort flag, all roles fall through to the common exit,
@@ -92,7 +95,7 @@ __device__ __forceinline__ void warp_arrive(uint32_t bar) {
 struct AttnParams {
   const float* lse; const float* delta;
   bf16* U; float* lse_out; bf16* dqkv;
-  int S, h; int* flags;
+  int S, h, B; int* flags;
   const float2* inv_rope;   // (cos, sin) table [S][d_h/2]: rotate dq, dk by -angle on the way out (or null)
 };
 
@@ -154,6 +157,24 @@ __device__ __forceinline__ void umma_ts_lo(uint32_t tmem_d, uint32_t tmem_a, uin
       : "memory");
 }
 
+// Work items (128 queries of one head of one sequence) are ordered heavy first - the last query
+// block of every (sequence, head), then the one before, ... - and dealt to the resident CTAs in
+// boustrophedon order, so every CTA gets a near-equal number of key blocks.  A CTA walks its items
+// without leaving: barriers, tensor memory and the K/V rings carry over, and the next item's Q
+// and first K/V tiles arrive while the current item's last blocks and its output drain.
+struct WorkItem { int qb, head, b; };
+__device__ __forceinline__ bool work_item(int k, int n_batch, int h, int nq, WorkItem& w) {
+  const int G = gridDim.x, cta = blockIdx.x;
+  const int t = k * G + ((k & 1) ? (G - 1 - cta) : cta);
+  const int hb = h * n_batch;
+  if (t >= nq * hb) return false;
+  w.qb = nq - 1 - t / hb;
+  const int rem = t % hb;
+  w.head = rem % h; w.b = rem / h;
+  return true;
+}
+
+constexpr int FWD_ALIGN_SLACK = 768;   // the full 1 KB would put the 128-wide head over the 227 KB limit
 template <int DH>
 __global__ void __launch_bounds__(FWD_THREADS, 1)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams p) {
@@ -161,26 +182,29 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align1k(smem_raw);
   const uint32_t Qs = smem_u32(smem), Ks = Qs + QT, Vs = Ks + NS * QT;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (1 + 2 * NS) * QT);
+  float2* exch = reinterpret_cast<float2*>(smem + (1 + 2 * NS) * QT);   // (reference, sum) of each row and group
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (1 + 2 * NS) * QT + 2 * 128 * 8);
   // P_FULL is indexed [group * 2 + buffer], PV_DONE by group
-  enum { Q_FULL = 0, K_FULL = 1, K_EMPTY = K_FULL + NS, V_FULL = K_EMPTY + NS, V_EMPTY = V_FULL + NS,
+  enum { Q_FULL = 0, Q_EMPTY, K_FULL, K_EMPTY = K_FULL + NS, V_FULL = K_EMPTY + NS, V_EMPTY = V_FULL + NS,
          S_FULL = V_EMPTY + NS, S_EMPTY = S_FULL + 2, P_FULL = S_EMPTY + 2, PV_DONE = P_FULL + 4,
-         ALL_DONE = PV_DONE + 2, MERGE, NBAR };
+         ALL_DONE = PV_DONE + 2, MERGE, O_EMPTY, NBAR };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  // (reference, sum) of each row and group; overlays the Q tile once every MMA has completed
-  float2* exch = reinterpret_cast<float2*>(smem);
   const uint32_t bar0 = smem_u32(bars);
   auto B = [&](int i) { return bar0 + 8u * i; };
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int qb = gridDim.x - 1 - blockIdx.x, head = blockIdx.y, b = blockIdx.z;
-  const int d = p.h * DH, S = p.S;
-  const int n = qb + 1;
+  const int d = p.h * DH, S = p.S, nq = (S + 127) / 128;
+  // the launch provides FWD_ALIGN_SLACK bytes for the 1 KB alignment of the tiles
+  if (smem - smem_raw > FWD_ALIGN_SLACK) {
+    if (threadIdx.x == 0 && p.flags) atomicExch(p.flags + PPU_FLAG_TIMEOUT, 1);
+    return;
+  }
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
     for (int i = 0; i < 4; ++i) mbar_init(B(P_FULL + i), 4);
     mbar_init(B(MERGE), 8);
+    mbar_init(B(O_EMPTY), 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -191,165 +215,184 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const uint32_t tS = tmem, tO = tmem + 256;   // S buffer s at tS + 128 s; O_g at tO + g * DH
+  // c counts the key blocks this CTA has gone through (every role keeps its own copy): it selects
+  // ring stages, score buffers and barrier phases across items
 
   if (warp == 0) {
     if (lane == 0) {
-      mbar_expect_tx(B(Q_FULL), QT);
-      for (int hf = 0; hf < NH; ++hf)
-        tma_load_3d(Qs + hf * 16384, &mapQKV, B(Q_FULL), head * DH + hf * 64, qb * 128, b);
-      for (int j = 0; j < n; ++j) {
-        const int st = j % NS; const uint32_t ph = (j / NS) & 1;
-        if (!mbar_wait(B(K_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) break;
-        mbar_expect_tx(B(K_FULL + st), QT);
+      WorkItem w; uint32_t c = 0; bool ok = true;
+      for (int k = 0; ok && work_item(k, p.B, p.h, nq, w); ++k) {
+        // the Q tile is free once the previous item's last S product is done
+        if (k > 0 && !mbar_wait(B(Q_EMPTY), (uint32_t)(k - 1) & 1u, abort_flag, p.flags)) break;
+        mbar_expect_tx(B(Q_FULL), QT);
         for (int hf = 0; hf < NH; ++hf)
-          tma_load_3d(Ks + st * QT + hf * 16384, &mapQKV, B(K_FULL + st), d + head * DH + hf * 64, j * 128, b);
-        if (!mbar_wait(B(V_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) break;
-        mbar_expect_tx(B(V_FULL + st), QT);
-        for (int hf = 0; hf < NH; ++hf)
-          tma_load_3d(Vs + st * QT + hf * 16384, &mapQKV, B(V_FULL + st), 2 * d + head * DH + hf * 64, j * 128, b);
+          tma_load_3d(Qs + hf * 16384, &mapQKV, B(Q_FULL), w.head * DH + hf * 64, w.qb * 128, w.b);
+        for (int j = 0; j <= w.qb; ++j, ++c) {
+          const int st = c % NS; const uint32_t ph = (c / NS) & 1;
+          if (!mbar_wait(B(K_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+          mbar_expect_tx(B(K_FULL + st), QT);
+          for (int hf = 0; hf < NH; ++hf)
+            tma_load_3d(Ks + st * QT + hf * 16384, &mapQKV, B(K_FULL + st), d + w.head * DH + hf * 64, j * 128, w.b);
+          if (!mbar_wait(B(V_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+          mbar_expect_tx(B(V_FULL + st), QT);
+          for (int hf = 0; hf < NH; ++hf)
+            tma_load_3d(Vs + st * QT + hf * 16384, &mapQKV, B(V_FULL + st), 2 * d + w.head * DH + hf * 64, j * 128, w.b);
+        }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
       const uint32_t q_lo = klo(Qs);
-      bool ok = mbar_wait(B(Q_FULL), 0, abort_flag, p.flags);
-      for (int j = 0; j < n && ok; ++j) {
-        const int st = j % NS, sb = j & 1;
-        if (!mbar_wait(B(K_FULL + st), (j / NS) & 1, abort_flag, p.flags)) break;
-        // buffer sb still holds the probabilities of block j-2 until their P V products are done
-        if (!mbar_wait(B(S_EMPTY + sb), ((j >> 1) & 1) ^ 1u, abort_flag, p.flags)) break;
-        tc_fence_after();
-        const uint32_t k_lo = klo(Ks + st * QT);
+      WorkItem w; uint32_t c = 0; bool ok = true;
+      for (int k = 0; ok && work_item(k, p.B, p.h, nq, w); ++k) {
+        if (!mbar_wait(B(Q_FULL), (uint32_t)k & 1u, abort_flag, p.flags)) break;
+        for (int j = 0; j <= w.qb; ++j, ++c) {
+          const int st = c % NS, sb = c & 1;
+          if (!mbar_wait(B(K_FULL + st), (c / NS) & 1, abort_flag, p.flags)) { ok = false; break; }
+          // buffer sb still holds the probabilities of two blocks ago until their P V products are done
+          if (!mbar_wait(B(S_EMPTY + sb), ((c >> 1) & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t k_lo = klo(Ks + st * QT);
 #pragma unroll
-        for (int ks = 0; ks < DH / 16; ++ks)
-          umma_lo(tS + sb * 128, q_lo + kstep<128>(ks), k_lo + kstep<128>(ks), idesc_s, ks > 0);
-        umma_commit(B(S_FULL + sb));
-        umma_commit(B(K_EMPTY + st));
+          for (int ks = 0; ks < DH / 16; ++ks)
+            umma_lo(tS + sb * 128, q_lo + kstep<128>(ks), k_lo + kstep<128>(ks), idesc_s, ks > 0);
+          umma_commit(B(S_FULL + sb));
+          umma_commit(B(K_EMPTY + st));
+        }
+        if (ok) umma_commit(B(Q_EMPTY));
       }
     }
   } else if (warp == 10) {
     if (lane == 0) {
       constexpr uint32_t idesc_o = make_idesc(128, DH, false, true);
-      bool ok = true;
-      for (int j = 0; j < n && ok; ++j) {
-        const int st = j % NS, sb = j & 1; const uint32_t ph = (j >> 1) & 1;
-        const uint32_t v_lo = mlo<128>(Vs + st * QT);
-        if (!mbar_wait(B(V_FULL + st), (j / NS) & 1, abort_flag, p.flags)) break;
+      WorkItem w; uint32_t c = 0; bool ok = true;
+      for (int k = 0; ok && work_item(k, p.B, p.h, nq, w); ++k) {
+        // the accumulators are free once the row threads have drained the previous item's output
+        if (k > 0 && !mbar_wait(B(O_EMPTY), (uint32_t)(k - 1) & 1u, abort_flag, p.flags)) break;
+        for (int j = 0; j <= w.qb && ok; ++j, ++c) {
+          const int st = c % NS, sb = c & 1; const uint32_t ph = (c >> 1) & 1;
+          const uint32_t v_lo = mlo<128>(Vs + st * QT);
+          if (!mbar_wait(B(V_FULL + st), (c / NS) & 1, abort_flag, p.flags)) { ok = false; break; }
 #pragma unroll
-        for (int g = 0; g < 2; ++g) {
-          if (!mbar_wait(B(P_FULL + g * 2 + sb), ph, abort_flag, p.flags)) { ok = false; break; }
-          tc_fence_after();
+          for (int g = 0; g < 2; ++g) {
+            if (!mbar_wait(B(P_FULL + g * 2 + sb), ph, abort_flag, p.flags)) { ok = false; break; }
+            tc_fence_after();
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
-            umma_ts_lo(tO + g * DH, tS + sb * 128 + 64 * g + 8 * ks, v_lo + mstep(4 * g + ks), idesc_o,
-                       (j > 0 || ks > 0));
-          umma_commit(B(PV_DONE + g));
+            for (int ks = 0; ks < 4; ++ks)
+              umma_ts_lo(tO + g * DH, tS + sb * 128 + 64 * g + 8 * ks, v_lo + mstep(4 * g + ks), idesc_o,
+                         (j > 0 || ks > 0));
+            umma_commit(B(PV_DONE + g));
+          }
+          if (!ok) break;
+          umma_commit(B(S_EMPTY + sb));
+          umma_commit(B(V_EMPTY + st));
         }
-        if (!ok) break;
-        umma_commit(B(S_EMPTY + sb));
-        umma_commit(B(V_EMPTY + st));
+        if (ok) umma_commit(B(ALL_DONE));
       }
-      if (ok) umma_commit(B(ALL_DONE));
     }
   } else {
     const int g = (warp - 2) >> 2;                // column group
     const int quarter = warp & 3;                 // TMEM lane quarter this warp may access
     const int row = quarter * 32 + lane;
-    const int grow = qb * 128 + row;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     const uint32_t tOg = tO + g * DH + lane_off;
     const float c = rsqrtf((float)DH) * LOG2E;
-    float m_ref = -INFINITY, l = 0.f;
-    bool ok = true;
-    for (int j = 0; j < n && ok; ++j) {
-      const int sb = j & 1; const uint32_t ph = (j >> 1) & 1;
-      const uint32_t tSg = tS + lane_off + sb * 128 + g * 64;
-      if (!mbar_wait(B(S_FULL + sb), ph, abort_flag, p.flags)) { ok = false; break; }
-      tc_fence_after();
-      uint32_t r[64];
-      tmem_ld32(tSg, r);
-      tmem_ld32(tSg + 32, r + 32);
-      tmem_ld_wait();
-      const int col0 = j * 128 + g * 64;
-      const bool diag = (j == qb) || ((j + 1) * 128 > S);
-      // eight independent partial maxima / sums: a single warp per scheduler cannot hide the
-      // latency of one long dependent chain
-      float mx8[8];
+    WorkItem w; uint32_t cb = 0; bool ok = true;
+    for (int k = 0; ok && work_item(k, p.B, p.h, nq, w); ++k) {
+      const int qb = w.qb, grow = qb * 128 + row;
+      float m_ref = -INFINITY, l = 0.f;
+      for (int j = 0; j <= qb && ok; ++j, ++cb) {
+        const int sb = cb & 1; const uint32_t ph = (cb >> 1) & 1;
+        const uint32_t tSg = tS + lane_off + sb * 128 + g * 64;
+        if (!mbar_wait(B(S_FULL + sb), ph, abort_flag, p.flags)) { ok = false; break; }
+        tc_fence_after();
+        uint32_t r[64];
+        tmem_ld32(tSg, r);
+        tmem_ld32(tSg + 32, r + 32);
+        tmem_ld_wait();
+        const int col0 = j * 128 + g * 64;
+        const bool diag = (j == qb) || ((j + 1) * 128 > S);
+        // eight independent partial maxima / sums: a single warp per scheduler cannot hide the
+        // latency of one long dependent chain
+        float mx8[8];
 #pragma unroll
-      for (int q = 0; q < 8; ++q) mx8[q] = -INFINITY;
-      if (!diag) {
+        for (int q = 0; q < 8; ++q) mx8[q] = -INFINITY;
+        if (!diag) {
 #pragma unroll
-        for (int e = 0; e < 64; ++e) mx8[e & 7] = fmaxf(mx8[e & 7], __uint_as_float(r[e]));
-      } else {
+          for (int e = 0; e < 64; ++e) mx8[e & 7] = fmaxf(mx8[e & 7], __uint_as_float(r[e]));
+        } else {
 #pragma unroll
-        for (int e = 0; e < 64; ++e) {
-          const int col = col0 + e;
-          if (col <= grow && col < S) mx8[e & 7] = fmaxf(mx8[e & 7], __uint_as_float(r[e]));
-        }
-      }
-      const float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
-                             fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
-      const float m_blk = mx * c;
-      const bool need = m_blk > m_ref + RESCALE_LOG2;
-      if (__any_sync(0xffffffffu, need)) {
-        const float new_ref = need ? m_blk : m_ref;
-        const float factor = need ? ex2(m_ref - new_ref) : 1.f;
-        if (j > 0) {
-          // O_g must be complete up to block j-1 before its rows are rescaled in place
-          if (!mbar_wait(B(PV_DONE + g), (uint32_t)(j - 1) & 1u, abort_flag, p.flags)) { ok = false; break; }
-          tc_fence_after();
-#pragma unroll 1
-          for (int cc = 0; cc < DH / 32; ++cc) {
-            uint32_t o[32];
-            tmem_ld32(tOg + cc * 32, o);
-            tmem_ld_wait();
-#pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
-            tmem_st32(tOg + cc * 32, o);
+          for (int e = 0; e < 64; ++e) {
+            const int col = col0 + e;
+            if (col <= grow && col < S) mx8[e & 7] = fmaxf(mx8[e & 7], __uint_as_float(r[e]));
           }
         }
-        l *= factor;
-        m_ref = new_ref;
-      }
-      float sum8[8];
+        const float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
+                               fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
+        const float m_blk = mx * c;
+        const bool need = m_blk > m_ref + RESCALE_LOG2;
+        if (__any_sync(0xffffffffu, need)) {
+          const float new_ref = need ? m_blk : m_ref;
+          const float factor = need ? ex2(m_ref - new_ref) : 1.f;
+          if (j > 0) {
+            // O_g must be complete up to the previous block before its rows are rescaled in place
+            if (!mbar_wait(B(PV_DONE + g), (cb - 1) & 1u, abort_flag, p.flags)) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll 1
+            for (int cc = 0; cc < DH / 32; ++cc) {
+              uint32_t o[32];
+              tmem_ld32(tOg + cc * 32, o);
+              tmem_ld_wait();
 #pragma unroll
-      for (int q = 0; q < 8; ++q) sum8[q] = 0.f;
-      // a group whose columns are all masked so far still has m_ref = -inf; the selects below
-      // discard whatever the exponential made of that
-      if (!diag) {
-#pragma unroll
-        for (int e = 0; e < 64; e += 2) {
-          const float p0 = ex2(fmaf(__uint_as_float(r[e]), c, -m_ref));
-          const float p1 = ex2(fmaf(__uint_as_float(r[e + 1]), c, -m_ref));
-          sum8[e & 7] += p0; sum8[(e + 1) & 7] += p1;
-          r[e >> 1] = pack2(p0, p1);
+              for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
+              tmem_st32(tOg + cc * 32, o);
+            }
+          }
+          l *= factor;
+          m_ref = new_ref;
         }
-      } else {
+        float sum8[8];
 #pragma unroll
-        for (int e = 0; e < 64; e += 2) {
-          const int col = col0 + e;
-          float p0 = ex2(fmaf(__uint_as_float(r[e]), c, -m_ref));
-          float p1 = ex2(fmaf(__uint_as_float(r[e + 1]), c, -m_ref));
-          if (col > grow || col >= S) p0 = 0.f;
-          if (col + 1 > grow || col + 1 >= S) p1 = 0.f;
-          sum8[e & 7] += p0; sum8[(e + 1) & 7] += p1;
-          r[e >> 1] = pack2(p0, p1);
+        for (int q = 0; q < 8; ++q) sum8[q] = 0.f;
+        // a group whose columns are all masked so far still has m_ref = -inf; the selects below
+        // discard whatever the exponential made of that
+        if (!diag) {
+#pragma unroll
+          for (int e = 0; e < 64; e += 2) {
+            const float p0 = ex2(fmaf(__uint_as_float(r[e]), c, -m_ref));
+            const float p1 = ex2(fmaf(__uint_as_float(r[e + 1]), c, -m_ref));
+            sum8[e & 7] += p0; sum8[(e + 1) & 7] += p1;
+            r[e >> 1] = pack2(p0, p1);
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 64; e += 2) {
+            const int col = col0 + e;
+            float p0 = ex2(fmaf(__uint_as_float(r[e]), c, -m_ref));
+            float p1 = ex2(fmaf(__uint_as_float(r[e + 1]), c, -m_ref));
+            if (col > grow || col >= S) p0 = 0.f;
+            if (col + 1 > grow || col + 1 >= S) p1 = 0.f;
+            sum8[e & 7] += p0; sum8[(e + 1) & 7] += p1;
+            r[e >> 1] = pack2(p0, p1);
+          }
         }
+        l += ((sum8[0] + sum8[1]) + (sum8[2] + sum8[3])) + ((sum8[4] + sum8[5]) + (sum8[6] + sum8[7]));
+        // the probabilities replace the first half of this thread's own scores
+        tmem_st32(tSg, r);
+        tmem_st_wait();
+        tc_fence_before();
+        warp_arrive(B(P_FULL + g * 2 + sb));
       }
-      l += ((sum8[0] + sum8[1]) + (sum8[2] + sum8[3])) + ((sum8[4] + sum8[5]) + (sum8[6] + sum8[7]));
-      // the probabilities replace the first half of this thread's own scores
-      tmem_st32(tSg, r);
-      tmem_st_wait();
-      tc_fence_before();
-      warp_arrive(B(P_FULL + g * 2 + sb));
-    }
-    // every MMA has completed: the Q tile is free to carry the groups' (reference, sum) pairs
-    if (ok && mbar_wait(B(ALL_DONE), 0, abort_flag, p.flags)) {
+      if (!ok) break;
+      // the item's last P V product is done: merge the two partial softmaxes and write the output
+      const uint32_t kp = (uint32_t)k & 1u;
+      if (!mbar_wait(B(ALL_DONE), kp, abort_flag, p.flags)) { ok = false; break; }
       tc_fence_after();
       exch[g * 128 + row] = make_float2(m_ref, l);
       warp_arrive(B(MERGE));
-      if (mbar_wait(B(MERGE), 0, abort_flag, p.flags)) {
+      if (!mbar_wait(B(MERGE), kp, abort_flag, p.flags)) { ok = false; break; }
+      {
         const float2 other = exch[(g ^ 1) * 128 + row];
         const float m = fmaxf(m_ref, other.x);
         // group A always has a finite reference (key 0 is visible to every query), so m is finite
@@ -357,7 +400,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
         const float l_tot = w_own * l + w_oth * other.y;
         const float inv = 1.f / l_tot;
         const float fa = (g == 0 ? w_own : w_oth) * inv, fb = (g == 0 ? w_oth : w_own) * inv;
-        bf16* out = p.U + ((int64_t)b * S + grow) * d + head * DH;
+        bf16* out = p.U + ((int64_t)w.b * S + grow) * d + w.head * DH;
         // each group writes half of the head's columns
 #pragma unroll 1
         for (int cc = g * (DH / 64); cc < (g + 1) * (DH / 64); ++cc) {
@@ -371,8 +414,12 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
           if (grow < S) drain32(out + cc * 32, oa, 1.f, nullptr, 0);
         }
         if (g == 0 && grow < S)
-          p.lse_out[((int64_t)b * p.h + head) * S + grow] = (m + log2f(l_tot)) * (1.f / LOG2E);
+          p.lse_out[((int64_t)w.b * p.h + w.head) * S + grow] = (m + log2f(l_tot)) * (1.f / LOG2E);
       }
+      // both accumulators have been read: the next item's P V products may overwrite them (this
+      // arrival also orders this thread's reads of the exchange buffer before the next item's writes)
+      tc_fence_before();
+      warp_arrive(B(O_EMPTY));
     }
   }
   if (*abort_flag) for (int i = 0; i < 64; ++i) __nanosleep(2000);
@@ -559,22 +606,26 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
 // One CTA owns 128 keys (K and V tiles resident) and streams 128-query slabs of Q and dU through
 // a two-deep TMA ring.  The transposed products S^T = K Q^T and dP^T = V dU^T of a slab land in
 // tensor memory; the 256 row threads (one key each, half of the slab's queries per group) turn
-// them into bf16 P^T and dS^T written back over the accumulators they came from (half their
-// columns), and dV += P^T dU, dK += dS^T Q take those as A operands straight from tensor memory.
-// The products of a slab are serial (the tensor-memory budget - two 128-column accumulators for
-// dV and dK plus the two score buffers - leaves no room to double-buffer the scores); the next
-// slab's Q and dU arrive meanwhile.
+// S^T into bf16 P^T and then dP^T into bf16 dS^T, each written back over the first half of the
+// thread's own accumulator columns, and dV += P^T dU, dK += dS^T Q take those as A operands
+// straight from tensor memory.  The tensor-memory budget (two 128-column accumulators for dV and
+// dK plus the two score buffers) leaves no room to double-buffer the scores, so the slab is
+// pipelined in halves instead: one thread issues S^T and dP^T, a second one dV and dK;
+// S^T of slab i+1 may start as soon as dV of slab i has consumed P^T (while the row threads are
+// still forming dS^T), and dP^T of slab i+1 as soon as dK of slab i is done.
 template <int DH>
-__global__ void __launch_bounds__(BWD_THREADS, 1)
+__global__ void __launch_bounds__(DQ_THREADS, 1)
 attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapG,
                    const AttnParams p) {
   constexpr int NH = DH / 64, QT = 128 * DH * 2, NS = 2;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align1k(smem_raw);
   const uint32_t Ks = smem_u32(smem), Vs = Ks + QT, Rs = Vs + QT;   // ring: Q then dU per stage
-  float* row_stat = reinterpret_cast<float*>(smem + (2 + 2 * NS) * QT);   // [parity][lse * log2e | delta][128]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (2 + 2 * NS) * QT + 2 * 2 * 128 * 4);
-  enum { KV_FULL = 0, QG_FULL = 1, QG_EMPTY = 1 + NS, SDP_FULL = 1 + 2 * NS, LOADED, PDS_FULL, OUT_FULL, NBAR };
+  // per-query statistics of a slab, staged one slab ahead: [slab % 3][lse * log2e | delta][128]
+  float* row_stat = reinterpret_cast<float*>(smem + (2 + 2 * NS) * QT);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (2 + 2 * NS) * QT + 3 * 2 * 128 * 4);
+  enum { KV_FULL = 0, QG_FULL = 1, QG_EMPTY = 1 + NS, S_FULL = 1 + 2 * NS, DP_FULL, P_FULL, DS_FULL, TS_EMPTY,
+         TP_EMPTY, OUT_FULL, NBAR };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar0 = smem_u32(bars);
@@ -583,15 +634,28 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
   const int kb = blockIdx.x, head = blockIdx.y, b = blockIdx.z;
   const int d = p.h * DH, S = p.S;
   const int n = (S + 127) / 128 - kb;      // 128-query slabs from the diagonal down
+  const float* lrow = p.lse + ((int64_t)b * p.h + head) * S;
+  const float* drow = p.delta + ((int64_t)b * p.h + head) * S;
+  // row thread (grp, row) fetches and stages the statistic `grp` of query `row` of slab `it`
+  auto fetch_stat = [&](int it, int grp, int row) -> float {
+    const int q = (kb + it) * 128 + row;
+    const int qc = q < S ? q : S - 1;
+    return grp == 0 ? __ldg(lrow + qc) * LOG2E : __ldg(drow + qc);
+  };
+  auto stage_stat = [&](int it, int grp, int row, float v) { row_stat[((it % 3) * 2 + grp) * 128 + row] = v; };
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
-    mbar_init(B(LOADED), 8); mbar_init(B(PDS_FULL), 8);
+    mbar_init(B(P_FULL), 8); mbar_init(B(DS_FULL), 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
   if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
+  if (warp >= 2 && warp < 10) {
+    const int g0 = (warp - 2) >> 2, r0 = (warp & 3) * 32 + lane;
+    stage_stat(0, g0, r0, fetch_stat(0, g0, r0));
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -618,33 +682,51 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
-      constexpr uint32_t idesc_o = make_idesc(128, DH, false, true);
       const uint32_t k_lo = klo(Ks), v_lo = klo(Vs);
       bool ok = mbar_wait(B(KV_FULL), 0, abort_flag, p.flags);
       for (int it = 0; it < n && ok; ++it) {
-        const int st = it % NS;
+        const int st = it % NS; const uint32_t prev = (uint32_t)(it - 1) & 1u;
         const uint32_t Qst = Rs + st * 2 * QT, Gst = Qst + QT;
         if (!mbar_wait(B(QG_FULL + st), (it / NS) & 1, abort_flag, p.flags)) break;
-        tc_fence_after();
-        // these overwrite P^T / dS^T of the previous slab: the products that read them were
-        // issued earlier by this thread and the tensor pipe runs its instructions in order
         const uint32_t q_lo = klo(Qst), g_lo = klo(Gst);
+        // S^T overwrites P^T of the previous slab: wait until dV has consumed it
+        if (it > 0 && !mbar_wait(B(TS_EMPTY), prev, abort_flag, p.flags)) break;
+        tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks)
           umma_lo(tS, k_lo + kstep<128>(ks), q_lo + kstep<128>(ks), idesc_s, ks > 0);
+        umma_commit(B(S_FULL));
+        // dP^T overwrites dS^T of the previous slab: wait until dK has consumed it
+        if (it > 0 && !mbar_wait(B(TP_EMPTY), prev, abort_flag, p.flags)) break;
+        tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks)
           umma_lo(tP, v_lo + kstep<128>(ks), g_lo + kstep<128>(ks), idesc_s, ks > 0);
-        umma_commit(B(SDP_FULL));
-        if (!mbar_wait(B(PDS_FULL), (uint32_t)it & 1u, abort_flag, p.flags)) break;
-        tc_fence_after();
+        umma_commit(B(DP_FULL));
+      }
+    }
+  } else if (warp == 10) {
+    if (lane == 0) {
+      constexpr uint32_t idesc_o = make_idesc(128, DH, false, true);
+      bool ok = true;
+      for (int it = 0; it < n && ok; ++it) {
+        const int st = it % NS; const uint32_t ph = (uint32_t)it & 1u;
+        const uint32_t Qst = Rs + st * 2 * QT, Gst = Qst + QT;
+        if (!mbar_wait(B(QG_FULL + st), (it / NS) & 1, abort_flag, p.flags)) break;
         const uint32_t gmn_lo = mlo<128>(Gst), qmn_lo = mlo<128>(Qst);
+        if (!mbar_wait(B(P_FULL), ph, abort_flag, p.flags)) break;
+        tc_fence_after();
+        // group g's 64 queries sit in the first 32 columns of its own half of the accumulator
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
-          umma_ts_lo(tV, tS + 8 * ks, gmn_lo + mstep(ks), idesc_o, (it > 0 || ks > 0));
+          umma_ts_lo(tV, tS + (ks >> 2) * 64 + (ks & 3) * 8, gmn_lo + mstep(ks), idesc_o, (it > 0 || ks > 0));
+        umma_commit(B(TS_EMPTY));
+        if (!mbar_wait(B(DS_FULL), ph, abort_flag, p.flags)) break;
+        tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
-          umma_ts_lo(tK, tP + 8 * ks, qmn_lo + mstep(ks), idesc_o, (it > 0 || ks > 0));
+          umma_ts_lo(tK, tP + (ks >> 2) * 64 + (ks & 3) * 8, qmn_lo + mstep(ks), idesc_o, (it > 0 || ks > 0));
+        umma_commit(B(TP_EMPTY));
         umma_commit(B(QG_EMPTY + st));
         if (it == n - 1) umma_commit(B(OUT_FULL));
       }
@@ -656,55 +738,67 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
     const int key = kb * 128 + row;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     const float scale = rsqrtf((float)DH), c = scale * LOG2E;
-    const float* lrow = p.lse + ((int64_t)b * p.h + head) * S;
-    const float* drow = p.delta + ((int64_t)b * p.h + head) * S;
     bool ok = true;
     for (int it = 0; it < n && ok; ++it) {
       const uint32_t ph = (uint32_t)it & 1u;
-      // per-query log-sum-exp and delta of this slab, staged once for all row threads
-      {
-        const int q = (kb + it) * 128 + row;
-        const int qc = q < S ? q : S - 1;
-        row_stat[(ph * 2 + grp) * 128 + row] = grp == 0 ? __ldg(lrow + qc) * LOG2E : __ldg(drow + qc);
-      }
-      if (!mbar_wait(B(SDP_FULL), ph, abort_flag, p.flags)) { ok = false; break; }
-      tc_fence_after();
-      uint32_t rs[64], rd[64];
-      tmem_ld32(tS + lane_off + 64 * grp, rs);
-      tmem_ld32(tS + lane_off + 64 * grp + 32, rs + 32);
-      tmem_ld32(tP + lane_off + 64 * grp, rd);
-      tmem_ld32(tP + lane_off + 64 * grp + 32, rd + 32);
-      tmem_ld_wait();
-      tc_fence_before();
-      // every row thread has its scores in registers (they may now be overwritten in place) and
-      // has staged its share of the slab's row statistics
-      warp_arrive(B(LOADED));
-      if (!mbar_wait(B(LOADED), ph, abort_flag, p.flags)) { ok = false; break; }
-      const float4* sl = reinterpret_cast<const float4*>(row_stat + (ph * 2 + 0) * 128 + 64 * grp);
-      const float4* sd = reinterpret_cast<const float4*>(row_stat + (ph * 2 + 1) * 128 + 64 * grp);
+      const float4* sl = reinterpret_cast<const float4*>(row_stat + ((it % 3) * 2 + 0) * 128 + 64 * grp);
+      const float4* sd = reinterpret_cast<const float4*>(row_stat + ((it % 3) * 2 + 1) * 128 + 64 * grp);
       const int q0 = (kb + it) * 128 + 64 * grp;
       const bool diag = (it == 0) || ((kb + it + 1) * 128 > S);
+      // the next slab's statistic is fetched now so that its latency hides behind this slab's work
+      const float next_stat = it + 1 < n ? fetch_stat(it + 1, grp, row) : 0.f;
+      // ---- P^T from S^T
+      if (!mbar_wait(B(S_FULL), ph, abort_flag, p.flags)) { ok = false; break; }
+      tc_fence_after();
+      uint32_t rs[64], pk[32];
+      tmem_ld32(tS + lane_off + 64 * grp, rs);
+      tmem_ld32(tS + lane_off + 64 * grp + 32, rs + 32);
+      tmem_ld_wait();
 #pragma unroll
       for (int e4 = 0; e4 < 16; ++e4) {
-        const float4 l4 = sl[e4], d4 = sd[e4];
-        const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dv[4] = {d4.x, d4.y, d4.z, d4.w};
-        float pe[4], de[4];
+        const float4 l4 = sl[e4];
+        const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const int e = 4 * e4 + u;
           float x = ex2(fmaf(__uint_as_float(rs[e]), c, -lv[u]));
           if (diag && (key > q0 + e || q0 + e >= S)) x = 0.f;
-          pe[u] = x;
-          de[u] = x * (__uint_as_float(rd[e]) - dv[u]);
+          rs[e] = __float_as_uint(x);
         }
-        rs[2 * e4] = pack2(pe[0], pe[1]); rs[2 * e4 + 1] = pack2(pe[2], pe[3]);
-        rd[2 * e4] = pack2(de[0], de[1]); rd[2 * e4 + 1] = pack2(de[2], de[3]);
+        pk[2 * e4] = pack2(__uint_as_float(rs[4 * e4]), __uint_as_float(rs[4 * e4 + 1]));
+        pk[2 * e4 + 1] = pack2(__uint_as_float(rs[4 * e4 + 2]), __uint_as_float(rs[4 * e4 + 3]));
       }
-      tmem_st32(tS + lane_off + 32 * grp, rs);
-      tmem_st32(tP + lane_off + 32 * grp, rd);
+      tmem_st32(tS + lane_off + 64 * grp, pk);
       tmem_st_wait();
       tc_fence_before();
-      warp_arrive(B(PDS_FULL));
+      // next slab's statistics: written before this arrival, they are visible to every thread
+      // that later sees the next slab's S^T (which is issued only after dV of this slab)
+      if (it + 1 < n) stage_stat(it + 1, grp, row, next_stat);
+      warp_arrive(B(P_FULL));
+      // ---- dS^T from dP^T
+      if (!mbar_wait(B(DP_FULL), ph, abort_flag, p.flags)) { ok = false; break; }
+      tc_fence_after();
+      {
+        uint32_t rd[64];
+        tmem_ld32(tP + lane_off + 64 * grp, rd);
+        tmem_ld32(tP + lane_off + 64 * grp + 32, rd + 32);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e4 = 0; e4 < 16; ++e4) {
+          const float4 d4 = sd[e4];
+          const float dv[4] = {d4.x, d4.y, d4.z, d4.w};
+          float de[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            de[u] = __uint_as_float(rs[4 * e4 + u]) * (__uint_as_float(rd[4 * e4 + u]) - dv[u]);
+          pk[2 * e4] = pack2(de[0], de[1]);
+          pk[2 * e4 + 1] = pack2(de[2], de[3]);
+        }
+      }
+      tmem_st32(tP + lane_off + 64 * grp, pk);
+      tmem_st_wait();
+      tc_fence_before();
+      warp_arrive(B(DS_FULL));
     }
     if (ok && mbar_wait(B(OUT_FULL), 0, abort_flag, p.flags)) {
       tc_fence_after();
@@ -741,6 +835,16 @@ bool encode3d(CUtensorMap* map, const bf16* base, int cols, int S, int B, int64_
              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+int sm_count() {
+  static int n_sm = 0;
+  if (n_sm == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (n_sm <= 0) n_sm = 148;
+  }
+  return n_sm;
+}
 template <typename K>
 bool set_smem(K kernel, int bytes) {
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
@@ -749,14 +853,14 @@ constexpr int EXTRA = 1024 + 256;   // alignment slack + barriers
 
 template <int DH>
 int fwd_t(const bf16* qkv, bf16* U, float* lse, int B, int S, int h, int* flags, cudaStream_t st) {
-  constexpr int SM = 7 * 128 * DH * 2 + EXTRA;
+  constexpr int SM = 7 * 128 * DH * 2 + 2 * 128 * 8 + 256 + FWD_ALIGN_SLACK;
   static bool ok = set_smem(attn_fwd_tc_kernel<DH>, SM);
   if (!ok) return -2;
   CUtensorMap m;
   if (!encode3d(&m, qkv, 3 * h * DH, S, B, 3 * (int64_t)h * DH, 128)) return -3;
-  AttnParams p{}; p.U = U; p.lse_out = lse; p.S = S; p.h = h; p.flags = flags;
-  dim3 grid((S + 127) / 128, h, B);
-  attn_fwd_tc_kernel<DH><<<grid, FWD_THREADS, SM, st>>>(m, p);
+  AttnParams p{}; p.U = U; p.lse_out = lse; p.S = S; p.h = h; p.B = B; p.flags = flags;
+  const int items = ((S + 127) / 128) * h * B;
+  attn_fwd_tc_kernel<DH><<<items < sm_count() ? items : sm_count(), FWD_THREADS, SM, st>>>(m, p);
   return 0;
 }
 
@@ -764,18 +868,18 @@ template <int DH>
 int bwd_t(const bf16* qkv, const float* lse, const bf16* dU, bf16* dqkv, const float* delta, int B,
           int S, int h, int* flags, cudaStream_t st, const float2* inv_rope) {
   constexpr int SM_DQ = 7 * 128 * DH * 2 + EXTRA;
-  constexpr int SM_KV = 6 * 128 * DH * 2 + 2 * 2 * 128 * 4 + EXTRA;
+  constexpr int SM_KV = 6 * 128 * DH * 2 + 3 * 2 * 128 * 4 + EXTRA;
   static bool ok = set_smem(attn_dq_tc_kernel<DH>, SM_DQ) && set_smem(attn_dkv_tc_kernel<DH>, SM_KV);
   if (!ok) return -2;
   const int d = h * DH;
   CUtensorMap mQKV, mG;
   if (!encode3d(&mQKV, qkv, 3 * d, S, B, 3 * (int64_t)d, 128) || !encode3d(&mG, dU, d, S, B, d, 128))
     return -3;
-  AttnParams p{}; p.lse = lse; p.delta = delta; p.dqkv = dqkv; p.S = S; p.h = h; p.flags = flags;
+  AttnParams p{}; p.lse = lse; p.delta = delta; p.dqkv = dqkv; p.S = S; p.h = h; p.B = B; p.flags = flags;
   p.inv_rope = inv_rope;
   dim3 grid((S + 127) / 128, h, B);
   attn_dq_tc_kernel<DH><<<grid, DQ_THREADS, SM_DQ, st>>>(mQKV, mG, p);
-  attn_dkv_tc_kernel<DH><<<grid, BWD_THREADS, SM_KV, st>>>(mQKV, mG, p);
+  attn_dkv_tc_kernel<DH><<<grid, DQ_THREADS, SM_KV, st>>>(mQKV, mG, p);
   return 0;
 }
 

@@ -24,8 +24,12 @@ using namespace tc;
 using namespace gemm_tc_detail;
 
 constexpr int PAIR_BN = 256;                 // accumulator columns (N of the pair's tile)
-constexpr int PAIR_STAGES = 6;
-constexpr int HALF_BYTES = 128 * BK * 2;     // one CTA's A (or B) slab: 128 rows x 64 k
+// A stage holds PAIR_KH slabs of 64 k: the issuing thread stalls while the tensor pipe is busy, so
+// a barrier wait per 64 k (four instructions) is not hidden behind the products; one per 128 k is.
+constexpr int PAIR_KH = 2;
+constexpr int PAIR_STAGES = 6 / PAIR_KH;
+constexpr int SLAB_BYTES = 128 * BK * 2;     // 128 rows x 64 k of one operand
+constexpr int HALF_BYTES = PAIR_KH * SLAB_BYTES;   // one CTA's A (or B) part of a stage
 constexpr int PAIR_STAGE_BYTES = 2 * HALF_BYTES;
 constexpr int PAIR_SMEM = PAIR_STAGES * PAIR_STAGE_BYTES + 1024 + 256;
 
@@ -115,7 +119,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
 
   const int n_pairs = gridDim.x >> 1, pair = blockIdx.x >> 1;
   const int num_tiles = p.tiles_m * p.tiles_n;
-  const int k_blocks = (p.K + BK - 1) / BK;
+  const int k_blocks = (p.K + PAIR_KH * BK - 1) / (PAIR_KH * BK);
 
   if (warp == 0) {
     if (lane == 0) {
@@ -132,17 +136,22 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
           const uint32_t b_dst = a_dst + HALF_BYTES;
           const uint32_t fb = map_to_rank(full_bar(s), 0);
           if (leader) mbar_expect_tx(full_bar(s), 2 * PAIR_STAGE_BYTES);
-          if (A_K) {
-            tma_load_2d_pair(a_dst, &mapA, fb, kb * BK, m0);
-          } else {
-            tma_load_2d_pair(a_dst, &mapA, fb, m0, kb * BK);
-            tma_load_2d_pair(a_dst + 8192, &mapA, fb, m0 + 64, kb * BK);
-          }
-          if (B_K) {
-            tma_load_2d_pair(b_dst, &mapB, fb, kb * BK, n0);
-          } else {
-            tma_load_2d_pair(b_dst, &mapB, fb, n0, kb * BK);
-            tma_load_2d_pair(b_dst + 8192, &mapB, fb, n0 + 64, kb * BK);
+          // (k past the end of the reduction reads zeros)
+#pragma unroll
+          for (int kh = 0; kh < PAIR_KH; ++kh) {
+            const int k0 = (kb * PAIR_KH + kh) * BK;
+            if (A_K) {
+              tma_load_2d_pair(a_dst + kh * SLAB_BYTES, &mapA, fb, k0, m0);
+            } else {
+              tma_load_2d_pair(a_dst + kh * SLAB_BYTES, &mapA, fb, m0, k0);
+              tma_load_2d_pair(a_dst + kh * SLAB_BYTES + 8192, &mapA, fb, m0 + 64, k0);
+            }
+            if (B_K) {
+              tma_load_2d_pair(b_dst + kh * SLAB_BYTES, &mapB, fb, k0, n0);
+            } else {
+              tma_load_2d_pair(b_dst + kh * SLAB_BYTES, &mapB, fb, n0, k0);
+              tma_load_2d_pair(b_dst + kh * SLAB_BYTES + 8192, &mapB, fb, n0 + 64, k0);
+            }
           }
           if (++s == ST) { s = 0; ph ^= 1u; }
         }
@@ -168,9 +177,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
           const uint32_t a_addr = smem_u32(smem + s * PAIR_STAGE_BYTES);
           const uint32_t b_addr = a_addr + HALF_BYTES;
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {
-            const uint64_t adesc = A_K ? make_desc(a_addr + k * 32, 16, 1024) : make_desc(a_addr + k * 2048, 8192, 1024);
-            const uint64_t bdesc = B_K ? make_desc(b_addr + k * 32, 16, 1024) : make_desc(b_addr + k * 2048, 8192, 1024);
+          for (int k = 0; k < PAIR_KH * (BK / UMMA_K); ++k) {
+            const uint32_t slab = (uint32_t)(k / (BK / UMMA_K)) * SLAB_BYTES, kk = (uint32_t)(k % (BK / UMMA_K));
+            const uint64_t adesc = A_K ? make_desc(a_addr + slab + kk * 32, 16, 1024) : make_desc(a_addr + slab + kk * 2048, 8192, 1024);
+            const uint64_t bdesc = B_K ? make_desc(b_addr + slab + kk * 32, 16, 1024) : make_desc(b_addr + slab + kk * 2048, 8192, 1024);
             umma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
           }
           umma_commit_pair(empty_bar(s));        // both CTAs' slots are free once these MMAs have read them
