@@ -7,16 +7,16 @@
 //             written back to TMEM over the scores, and P V (A operand from TMEM) accumulates in
 //             TMEM, one accumulator per group, with lazy online-softmax rescaling; the two
 //             partial softmaxes are merged at the end.
-//   dq        one CTA per 128 queries, 128-key slabs; S = Q K^T and dP = dU V^T in TMEM, the
+//   dq        128 queries per work item, 128-key slabs; S = Q K^T and dP = dU V^T in TMEM, the
 //             threads form dS = P (dP - delta) and write it back to TMEM as bf16, from where it is
 //             the A operand of dQ += dS K, which accumulates in TMEM over all slabs (no rescaling
 //             is needed in the backward).
-//   dk, dv    one CTA per 128 keys, 128-query slabs; the transposed products S^T = K Q^T,
+//   dk, dv    128 keys per work item, 128-query slabs; the transposed products S^T = K Q^T,
 //             dP^T = V dU^T; P^T and dS^T overwrite them in TMEM as bf16 and feed dV += P^T dU and
 //             dK += dS^T Q, which accumulate in TMEM.
-// The forward kernel is persistent: one CTA per SM walks a balanced list of (sequence, head,
-// query block) items, so set-up, the first loads and the output drain of an item overlap with
-// the products of its neighbours.
+// All three kernels are persistent: one CTA per SM walks a balanced list of (sequence, head,
+// query or key block) items, so set-up, the first loads and the output drain of an item overlap
+// with the products of its neighbours.
 // The two backward kernels recompute P from q, k and the saved log-sum-exp; nothing is
 // accumulated with atomics, so results are bitwise reproducible.  (Appendix C.1, MHA.)
 //
@@ -51,12 +51,16 @@ __device__ __forceinline__ void drain32(bf16* out, const uint32_t* r, float f, c
 #pragma unroll
   for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]) * f;
   if (cs_row) {
+    // the chunk's 16 (cos, sin) pairs are 128 contiguous, 128-byte aligned bytes of the table
+    const float4* w4 = reinterpret_cast<const float4*>(cs_row + c0 / 2);
 #pragma unroll
-    for (int q = 0; q < 16; ++q) {
-      const float2 w = __ldg(cs_row + c0 / 2 + q);
-      const float a = v[2 * q], b = v[2 * q + 1];
-      v[2 * q] = a * w.x + b * w.y;
-      v[2 * q + 1] = b * w.x - a * w.y;
+    for (int q = 0; q < 8; ++q) {
+      const float4 w = __ldg(w4 + q);
+      const float a0 = v[4 * q], b0 = v[4 * q + 1], a1 = v[4 * q + 2], b1 = v[4 * q + 3];
+      v[4 * q] = a0 * w.x + b0 * w.y;
+      v[4 * q + 1] = b0 * w.x - a0 * w.y;
+      v[4 * q + 2] = a1 * w.z + b1 * w.w;
+      v[4 * q + 3] = b1 * w.z - a1 * w.w;
     }
   }
 #pragma unroll
@@ -132,7 +136,7 @@ __device__ __forceinline__ uint8_t* align1k(uint8_t* p) {
 }
 
 // ------------------------------------------------------------------ forward
-// One CTA per 128 queries, 128-key blocks.  S = Q K^T of block j+1 is issued into the second TMEM
+// A work item is 128 queries, walked in 128-key blocks.  S = Q K^T of block j+1 is issued into the second TMEM
 // buffer while the row threads work on block j.  Two groups of 128 row threads share a block by
 // key columns: group g owns columns [64g, 64g+64) of every block, keeps its own softmax
 // reference and row sum, writes its bf16 probabilities back into tensor memory over the first
@@ -429,7 +433,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const AttnParams 
 }
 
 // ------------------------------------------------------------------ backward: dq
-// One CTA owns 128 queries (Q and dU tiles resident) and streams 128-key slabs of K and V through
+// A work item owns 128 queries (Q and dU tiles resident) and streams 128-key slabs of K and V through
 // a two-deep TMA ring.  S = Q K^T and dP = dU V^T of a slab land in tensor memory; the 256 row
 // threads (one query row each, half of the slab's key columns per group) pull them into
 // registers, which frees the two accumulators for the next slab, form dS = P (dP - delta) and
@@ -445,20 +449,18 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
   uint8_t* smem = align1k(smem_raw);
   const uint32_t Qs = smem_u32(smem), Gs = Qs + QT, Kr = Gs + QT, Vr = Kr + NK * QT;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (2 + NK + NV) * QT);
-  enum { Q_FULL = 0, K_FULL = 1, V_FULL = K_FULL + NK, K_EMPTY = V_FULL + NV, V_EMPTY = K_EMPTY + NK,
-         SDP_FULL = V_EMPTY + NV, SDP_EMPTY, DS_FULL, DS_EMPTY = DS_FULL + 2, DQ_FULL = DS_EMPTY + 2, NBAR };
+  enum { Q_FULL = 0, QG_EMPTY, K_FULL, V_FULL = K_FULL + NK, K_EMPTY = V_FULL + NV, V_EMPTY = K_EMPTY + NK,
+         SDP_FULL = V_EMPTY + NV, SDP_EMPTY, DS_FULL, DS_EMPTY = DS_FULL + 2, DQ_FULL = DS_EMPTY + 2, TQ_EMPTY, NBAR };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar0 = smem_u32(bars);
   auto B = [&](int i) { return bar0 + 8u * i; };
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int qb = gridDim.x - 1 - blockIdx.x, head = blockIdx.y, b = blockIdx.z;
-  const int d = p.h * DH, S = p.S;
-  const int n = min(qb + 1, (S + 127) / 128);      // 128-key slabs up to the diagonal
+  const int d = p.h * DH, S = p.S, nq = (S + 127) / 128;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
-    mbar_init(B(SDP_EMPTY), 8); mbar_init(B(DS_FULL), 8); mbar_init(B(DS_FULL + 1), 8);
+    mbar_init(B(SDP_EMPTY), 8); mbar_init(B(DS_FULL), 8); mbar_init(B(DS_FULL + 1), 8); mbar_init(B(TQ_EMPTY), 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -469,49 +471,57 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const uint32_t tS = tmem, tP = tmem + 128, tD = tmem + 256, tQ = tmem + 384;   // dS buffer b at tD + 64 b
+  // c counts the key slabs this CTA has gone through (every role keeps its own copy)
 
   if (warp == 0) {
     if (lane == 0) {
-      mbar_expect_tx(B(Q_FULL), 2 * QT);
-      for (int hf = 0; hf < NH; ++hf) {
-        tma_load_3d(Qs + hf * 16384, &mapQKV, B(Q_FULL), head * DH + hf * 64, qb * 128, b);
-        tma_load_3d(Gs + hf * 16384, &mapG, B(Q_FULL), head * DH + hf * 64, qb * 128, b);
-      }
-      for (int it = 0; it < n; ++it) {
-        const int sk = it % NK, sv = it % NV;
-        if (!mbar_wait(B(K_EMPTY + sk), ((it / NK) & 1) ^ 1u, abort_flag, p.flags)) break;
-        mbar_expect_tx(B(K_FULL + sk), QT);
-        for (int hf = 0; hf < NH; ++hf)
-          tma_load_3d(Kr + sk * QT + hf * 16384, &mapQKV, B(K_FULL + sk), d + head * DH + hf * 64, it * 128, b);
-        if (!mbar_wait(B(V_EMPTY + sv), ((it / NV) & 1) ^ 1u, abort_flag, p.flags)) break;
-        mbar_expect_tx(B(V_FULL + sv), QT);
-        for (int hf = 0; hf < NH; ++hf)
-          tma_load_3d(Vr + sv * QT + hf * 16384, &mapQKV, B(V_FULL + sv), 2 * d + head * DH + hf * 64, it * 128, b);
+      WorkItem w; uint32_t c = 0; bool ok = true;
+      for (int k = 0; ok && work_item(k, p.B, p.h, nq, w); ++k) {
+        // the Q and dU tiles are free once the previous item's last S / dP products are done
+        if (k > 0 && !mbar_wait(B(QG_EMPTY), (uint32_t)(k - 1) & 1u, abort_flag, p.flags)) break;
+        mbar_expect_tx(B(Q_FULL), 2 * QT);
+        for (int hf = 0; hf < NH; ++hf) {
+          tma_load_3d(Qs + hf * 16384, &mapQKV, B(Q_FULL), w.head * DH + hf * 64, w.qb * 128, w.b);
+          tma_load_3d(Gs + hf * 16384, &mapG, B(Q_FULL), w.head * DH + hf * 64, w.qb * 128, w.b);
+        }
+        for (int it = 0; it <= w.qb; ++it, ++c) {
+          const int sk = c % NK, sv = c % NV;
+          if (!mbar_wait(B(K_EMPTY + sk), ((c / NK) & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+          mbar_expect_tx(B(K_FULL + sk), QT);
+          for (int hf = 0; hf < NH; ++hf)
+            tma_load_3d(Kr + sk * QT + hf * 16384, &mapQKV, B(K_FULL + sk), d + w.head * DH + hf * 64, it * 128, w.b);
+          if (!mbar_wait(B(V_EMPTY + sv), ((c / NV) & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+          mbar_expect_tx(B(V_FULL + sv), QT);
+          for (int hf = 0; hf < NH; ++hf)
+            tma_load_3d(Vr + sv * QT + hf * 16384, &mapQKV, B(V_FULL + sv), 2 * d + w.head * DH + hf * 64, it * 128, w.b);
+        }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
       const uint32_t q_lo = klo(Qs), g_lo = klo(Gs);
-      auto issue_sdp = [&](int it) -> bool {
-        const int sk = it % NK, sv = it % NV;
-        if (!mbar_wait(B(K_FULL + sk), (it / NK) & 1, abort_flag, p.flags)) return false;
-        if (!mbar_wait(B(V_FULL + sv), (it / NV) & 1, abort_flag, p.flags)) return false;
-        if (it > 0 && !mbar_wait(B(SDP_EMPTY), (uint32_t)(it - 1) & 1u, abort_flag, p.flags)) return false;
-        tc_fence_after();
-        const uint32_t k_lo = klo(Kr + sk * QT), v_lo = klo(Vr + sv * QT);
+      WorkItem w; uint32_t c = 0; bool ok = true;
+      for (int k = 0; ok && work_item(k, p.B, p.h, nq, w); ++k) {
+        if (!mbar_wait(B(Q_FULL), (uint32_t)k & 1u, abort_flag, p.flags)) break;
+        for (int it = 0; it <= w.qb; ++it, ++c) {
+          const int sk = c % NK, sv = c % NV;
+          if (!mbar_wait(B(K_FULL + sk), (c / NK) & 1, abort_flag, p.flags)) { ok = false; break; }
+          if (!mbar_wait(B(V_FULL + sv), (c / NV) & 1, abort_flag, p.flags)) { ok = false; break; }
+          if (c > 0 && !mbar_wait(B(SDP_EMPTY), (c - 1) & 1u, abort_flag, p.flags)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t k_lo = klo(Kr + sk * QT), v_lo = klo(Vr + sv * QT);
 #pragma unroll
-        for (int ks = 0; ks < DH / 16; ++ks)
-          umma_lo(tS, q_lo + kstep<128>(ks), k_lo + kstep<128>(ks), idesc_s, ks > 0);
+          for (int ks = 0; ks < DH / 16; ++ks)
+            umma_lo(tS, q_lo + kstep<128>(ks), k_lo + kstep<128>(ks), idesc_s, ks > 0);
 #pragma unroll
-        for (int ks = 0; ks < DH / 16; ++ks)
-          umma_lo(tP, g_lo + kstep<128>(ks), v_lo + kstep<128>(ks), idesc_s, ks > 0);
-        umma_commit(B(SDP_FULL));
-        umma_commit(B(V_EMPTY + sv));
-        return true;
-      };
-      bool ok = mbar_wait(B(Q_FULL), 0, abort_flag, p.flags);
-      for (int it = 0; it < n && ok; ++it) ok = issue_sdp(it);
+          for (int ks = 0; ks < DH / 16; ++ks)
+            umma_lo(tP, g_lo + kstep<128>(ks), v_lo + kstep<128>(ks), idesc_s, ks > 0);
+          umma_commit(B(SDP_FULL));
+          umma_commit(B(V_EMPTY + sv));
+        }
+        if (ok) umma_commit(B(QG_EMPTY));
+      }
     }
   } else if (warp == 10) {
     // second issuing thread: its waits overlap the first thread's instructions and vice versa
@@ -519,73 +529,79 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
     // serialise every wait with the products)
     if (lane == 0) {
       constexpr uint32_t idesc_q = make_idesc(128, DH, false, true);
-      bool ok = true;
-      for (int it = 0; it < n && ok; ++it) {
-        const int sk = it % NK, db = it & 1;
-        if (!mbar_wait(B(K_FULL + sk), (it / NK) & 1, abort_flag, p.flags)) break;
-        if (!mbar_wait(B(DS_FULL + db), (it >> 1) & 1, abort_flag, p.flags)) break;
-        tc_fence_after();
-        const uint32_t kmn_lo = mlo<128>(Kr + sk * QT);
+      WorkItem w; uint32_t c = 0; bool ok = true;
+      for (int k = 0; ok && work_item(k, p.B, p.h, nq, w); ++k) {
+        // the accumulator is free once the row threads have drained the previous item's dQ
+        if (k > 0 && !mbar_wait(B(TQ_EMPTY), (uint32_t)(k - 1) & 1u, abort_flag, p.flags)) break;
+        for (int it = 0; it <= w.qb; ++it, ++c) {
+          const int sk = c % NK, db = c & 1;
+          if (!mbar_wait(B(K_FULL + sk), (c / NK) & 1, abort_flag, p.flags)) { ok = false; break; }
+          if (!mbar_wait(B(DS_FULL + db), (c >> 1) & 1, abort_flag, p.flags)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t kmn_lo = mlo<128>(Kr + sk * QT);
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          umma_ts_lo(tQ, tD + 64 * db + 8 * ks, kmn_lo + mstep(ks), idesc_q, (it > 0 || ks > 0));
-        umma_commit(B(DS_EMPTY + db));
-        umma_commit(B(K_EMPTY + sk));
-        if (it == n - 1) umma_commit(B(DQ_FULL));
+          for (int ks = 0; ks < 8; ++ks)
+            umma_ts_lo(tQ, tD + 64 * db + 8 * ks, kmn_lo + mstep(ks), idesc_q, (it > 0 || ks > 0));
+          umma_commit(B(DS_EMPTY + db));
+          umma_commit(B(K_EMPTY + sk));
+        }
+        if (ok) umma_commit(B(DQ_FULL));
       }
     }
   } else {
     const int grp = (warp - 2) >> 2;               // column half of every slab this thread handles
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
-    const int grow = qb * 128 + row;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     const float scale = rsqrtf((float)DH), c = scale * LOG2E;
-    const int64_t si = ((int64_t)b * p.h + head) * S + (grow < S ? grow : S - 1);
-    const float l2 = p.lse[si] * LOG2E, dl = p.delta[si];
-    bool ok = true;
-    for (int it = 0; it < n && ok; ++it) {
-      const int db = it & 1;
-      if (!mbar_wait(B(SDP_FULL), (uint32_t)it & 1u, abort_flag, p.flags)) { ok = false; break; }
-      tc_fence_after();
-      uint32_t rs[64], rd[64];
-      tmem_ld32(tS + lane_off + 64 * grp, rs);
-      tmem_ld32(tS + lane_off + 64 * grp + 32, rs + 32);
-      tmem_ld32(tP + lane_off + 64 * grp, rd);
-      tmem_ld32(tP + lane_off + 64 * grp + 32, rd + 32);
-      tmem_ld_wait();
-      tc_fence_before();
-      warp_arrive(B(SDP_EMPTY));               // the accumulators are in registers: free them early
-      const bool diag = (it == qb) || ((it + 1) * 128 > S);
-      const int col0 = it * 128 + 64 * grp;
-      if (!diag) {
+    WorkItem w; uint32_t cs = 0; bool ok = true;
+    for (int k = 0; ok && work_item(k, p.B, p.h, nq, w); ++k) {
+      const int qb = w.qb, grow = qb * 128 + row;
+      const int64_t si = ((int64_t)w.b * p.h + w.head) * S + (grow < S ? grow : S - 1);
+      const float l2 = p.lse[si] * LOG2E, dl = p.delta[si];
+      for (int it = 0; it <= qb && ok; ++it, ++cs) {
+        const int db = cs & 1;
+        if (!mbar_wait(B(SDP_FULL), cs & 1u, abort_flag, p.flags)) { ok = false; break; }
+        tc_fence_after();
+        uint32_t rs[64], rd[64];
+        tmem_ld32(tS + lane_off + 64 * grp, rs);
+        tmem_ld32(tS + lane_off + 64 * grp + 32, rs + 32);
+        tmem_ld32(tP + lane_off + 64 * grp, rd);
+        tmem_ld32(tP + lane_off + 64 * grp + 32, rd + 32);
+        tmem_ld_wait();
+        tc_fence_before();
+        warp_arrive(B(SDP_EMPTY));               // the accumulators are in registers: free them early
+        const bool diag = (it == qb) || ((it + 1) * 128 > S);
+        const int col0 = it * 128 + 64 * grp;
+        if (!diag) {
 #pragma unroll
-        for (int e = 0; e < 64; e += 2) {
-          const float p0 = ex2(fmaf(__uint_as_float(rs[e]), c, -l2));
-          const float p1 = ex2(fmaf(__uint_as_float(rs[e + 1]), c, -l2));
-          rs[e >> 1] = pack2(p0 * (__uint_as_float(rd[e]) - dl), p1 * (__uint_as_float(rd[e + 1]) - dl));
-        }
-      } else {
+          for (int e = 0; e < 64; e += 2) {
+            const float p0 = ex2(fmaf(__uint_as_float(rs[e]), c, -l2));
+            const float p1 = ex2(fmaf(__uint_as_float(rs[e + 1]), c, -l2));
+            rs[e >> 1] = pack2(p0 * (__uint_as_float(rd[e]) - dl), p1 * (__uint_as_float(rd[e + 1]) - dl));
+          }
+        } else {
 #pragma unroll
-        for (int e = 0; e < 64; e += 2) {
-          const int col = col0 + e;
-          float p0 = ex2(fmaf(__uint_as_float(rs[e]), c, -l2));
-          float p1 = ex2(fmaf(__uint_as_float(rs[e + 1]), c, -l2));
-          if (col > grow || col >= S) p0 = 0.f;
-          if (col + 1 > grow || col + 1 >= S) p1 = 0.f;
-          rs[e >> 1] = pack2(p0 * (__uint_as_float(rd[e]) - dl), p1 * (__uint_as_float(rd[e + 1]) - dl));
+          for (int e = 0; e < 64; e += 2) {
+            const int col = col0 + e;
+            float p0 = ex2(fmaf(__uint_as_float(rs[e]), c, -l2));
+            float p1 = ex2(fmaf(__uint_as_float(rs[e + 1]), c, -l2));
+            if (col > grow || col >= S) p0 = 0.f;
+            if (col + 1 > grow || col + 1 >= S) p1 = 0.f;
+            rs[e >> 1] = pack2(p0 * (__uint_as_float(rd[e]) - dl), p1 * (__uint_as_float(rd[e + 1]) - dl));
+          }
         }
+        if (!mbar_wait(B(DS_EMPTY + db), ((cs >> 1) & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+        tc_fence_after();
+        tmem_st32(tD + 64 * db + lane_off + 32 * grp, rs);
+        tmem_st_wait();
+        tc_fence_before();
+        warp_arrive(B(DS_FULL + db));
       }
-      if (!mbar_wait(B(DS_EMPTY + db), ((it >> 1) & 1) ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+      if (!ok) break;
+      if (!mbar_wait(B(DQ_FULL), (uint32_t)k & 1u, abort_flag, p.flags)) { ok = false; break; }
       tc_fence_after();
-      tmem_st32(tD + 64 * db + lane_off + 32 * grp, rs);
-      tmem_st_wait();
-      tc_fence_before();
-      warp_arrive(B(DS_FULL + db));
-    }
-    if (ok && mbar_wait(B(DQ_FULL), 0, abort_flag, p.flags)) {
-      tc_fence_after();
-      bf16* out = p.dqkv + ((int64_t)b * S + grow) * (3 * d) + head * DH;
+      bf16* out = p.dqkv + ((int64_t)w.b * S + grow) * (3 * d) + w.head * DH;
 #pragma unroll 1
       for (int cc = grp; cc < DH / 32; cc += 2) {       // the two groups drain alternate column chunks
         uint32_t r[32];
@@ -594,6 +610,8 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
         if (grow < S)
           drain32(out + cc * 32, r, scale, p.inv_rope ? p.inv_rope + (int64_t)grow * (DH / 2) : nullptr, cc * 32);
       }
+      tc_fence_before();
+      warp_arrive(B(TQ_EMPTY));                 // the next item's dQ products may overwrite the accumulator
     }
   }
   if (*abort_flag) for (int i = 0; i < 64; ++i) __nanosleep(2000);
@@ -603,7 +621,7 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
 }
 
 // ------------------------------------------------------------------ backward: dk, dv
-// One CTA owns 128 keys (K and V tiles resident) and streams 128-query slabs of Q and dU through
+// A work item owns 128 keys (K and V tiles resident) and streams 128-query slabs of Q and dU through
 // a two-deep TMA ring.  The transposed products S^T = K Q^T and dP^T = V dU^T of a slab land in
 // tensor memory; the 256 row threads (one key each, half of the slab's queries per group) turn
 // S^T into bf16 P^T and then dP^T into bf16 dS^T, each written back over the first half of the
@@ -613,6 +631,19 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
 // pipelined in halves instead: one thread issues S^T and dP^T, a second one dV and dK;
 // S^T of slab i+1 may start as soon as dV of slab i has consumed P^T (while the row threads are
 // still forming dS^T), and dP^T of slab i+1 as soon as dK of slab i is done.
+// Work items of the dk/dv kernel: 128 keys of one head of one sequence, heavy (first key block)
+// first; qb of the item is its key block.
+__device__ __forceinline__ bool work_item_kv(int k, int n_batch, int h, int nq, WorkItem& w) {
+  const int G = gridDim.x, cta = blockIdx.x;
+  const int t = k * G + ((k & 1) ? (G - 1 - cta) : cta);
+  const int hb = h * n_batch;
+  if (t >= nq * hb) return false;
+  w.qb = t / hb;
+  const int rem = t % hb;
+  w.head = rem % h; w.b = rem / h;
+  return true;
+}
+
 template <int DH>
 __global__ void __launch_bounds__(DQ_THREADS, 1)
 attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapG,
@@ -624,58 +655,63 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
   // per-query statistics of a slab, staged one slab ahead: [slab % 3][lse * log2e | delta][128]
   float* row_stat = reinterpret_cast<float*>(smem + (2 + 2 * NS) * QT);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (2 + 2 * NS) * QT + 3 * 2 * 128 * 4);
-  enum { KV_FULL = 0, QG_FULL = 1, QG_EMPTY = 1 + NS, S_FULL = 1 + 2 * NS, DP_FULL, P_FULL, DS_FULL, TS_EMPTY,
-         TP_EMPTY, OUT_FULL, NBAR };
+  enum { KV_FULL = 0, KV_EMPTY, QG_FULL, QG_EMPTY = QG_FULL + NS, S_FULL = QG_EMPTY + NS, DP_FULL, P_FULL, DS_FULL,
+         TS_EMPTY, TP_EMPTY, OUT_FULL, ACC_EMPTY, NBAR };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar0 = smem_u32(bars);
   auto B = [&](int i) { return bar0 + 8u * i; };
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int kb = blockIdx.x, head = blockIdx.y, b = blockIdx.z;
-  const int d = p.h * DH, S = p.S;
-  const int n = (S + 127) / 128 - kb;      // 128-query slabs from the diagonal down
-  const float* lrow = p.lse + ((int64_t)b * p.h + head) * S;
-  const float* drow = p.delta + ((int64_t)b * p.h + head) * S;
-  // row thread (grp, row) fetches and stages the statistic `grp` of query `row` of slab `it`
-  auto fetch_stat = [&](int it, int grp, int row) -> float {
-    const int q = (kb + it) * 128 + row;
-    const int qc = q < S ? q : S - 1;
-    return grp == 0 ? __ldg(lrow + qc) * LOG2E : __ldg(drow + qc);
+  const int d = p.h * DH, S = p.S, nq = (S + 127) / 128;
+  // row thread (grp, row) fetches the statistic `grp` of query `row` of query block qblk
+  auto fetch_stat = [&](const WorkItem& w, int qblk, int grp, int row) -> float {
+    const int q = qblk * 128 + row;
+    const int64_t i = ((int64_t)w.b * p.h + w.head) * S + (q < S ? q : S - 1);
+    return grp == 0 ? __ldg(p.lse + i) * LOG2E : __ldg(p.delta + i);
   };
-  auto stage_stat = [&](int it, int grp, int row, float v) { row_stat[((it % 3) * 2 + grp) * 128 + row] = v; };
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
-    mbar_init(B(P_FULL), 8); mbar_init(B(DS_FULL), 8);
+    mbar_init(B(P_FULL), 8); mbar_init(B(DS_FULL), 8); mbar_init(B(ACC_EMPTY), 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
   if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
   if (warp >= 2 && warp < 10) {
-    const int g0 = (warp - 2) >> 2, r0 = (warp & 3) * 32 + lane;
-    stage_stat(0, g0, r0, fetch_stat(0, g0, r0));
+    WorkItem w0;
+    if (work_item_kv(0, p.B, p.h, nq, w0)) {
+      const int g0 = (warp - 2) >> 2, r0 = (warp & 3) * 32 + lane;
+      row_stat[g0 * 128 + r0] = fetch_stat(w0, w0.qb, g0, r0);
+    }
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const uint32_t tS = tmem, tP = tmem + 128, tV = tmem + 256, tK = tmem + 384;   // P^T overlays S^T, dS^T overlays dP^T
+  // c counts the query slabs this CTA has gone through (every role keeps its own copy)
 
   if (warp == 0) {
     if (lane == 0) {
-      mbar_expect_tx(B(KV_FULL), 2 * QT);
-      for (int hf = 0; hf < NH; ++hf) {
-        tma_load_3d(Ks + hf * 16384, &mapQKV, B(KV_FULL), d + head * DH + hf * 64, kb * 128, b);
-        tma_load_3d(Vs + hf * 16384, &mapQKV, B(KV_FULL), 2 * d + head * DH + hf * 64, kb * 128, b);
-      }
-      for (int it = 0; it < n; ++it) {
-        const int st = it % NS; const uint32_t ph = (it / NS) & 1;
-        if (!mbar_wait(B(QG_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) break;
-        mbar_expect_tx(B(QG_FULL + st), 2 * QT);
+      WorkItem w; uint32_t c = 0; bool ok = true;
+      for (int k = 0; ok && work_item_kv(k, p.B, p.h, nq, w); ++k) {
+        const int kb = w.qb;
+        // the K and V tiles are free once the previous item's last S^T / dP^T products are done
+        if (k > 0 && !mbar_wait(B(KV_EMPTY), (uint32_t)(k - 1) & 1u, abort_flag, p.flags)) break;
+        mbar_expect_tx(B(KV_FULL), 2 * QT);
         for (int hf = 0; hf < NH; ++hf) {
-          tma_load_3d(Rs + st * 2 * QT + hf * 16384, &mapQKV, B(QG_FULL + st), head * DH + hf * 64, (kb + it) * 128, b);
-          tma_load_3d(Rs + st * 2 * QT + QT + hf * 16384, &mapG, B(QG_FULL + st), head * DH + hf * 64, (kb + it) * 128, b);
+          tma_load_3d(Ks + hf * 16384, &mapQKV, B(KV_FULL), d + w.head * DH + hf * 64, kb * 128, w.b);
+          tma_load_3d(Vs + hf * 16384, &mapQKV, B(KV_FULL), 2 * d + w.head * DH + hf * 64, kb * 128, w.b);
+        }
+        for (int it = 0; it < nq - kb; ++it, ++c) {
+          const int st = c % NS; const uint32_t ph = (c / NS) & 1;
+          if (!mbar_wait(B(QG_EMPTY + st), ph ^ 1u, abort_flag, p.flags)) { ok = false; break; }
+          mbar_expect_tx(B(QG_FULL + st), 2 * QT);
+          for (int hf = 0; hf < NH; ++hf) {
+            tma_load_3d(Rs + st * 2 * QT + hf * 16384, &mapQKV, B(QG_FULL + st), w.head * DH + hf * 64, (kb + it) * 128, w.b);
+            tma_load_3d(Rs + st * 2 * QT + QT + hf * 16384, &mapG, B(QG_FULL + st), w.head * DH + hf * 64, (kb + it) * 128, w.b);
+          }
         }
       }
     }
@@ -683,126 +719,141 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
       const uint32_t k_lo = klo(Ks), v_lo = klo(Vs);
-      bool ok = mbar_wait(B(KV_FULL), 0, abort_flag, p.flags);
-      for (int it = 0; it < n && ok; ++it) {
-        const int st = it % NS; const uint32_t prev = (uint32_t)(it - 1) & 1u;
-        const uint32_t Qst = Rs + st * 2 * QT, Gst = Qst + QT;
-        if (!mbar_wait(B(QG_FULL + st), (it / NS) & 1, abort_flag, p.flags)) break;
-        const uint32_t q_lo = klo(Qst), g_lo = klo(Gst);
-        // S^T overwrites P^T of the previous slab: wait until dV has consumed it
-        if (it > 0 && !mbar_wait(B(TS_EMPTY), prev, abort_flag, p.flags)) break;
-        tc_fence_after();
+      WorkItem w; uint32_t c = 0; bool ok = true;
+      for (int k = 0; ok && work_item_kv(k, p.B, p.h, nq, w); ++k) {
+        if (!mbar_wait(B(KV_FULL), (uint32_t)k & 1u, abort_flag, p.flags)) break;
+        for (int it = 0; it < nq - w.qb; ++it, ++c) {
+          const int st = c % NS; const uint32_t prev = (c - 1) & 1u;
+          const uint32_t Qst = Rs + st * 2 * QT, Gst = Qst + QT;
+          if (!mbar_wait(B(QG_FULL + st), (c / NS) & 1, abort_flag, p.flags)) { ok = false; break; }
+          const uint32_t q_lo = klo(Qst), g_lo = klo(Gst);
+          // S^T overwrites P^T of the previous slab: wait until dV has consumed it
+          if (c > 0 && !mbar_wait(B(TS_EMPTY), prev, abort_flag, p.flags)) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll
-        for (int ks = 0; ks < DH / 16; ++ks)
-          umma_lo(tS, k_lo + kstep<128>(ks), q_lo + kstep<128>(ks), idesc_s, ks > 0);
-        umma_commit(B(S_FULL));
-        // dP^T overwrites dS^T of the previous slab: wait until dK has consumed it
-        if (it > 0 && !mbar_wait(B(TP_EMPTY), prev, abort_flag, p.flags)) break;
-        tc_fence_after();
+          for (int ks = 0; ks < DH / 16; ++ks)
+            umma_lo(tS, k_lo + kstep<128>(ks), q_lo + kstep<128>(ks), idesc_s, ks > 0);
+          umma_commit(B(S_FULL));
+          // dP^T overwrites dS^T of the previous slab: wait until dK has consumed it
+          if (c > 0 && !mbar_wait(B(TP_EMPTY), prev, abort_flag, p.flags)) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll
-        for (int ks = 0; ks < DH / 16; ++ks)
-          umma_lo(tP, v_lo + kstep<128>(ks), g_lo + kstep<128>(ks), idesc_s, ks > 0);
-        umma_commit(B(DP_FULL));
+          for (int ks = 0; ks < DH / 16; ++ks)
+            umma_lo(tP, v_lo + kstep<128>(ks), g_lo + kstep<128>(ks), idesc_s, ks > 0);
+          umma_commit(B(DP_FULL));
+        }
+        if (ok) umma_commit(B(KV_EMPTY));
       }
     }
   } else if (warp == 10) {
     if (lane == 0) {
       constexpr uint32_t idesc_o = make_idesc(128, DH, false, true);
-      bool ok = true;
-      for (int it = 0; it < n && ok; ++it) {
-        const int st = it % NS; const uint32_t ph = (uint32_t)it & 1u;
-        const uint32_t Qst = Rs + st * 2 * QT, Gst = Qst + QT;
-        if (!mbar_wait(B(QG_FULL + st), (it / NS) & 1, abort_flag, p.flags)) break;
-        const uint32_t gmn_lo = mlo<128>(Gst), qmn_lo = mlo<128>(Qst);
-        if (!mbar_wait(B(P_FULL), ph, abort_flag, p.flags)) break;
-        tc_fence_after();
-        // group g's 64 queries sit in the first 32 columns of its own half of the accumulator
+      WorkItem w; uint32_t c = 0; bool ok = true;
+      for (int k = 0; ok && work_item_kv(k, p.B, p.h, nq, w); ++k) {
+        // the accumulators are free once the row threads have drained the previous item's dV, dK
+        if (k > 0 && !mbar_wait(B(ACC_EMPTY), (uint32_t)(k - 1) & 1u, abort_flag, p.flags)) break;
+        for (int it = 0; it < nq - w.qb; ++it, ++c) {
+          const int st = c % NS; const uint32_t ph = c & 1u;
+          const uint32_t Qst = Rs + st * 2 * QT, Gst = Qst + QT;
+          if (!mbar_wait(B(QG_FULL + st), (c / NS) & 1, abort_flag, p.flags)) { ok = false; break; }
+          const uint32_t gmn_lo = mlo<128>(Gst), qmn_lo = mlo<128>(Qst);
+          if (!mbar_wait(B(P_FULL), ph, abort_flag, p.flags)) { ok = false; break; }
+          tc_fence_after();
+          // group g's 64 queries sit in the first 32 columns of its own half of the accumulator
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          umma_ts_lo(tV, tS + (ks >> 2) * 64 + (ks & 3) * 8, gmn_lo + mstep(ks), idesc_o, (it > 0 || ks > 0));
-        umma_commit(B(TS_EMPTY));
-        if (!mbar_wait(B(DS_FULL), ph, abort_flag, p.flags)) break;
-        tc_fence_after();
+          for (int ks = 0; ks < 8; ++ks)
+            umma_ts_lo(tV, tS + (ks >> 2) * 64 + (ks & 3) * 8, gmn_lo + mstep(ks), idesc_o, (it > 0 || ks > 0));
+          umma_commit(B(TS_EMPTY));
+          if (!mbar_wait(B(DS_FULL), ph, abort_flag, p.flags)) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          umma_ts_lo(tK, tP + (ks >> 2) * 64 + (ks & 3) * 8, qmn_lo + mstep(ks), idesc_o, (it > 0 || ks > 0));
-        umma_commit(B(TP_EMPTY));
-        umma_commit(B(QG_EMPTY + st));
-        if (it == n - 1) umma_commit(B(OUT_FULL));
+          for (int ks = 0; ks < 8; ++ks)
+            umma_ts_lo(tK, tP + (ks >> 2) * 64 + (ks & 3) * 8, qmn_lo + mstep(ks), idesc_o, (it > 0 || ks > 0));
+          umma_commit(B(TP_EMPTY));
+          umma_commit(B(QG_EMPTY + st));
+        }
+        if (ok) umma_commit(B(OUT_FULL));
       }
     }
   } else {
     const int grp = (warp - 2) >> 2;               // query half of every slab this thread handles
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
-    const int key = kb * 128 + row;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     const float scale = rsqrtf((float)DH), c = scale * LOG2E;
-    bool ok = true;
-    for (int it = 0; it < n && ok; ++it) {
-      const uint32_t ph = (uint32_t)it & 1u;
-      const float4* sl = reinterpret_cast<const float4*>(row_stat + ((it % 3) * 2 + 0) * 128 + 64 * grp);
-      const float4* sd = reinterpret_cast<const float4*>(row_stat + ((it % 3) * 2 + 1) * 128 + 64 * grp);
-      const int q0 = (kb + it) * 128 + 64 * grp;
-      const bool diag = (it == 0) || ((kb + it + 1) * 128 > S);
-      // the next slab's statistic is fetched now so that its latency hides behind this slab's work
-      const float next_stat = it + 1 < n ? fetch_stat(it + 1, grp, row) : 0.f;
-      // ---- P^T from S^T
-      if (!mbar_wait(B(S_FULL), ph, abort_flag, p.flags)) { ok = false; break; }
-      tc_fence_after();
-      uint32_t rs[64], pk[32];
-      tmem_ld32(tS + lane_off + 64 * grp, rs);
-      tmem_ld32(tS + lane_off + 64 * grp + 32, rs + 32);
-      tmem_ld_wait();
-#pragma unroll
-      for (int e4 = 0; e4 < 16; ++e4) {
-        const float4 l4 = sl[e4];
-        const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int e = 4 * e4 + u;
-          float x = ex2(fmaf(__uint_as_float(rs[e]), c, -lv[u]));
-          if (diag && (key > q0 + e || q0 + e >= S)) x = 0.f;
-          rs[e] = __float_as_uint(x);
-        }
-        pk[2 * e4] = pack2(__uint_as_float(rs[4 * e4]), __uint_as_float(rs[4 * e4 + 1]));
-        pk[2 * e4 + 1] = pack2(__uint_as_float(rs[4 * e4 + 2]), __uint_as_float(rs[4 * e4 + 3]));
-      }
-      tmem_st32(tS + lane_off + 64 * grp, pk);
-      tmem_st_wait();
-      tc_fence_before();
-      // next slab's statistics: written before this arrival, they are visible to every thread
-      // that later sees the next slab's S^T (which is issued only after dV of this slab)
-      if (it + 1 < n) stage_stat(it + 1, grp, row, next_stat);
-      warp_arrive(B(P_FULL));
-      // ---- dS^T from dP^T
-      if (!mbar_wait(B(DP_FULL), ph, abort_flag, p.flags)) { ok = false; break; }
-      tc_fence_after();
-      {
-        uint32_t rd[64];
-        tmem_ld32(tP + lane_off + 64 * grp, rd);
-        tmem_ld32(tP + lane_off + 64 * grp + 32, rd + 32);
+    WorkItem w, wn; uint32_t cs = 0; bool ok = true;
+    bool have = work_item_kv(0, p.B, p.h, nq, w);
+    for (int k = 0; ok && have; ++k) {
+      const int kb = w.qb, n = nq - kb, key = kb * 128 + row;
+      const bool have_next = work_item_kv(k + 1, p.B, p.h, nq, wn);
+      for (int it = 0; it < n && ok; ++it, ++cs) {
+        const uint32_t ph = cs & 1u;
+        const float4* sl = reinterpret_cast<const float4*>(row_stat + ((cs % 3) * 2 + 0) * 128 + 64 * grp);
+        const float4* sd = reinterpret_cast<const float4*>(row_stat + ((cs % 3) * 2 + 1) * 128 + 64 * grp);
+        const int q0 = (kb + it) * 128 + 64 * grp;
+        const bool diag = (it == 0) || ((kb + it + 1) * 128 > S);
+        // the next slab's statistic (of this item or of the next one) is fetched now so that its
+        // latency hides behind this slab's work
+        const bool more = it + 1 < n || have_next;
+        const float next_stat = it + 1 < n ? fetch_stat(w, kb + it + 1, grp, row)
+                                           : (have_next ? fetch_stat(wn, wn.qb, grp, row) : 0.f);
+        // ---- P^T from S^T
+        if (!mbar_wait(B(S_FULL), ph, abort_flag, p.flags)) { ok = false; break; }
+        tc_fence_after();
+        uint32_t rs[64], pk[32];
+        tmem_ld32(tS + lane_off + 64 * grp, rs);
+        tmem_ld32(tS + lane_off + 64 * grp + 32, rs + 32);
         tmem_ld_wait();
 #pragma unroll
         for (int e4 = 0; e4 < 16; ++e4) {
-          const float4 d4 = sd[e4];
-          const float dv[4] = {d4.x, d4.y, d4.z, d4.w};
-          float de[4];
+          const float4 l4 = sl[e4];
+          const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
 #pragma unroll
-          for (int u = 0; u < 4; ++u)
-            de[u] = __uint_as_float(rs[4 * e4 + u]) * (__uint_as_float(rd[4 * e4 + u]) - dv[u]);
-          pk[2 * e4] = pack2(de[0], de[1]);
-          pk[2 * e4 + 1] = pack2(de[2], de[3]);
+          for (int u = 0; u < 4; ++u) {
+            const int e = 4 * e4 + u;
+            float x = ex2(fmaf(__uint_as_float(rs[e]), c, -lv[u]));
+            if (diag && (key > q0 + e || q0 + e >= S)) x = 0.f;
+            rs[e] = __float_as_uint(x);
+          }
+          pk[2 * e4] = pack2(__uint_as_float(rs[4 * e4]), __uint_as_float(rs[4 * e4 + 1]));
+          pk[2 * e4 + 1] = pack2(__uint_as_float(rs[4 * e4 + 2]), __uint_as_float(rs[4 * e4 + 3]));
         }
+        tmem_st32(tS + lane_off + 64 * grp, pk);
+        tmem_st_wait();
+        tc_fence_before();
+        // next slab's statistics: written before this arrival, they are visible to every thread
+        // that later sees the next slab's S^T (which is issued only after dV of this slab)
+        if (more) row_stat[(((cs + 1) % 3) * 2 + grp) * 128 + row] = next_stat;
+        warp_arrive(B(P_FULL));
+        // ---- dS^T from dP^T
+        if (!mbar_wait(B(DP_FULL), ph, abort_flag, p.flags)) { ok = false; break; }
+        tc_fence_after();
+        {
+          uint32_t rd[64];
+          tmem_ld32(tP + lane_off + 64 * grp, rd);
+          tmem_ld32(tP + lane_off + 64 * grp + 32, rd + 32);
+          tmem_ld_wait();
+#pragma unroll
+          for (int e4 = 0; e4 < 16; ++e4) {
+            const float4 d4 = sd[e4];
+            const float dv[4] = {d4.x, d4.y, d4.z, d4.w};
+            float de[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+              de[u] = __uint_as_float(rs[4 * e4 + u]) * (__uint_as_float(rd[4 * e4 + u]) - dv[u]);
+            pk[2 * e4] = pack2(de[0], de[1]);
+            pk[2 * e4 + 1] = pack2(de[2], de[3]);
+          }
+        }
+        tmem_st32(tP + lane_off + 64 * grp, pk);
+        tmem_st_wait();
+        tc_fence_before();
+        warp_arrive(B(DS_FULL));
       }
-      tmem_st32(tP + lane_off + 64 * grp, pk);
-      tmem_st_wait();
-      tc_fence_before();
-      warp_arrive(B(DS_FULL));
-    }
-    if (ok && mbar_wait(B(OUT_FULL), 0, abort_flag, p.flags)) {
+      if (!ok) break;
+      if (!mbar_wait(B(OUT_FULL), (uint32_t)k & 1u, abort_flag, p.flags)) { ok = false; break; }
       tc_fence_after();
-      bf16* out = p.dqkv + ((int64_t)b * S + key) * (3 * d) + head * DH;
+      bf16* out = p.dqkv + ((int64_t)w.b * S + key) * (3 * d) + w.head * DH;
 #pragma unroll 1
       for (int cc = grp; cc < 2 * DH / 32; cc += 2) {
         const bool is_k = cc >= DH / 32;
@@ -814,6 +865,9 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
           drain32(out + (is_k ? d : 2 * d) + c0, r, is_k ? scale : 1.f,
                   (is_k && p.inv_rope) ? p.inv_rope + (int64_t)key * (DH / 2) : nullptr, c0);
       }
+      tc_fence_before();
+      warp_arrive(B(ACC_EMPTY));                // the next item's products may overwrite dV, dK
+      w = wn; have = have_next;
     }
   }
   if (*abort_flag) for (int i = 0; i < 64; ++i) __nanosleep(2000);
@@ -877,9 +931,9 @@ int bwd_t(const bf16* qkv, const float* lse, const bf16* dU, bf16* dqkv, const f
     return -3;
   AttnParams p{}; p.lse = lse; p.delta = delta; p.dqkv = dqkv; p.S = S; p.h = h; p.B = B; p.flags = flags;
   p.inv_rope = inv_rope;
-  dim3 grid((S + 127) / 128, h, B);
-  attn_dq_tc_kernel<DH><<<grid, DQ_THREADS, SM_DQ, st>>>(mQKV, mG, p);
-  attn_dkv_tc_kernel<DH><<<grid, DQ_THREADS, SM_KV, st>>>(mQKV, mG, p);
+  const int items = ((S + 127) / 128) * h * B, ctas = items < sm_count() ? items : sm_count();
+  attn_dq_tc_kernel<DH><<<ctas, DQ_THREADS, SM_DQ, st>>>(mQKV, mG, p);
+  attn_dkv_tc_kernel<DH><<<ctas, DQ_THREADS, SM_KV, st>>>(mQKV, mG, p);
   return 0;
 }
 

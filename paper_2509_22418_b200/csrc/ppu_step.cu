@@ -200,18 +200,17 @@ struct Sched {
         const double fl = 10.0 * B * h * dh * 0.5 * S * (double)(S + 1);
         EvScope ev(c, 1, fl);
         const int kind = attn_kind();
-        if (kind == 0)
-          rc |= launch_attn_bwd_tc(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, c->flags, st);
+        if (kind == 0)   // rotates dq, dk back on the way out (the output drain overlaps the next item's products)
+          rc |= launch_attn_bwd_tc(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, c->flags, st,
+                                   c->rope_cs);
         else if (kind == 2)
           rc |= launch_attn_bwd_mma(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, st);
         else
           rc |= launch_attn_bwd_simt(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, st);
         c->launches += kind == 1 ? 2 : 3;
         c->flops_dgrad += fl;
+        if (kind != 0) { launch_rope(c->dqkv, c->rope_cs, B, S, h, dh, 1, st); c->launches++; }
       }
-      // (the tcgen05 kernels can rotate dq, dk on the way out, but the table lookups sit on each
-      // CTA's critical path and cost more than this separate pass)
-      launch_rope(c->dqkv, c->rope_cs, B, S, h, dh, 1, st); c->launches++;
       gemm(c->dqkv, 3 * d, 1, W(l, c->rel_wq), d, 0, T, d, 3 * d, EPI_STORE_BF16, c->t16, d, nullptr,
            nullptr, 0, &c->flops_dgrad);
       launch_ln_bwd(c->t16, a.x, a.st1, Pf(l, c->rel_ln1g), c->g, c->g, c->g16, T, d, st);
