@@ -39,6 +39,9 @@ WORKLOADS = {
 ADAM = dict(lr=3e-4, beta1=0.9, beta2=0.99, eps=1e-8, wd=0.1)     # Section 3.1
 OUTER = dict(lr=0.7, momentum=0.9)
 SEED = 1234
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant GEMM kernel (SM-pair
+# kernel, 128-k stages); set to None whenever that kernel changes after the capture
+GEMM_TRAFFIC_BYTES = 183.8e6
 
 
 def peaks():
@@ -342,12 +345,14 @@ def main():
                         gbs=st.outer_bytes / (outer_ms * 1e-3) / 1e9, peak_gbs=pk["hbm"],
                         frac=st.outer_bytes / (outer_ms * 1e-3) / 1e9 / pk["hbm"], of=pk["src"]),
         step_flops=dict(fwd=st.flops_fwd, dgrad=st.flops_dgrad, wgrad=st.flops_wgrad),
-        roofline=dict(bound="tensor", kernel="gemm_tc_kernel (tcgen05 bf16 GEMM, all products of the step)",
+        roofline=dict(bound="tensor", kernel="gemm_tc_pair_kernel / gemm_tc_kernel (tcgen05 bf16 GEMM, all products of the step)",
                       achieved=gemm_tflops, peak=pk["tensor"], unit="TFLOP/s",
                       frac=gemm_tflops / pk["tensor"], peak_kind=f"sustained bf16, {pk['src']}",
                       frac_of_burst=gemm_tflops / pk["tensor_burst"], frac_of_nominal=gemm_tflops / 2250.0,
                       launches=int(prof.gemm_launches), avg_launch_ms=prof.gemm_ms / max(1, prof.gemm_launches),
-                      gemm_share_of_step=prof.gemm_ms / steps_ms, traffic=None),
+                      gemm_share_of_step=prof.gemm_ms / steps_ms, traffic=GEMM_TRAFFIC_BYTES,
+                      traffic_of="one launch of the 8192 x 8192 x 2048 forward product (FFN up), ncu capture "
+                                 "in profiles/gemm_tc_pair_8192x8192x2048.md; algorithmic 201.3e6 bytes"),
         attention=dict(tflops=attn_tflops, ms_per_step=prof.attn_ms / args.steps,
                        share_of_step=prof.attn_ms / steps_ms),
         e2e=dict(value=tokens / (e2e_ms * 1e-3), unit="tokens/s", h2d_bytes_per_step=B * S * 4,
