@@ -83,7 +83,7 @@ struct TcParams {
 // host side (gemm_tc.cu / gemm_tc_pair.cu)
 bool encode_map(CUtensorMap* map, const bf16* base, long long ld, bool kmajor, int rows, int K, int box_rows);
 TcParams make_params(const GemmArgs& g);
-int launch_gemm_tc_pair(const GemmArgs& g, const TcParams& p, cudaStream_t st);
+int launch_gemm_tc_pair(const GemmArgs& g, const TcParams& p, int bn, cudaStream_t st);   // bn: 256 or 128
 
 // Drains rows [m0 + 32 quarter, +32) x columns [n0 + half BN/2, + BN/2) of the accumulator at
 // TMEM column t_acc through registers into global memory, applying the epilogue p.epilogue.

@@ -23,15 +23,21 @@ namespace {
 using namespace tc;
 using namespace gemm_tc_detail;
 
-constexpr int PAIR_BN = 256;                 // accumulator columns (N of the pair's tile)
+// The pair's tile is 256 rows x BN columns, BN = 256 or 128.  The narrow tile is for outputs whose
+// 256-wide tiling leaves the last wave of SM pairs half empty (N = 2048 with 8192 rows: 256 tiles
+// on 74 pairs).
 // A stage holds PAIR_KH slabs of 64 k: the issuing thread stalls while the tensor pipe is busy, so
 // a barrier wait per 64 k (four instructions) is not hidden behind the products; one per 128 k is.
 constexpr int PAIR_KH = 2;
-constexpr int PAIR_STAGES = 6 / PAIR_KH;
 constexpr int SLAB_BYTES = 128 * BK * 2;     // 128 rows x 64 k of one operand
-constexpr int HALF_BYTES = PAIR_KH * SLAB_BYTES;   // one CTA's A (or B) part of a stage
-constexpr int PAIR_STAGE_BYTES = 2 * HALF_BYTES;
-constexpr int PAIR_SMEM = PAIR_STAGES * PAIR_STAGE_BYTES + 1024 + 256;
+template <int BN> struct PairCfg {
+  static constexpr int STAGES = BN == 256 ? 3 : 4;
+  static constexpr int A_HALF = PAIR_KH * SLAB_BYTES;            // this CTA's 128 rows of A
+  static constexpr int B_SLAB = (BN / 2) * BK * 2;               // this CTA's BN/2 rows of B, 64 k
+  static constexpr int B_HALF = PAIR_KH * B_SLAB;
+  static constexpr int STAGE_BYTES = A_HALF + B_HALF;
+  static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 + 256;
+};
 
 __device__ __forceinline__ uint32_t cluster_rank() {
   uint32_t r;
@@ -77,11 +83,12 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
       : "memory");
 }
 
-template <bool A_K, bool B_K>
+template <int PAIR_BN, bool A_K, bool B_K>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                     const TcParams p) {
-  constexpr int ST = PAIR_STAGES;
+  using PC = PairCfg<PAIR_BN>;
+  constexpr int ST = PC::STAGES, PAIR_STAGE_BYTES = PC::STAGE_BYTES, HALF_BYTES = PC::A_HALF, B_SLAB = PC::B_SLAB;
   extern __shared__ uint8_t smem_raw[];
   // the dynamic window starts at the same offset in both CTAs, so aligned offsets match too
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -128,7 +135,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
       bool ok = true;
       for (int tile = pair; tile < num_tiles && ok; tile += n_pairs) {
         const int m0 = (tile % p.tiles_m) * 256 + (int)rank * 128;
-        const int n0 = (tile / p.tiles_m) * PAIR_BN + (int)rank * 128;
+        const int n0 = (tile / p.tiles_m) * PAIR_BN + (int)rank * (PAIR_BN / 2);
         for (int kb = 0; kb < k_blocks; ++kb) {
           ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.flags);
           if (!ok) break;
@@ -147,10 +154,11 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
               tma_load_2d_pair(a_dst + kh * SLAB_BYTES + 8192, &mapA, fb, m0 + 64, k0);
             }
             if (B_K) {
-              tma_load_2d_pair(b_dst + kh * SLAB_BYTES, &mapB, fb, k0, n0);
+              tma_load_2d_pair(b_dst + kh * B_SLAB, &mapB, fb, k0, n0);
             } else {
-              tma_load_2d_pair(b_dst + kh * SLAB_BYTES, &mapB, fb, n0, k0);
-              tma_load_2d_pair(b_dst + kh * SLAB_BYTES + 8192, &mapB, fb, n0 + 64, k0);
+#pragma unroll
+              for (int i = 0; i < PAIR_BN / 128; ++i)
+                tma_load_2d_pair(b_dst + kh * B_SLAB + i * 8192, &mapB, fb, n0 + 64 * i, k0);
             }
           }
           if (++s == ST) { s = 0; ph ^= 1u; }
@@ -178,9 +186,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
           const uint32_t b_addr = a_addr + HALF_BYTES;
 #pragma unroll
           for (int k = 0; k < PAIR_KH * (BK / UMMA_K); ++k) {
-            const uint32_t slab = (uint32_t)(k / (BK / UMMA_K)) * SLAB_BYTES, kk = (uint32_t)(k % (BK / UMMA_K));
+            const uint32_t kh = (uint32_t)(k / (BK / UMMA_K)), kk = (uint32_t)(k % (BK / UMMA_K));
+            const uint32_t slab = kh * SLAB_BYTES, slab_b = kh * B_SLAB;
             const uint64_t adesc = A_K ? make_desc(a_addr + slab + kk * 32, 16, 1024) : make_desc(a_addr + slab + kk * 2048, 8192, 1024);
-            const uint64_t bdesc = B_K ? make_desc(b_addr + slab + kk * 32, 16, 1024) : make_desc(b_addr + slab + kk * 2048, 8192, 1024);
+            const uint64_t bdesc = B_K ? make_desc(b_addr + slab_b + kk * 32, 16, 1024) : make_desc(b_addr + slab_b + kk * 2048, 8192, 1024);
             umma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
           }
           umma_commit_pair(empty_bar(s));        // both CTAs' slots are free once these MMAs have read them
@@ -222,18 +231,18 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
   }
 }
 
-template <bool A_K, bool B_K>
+template <int PAIR_BN, bool A_K, bool B_K>
 int launch_pair_t(const GemmArgs& g, const TcParams& p0, cudaStream_t st) {
   static bool attr_done = false;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(gemm_tc_pair_kernel<A_K, B_K>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             PAIR_SMEM) != cudaSuccess)
+    if (cudaFuncSetAttribute(gemm_tc_pair_kernel<PAIR_BN, A_K, B_K>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             PairCfg<PAIR_BN>::SMEM) != cudaSuccess)
       return -1;
     attr_done = true;
   }
   CUtensorMap mapA, mapB;
   if (!encode_map(&mapA, g.A, g.lda, A_K, g.M, g.K, 128)) return -2;
-  if (!encode_map(&mapB, g.B, g.ldb, B_K, g.N, g.K, 128)) return -2;
+  if (!encode_map(&mapB, g.B, g.ldb, B_K, g.N, g.K, PAIR_BN / 2)) return -2;
   TcParams p = p0;
   p.tiles_m = (g.M + 255) / 256;
   p.tiles_n = (g.N + PAIR_BN - 1) / PAIR_BN;
@@ -247,17 +256,24 @@ int launch_pair_t(const GemmArgs& g, const TcParams& p0, cudaStream_t st) {
     if (n_sm <= 0) n_sm = 148;
   }
   const int pairs = tiles < n_sm / 2 ? tiles : n_sm / 2;
-  gemm_tc_pair_kernel<A_K, B_K><<<2 * pairs, GEMM_THREADS, PAIR_SMEM, st>>>(mapA, mapB, p);
+  gemm_tc_pair_kernel<PAIR_BN, A_K, B_K><<<2 * pairs, GEMM_THREADS, PairCfg<PAIR_BN>::SMEM, st>>>(mapA, mapB, p);
   return cudaGetLastError() == cudaSuccess ? 0 : -3;
 }
 
 }  // namespace
 
+namespace {
+template <int PAIR_BN>
+int launch_pair_bn(const GemmArgs& g, const TcParams& p, cudaStream_t st) {
+  if (g.a_kmajor && g.b_kmajor) return launch_pair_t<PAIR_BN, true, true>(g, p, st);
+  if (g.a_kmajor && !g.b_kmajor) return launch_pair_t<PAIR_BN, true, false>(g, p, st);
+  if (!g.a_kmajor && g.b_kmajor) return launch_pair_t<PAIR_BN, false, true>(g, p, st);
+  return launch_pair_t<PAIR_BN, false, false>(g, p, st);
+}
+}  // namespace
+
 namespace gemm_tc_detail {
-int launch_gemm_tc_pair(const GemmArgs& g, const TcParams& p, cudaStream_t st) {
-  if (g.a_kmajor && g.b_kmajor) return launch_pair_t<true, true>(g, p, st);
-  if (g.a_kmajor && !g.b_kmajor) return launch_pair_t<true, false>(g, p, st);
-  if (!g.a_kmajor && g.b_kmajor) return launch_pair_t<false, true>(g, p, st);
-  return launch_pair_t<false, false>(g, p, st);
+int launch_gemm_tc_pair(const GemmArgs& g, const TcParams& p, int bn, cudaStream_t st) {
+  return bn == 128 ? launch_pair_bn<128>(g, p, st) : launch_pair_bn<256>(g, p, st);
 }
 }  // namespace gemm_tc_detail

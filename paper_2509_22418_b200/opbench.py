@@ -27,7 +27,7 @@ def main():
     ap.add_argument("--heads", type=int, default=16)
     ap.add_argument("--dh", type=int, default=128)
     ap.add_argument("--backend", type=int, default=0, help="attention: 0 tcgen05, 1 SIMT, 2 mma.sync; gemm: 0 tcgen05 (shape chosen), 1 SIMT, "
-                         "2 tcgen05 one CTA per tile, 3 tcgen05 SM pairs")
+                         "2 tcgen05 one CTA per tile, 3 tcgen05 SM pairs 256 x 256, 4 SM pairs 256 x 128")
     ap.add_argument("--iters", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     a = ap.parse_args()

@@ -29,8 +29,8 @@ GEMM_SHAPES = [
 
 
 # backends: 0 tcgen05 with the tile shape the step would choose, 1 SIMT, 2 tcgen05 one CTA per tile,
-# 3 tcgen05 SM pairs (cta_group::2)
-@pytest.mark.parametrize("backend", [0, 1, 2, 3])
+# 3 tcgen05 SM pairs (cta_group::2) on 256 x 256 tiles, 4 the same on 256 x 128 tiles
+@pytest.mark.parametrize("backend", [0, 1, 2, 3, 4])
 @pytest.mark.parametrize("a_k,b_k", [(1, 1), (1, 0), (0, 1), (0, 0)])
 @pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
 def test_gemm_against_oracle_matmul(backend, a_k, b_k, M, N, K):
@@ -59,7 +59,7 @@ def test_gemm_strided_operands_and_column_offset():
     dH, dH64 = _bf16_tensor(rng, (T, F))
     b, b64 = _bf16_tensor(rng, (T, d))
     ref = dH64[:, lo:hi].T @ b64                       # dW_in[lo:hi, :]
-    for backend in (0, 1, 2, 3):
+    for backend in (0, 1, 2, 3, 4):
         got = ppu.ppu_gemm(dH[:, lo:hi], 0, b, 0, hi - lo, d, T, out_f32=True, backend=backend)
         torch.cuda.synchronize()
         err = np.abs(got.cpu().numpy() - ref)
