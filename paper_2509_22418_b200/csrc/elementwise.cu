@@ -246,8 +246,16 @@ ln_bwd_warp_kernel(const bf16* __restrict__ dy, const float* __restrict__ x,
       s2 += a[i][j] * hh[i][j];
     }
   }
-  const float m1 = warp_sum(s1) * (1.f / d), m2 = warp_sum(s2) * (1.f / d);
+  // the incoming gradient is fetched before the reductions, so that its latency overlaps them
   const float4* gsrc = gin ? reinterpret_cast<const float4*>(gin + t * d) : nullptr;
+  float4 pin[NV][2];
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int c = lane + 32 * i;
+    if (gsrc) { pin[i][0] = gsrc[2 * c]; pin[i][1] = gsrc[2 * c + 1]; }
+    else { pin[i][0] = pin[i][1] = make_float4(0.f, 0.f, 0.f, 0.f); }
+  }
+  const float m1 = warp_sum(s1) * (1.f / d), m2 = warp_sum(s2) * (1.f / d);
   float4* gdst = reinterpret_cast<float4*>(gout + t * d);
   uint4* g16 = reinterpret_cast<uint4*>(gout16 + t * d);
 #pragma unroll
@@ -256,11 +264,8 @@ ln_bwd_warp_kernel(const bf16* __restrict__ dy, const float* __restrict__ x,
     float f[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) f[j] = st.y * (a[i][j] - m1 - hh[i][j] * m2);
-    if (gsrc) {
-      const float4 p0 = gsrc[2 * c], p1 = gsrc[2 * c + 1];
-      f[0] += p0.x; f[1] += p0.y; f[2] += p0.z; f[3] += p0.w;
-      f[4] += p1.x; f[5] += p1.y; f[6] += p1.z; f[7] += p1.w;
-    }
+    f[0] += pin[i][0].x; f[1] += pin[i][0].y; f[2] += pin[i][0].z; f[3] += pin[i][0].w;
+    f[4] += pin[i][1].x; f[5] += pin[i][1].y; f[6] += pin[i][1].z; f[7] += pin[i][1].w;
     gdst[2 * c] = make_float4(f[0], f[1], f[2], f[3]);
     gdst[2 * c + 1] = make_float4(f[4], f[5], f[6], f[7]);
     g16[c] = pack8(f);
