@@ -951,9 +951,9 @@ int launch_attn_fwd_tc(const bf16* qkv, bf16* U, float* lse, int B, int S, int h
 
 int launch_attn_bwd_tc(const bf16* qkv, const bf16* U, const float* lse, const bf16* dU, bf16* dqkv,
                        float* scratch, int B, int S, int h, int dh, int* flags, cudaStream_t st,
-                       const float2* inv_rope_cs) {
+                       const float2* inv_rope_cs, bool delta_done) {
   if (gemm_tc_init() != 0) return -1;
-  launch_attn_delta(U, dU, scratch, B, S, h, dh, st);
+  if (!delta_done) launch_attn_delta(U, dU, scratch, B, S, h, dh, st);
   if (dh == 64) return bwd_t<64>(qkv, lse, dU, dqkv, scratch, B, S, h, flags, st, inv_rope_cs);
   if (dh == 128) return bwd_t<128>(qkv, lse, dU, dqkv, scratch, B, S, h, flags, st, inv_rope_cs);
   return -1;

@@ -16,7 +16,11 @@ enum GemmEpilogue {
   EPI_GELU_DUAL = 2,   // C bf16 = acc (pre-activation), C2 bf16 = gelu(acc)
   EPI_RESID_F32 = 3,   // C fp32 = aux fp32 + acc (residual stream)
   EPI_DGELU = 4,       // C bf16 = acc * gelu'(aux bf16)
-  EPI_ROPE_BF16 = 5    // C bf16 = acc with rotary positions applied to the columns < rope_cols
+  EPI_ROPE_BF16 = 5,   // C bf16 = acc with rotary positions applied to the columns < rope_cols
+  // C bf16 = acc (the attention output's gradient dU), and per (token, head)
+  // C3 fp32 [batch, heads, rope_S] = sum over the head's rope_dh columns of C * aux (aux = U bf16):
+  // the row term of the softmax backward, formed while dU is still in registers
+  EPI_DELTA_BF16 = 6
 };
 
 struct GemmArgs {
@@ -43,6 +47,9 @@ struct GemmArgs {
 
 int launch_gemm_simt(const GemmArgs& g, cudaStream_t st);
 int launch_gemm_tc(const GemmArgs& g, cudaStream_t st);   // tcgen05 / TMEM / TMA
+// whether launch_gemm_tc accepts EPI_DELTA_BF16 for this product (tile shape and alignment allow
+// a thread to own whole heads of its row); otherwise the caller runs launch_attn_delta
+bool gemm_tc_fuses_delta(const GemmArgs& g);
 int gemm_tc_init();                                        // resolves the tensor-map encoder
 
 // ---- attention -------------------------------------------------------------
@@ -61,7 +68,8 @@ int launch_attn_fwd_tc(const bf16* qkv, bf16* U, float* lse, int B, int S, int h
                        cudaStream_t st);
 int launch_attn_bwd_tc(const bf16* qkv, const bf16* U, const float* lse, const bf16* dU, bf16* dqkv,
                        float* scratch, int B, int S, int h, int dh, int* flags, cudaStream_t st,
-                       const float2* inv_rope_cs = nullptr);   // non-null: rotate dq, dk back by -angle
+                       const float2* inv_rope_cs = nullptr,    // non-null: rotate dq, dk back by -angle
+                       bool delta_done = false);               // scratch already holds delta
 // delta[b,h,s] = sum_e dU * U of the head's slice
 void launch_attn_delta(const bf16* U, const bf16* dU, float* delta, int B, int S, int h, int dh,
                        cudaStream_t st);

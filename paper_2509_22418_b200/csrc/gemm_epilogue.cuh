@@ -94,6 +94,7 @@ __device__ __forceinline__ void drain_tile(const TcParams& p, int m0, int n0, in
   const int m = m0 + quarter * 32 + lane;
   const bool row_ok = m < p.M;
   const uint32_t t_row = t_acc + ((uint32_t)(quarter * 32) << 16);
+  float head_dot = 0.f;   // EPI_DELTA_BF16: running sum over the current head's columns
 #pragma unroll 1
   for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
     const int nb = n0 + c0;
@@ -141,6 +142,11 @@ __device__ __forceinline__ void drain_tile(const TcParams& p, int m0, int n0, in
           for (int j = 0; j < 4; ++j) st_v8((float*)p.C + ci + 8 * j, r + 8 * j);
         }
       } else {
+        uint32_t uv[16];
+        if (p.epilogue == EPI_DELTA_BF16 && row_ok) {
+          const bf16* us = (const bf16*)p.aux + (long long)m * p.ldaux + nb;
+          ld_v8(uv, us); ld_v8(uv + 8, us + 16);
+        }
         tmem_ld_wait();
         if (row_ok) {
           if (p.epilogue == EPI_ROPE_BF16 && nb < p.rope_cols) {
@@ -167,6 +173,20 @@ __device__ __forceinline__ void drain_tile(const TcParams& p, int m0, int n0, in
           for (int j = 0; j < 16; ++j) o[j] = pack2_bf16(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
           st_v8((bf16*)p.C + ci, o);
           st_v8((bf16*)p.C + ci + 16, o + 8);
+          if (p.epilogue == EPI_DELTA_BF16) {
+            // the product uses the stored (rounded) values, as the attention kernels will
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float2 gv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&o[j]));
+              const float2 u2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&uv[j]));
+              head_dot = fmaf(gv.x, u2.x, fmaf(gv.y, u2.y, head_dot));
+            }
+            if ((nb + 32) % p.rope_dh == 0) {
+              const int heads = p.N / p.rope_dh;
+              ((float*)p.C3)[((long long)(m / p.rope_S) * heads + nb / p.rope_dh) * p.rope_S + m % p.rope_S] = head_dot;
+              head_dot = 0.f;
+            }
+          }
           if (p.epilogue == EPI_GELU_DUAL) {
 #pragma unroll
             for (int j = 0; j < 16; ++j)

@@ -211,6 +211,7 @@ TcParams make_params(const GemmArgs& g) {
   if (g.epilogue == EPI_GELU_DUAL) w = w && (reinterpret_cast<uintptr_t>(g.C2) % 32 == 0);
   if (g.epilogue == EPI_RESID_F32) w = w && (reinterpret_cast<uintptr_t>(g.aux) % 32 == 0) && (g.ldaux % 8 == 0);
   if (g.epilogue == EPI_DGELU) w = w && (reinterpret_cast<uintptr_t>(g.aux) % 32 == 0) && (g.ldaux % 16 == 0);
+  if (g.epilogue == EPI_DELTA_BF16) w = w && (reinterpret_cast<uintptr_t>(g.aux) % 32 == 0) && (g.ldaux % 16 == 0);
   p.wide = w ? 1 : 0;
   return p;
 }
@@ -270,9 +271,28 @@ int gemm_tc_init() {
   return 0;
 }
 
+namespace {
+// the SM-pair kernel on 256 x 256 tiles is chosen for this product
+bool picks_pair256(const GemmArgs& g) {
+  const long long tiles_pair = (long long)((g.M + 255) / 256) * ((g.N + 255) / 256);
+  return g.tile_shape == 2 || (g.tile_shape == 0 && g.splits <= 1 && g.M > 128 && g.N > 128 && tiles_pair >= 74);
+}
+}  // namespace
+
+bool gemm_tc_fuses_delta(const GemmArgs& g) {
+  // a thread drains 128 consecutive columns of its row in 32-column chunks with 32-byte accesses:
+  // heads must be whole multiples of a chunk and must not straddle the 128-column boundary
+  GemmArgs probe = g;
+  probe.epilogue = EPI_DELTA_BF16;
+  const int dh = g.rope_dh;
+  return picks_pair256(g) && (dh == 32 || dh == 64 || dh == 128) && g.N % dh == 0 && g.N % 32 == 0 &&
+         g.rope_S > 0 && g.M % g.rope_S == 0 && g.aux && g.C3 && gemm_tc_detail::make_params(probe).wide;
+}
+
 int launch_gemm_tc(const GemmArgs& g, cudaStream_t st) {
   if (g.M <= 0 || g.N <= 0 || g.K <= 0) return 0;
   if (gemm_tc_init() != 0) return -1;
+  if (g.epilogue == EPI_DELTA_BF16 && !gemm_tc_fuses_delta(g)) return -4;
   if ((g.lda % 8) || (g.ldb % 8) || (g.ldc % 8) || (g.N % 8) ||
       (reinterpret_cast<uintptr_t>(g.A) & 15) || (reinterpret_cast<uintptr_t>(g.B) & 15) ||
       (reinterpret_cast<uintptr_t>(g.C) & 15))
@@ -282,11 +302,9 @@ int launch_gemm_tc(const GemmArgs& g, cudaStream_t st) {
   // (256 x 128 pair tiles would fill the last wave of the N = 2048 products better - 512 tiles
   // instead of 256 on 74 pairs - but their narrower instruction measured 25 % slower, so they are
   // never chosen here; tile_shape 3 keeps them testable.)
-  const long long tiles_pair = (long long)((g.M + 255) / 256) * ((g.N + 255) / 256);
   if ((g.tile_shape == 2 || g.tile_shape == 3) && g.splits > 1) return -4;
   if (g.tile_shape == 3) return launch_gemm_tc_pair(g, make_params(g), 128, st);
-  if (g.tile_shape == 2 || (g.tile_shape == 0 && g.splits <= 1 && g.M > 128 && g.N > 128 && tiles_pair >= 74))
-    return launch_gemm_tc_pair(g, make_params(g), 256, st);
+  if (picks_pair256(g)) return launch_gemm_tc_pair(g, make_params(g), 256, st);
   const long long tiles256 = (long long)((g.M + BM - 1) / BM) * ((g.N + 255) / 256) * (g.splits > 1 ? g.splits : 1);
   if (g.N > 128 && tiles256 >= 148) return launch_bn<256>(g, st);
   return launch_bn<128>(g, st);

@@ -194,20 +194,34 @@ struct Sched {
            nullptr, 0, &c->flops_dgrad);
       launch_ln_bwd(c->t16, a.x1, a.st2, Pf(l, c->rel_ln2g), c->g, c->g, c->g16, T, d, st);
       c->launches++;
-      gemm(c->g16, d, 1, W(l, c->rel_wo), d, 0, T, d, d, EPI_STORE_BF16, c->t16, d, nullptr, nullptr,
-           0, &c->flops_dgrad);
+      // dU = g1 W_O^T; where the tile shape allows, its epilogue also forms delta = rowsum(dU * U)
+      // per (token, head) for the attention backward
+      const int kind = attn_kind();
+      bool delta_fused = false;
+      if (kind == 0 && c->gemm_backend == 0) {
+        GemmArgs q;
+        q.A = c->g16; q.lda = d; q.a_kmajor = 1; q.B = W(l, c->rel_wo); q.ldb = d; q.b_kmajor = 0;
+        q.M = T; q.N = d; q.K = d; q.epilogue = EPI_DELTA_BF16; q.C = c->t16; q.ldc = d; q.C2 = nullptr;
+        q.aux = a.U; q.ldaux = d; q.flags = c->flags; q.C3 = c->attn_scratch; q.rope_S = S; q.rope_dh = dh;
+        delta_fused = gemm_tc_fuses_delta(q);
+      }
+      if (delta_fused)
+        gemm(c->g16, d, 1, W(l, c->rel_wo), d, 0, T, d, d, EPI_DELTA_BF16, c->t16, d, nullptr, a.U, d,
+             &c->flops_dgrad, 1, 0, 0, c->attn_scratch);
+      else
+        gemm(c->g16, d, 1, W(l, c->rel_wo), d, 0, T, d, d, EPI_STORE_BF16, c->t16, d, nullptr, nullptr,
+             0, &c->flops_dgrad);
       {
         const double fl = 10.0 * B * h * dh * 0.5 * S * (double)(S + 1);
         EvScope ev(c, 1, fl);
-        const int kind = attn_kind();
         if (kind == 0)   // rotates dq, dk back on the way out (the output drain overlaps the next item's products)
           rc |= launch_attn_bwd_tc(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, c->flags, st,
-                                   c->rope_cs);
+                                   c->rope_cs, delta_fused);
         else if (kind == 2)
           rc |= launch_attn_bwd_mma(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, st);
         else
           rc |= launch_attn_bwd_simt(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, st);
-        c->launches += kind == 1 ? 2 : 3;
+        c->launches += (kind == 1 ? 2 : 3) - (delta_fused ? 1 : 0);
         c->flops_dgrad += fl;
         if (kind != 0) { launch_rope(c->dqkv, c->rope_cs, B, S, h, dh, 1, st); c->launches++; }
       }

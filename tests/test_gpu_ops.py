@@ -86,7 +86,10 @@ def _attention_case(B, S, h, dh, seed):
 @pytest.mark.parametrize("backend", [1, 2, 0])
 @pytest.mark.parametrize("B,S,h,dh", [(2, 64, 4, 16), (1, 200, 2, 64), (2, 256, 2, 128), (1, 130, 3, 32),
                                       (1, 1024, 2, 128), (2, 333, 2, 64), (1, 2048, 1, 128), (1, 64, 1, 64),
-                                      (1, 7, 2, 64)])
+                                      (1, 7, 2, 64),
+                                      # more work items than SMs: every persistent CTA walks several
+                                      # items of different lengths, with a ragged last block
+                                      (3, 777, 16, 64), (2, 640, 40, 128)])
 def test_attention_forward_backward(backend, B, S, h, dh):
     import torch
     from paper_2509_22418_b200 import ppu
