@@ -485,25 +485,58 @@ class Replica:
 # --------------------------------------------------------------------------
 # outer synchronisation (Algorithm 1 lines 12-15; Eq. 2.4-2.5)
 # --------------------------------------------------------------------------
-def outer_sync(theta, buf, replicas, hp: Outer):
+def sync_group_mask(cfg: Model, group: int, n_groups: int) -> np.ndarray:
+    """Positions synchronised together under streaming synchronisation by layers
+    (Appendix "Streaming Synchronization"; Section 3.1): the L transformer
+    layers are split, in order, into n_groups groups of L / n_groups layers
+    (every tensor of those layers); one more group, index n_groups, holds the
+    embeddings and the outer normalisation.  The paper's 1.3B runs use 8 groups
+    of 3 layers plus that ninth group."""
+    L = cfg.n_layer
+    if n_groups < 1 or L % n_groups != 0 or not (0 <= group <= n_groups):
+        raise ValueError("bad group")
+    mask = np.zeros(n_params(cfg), dtype=bool)
+    per = L // n_groups
+    for name, off, shape in layout(cfg):
+        size = int(np.prod(shape))
+        if name.startswith("l") and "." in name and name[1:name.index(".")].isdigit():
+            layer = int(name[1:name.index(".")])
+            inside = group < n_groups and group * per <= layer < (group + 1) * per
+        else:                                   # E, lnf_g, lnf_b
+            inside = group == n_groups
+        if inside:
+            mask[off:off + size] = True
+    return mask
+
+
+def outer_sync(theta, buf, replicas, hp: Outer, mask=None):
     """Dense definition.  Delta_k is theta_k^(t,H) - theta^(t) on I_k^train and
     0 elsewhere; Delta = sum_k Delta_k / m with 0/0 := 0; the outer optimizer
     is SGD with Nesterov momentum on the pseudo-gradient g = -Delta.  Every
     listed replica restarts from the new global parameters.
-    Returns (theta_new, buf_new, m)."""
+    With a mask (streaming synchronisation: one group of positions at a time)
+    the step is taken on the masked positions only: elsewhere the global
+    parameters, the outer momentum and the replicas' own values stay as they
+    are.  Returns (theta_new, buf_new, m); m is counted on the masked
+    positions."""
     n = theta.shape[0]
+    sel = np.ones(n, dtype=bool) if mask is None else np.asarray(mask, dtype=bool)
     total = np.zeros(n, dtype=theta.dtype)
     for r in replicas:
         dk = np.zeros(n, dtype=theta.dtype)
         dk[r.idx] = r.theta_sub - theta[r.idx]
         total += dk
     m = count_vector(n, [r.idx for r in replicas])
+    m = np.where(sel, m, 0)
     delta = np.where(m > 0, total / np.maximum(m, 1), 0.0)
     g = -delta
-    buf_new = hp.momentum * buf + g
-    theta_new = theta - hp.lr * (g + hp.momentum * buf_new)
+    buf_step = hp.momentum * buf + g
+    theta_step = theta - hp.lr * (g + hp.momentum * buf_step)
+    buf_new = np.where(sel, buf_step, buf)
+    theta_new = np.where(sel, theta_step, theta)
     for r in replicas:
-        r.theta_sub = theta_new[r.idx].copy()
+        inside = sel[r.idx]
+        r.theta_sub = np.where(inside, theta_new[r.idx], r.theta_sub)
     return theta_new, buf_new, m
 
 

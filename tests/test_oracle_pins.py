@@ -172,3 +172,67 @@ def test_loss_at_init_is_log_vocab():
     cfg, th, tok = tiny()
     loss, _ = O.forward(cfg, th, tok, keep=False)
     assert abs(loss - math.log(cfg.vocab)) < 0.01 * math.log(cfg.vocab)
+
+
+# ---- streaming synchronisation by layer groups (Appendix "Streaming Synchronization") ------
+def test_sync_groups_partition_the_parameters_as_the_paper_describes():
+    # the paper's run: 24 layers in 8 groups of 3, plus a ninth group for the embeddings and
+    # the outer normalisation
+    cfg = O.Model(24, 32, 2, 64, 48)
+    P, d, F, V = O.n_params(cfg), 32, 64, 48
+    per_layer = 4 * d * d + 2 * d * F + 4 * d
+    masks = [O.sync_group_mask(cfg, g, 8) for g in range(9)]
+    assert np.array_equal(np.sum(masks, axis=0), np.ones(P, dtype=np.int64))       # disjoint cover
+    assert all(int(m.sum()) == 3 * per_layer for m in masks[:8])
+    assert int(masks[8].sum()) == V * d + 2 * d
+    views = O.views(cfg, masks[2].astype(np.int64))
+    assert np.all(views["l6.W_q"] == 1) and np.all(views["l8.ln2_b"] == 1) and np.all(views["l8.W_out"] == 1)
+    assert not views["l5.W_out"].any() and not views["l9.ln1_g"].any() and not views["E"].any()
+    with pytest.raises(ValueError):
+        O.sync_group_mask(cfg, 0, 5)           # 24 layers do not split into 5 groups
+
+
+def test_streaming_sync_is_the_full_step_taken_group_by_group():
+    cfg, th, tok = tiny()
+    hp = O.Outer(lr=0.7, momentum=0.9)
+    rng = np.random.default_rng(5)
+    buf0 = rng.normal(0, 1e-3, len(th))
+
+    def moved_replicas():
+        reps = [O.Replica(cfg, th, O.slice_ranges(cfg, 2, k), train_non_mlp=True) for k in range(4)]
+        r2 = np.random.default_rng(9)
+        for r in reps:
+            r.theta_sub = r.theta_sub + r2.normal(0, 1e-2, r.theta_sub.shape)
+        return reps
+
+    full = moved_replicas()
+    th_full, buf_full, m_full = O.outer_sync(th, buf0, full, hp)
+    for order in ([0, 1, 2], [2, 0, 1]):
+        reps = moved_replicas()
+        th_s, buf_s = th.copy(), buf0.copy()
+        for g in order:
+            mask = O.sync_group_mask(cfg, g, 2)
+            before = (th_s.copy(), buf_s.copy(), [r.theta_sub.copy() for r in reps])
+            th_s, buf_s, m = O.outer_sync(th_s, buf_s, reps, hp, mask=mask)
+            # outside the group nothing moves: global parameters, momentum, replicas' values
+            assert np.array_equal(th_s[~mask], before[0][~mask])
+            assert np.array_equal(buf_s[~mask], before[1][~mask])
+            assert np.array_equal(m, np.where(mask, m_full, 0))
+            for r, old in zip(reps, before[2]):
+                out = ~mask[r.idx]
+                assert np.array_equal(r.theta_sub[out], old[out])
+                assert np.array_equal(r.theta_sub[~out], th_s[r.idx][~out])
+        # positions do not interact in the outer step: every group once == the full step, exactly
+        assert np.array_equal(th_s, th_full) and np.array_equal(buf_s, buf_full)
+        for r, rf in zip(reps, full):
+            assert np.array_equal(r.theta_sub, rf.theta_sub)
+    # closed form of a first step on a group (momentum buffer zero): theta + eta (1 + mu) Delta
+    reps = moved_replicas()
+    mask = O.sync_group_mask(cfg, 1, 2)
+    # (the replicas' index lists agree on the non-MLP tail: equal slice widths put it at the same offsets)
+    delta = np.mean([r.theta_sub for r in reps], axis=0) - th[reps[0].idx]
+    idx = reps[0].idx
+    th1, _, m = O.outer_sync(th, np.zeros_like(th), reps, hp, mask=mask)
+    shared = (m[idx] == 4)                     # the non-MLP positions, trained by all four replicas
+    assert shared.any()
+    assert np.allclose((th1 - th)[idx][shared], (0.7 * 1.9 * delta)[shared], rtol=1e-9, atol=1e-15)
