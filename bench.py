@@ -233,12 +233,25 @@ def run_round(args):
     st = ctx.ppu_stats()
     steps_ms, outer_ms = ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2])
     pk = peaks()
+    # the same sync taken as a streaming sync: 8 groups of 3 layers plus the embeddings / final norm
+    # group (Appendix "Streaming Synchronization"), each group timed on its own
+    G, groups = 8, []
+    for g in range(G + 1):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        ctx.ppu_outer_sync_group(list(range(K)), g, G)
+        b.record()
+        torch.cuda.synchronize()
+        by = ctx.ppu_stats().outer_bytes
+        groups.append(dict(group=g, ms=a.elapsed_time(b), algorithmic_bytes=by,
+                           gbs=by / (a.elapsed_time(b) * 1e-3) / 1e9))
     print(json.dumps(dict(
         metric="full outer round, 1.3B", replicas=K, inner_steps=H, round_s=(steps_ms + outer_ms) * 1e-3,
         tokens_per_s=K * H * B * S / ((steps_ms + outer_ms) * 1e-3), local_step_ms=steps_ms / (K * H),
         outer_sync=dict(ms=outer_ms, algorithmic_bytes=st.outer_bytes,
                         gbs=st.outer_bytes / (outer_ms * 1e-3) / 1e9, peak_gbs=pk["hbm"],
                         frac=st.outer_bytes / (outer_ms * 1e-3) / 1e9 / pk["hbm"], of=pk["src"]),
+        streaming_sync=dict(n_groups=G + 1, total_ms=sum(g["ms"] for g in groups), groups=groups),
         last_losses=losses, data="synthetic", hbm_bytes=st.arena_bytes)))
 
 

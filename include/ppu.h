@@ -126,6 +126,18 @@ int ppu_local_step_host(ppu_ctx* ctx, int replica, const int32_t* tokens_host, i
  * 6).  AdamW moments and step counts are kept.  Asynchronous. */
 int ppu_outer_sync(ppu_ctx* ctx, const int32_t* replicas, int n);
 
+/* Streaming synchronisation by layers (Appendix "Streaming Synchronization", Section
+ * 3.1): the same outer step, taken on one group of positions only.  The n_layer
+ * layers are split in order into n_groups groups of n_layer / n_groups layers (every
+ * tensor of those layers); group == n_groups is one more group holding the embeddings
+ * and the final LayerNorm (the paper: 24 layers as 8 groups of 3, plus that ninth
+ * group).  Outside the group nothing changes: not the global parameters, not the
+ * outer momentum, not the listed replicas' own values (they keep training from where
+ * they are).  The caller owns the schedule (which group after which local steps).
+ * n_layer must be a multiple of n_groups and 0 <= group <= n_groups, else PPU_EINVAL.
+ * replicas: HOST array, no duplicates.  Asynchronous. */
+int ppu_outer_sync_group(ppu_ctx* ctx, const int32_t* replicas, int n, int group, int n_groups);
+
 /* Loss of the replica's most recent local step: Eq. 2.2 as the mean negative
  * log-likelihood (nats) over the batch*(seq-1) predicted tokens.  Waits for the
  * stream.  loss_out: HOST. */

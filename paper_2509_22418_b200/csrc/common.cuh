@@ -129,5 +129,9 @@ struct OuterTables {
   int64_t P, e_size, layer_size, win_rel, wout_rel;  // canonical geometry
   int32_t L, d, F;
 };
+// Segments of the canonical vector the outer sweep works through: 0-3 quarters of E, then three
+// per layer (non-FFN block, W_in, W_out), then the final LayerNorm.  The sweep covers segments
+// [seg_lo, seg_lo + seg_count).
+inline int outer_segments(int n_layer) { return 4 + 3 * n_layer + 1; }
 void launch_outer(const OuterTables& t, float* theta, float* buf, bf16* w16, float lr, float mu,
-                  cudaStream_t st);
+                  int seg_lo, int seg_count, cudaStream_t st);

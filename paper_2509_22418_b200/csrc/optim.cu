@@ -105,9 +105,9 @@ __device__ __forceinline__ void outer_update(float4& th, float4& bu, const float
 
 __global__ void __launch_bounds__(256)
 outer_kernel(OuterTables t, float* __restrict__ theta, float* __restrict__ buf,
-             bf16* __restrict__ w16, float lr, float mu) {
+             bf16* __restrict__ w16, float lr, float mu, int seg_lo) {
   // ---- segment decoding (uniform per block) ----
-  const int seg = blockIdx.y;
+  const int seg = seg_lo + blockIdx.y;
   int64_t start; int64_t len; int kind = 0, layer = 0;
   const int64_t fd = (int64_t)t.F * t.d;
   if (seg < 4) {
@@ -226,8 +226,13 @@ void launch_slices_scatter_f32(const SliceSeg* segs, int n_seg, const float* pac
 }
 
 void launch_outer(const OuterTables& t, float* theta, float* buf, bf16* w16, float lr, float mu,
-                  cudaStream_t st) {
-  // 4 segments for E, 3 per layer, 1 for the final LayerNorm; ~2 waves of 256-thread blocks
-  dim3 grid(32, 4 + 3 * t.L + 1);
-  outer_kernel<<<grid, 256, 0, st>>>(t, theta, buf, w16, lr, mu);
+                  int seg_lo, int seg_count, cudaStream_t st) {
+  if (seg_count <= 0) return;
+  // 4 segments for E, 3 per layer, 1 for the final LayerNorm
+  // enough blocks for about four waves of three resident blocks per SM, never fewer than 32 per
+  // segment (a streaming-sync group has few segments)
+  int gx = (4 * 3 * 148 + seg_count - 1) / seg_count;
+  gx = gx < 32 ? 32 : (gx > 256 ? 256 : gx);
+  dim3 grid(gx, seg_count);
+  outer_kernel<<<grid, 256, 0, st>>>(t, theta, buf, w16, lr, mu, seg_lo);
 }

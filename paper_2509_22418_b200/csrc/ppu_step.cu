@@ -320,9 +320,14 @@ extern "C" int ppu_eval_loss(ppu_ctx* c, int replica, const int32_t* tokens, int
   return ppu_check_flags(c);
 }
 
-extern "C" int ppu_outer_sync(ppu_ctx* c, const int32_t* replicas, int n) {
+namespace {
+// Outer step over the listed replicas on one group of positions (group < 0: every position).
+int outer_sync_impl(ppu_ctx* c, const int32_t* replicas, int n, int group, int n_groups) {
   if (!c) return ppu_fail(PPU_EINVAL, "ctx is null");
   if (n < 0 || (n > 0 && !replicas)) return ppu_fail(PPU_EINVAL, "bad replica list");
+  const int L = c->cfg.n_layer, F = c->cfg.d_ff, d = c->cfg.d_model;
+  if (group >= 0 && (n_groups < 1 || L % n_groups != 0 || group > n_groups))
+    return ppu_fail(PPU_EINVAL, "group %d of %d does not divide %d layers", group, n_groups, L);
   std::vector<int32_t> list(replicas, replicas + n);
   {
     std::vector<int32_t> sorted = list;
@@ -332,10 +337,17 @@ extern "C" int ppu_outer_sync(ppu_ctx* c, const int32_t* replicas, int n) {
       if (i && sorted[i] == sorted[i - 1]) return ppu_fail(PPU_EINVAL, "replica %d listed twice", sorted[i]);
     }
   }
-  const int L = c->cfg.n_layer, F = c->cfg.d_ff, d = c->cfg.d_model;
   const int64_t launches0 = c->launches;
+  // layers [l0, l1) and, for the last group, the embeddings and the final LayerNorm
+  const bool all = group < 0, tail = all || group == n_groups;
+  const int per = all ? L : L / n_groups;
+  const int l0 = all ? 0 : (tail ? L : group * per), l1 = all ? L : (tail ? L : l0 + per);
   double owned = 0;
-  for (int k : list) owned += (double)c->reps[k].n_sub;
+  for (int k : list) {
+    const ReplicaState& r = c->reps[k];
+    for (size_t i = 0; i < r.segs.size(); ++i)
+      if (r.seg_layer[i] >= l0 && r.seg_layer[i] < l1) owned += 2.0 * (double)(r.segs[i].hi - r.segs[i].lo) * d;
+  }
   if (list != c->cached_sync_list || list.empty()) {
     std::vector<OuterOwner> owners;
     std::vector<std::vector<int32_t>> per_group((size_t)L * (F / 8));
@@ -367,17 +379,46 @@ extern "C" int ppu_outer_sync(ppu_ctx* c, const int32_t* replicas, int n) {
       CUDA_OK(cudaMemcpy(c->d_unit_owner, flat.data(), flat.size() * 4, cudaMemcpyHostToDevice));
     c->cached_sync_list = list;
   }
+  // a group step rewrites the working copy only on its own positions: everywhere else it must
+  // already hold the global values, not the resident replica's
+  if (!all) ppu_make_resident(c, -1);
   OuterTables t;
   t.owners = c->d_owners; t.unit_begin = c->d_unit_begin; t.unit_owner = c->d_unit_owner;
   t.P = c->P; t.e_size = c->e_size; t.layer_size = c->layer_size; t.win_rel = c->rel_win;
   t.wout_rel = c->rel_wout; t.L = L; t.d = d; t.F = F;
-  launch_outer(t, c->theta, c->buf, c->w16, c->cfg.outer_lr, c->cfg.outer_momentum, c->stream);
-  c->launches++;
-  c->resident = -1;   // the working copy now holds the new global parameters everywhere
+  const int n_seg = outer_segments(L);
+  double swept = 0;
+  auto sweep = [&](int seg_lo, int seg_count) {
+    if (seg_count <= 0) return;
+    launch_outer(t, c->theta, c->buf, c->w16, c->cfg.outer_lr, c->cfg.outer_momentum, seg_lo, seg_count, c->stream);
+    c->launches++;
+  };
+  if (all) {
+    sweep(0, n_seg);
+    swept = (double)c->P;
+  } else if (tail) {
+    sweep(0, 4);                // embeddings
+    sweep(n_seg - 1, 1);        // final LayerNorm
+    swept = (double)c->e_size + (double)(c->P - c->e_size - (int64_t)L * c->layer_size);
+  } else {
+    sweep(4 + 3 * l0, 3 * (l1 - l0));
+    swept = (double)(l1 - l0) * (double)c->layer_size;
+  }
+  c->resident = -1;   // the working copy now holds the global parameters everywhere
   c->launches_last_sync = c->launches - launches0;
-  c->outer_bytes = 18.0 * (double)c->P + 8.0 * owned;
+  c->outer_bytes = 18.0 * swept + 8.0 * owned;
   CUDA_OK(cudaGetLastError());
   return PPU_OK;
+}
+}  // namespace
+
+extern "C" int ppu_outer_sync(ppu_ctx* c, const int32_t* replicas, int n) {
+  return outer_sync_impl(c, replicas, n, -1, 0);
+}
+
+extern "C" int ppu_outer_sync_group(ppu_ctx* c, const int32_t* replicas, int n, int group, int n_groups) {
+  if (group < 0) return ppu_fail(PPU_EINVAL, "group %d is negative", group);
+  return outer_sync_impl(c, replicas, n, group, n_groups);
 }
 
 extern "C" int ppu_profile_enable(ppu_ctx* c, int enable) {

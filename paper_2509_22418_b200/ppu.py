@@ -150,6 +150,10 @@ class Context:
         r = np.ascontiguousarray(list(replicas), dtype=np.int32)
         _check(lib().ppu_outer_sync(self._h, _np_ptr(r, C.c_int32), len(r)))
 
+    def ppu_outer_sync_group(self, replicas, group: int, n_groups: int) -> None:
+        r = np.ascontiguousarray(list(replicas), dtype=np.int32)
+        _check(lib().ppu_outer_sync_group(self._h, _np_ptr(r, C.c_int32), len(r), group, n_groups))
+
     def ppu_loss(self, replica: int) -> float:
         out = C.c_double()
         _check(lib().ppu_loss(self._h, replica, C.byref(out)))

@@ -222,3 +222,64 @@ def test_host_entry_point_and_argument_errors():
     spec, _ = ppu.make_spec(6, n_slices=4)                                   # K not a multiple of N
     with pytest.raises(ppu.PpuError):
         ppu.ppu_query_bytes(cfg, spec)
+
+
+def _check_outer_group(P: Pair, replicas, group, n_groups):
+    """One streaming-sync step on a group of layers against the oracle's masked outer step."""
+    theta_before = P.ctx.ppu_get_params(-1)
+    buf_before = P.ctx.ppu_get_outer_momentum()
+    local_before = {k: P.ctx.ppu_get_params(k) for k in replicas}
+    P.ctx.ppu_outer_sync_group(replicas, group, n_groups)
+    P.ctx.ppu_sync()
+    th_gpu = P.ctx.ppu_get_params(-1)
+    buf_gpu = P.ctx.ppu_get_outer_momentum()
+    mask = O.sync_group_mask(P.ocfg, group, n_groups)
+    P.theta, P.buf, m = O.outer_sync(P.theta, P.buf, [P.reps[k] for k in replicas], P.outer, mask=mask)
+    # outside the group, and where no listed replica trains: the same bits as before
+    still = ~mask | (m == 0)
+    assert np.array_equal(th_gpu[still], theta_before[still])
+    assert np.array_equal(buf_gpu[still], buf_before[still])
+    tr = m > 0
+    if tr.any():
+        assert max_abs_over_norm(th_gpu[tr], P.theta[tr]) <= TENSOR_TOL
+        assert max_abs_over_norm(buf_gpu[tr], P.buf[tr]) <= TENSOR_TOL
+    assert np.array_equal(P.ctx.ppu_get_working_bf16(), bf16_bits(th_gpu))
+    for k in replicas:
+        now = P.ctx.ppu_get_params(k)
+        idx = P.reps[k].idx
+        inside = np.zeros(len(now), bool)
+        inside[idx] = mask[idx]
+        assert np.array_equal(now[inside], th_gpu[inside])                     # restarted in the group
+        assert np.array_equal(now[~inside], np.where(mask, th_gpu, local_before[k])[~inside])   # kept elsewhere
+        assert max_abs_over_norm(now[idx], P.reps[k].theta_sub) <= TENSOR_TOL
+
+
+def test_streaming_sync_by_layer_groups():
+    """Appendix "Streaming Synchronization": the outer step taken on one group of layers at a time,
+    with local steps in between; a group that no replica trains (embeddings, final norm) moves
+    nothing."""
+    dims = (4, 64, 4, 256, 512)
+    ranges = [O.slice_ranges(O.Model(*dims), 4, k) for k in range(4)]
+    P = Pair(dims, ranges, 4, 64, seed=5, adam=O.AdamW(1e-3, 0.9, 0.95, 1e-8, 0.1),
+             outer=O.Outer(0.7, 0.9))
+    try:
+        order = [(k, h) for k in range(4) for h in range(2)]
+        for k, h in order:
+            tok = P.tokens(k, 0, h, 4, 64)
+            P.gpu_step(k, tok)
+            P.reps[k].local_step(P.theta, tok, P.adam)
+        _check_outer_group(P, [0, 1, 2, 3], 0, 2)          # layers 0-1
+        for k in range(4):                                  # replicas go on from mixed parameters
+            tok = P.tokens(k, 1, 0, 4, 64)
+            loss_gpu, _ = P.gpu_step(k, tok)
+            loss_ref = P.reps[k].local_step(P.theta, tok, P.adam)
+            assert abs(loss_gpu - loss_ref) <= LOSS_RTOL * abs(loss_ref)
+        _check_outer_group(P, [0, 1, 3], 1, 2)              # layers 2-3, replica 2 sits out
+        _check_outer_group(P, [0, 1, 2, 3], 2, 2)           # embeddings + final norm: nothing trained
+        _check_outer_group(P, [0, 1, 2, 3], 0, 4)           # a finer grouping: layer 0 alone
+        with pytest.raises(P.ppu.PpuError):
+            P.ctx.ppu_outer_sync_group([0], 0, 3)           # 4 layers do not split into 3 groups
+        with pytest.raises(P.ppu.PpuError):
+            P.ctx.ppu_outer_sync_group([0], 3, 2)           # only groups 0..2 exist
+    finally:
+        P.close()
