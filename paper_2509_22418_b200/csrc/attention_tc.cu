@@ -31,8 +31,9 @@
 namespace {
 using namespace tc;
 
-constexpr int DQ_THREADS = 352;   // as BWD_THREADS plus warp 10: second MMA-issuing thread
-constexpr int BWD_THREADS = 320;  // warp 0 TMA, warp 1 MMA, warps 2-5 and 6-9: two row groups, half the slab columns each
+// backward kernels: warp 0 TMA, warp 1 first MMA-issuing thread, warps 2-5 and 6-9 two row groups (half
+// the slab columns each), warp 10 second MMA-issuing thread
+constexpr int DQ_THREADS = 352;
 constexpr float LOG2E = 1.4426950408889634f;
 
 __device__ __forceinline__ float ex2(float x) {
