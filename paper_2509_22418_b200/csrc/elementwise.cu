@@ -192,6 +192,14 @@ ln_fwd_warp_kernel(const float* __restrict__ x, const float* __restrict__ g,
 #pragma unroll
     for (int j = 0; j < 8; ++j) s += v[i][j];
   }
+  // gain and bias are fetched before the reductions, so that their latency overlaps them
+  float4 gq[NV][2], bq2[NV][2];
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int c = lane + 32 * i;
+    gq[i][0] = reinterpret_cast<const float4*>(g)[2 * c]; gq[i][1] = reinterpret_cast<const float4*>(g)[2 * c + 1];
+    bq2[i][0] = reinterpret_cast<const float4*>(b)[2 * c]; bq2[i][1] = reinterpret_cast<const float4*>(b)[2 * c + 1];
+  }
   const float mean = warp_sum(s) * (1.f / d);
   float q = 0.f;
 #pragma unroll
@@ -204,10 +212,8 @@ ln_fwd_warp_kernel(const float* __restrict__ x, const float* __restrict__ g,
 #pragma unroll
   for (int i = 0; i < NV; ++i) {
     const int c = lane + 32 * i;
-    const float4 g0 = reinterpret_cast<const float4*>(g)[2 * c], g1 = reinterpret_cast<const float4*>(g)[2 * c + 1];
-    const float4 b0 = reinterpret_cast<const float4*>(b)[2 * c], b1 = reinterpret_cast<const float4*>(b)[2 * c + 1];
-    const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-    const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+    const float gg[8] = {gq[i][0].x, gq[i][0].y, gq[i][0].z, gq[i][0].w, gq[i][1].x, gq[i][1].y, gq[i][1].z, gq[i][1].w};
+    const float bb[8] = {bq2[i][0].x, bq2[i][0].y, bq2[i][0].z, bq2[i][0].w, bq2[i][1].x, bq2[i][1].y, bq2[i][1].z, bq2[i][1].w};
     float f[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) f[j] = (v[i][j] - mean) * rstd * gg[j] + bb[j];
