@@ -49,6 +49,35 @@ def test_125m_two_replicas_one_step_and_outer_sync():
         assert np.array_equal(th_gpu[m == 0], theta0[m == 0])
         assert max_abs_over_norm(th_gpu[m > 0], P.theta[m > 0]) <= TENSOR_TOL
         assert np.array_equal(P.ctx.ppu_get_working_bf16(), bf16_bits(th_gpu))
+        # streaming synchronisation at this size: another step of replica 5 (the GPU step runs at
+        # full size; the oracle only needs the replica's new values, taken from the GPU within
+        # the tolerance checked above, like the global parameters and momentum), then the outer
+        # step on one group of three layers only
+        tok = P.tokens(5, 1, 0, 8, 1024)
+        P.gpu_step(5, tok)
+        th5 = P.ctx.ppu_get_params(5)
+        P.reps[5].theta_sub = th5[P.reps[5].idx].astype(np.float64)
+        P.reps[0].theta_sub = P.ctx.ppu_get_params(0)[P.reps[0].idx].astype(np.float64)
+        P.theta = th_gpu.astype(np.float64)
+        buf_before = P.ctx.ppu_get_outer_momentum()
+        P.buf = buf_before.astype(np.float64)
+        P.ctx.ppu_outer_sync_group([0, 5], 2, 4)          # layers 6-8
+        P.ctx.ppu_sync()
+        th2 = P.ctx.ppu_get_params(-1)
+        buf2 = P.ctx.ppu_get_outer_momentum()
+        mask = O.sync_group_mask(P.ocfg, 2, 4)
+        ref_th, ref_buf, m = O.outer_sync(P.theta, P.buf, [P.reps[0], P.reps[5]], P.outer, mask=mask)
+        still = ~mask | (m == 0)
+        assert np.array_equal(th2[still], th_gpu[still]) and np.array_equal(buf2[still], buf_before[still])
+        assert (m > 0).any()
+        assert max_abs_over_norm(th2[m > 0], ref_th[m > 0]) <= 1e-5      # same inputs: fp32 rounding only
+        assert max_abs_over_norm(buf2[m > 0], ref_buf[m > 0]) <= 1e-5
+        assert np.array_equal(P.ctx.ppu_get_working_bf16(), bf16_bits(th2))
+        now5 = P.ctx.ppu_get_params(5)
+        inside = np.zeros(len(now5), bool)
+        inside[P.reps[5].idx] = mask[P.reps[5].idx]
+        assert np.array_equal(now5[inside], th2[inside])                   # restarted inside the group
+        assert np.array_equal(now5[~inside & ~mask], th5[~inside & ~mask])  # kept outside it
     finally:
         P.close()
 
