@@ -473,13 +473,19 @@ class Replica:
         g = np.concatenate(parts) if parts else np.zeros(0, dtype=th.dtype)
         return loss, g
 
-    def local_step(self, theta_global, tokens, hp: AdamW, mode="restricted"):
-        loss, g = self.gradient(theta_global, tokens, mode)
+    def apply_gradient(self, loss, g, hp: AdamW):
+        """Algorithm 1 line 10 for a gradient g[I_train] that is already known (several
+        nodes that start from the same parameters and see the same batch share one full
+        backward pass: each takes its own entries of it)."""
         self.t += 1
         self.theta_sub, self.m, self.v = adamw_update(self.theta_sub, g, self.m,
                                                       self.v, self.t, hp)
         self.last_loss, self.last_grad = loss, g
         return loss
+
+    def local_step(self, theta_global, tokens, hp: AdamW, mode="restricted"):
+        loss, g = self.gradient(theta_global, tokens, mode)
+        return self.apply_gradient(loss, g, hp)
 
 
 # --------------------------------------------------------------------------

@@ -36,12 +36,14 @@ def normal_tensor(seed: int, tensor_id: int, n: int, std: float,
     return out.astype(dtype, copy=False)
 
 
-def init_params(seed: int, tensors, std: float = 0.02) -> np.ndarray:
+def init_params(seed: int, tensors, std: float = 0.02, ln_jitter: float = 0.0) -> np.ndarray:
     """Flat fp32 parameter vector for a list of (name, offset, shape) records.
 
     Tensors whose name ends in '_g' are LayerNorm gains (ones), '_b' shifts
-    (zeros); everything else is N(0, std).  The caller supplies the records
-    (each side derives them from its own layout code).
+    (zeros); everything else is N(0, std).  With ln_jitter > 0 the gains are
+    1 + N(0, ln_jitter) and the shifts N(0, ln_jitter), as after some training,
+    so that a gain or shift that is ignored or swapped changes the result.  The
+    caller supplies the records (each side derives them from its own layout code).
     """
     total = max(off + int(np.prod(shape)) for _, off, shape in tensors)
     theta = np.empty(total, dtype=np.float32)
@@ -49,8 +51,12 @@ def init_params(seed: int, tensors, std: float = 0.02) -> np.ndarray:
         n = int(np.prod(shape))
         if name.endswith("_g"):
             theta[off:off + n] = 1.0
+            if ln_jitter > 0:
+                theta[off:off + n] += normal_tensor(seed, tid, n, ln_jitter)
         elif name.endswith("_b"):
             theta[off:off + n] = 0.0
+            if ln_jitter > 0:
+                theta[off:off + n] += normal_tensor(seed, tid, n, ln_jitter)
         else:
             theta[off:off + n] = normal_tensor(seed, tid, n, std)
     return theta

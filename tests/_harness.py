@@ -1,5 +1,19 @@
 """Shared pieces of the GPU parity tests: build a library context and the matching oracle
-state from the same seeded inputs, and the error metrics the tolerances are stated in."""
+state from the same seeded inputs, and the gates the tolerances are stated in.
+
+Gates.  The stated tolerance for gradients and updated weights is 2e-2 in max-abs over
+l2-norm.  That metric shrinks with the square root of the vector length (an all-zero gradient of
+a 25M-element subset scores 1e-3), so every gate here pairs it with one that cannot be passed
+by a wrong result at any size:
+  * gradients, AdamW moments: relative l2 error <= 2e-2 as well;
+  * updates (the change of the trained values over one step, not the values themselves):
+    AdamW's early updates are lr * sign-like, so an element whose gradient is below the bf16
+    noise floor may legitimately move the other way.  Elements whose update differs from the
+    oracle's by more than 10 % of the step scale must all be such knife-edge elements
+    (|g_ref| <= 0.05 rms(g_ref) at some step so far) and fewer than 2 % of the vector; the
+    rest must agree to 2e-2 in relative l2.
+tests/test_gates_can_fail.py plants mistakes in the oracle and checks that each gate rejects them.
+"""
 from __future__ import annotations
 
 import numpy as np
@@ -8,7 +22,10 @@ from oracle import ppu_oracle as O
 from paper_2509_22418_b200 import synth
 
 LOSS_RTOL = 1e-3        # losses: relative
-TENSOR_TOL = 2e-2       # subset gradients and updated weights: max-abs over l2-norm
+TENSOR_TOL = 2e-2       # subset gradients and updated weights: max-abs over l2-norm, and relative l2
+KNIFE_TAU = 0.05        # |g_ref| <= KNIFE_TAU * rms(g_ref): the sign of an AdamW step may differ
+KNIFE_FRAC = 0.02       # at most this share of a vector may differ by more than UPDATE_TOL * scale
+UPDATE_TOL = 0.10
 
 
 def max_abs_over_norm(a, b):
@@ -33,11 +50,54 @@ def bf16_bits(x):
     return ((u + 0x7FFF + ((u >> 16) & 1)) >> 16).astype(np.uint16)
 
 
+# ---- gates ---------------------------------------------------------------------------------
+def gate_vector(got, ref, what="gradient", tol=TENSOR_TOL):
+    """The stated metric and the relative l2 error, both <= tol.  Returns the two numbers."""
+    a, b = max_abs_over_norm(got, ref), rel_l2(got, ref)
+    assert a <= tol, f"{what}: max-abs over norm {a:.3e} > {tol}"
+    assert b <= tol, f"{what}: relative l2 {b:.3e} > {tol}"
+    return a, b
+
+
+def knife_edge(g_ref, tau=KNIFE_TAU):
+    """Elements whose reference gradient is small enough for bf16 noise to turn its sign."""
+    g = np.asarray(g_ref, dtype=np.float64)
+    rms = float(np.sqrt(np.mean(g * g))) if g.size else 0.0
+    return np.abs(g) <= tau * rms
+
+
+def gate_update(d_got, d_ref, scale, knife, what="update", tol=TENSOR_TOL):
+    """d_got, d_ref: change of the trained values over the step(s); scale: size of one full step
+    (the learning rate for AdamW); knife: boolean mask of knife-edge candidates.  Returns
+    (share of elements off by more than UPDATE_TOL * scale, relative l2 of the others)."""
+    d_got = np.asarray(d_got, dtype=np.float64)
+    d_ref = np.asarray(d_ref, dtype=np.float64)
+    assert d_got.shape == d_ref.shape
+    assert np.linalg.norm(d_ref) > 0, f"{what}: the reference did not move"
+    off = np.abs(d_got - d_ref) > UPDATE_TOL * scale
+    share = float(off.mean()) if off.size else 0.0
+    assert share < KNIFE_FRAC, f"{what}: {share:.2%} of the elements differ by more than {UPDATE_TOL} x step"
+    assert knife[off].all(), (f"{what}: {int((off & ~knife).sum())} elements differ by more than "
+                              f"{UPDATE_TOL} x step although their gradient is not near zero")
+    r = rel_l2(d_got[~off], d_ref[~off])
+    assert r <= tol, f"{what}: relative l2 {r:.3e} > {tol} outside the knife-edge elements"
+    return share, r
+
+
+def gate_adam_state(m_got, v_got, step_got, rep, tol=TENSOR_TOL):
+    """AdamW moments and step count of the library against the oracle replica's."""
+    assert step_got == rep.t, f"AdamW step count {step_got} != {rep.t}"
+    gate_vector(m_got, rep.m, "AdamW first moment", tol)
+    # v is quadratic in the gradient: its elementwise relative error is twice the gradient's
+    gate_vector(v_got, rep.v, "AdamW second moment", 2 * tol)
+
+
 class Pair:
     """A library context and the oracle's state for the same model, subset and seed."""
 
     def __init__(self, dims, ranges, max_batch, max_seq, seed=11, adam=None, outer=None,
-                 mode=None, n_slices=1, layer_stride=1, dtype=np.float64):
+                 mode=None, n_slices=1, layer_stride=1, dtype=np.float64, ln_jitter=0.0,
+                 train_non_mlp=False, head_ranges=None):
         from paper_2509_22418_b200 import ppu
         self.ppu = ppu
         L, d, h, F, V = dims
@@ -50,18 +110,31 @@ class Pair:
                            adam_beta1=self.adam.beta1, adam_beta2=self.adam.beta2,
                            adam_eps=self.adam.eps, adam_wd=self.adam.wd, outer_lr=self.outer.lr,
                            outer_momentum=self.outer.momentum)
+        extra = {}
+        if train_non_mlp:
+            extra["train_non_mlp"] = 1
+        if head_ranges is not None:
+            extra["head_ranges"] = np.asarray(head_ranges, np.int32)
         if mode is None:
-            spec, keep = ppu.make_spec(K, ppu.SUBSET_EXPLICIT, ranges=np.asarray(ranges, np.int32))
+            spec, keep = ppu.make_spec(K, ppu.SUBSET_EXPLICIT, ranges=np.asarray(ranges, np.int32), **extra)
         else:
-            spec, keep = ppu.make_spec(K, mode, n_slices=n_slices, layer_stride=layer_stride)
+            spec, keep = ppu.make_spec(K, mode, n_slices=n_slices, layer_stride=layer_stride, **extra)
         self.ctx = ppu.Context(cfg, spec, keep)
         recs = self.ctx.tensors()
         assert [(n, o, tuple(s)) for n, o, s in recs] == [(n, o, tuple(s)) for n, o, s in O.layout(self.ocfg)]
-        self.theta32 = synth.init_params(seed, recs)
+        self.theta32 = synth.init_params(seed, recs, ln_jitter=ln_jitter)
         self.ctx.ppu_set_params(self.theta32)
         self.theta = self.theta32.astype(dtype)          # oracle's global parameters
         self.buf = np.zeros_like(self.theta)
-        self.reps = [O.Replica(self.ocfg, self.theta, r) for r in ranges]
+        okw = {}
+        if train_non_mlp:
+            okw["train_non_mlp"] = True
+        if head_ranges is not None:
+            self.reps = [O.Replica(self.ocfg, self.theta, r, head_range=tuple(hr), **okw)
+                         for r, hr in zip(ranges, head_ranges)]
+        else:
+            self.reps = [O.Replica(self.ocfg, self.theta, r, **okw) for r in ranges]
+        self.knife = [np.zeros(len(r.idx), bool) for r in self.reps]   # knife-edge candidates so far
         self.seed = seed
 
     def tokens(self, k, rnd, step, B, S):
@@ -73,6 +146,33 @@ class Pair:
         self.ctx.ppu_local_step(k, t)
         loss = self.ctx.ppu_loss(k)
         return loss, t
+
+    def step_and_gate(self, k, tok, oracle_tok=None, check=True):
+        """One local step of replica k on both sides, every per-step gate applied.  oracle_tok:
+        the batch the oracle sees when it differs from the library's (a batch of identical
+        sequences has the loss and gradient of one of them).  Returns a record of the numbers."""
+        rep = self.reps[k]
+        before = self.ctx.ppu_get_params(k)[rep.idx].astype(np.float64)
+        sub_before = rep.theta_sub.astype(np.float64)
+        loss_gpu, _ = self.gpu_step(k, tok)
+        loss_ref = rep.local_step(self.theta, tok if oracle_tok is None else oracle_tok, self.adam)
+        self.knife[k] |= knife_edge(rep.last_grad)
+        g_gpu = self.ctx.ppu_get_subset_grads(k)
+        after = self.ctx.ppu_get_params(k)[rep.idx].astype(np.float64)
+        m_gpu, v_gpu, t_gpu = self.ctx.ppu_get_subset_state(k)
+        rec = dict(k=k, loss_gpu=loss_gpu, loss_ref=loss_ref,
+                   grad_err=max_abs_over_norm(g_gpu, rep.last_grad), grad_l2=rel_l2(g_gpu, rep.last_grad),
+                   w_err=max_abs_over_norm(after, rep.theta_sub),
+                   m_l2=rel_l2(m_gpu, rep.m), v_l2=rel_l2(v_gpu, rep.v))
+        if check:
+            assert abs(loss_gpu - loss_ref) <= LOSS_RTOL * abs(loss_ref), rec
+            gate_vector(g_gpu, rep.last_grad, "subset gradient")
+            assert rec["w_err"] <= TENSOR_TOL, rec
+            rec["upd_off"], rec["upd_l2"] = gate_update(
+                after - before, rep.theta_sub.astype(np.float64) - sub_before, self.adam.lr,
+                self.knife[k], "AdamW update")
+            gate_adam_state(m_gpu, v_gpu, t_gpu, rep)
+        return rec
 
     def close(self):
         self.ctx.close()

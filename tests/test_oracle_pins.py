@@ -236,3 +236,56 @@ def test_streaming_sync_is_the_full_step_taken_group_by_group():
     shared = (m[idx] == 4)                     # the non-MLP positions, trained by all four replicas
     assert shared.any()
     assert np.allclose((th1 - th)[idx][shared], (0.7 * 1.9 * delta)[shared], rtol=1e-9, atol=1e-15)
+
+
+# ---- the fp32-storage path used at the 1.3B shapes ------------------------------------------
+def test_float32_storage_path_agrees_with_float64():
+    """At the largest shapes the oracle stores parameters and activations in float32 (numpy's
+    products then accumulate in float32 as well).  On a mid-size model the same functions in
+    float32 must reproduce their float64 results to float32 accuracy: loss, restricted gradient,
+    AdamW step."""
+    cfg = O.Model(4, 256, 4, 1024, 2048)
+    th64 = synth.init_params(5, O.layout(cfg), ln_jitter=0.1).astype(np.float64)
+    th32 = th64.astype(np.float32)
+    tok = synth.tokens(5, 0, 0, 0, 2, 128, cfg.vocab)
+    ranges = O.slice_ranges(cfg, 4, 2)
+    hp = O.AdamW(3e-4, 0.9, 0.99, 1e-8, 0.1)
+    r64, r32 = O.Replica(cfg, th64, ranges), O.Replica(cfg, th32, ranges)
+    l64 = r64.local_step(th64, tok, hp)
+    l32 = r32.local_step(th32, tok, hp)
+    assert r32.last_grad.dtype == np.float32 and r32.theta_sub.dtype == np.float32
+    assert abs(l32 - l64) <= 2e-6 * l64
+    g64, g32 = r64.last_grad, r32.last_grad.astype(np.float64)
+    assert np.linalg.norm(g32 - g64) <= 2e-5 * np.linalg.norm(g64)
+    assert np.abs(g32 - g64).max() <= 1e-4 * np.abs(g64).max()
+    # the first AdamW step is lr * (sign(g) + wd * theta): equal wherever the sign is decided
+    d64, d32 = r64.theta_sub - th64[r64.idx], r32.theta_sub.astype(np.float64) - th64[r64.idx]
+    decided = np.abs(g64) > 1e-4 * np.abs(g64).max()
+    assert np.abs(d32 - d64)[decided].max() <= 1e-3 * hp.lr
+    _, gf32 = O.grad_full(cfg, th32, tok)
+    _, gf64 = O.grad_full(cfg, th64, tok)
+    assert np.linalg.norm(gf32 - gf64) <= 2e-5 * np.linalg.norm(gf64)
+
+
+def test_whole_layer_assignment_geometry():
+    """"Every 4th block": the node with index n trains the complete W_in and W_out of the blocks
+    n, n + 4, ... and nothing else; the four index sets tile the FFN parameters exactly once."""
+    cfg = O.Model(8, 16, 2, 32, 24)
+    recs = {name: (off, int(np.prod(shape))) for name, off, shape in O.layout(cfg)}
+    sets = []
+    for n in range(4):
+        ranges = O.layer_ranges(cfg, 4, n)
+        assert [l for l, (lo, hi) in enumerate(ranges) if hi > lo] == [n, n + 4]
+        assert all((lo, hi) in ((0, 0), (0, cfg.d_ff)) for lo, hi in ranges)
+        idx = O.train_index(cfg, ranges)
+        want = np.concatenate([np.arange(recs[f"l{l}.{w}"][0], sum(recs[f"l{l}.{w}"]))
+                               for l in (n, n + 4) for w in ("W_in", "W_out")])
+        assert np.array_equal(np.sort(idx), want) and len(np.unique(idx)) == len(idx)
+        assert O.layer_ranges(cfg, 4, n + 4) == ranges              # replica k uses n = k mod stride
+        sets.append(idx)
+    m = O.count_vector(O.n_params(cfg), sets)
+    ffn = np.zeros(O.n_params(cfg), bool)
+    for name, (off, size) in recs.items():
+        if name.endswith("W_in") or name.endswith("W_out"):
+            ffn[off:off + size] = True
+    assert np.array_equal(m == 1, ffn) and m.max() == 1
