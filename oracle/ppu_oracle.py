@@ -11,8 +11,10 @@ What it computes, all in numpy (float64 unless a dtype is passed), following
 * the decoder forward pass on all parameters and the loss of Eq. 2.2;
 * the gradient of Algorithm 1 line 9 in two ways: the definition (full
   backward, then mask to the trainable index set) and the restricted backward
-  of Appendix C.1 (weight gradients only for the trained FFN slice, input
-  gradients through every slice, nothing below the lowest trained layer);
+  of Appendix C.1 (weight gradients only for the trained FFN slice and, under
+  head slicing, for the trained heads' query / key / value projections; input
+  gradients through every slice and head; nothing below the lowest trained
+  layer when only FFN slices are trained);
 * the inner AdamW update on the subset (Algorithm 1 line 10, Section 3.1);
 * per-node deltas, the count vector m, the count-normalised average and the
   outer Nesterov step (Algorithm 1 lines 12-15, Eq. 2.4-2.5);
@@ -26,7 +28,8 @@ weights are stored [out, in] (y = x W^T), so the paper's W in R^{4d x d} is
 W_in and V in R^{d x 4d} is W_out; pre-LayerNorm blocks; GELU in its tanh form;
 rotary positions on adjacent pairs with base 1e4; tied input/output embedding;
 no linear biases; loss = mean over the B*(S-1) predicted tokens; AdamW with
-bias correction and eps = 1e-8; Nesterov in the "buf = mu*buf + g, step with
+bias correction and eps = 1e-8, weight decay on matrices only (not on the
+normalisation layers' gains and shifts); Nesterov in the "buf = mu*buf + g, step with
 g + mu*buf" form with g = -Delta.
 
 Parity pins live in tests/test_oracle_*.py.  Conventions above that no printed
@@ -319,32 +322,55 @@ def grad_full(cfg: Model, theta: np.ndarray, tokens: np.ndarray):
     return loss, g
 
 
-def grad_restricted(cfg: Model, theta: np.ndarray, tokens: np.ndarray, ranges):
-    """Restricted backward of Appendix C.1 for FFN hidden-unit slices.
+def head_rows(cfg: Model, head_range):
+    """Rows of W_q / W_k / W_v (stored [out, in]) that belong to the heads
+    [h_lo, h_hi): the paper's columns W_Q[:, H_n] of Section 2.2.1."""
+    h_lo, h_hi = head_range
+    return h_lo * cfg.d_head, h_hi * cfg.d_head
 
-    ranges[l] = (lo, hi): hidden units of layer l this node trains (lo == hi:
-    none).  Returns (loss, {l: (dW_in[lo:hi, :], dW_out[:, lo:hi])}).
-    Weight gradients are formed for the trained slice only; the input gradient
-    runs through every slice and every head; below the lowest trained layer
-    nothing is computed, and at that layer only its own slice's part.
+
+def grad_restricted(cfg: Model, theta: np.ndarray, tokens: np.ndarray, ranges,
+                    head_range=None, train_rest=False):
+    """Restricted backward of Appendix C.1.
+
+    ranges[l] = (lo, hi): FFN hidden units of layer l this node trains (lo ==
+    hi: none) - "MLP" part of the appendix.  head_range = (h_lo, h_hi): heads
+    whose query / key / value projections it trains - "MHA" part: the weight
+    gradients of the other heads are not formed, the input gradient still sums
+    over every head.  train_rest: the node also trains what Section 2.2.1 never
+    slices (embedding tied to the output head, W_o, every normalisation layer).
+
+    Returns (loss, out): out[l] = (dW_in[lo:hi, :], dW_out[:, lo:hi]);
+    out["qkv", l] = the trained rows of (dW_q, dW_k, dW_v); with train_rest
+    also out["W_o", l], out["ln1", l] and out["ln2", l] = (dgamma, dbeta),
+    out["lnf"] and out["E"].  Input gradients run through every slice and every
+    head.  When only FFN slices are trained nothing is computed below the
+    lowest trained layer, and at that layer only its own slice's part.
     """
     loss, c = forward(cfg, theta, tokens)
     P = views(cfg, theta)
     B, S = tokens.shape
+    d = cfg.d_model
+    heads = head_range is not None and head_range[1] > head_range[0]
+    deep = heads or train_rest                      # the backward pass reaches layer 0
     trained = [l for l in range(cfg.n_layer) if ranges[l][1] > ranges[l][0]]
     out = {}
-    if not trained:
+    if not trained and not deep:
         return loss, out
-    l0 = min(trained)
-    dl = _dlogits(cfg, c)
-    df = _mm(dl, P["E"])
-    gx, _, _ = layernorm_bwd(df, P["lnf_g"], c["lnf"])
+    l0 = 0 if deep else min(trained)
     T2 = lambda t: t.reshape(B * S, -1)
+    dl = _dlogits(cfg, c)
+    if train_rest:
+        out["E"] = T2(dl).T @ T2(c["f"])            # output head, tied to the embedding
+    df = _mm(dl, P["E"])
+    gx, dgam, dbet = layernorm_bwd(df, P["lnf_g"], c["lnf"])
+    if train_rest:
+        out["lnf"] = (dgam, dbet)
     for l in reversed(range(l0, cfg.n_layer)):
         p = f"l{l}."
         L = c["layers"][l]
         lo, hi = ranges[l]
-        if l == l0:
+        if l == l0 and not deep:
             dA_n = _mm(gx, P[p + "W_out"][:, lo:hi])
             dH_n = dA_n * gelu_grad(L["Hd"][..., lo:hi])
             out[l] = (T2(dH_n).T @ T2(L["b"]), T2(gx).T @ T2(L["Ac"][..., lo:hi]))
@@ -355,17 +381,30 @@ def grad_restricted(cfg: Model, theta: np.ndarray, tokens: np.ndarray, ranges):
             out[l] = (T2(dH[..., lo:hi]).T @ T2(L["b"]),
                       T2(gx).T @ T2(L["Ac"][..., lo:hi]))
         db = _mm(dH, P[p + "W_in"])
-        dx1, _, _ = layernorm_bwd(db, P[p + "ln2_g"], L["ln2"])
+        dx1, dgam, dbet = layernorm_bwd(db, P[p + "ln2_g"], L["ln2"])
+        if train_rest:
+            out["ln2", l] = (dgam, dbet)
         g1 = gx + dx1
+        if train_rest:
+            out["W_o", l] = T2(g1).T @ T2(L["U"])
         dU = _mm(g1, P[p + "W_o"])
         dq, dk, dv = _attention_bwd(cfg, L, dU, c)
         dq = rope(dq, c["cos"], c["sin"], inverse=True)
         dk = rope(dk, c["cos"], c["sin"], inverse=True)
-        d = cfg.d_model
+        if heads:
+            r0, r1 = head_rows(cfg, head_range)
+            a2 = T2(L["a"])
+            out["qkv", l] = tuple(T2(t)[:, r0:r1].T @ a2 for t in (dq, dk, dv))
+        if l == 0 and not train_rest:
+            break                                   # nothing below needs the input gradient
         da = (_mm(dq.reshape(B, S, d), P[p + "W_q"]) + _mm(dk.reshape(B, S, d), P[p + "W_k"])
               + _mm(dv.reshape(B, S, d), P[p + "W_v"]))
-        dx0, _, _ = layernorm_bwd(da, P[p + "ln1_g"], L["ln1"])
+        dx0, dgam, dbet = layernorm_bwd(da, P[p + "ln1_g"], L["ln1"])
+        if train_rest:
+            out["ln1", l] = (dgam, dbet)
         gx = g1 + dx0
+    if train_rest:
+        np.add.at(out["E"], tokens.reshape(-1), gx.reshape(B * S, d))
     return loss, out
 
 
@@ -387,11 +426,15 @@ def layer_ranges(cfg: Model, stride: int, replica: int):
     return [(0, cfg.d_ff) if l % stride == n else (0, 0) for l in range(cfg.n_layer)]
 
 
-def train_index(cfg: Model, ranges, train_non_mlp=False) -> np.ndarray:
+def train_index(cfg: Model, ranges, train_non_mlp=False, head_range=None) -> np.ndarray:
     """Flat indices of I_k^train in a fixed order: for each layer the W_in rows
-    block, then the W_out column block (row-major over [d, hi-lo]); when
-    train_non_mlp is set, every non-FFN parameter follows (the paper's
-    MLP-only slicing trains those on all nodes)."""
+    block, then the W_out column block (row-major over [d, hi-lo]); then, in
+    the order of the parameter vector, what the node trains outside the FFNs.
+    train_non_mlp: every non-FFN parameter (the paper's MLP-only slicing
+    trains those on all nodes).  head_range = (h_lo, h_hi): of W_q, W_k, W_v
+    only the rows of those heads (MLP + attention-head slicing: the columns
+    W_{Q,K,V}[:, H_n] of Section 2.2.1; W_o is not sliced); it may be combined
+    with train_non_mlp or stand alone."""
     recs = {name: (off, shape) for name, off, shape in layout(cfg)}
     d, F = cfg.d_model, cfg.d_ff
     parts = []
@@ -405,12 +448,27 @@ def train_index(cfg: Model, ranges, train_non_mlp=False) -> np.ndarray:
         rows = np.arange(d, dtype=np.int64)[:, None] * F
         cols = np.arange(lo, hi, dtype=np.int64)[None, :]
         parts.append((off_out + rows + cols).reshape(-1))
-    if train_non_mlp:
-        for name, off, shape in layout(cfg):
-            if name.endswith("W_in") or name.endswith("W_out"):
-                continue
+    for name, off, shape in layout(cfg):
+        if name.endswith("W_in") or name.endswith("W_out"):
+            continue
+        if name.endswith(("W_q", "W_k", "W_v")) and head_range is not None:
+            r0, r1 = head_rows(cfg, head_range)
+            if r1 > r0:
+                parts.append(off + np.arange(r0 * d, r1 * d, dtype=np.int64))
+        elif train_non_mlp:
             parts.append(off + np.arange(int(np.prod(shape)), dtype=np.int64))
     return np.concatenate(parts) if parts else np.zeros(0, dtype=np.int64)
+
+
+def decay_flags(cfg: Model, idx: np.ndarray) -> np.ndarray:
+    """True where weight decay applies: positions inside matrices.  Section 3.1
+    gives AdamW's weight decay (0.1) without saying which tensors it covers;
+    the reading taken here is the usual one - matrices decay, the gains and
+    shifts of the normalisation layers do not."""
+    recs = layout(cfg)
+    starts = np.array([off for _, off, _ in recs], dtype=np.int64)
+    is_matrix = np.array([len(shape) == 2 for _, _, shape in recs])
+    return is_matrix[np.searchsorted(starts, idx, side="right") - 1]
 
 
 def count_vector(n_total: int, index_sets) -> np.ndarray:
@@ -424,14 +482,16 @@ def count_vector(n_total: int, index_sets) -> np.ndarray:
 # --------------------------------------------------------------------------
 # inner optimizer (Algorithm 1 line 10; AdamW, Section 3.1)
 # --------------------------------------------------------------------------
-def adamw_update(p, g, m, v, t, hp: AdamW):
+def adamw_update(p, g, m, v, t, hp: AdamW, decay=None):
     """One decoupled-weight-decay Adam step on arrays of equal shape; t is the
-    1-based step count.  Returns new (p, m, v)."""
+    1-based step count; decay (optional, boolean) marks the elements the weight
+    decay applies to (all of them when omitted).  Returns new (p, m, v)."""
     m = hp.beta1 * m + (1.0 - hp.beta1) * g
     v = hp.beta2 * v + (1.0 - hp.beta2) * g * g
     mhat = m / (1.0 - hp.beta1 ** t)
     vhat = v / (1.0 - hp.beta2 ** t)
-    p = p - hp.lr * (mhat / (np.sqrt(vhat) + hp.eps) + hp.wd * p)
+    shrink = hp.wd * p if decay is None else np.where(decay, hp.wd * p, 0.0)
+    p = p - hp.lr * (mhat / (np.sqrt(vhat) + hp.eps) + shrink)
     return p, m, v
 
 
@@ -441,11 +501,14 @@ class Replica:
     from the global vector and never written."""
 
     def __init__(self, cfg: Model, theta_global: np.ndarray, ranges,
-                 train_non_mlp=False):
+                 train_non_mlp=False, head_range=None):
         self.cfg = cfg
         self.ranges = list(ranges)
         self.train_non_mlp = train_non_mlp
-        self.idx = train_index(cfg, ranges, train_non_mlp)
+        self.head_range = head_range if head_range is not None else (
+            (0, cfg.n_head) if train_non_mlp else None)
+        self.idx = train_index(cfg, ranges, train_non_mlp, head_range)
+        self.decay = decay_flags(cfg, self.idx)
         self.theta_sub = theta_global[self.idx].copy()     # theta_k^(t,0) <- theta^(t)
         self.m = np.zeros_like(self.theta_sub)
         self.v = np.zeros_like(self.theta_sub)
@@ -459,17 +522,33 @@ class Replica:
         return th
 
     def gradient(self, theta_global, tokens, mode="restricted"):
-        """g_k[I_train] of Algorithm 1 line 9, in the order of self.idx."""
+        """g_k[I_train] of Algorithm 1 line 9, in the order of self.idx: by the
+        definition (mode "masked_full": the full gradient, then the mask) or by
+        the restricted backward of Appendix C.1."""
         th = self.materialise(theta_global)
-        if mode == "masked_full" or self.train_non_mlp:
+        if mode == "masked_full":
             loss, g = grad_full(self.cfg, th, tokens)
             return loss, g[self.idx]
-        loss, sl = grad_restricted(self.cfg, th, tokens, self.ranges)
+        loss, out = grad_restricted(self.cfg, th, tokens, self.ranges, self.head_range,
+                                    self.train_non_mlp)
         parts = []
         for l in range(self.cfg.n_layer):
-            if l in sl:
-                parts.append(sl[l][0].reshape(-1))
-                parts.append(sl[l][1].reshape(-1))
+            if l in out:
+                parts.append(out[l][0].reshape(-1))
+                parts.append(out[l][1].reshape(-1))
+        if ("qkv", 0) in out or self.train_non_mlp:       # non-FFN part, in the order of the vector
+            if self.train_non_mlp:
+                parts.append(out["E"].reshape(-1))
+            for l in range(self.cfg.n_layer):
+                if self.train_non_mlp:
+                    parts.extend(out["ln1", l])
+                if ("qkv", l) in out:
+                    parts.extend(t.reshape(-1) for t in out["qkv", l])
+                if self.train_non_mlp:
+                    parts.append(out["W_o", l].reshape(-1))
+                    parts.extend(out["ln2", l])
+            if self.train_non_mlp:
+                parts.extend(out["lnf"])
         g = np.concatenate(parts) if parts else np.zeros(0, dtype=th.dtype)
         return loss, g
 
@@ -479,7 +558,7 @@ class Replica:
         backward pass: each takes its own entries of it)."""
         self.t += 1
         self.theta_sub, self.m, self.v = adamw_update(self.theta_sub, g, self.m,
-                                                      self.v, self.t, hp)
+                                                      self.v, self.t, hp, self.decay)
         self.last_loss, self.last_grad = loss, g
         return loss
 

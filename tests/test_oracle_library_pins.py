@@ -115,18 +115,23 @@ def test_full_subset_is_plain_local_sgd_round():
         for h in range(H):
             reps[k].local_step(th, toks[k][h], hp_in)
     th_new, _, _ = O.outer_sync(th, np.zeros_like(th), reps, hp_out)
-    # plain loop
+    # plain loop: one torch tensor per parameter tensor, matrices in a group with weight decay,
+    # the normalisation layers' gains and shifts in a group without
+    recs = O.layout(cfg)
     ends = []
     for k in range(K):
-        order = np.argsort(reps[k].idx)
-        tk = torch.tensor(th, dtype=torch.float64, requires_grad=True)
-        opt = torch.optim.AdamW([tk], lr=hp_in.lr, betas=(hp_in.beta1, hp_in.beta2),
-                                eps=hp_in.eps, weight_decay=hp_in.wd)
+        ps = [torch.tensor(th[off:off + int(np.prod(sh))].copy(), dtype=torch.float64, requires_grad=True)
+              for _, off, sh in recs]
+        groups = [dict(params=[p for p, (_, _, sh) in zip(ps, recs) if len(sh) == 2], weight_decay=hp_in.wd),
+                  dict(params=[p for p, (_, _, sh) in zip(ps, recs) if len(sh) == 1], weight_decay=0.0)]
+        opt = torch.optim.AdamW(groups, lr=hp_in.lr, betas=(hp_in.beta1, hp_in.beta2), eps=hp_in.eps)
         for h in range(H):
-            _, g = O.grad_full(cfg, tk.detach().numpy().copy(), toks[k][h])
-            tk.grad = torch.tensor(g)
+            flat = np.concatenate([p.detach().numpy() for p in ps])
+            _, g = O.grad_full(cfg, flat, toks[k][h])
+            for p, (_, off, sh) in zip(ps, recs):
+                p.grad = torch.tensor(g[off:off + int(np.prod(sh))])
             opt.step()
-        ends.append(tk.detach().numpy().copy())
+        ends.append(np.concatenate([p.detach().numpy() for p in ps]))
     delta = np.mean([e - th for e in ends], axis=0)
     tt = torch.tensor(th, dtype=torch.float64, requires_grad=True)
     out = torch.optim.SGD([tt], lr=hp_out.lr, momentum=hp_out.momentum, nesterov=True)

@@ -289,3 +289,114 @@ def test_whole_layer_assignment_geometry():
         if name.endswith("W_in") or name.endswith("W_out"):
             ffn[off:off + size] = True
     assert np.array_equal(m == 1, ffn) and m.max() == 1
+
+
+# ---- MLP + attention-head slicing (Section 2.2.1, Appendix C.1 "MHA") ---------------------------
+@pytest.mark.parametrize("rho,printed", [(0.5, 0.72), (0.25, 0.44)])
+def test_table1_head_slicing_rows_through_the_index_sets(rho, printed):
+    """Table 1, "1/2 mlps + 1/2 heads" and "1/4 mlps + 1/4 heads": the size of the actual index
+    set of a node (its FFN slice, the query / key / value rows of its head group, and everything
+    that is never sliced) at the paper's shapes, in billions, to the two printed digits."""
+    cfg = O.Model(24, 2048, 16, 8192, 32000)
+    N = int(round(1 / rho))
+    n = N - 1                                              # the last slice and head group
+    ranges = O.slice_ranges(cfg, N, n)
+    hg = cfg.n_head // N
+    idx = O.train_index(cfg, ranges, train_non_mlp=True, head_range=(n * hg, (n + 1) * hg))
+    assert round(len(idx) / 1e9, 2) == printed
+    assert len(idx) == O.trainable_params(cfg, rho, rho)
+    assert idx.min() >= 0 and idx.max() < O.n_params(cfg)
+    # no position twice: the FFN part ascends layer by layer, the rest follows the vector's order
+    rest = idx[24 * 2 * (cfg.d_ff // N) * cfg.d_model:]
+    assert np.all(np.diff(rest) > 0)
+    del idx, rest
+
+
+def test_head_slicing_index_geometry():
+    """Head group n owns rows [n d_h g, (n+1) d_h g) of W_q, W_k and W_v in every layer (the
+    paper's columns W_{Q,K,V}[:, H_n] in this storage order), W_o whole; the groups tile the
+    three projections exactly once and share everything else."""
+    cfg = O.Model(3, 16, 4, 32, 24)
+    recs = {name: (off, shape) for name, off, shape in O.layout(cfg)}
+    d, dh = cfg.d_model, cfg.d_head
+    sets = []
+    for n in range(2):
+        hr = (2 * n, 2 * n + 2)
+        idx = O.train_index(cfg, [(0, 0)] * 3, head_range=hr)
+        want = np.concatenate([recs[f"l{l}.{w}"][0] + np.arange(hr[0] * dh * d, hr[1] * dh * d)
+                               for l in range(3) for w in ("W_q", "W_k", "W_v")])
+        assert np.array_equal(idx, want)
+        full = O.train_index(cfg, [(0, 0)] * 3, train_non_mlp=True, head_range=hr)
+        assert set(idx) <= set(full) and len(np.unique(full)) == len(full)
+        sets.append(full)
+    m = O.count_vector(O.n_params(cfg), sets)
+    qkv = np.zeros(O.n_params(cfg), bool)
+    ffn = np.zeros(O.n_params(cfg), bool)
+    for name, (off, shape) in recs.items():
+        size = int(np.prod(shape))
+        if name.endswith(("W_q", "W_k", "W_v")):
+            qkv[off:off + size] = True
+        if name.endswith(("W_in", "W_out")):
+            ffn[off:off + size] = True
+    assert np.all(m[qkv] == 1) and np.all(m[ffn] == 0) and np.all(m[~qkv & ~ffn] == 2)
+    # no head range and train_non_mlp: every head, i.e. the MLP-only scheme's non-FFN set
+    a = O.train_index(cfg, [(0, 8)] * 3, train_non_mlp=True)
+    b = O.train_index(cfg, [(0, 8)] * 3, train_non_mlp=True, head_range=(0, cfg.n_head))
+    assert np.array_equal(a, b)
+
+
+@pytest.mark.parametrize("train_rest,head_range,ranges", [
+    (False, (1, 2), [(8, 16), (8, 16)]),        # FFN slice + one head, everything else frozen
+    (True, (0, 1), [(0, 8), (16, 32)]),         # the paper's MLP + head slicing
+    (True, None, [(8, 16), (0, 0)]),            # the paper's MLP-only slicing: all heads trained
+    (False, (0, 2), [(0, 0), (0, 0)]),          # heads only
+])
+def test_head_sliced_restricted_gradient(train_rest, head_range, ranges):
+    """The restricted backward with head slicing against central differences and against the
+    definition (full gradient, then the mask)."""
+    cfg, th, tok = micro()
+    r = O.Replica(cfg, th, ranges, train_non_mlp=train_rest, head_range=head_range)
+    loss, g = r.gradient(th, tok, "restricted")
+    loss2, g2 = r.gradient(th, tok, "masked_full")
+    assert loss == loss2 and len(g) == len(r.idx)
+    assert np.abs(g - g2).max() <= 1e-12 * max(1.0, np.abs(g2).max())
+    rng = np.random.default_rng(2)
+    for j in rng.choice(len(r.idx), size=40, replace=False):
+        i, e = r.idx[j], 1e-5
+        tp, tm = th.copy(), th.copy()
+        tp[i] += e
+        tm[i] -= e
+        fd = (O.forward(cfg, tp, tok, keep=False)[0]
+              - O.forward(cfg, tm, tok, keep=False)[0]) / (2 * e)
+        assert abs(fd - g[j]) <= 1e-6 * max(1.0, abs(fd)) + 1e-9
+
+
+def test_frozen_heads_keep_their_bits_and_counts_under_head_slicing():
+    cfg, th, tok = micro()
+    hp = O.AdamW()
+    reps = [O.Replica(cfg, th, [(0, 16), (0, 16)] if n == 0 else [(16, 32), (16, 32)],
+                      train_non_mlp=True, head_range=(n, n + 1)) for n in (0, 1, 0, 1)]
+    for r in reps:
+        r.local_step(th, tok, hp)
+    after = reps[0].materialise(th)
+    own = np.zeros(len(th), bool)
+    own[reps[0].idx] = True
+    assert np.array_equal(after[~own], th[~own]) and np.all(after[own] != th[own])
+    m = O.count_vector(len(th), [r.idx for r in reps])
+    # K = 4 nodes, N = 2 slices: sliced parameters (FFN and q/k/v) are trained by K / N nodes,
+    # all others by K (Section 2.2.1)
+    recs = O.layout(cfg)
+    for name, off, shape in recs:
+        size = int(np.prod(shape))
+        sliced = name.endswith(("W_in", "W_out", "W_q", "W_k", "W_v"))
+        assert np.all(m[off:off + size] == (2 if sliced else 4)), name
+
+
+def test_decay_flags_follow_tensor_rank():
+    cfg = O.Model(2, 16, 2, 32, 24)
+    idx = np.arange(O.n_params(cfg))
+    fl = O.decay_flags(cfg, idx)
+    for name, off, shape in O.layout(cfg):
+        assert np.all(fl[off:off + int(np.prod(shape))] == (len(shape) == 2)), name
+    sub = np.array([0, 24 * 16, 24 * 16 + 15, 24 * 16 + 32, O.n_params(cfg) - 1])   # E, ln1_g, ln1_g, W_q, lnf_b
+    assert O.decay_flags(cfg, sub).tolist() == [True, False, False, True, False]
