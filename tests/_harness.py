@@ -7,11 +7,14 @@ a 25M-element subset scores 1e-3), so every gate here pairs it with one that can
 by a wrong result at any size:
   * gradients, AdamW moments: relative l2 error <= 2e-2 as well;
   * updates (the change of the trained values over one step, not the values themselves):
-    AdamW's early updates are lr * sign-like, so an element whose gradient is below the bf16
-    noise floor may legitimately move the other way.  Elements whose update differs from the
-    oracle's by more than 10 % of the step scale must all be such knife-edge elements
-    (|g_ref| <= 0.05 rms(g_ref) at some step so far) and fewer than 2 % of the vector; the
-    rest must agree to 2e-2 in relative l2.
+    AdamW's update is lr times a quotient of gradient averages, so an element's update carries
+    the relative error of its gradient, and where the gradient is below the bf16 noise floor
+    it may legitimately move the other way.  Element i may differ from the oracle's update by
+    step * (0.1 + 0.08 / r_i), r_i = the largest |g_ref,i| / rms(g_ref) over the steps so far
+    (gradients accurate to 1e-2 rms - half the gradient gate - at eight sigma), and by 2.2 steps
+    (a full step the other way) where r_i <= 0.08, i.e. where that noise can turn the sign;
+    fewer than 2 % of the elements may differ by more than 0.1 step; the rest must agree to
+    2e-2 in relative l2.
 tests/test_gates_can_fail.py plants mistakes in the oracle and checks that each gate rejects them.
 """
 from __future__ import annotations
@@ -23,9 +26,11 @@ from paper_2509_22418_b200 import synth
 
 LOSS_RTOL = 1e-3        # losses: relative
 TENSOR_TOL = 2e-2       # subset gradients and updated weights: max-abs over l2-norm, and relative l2
-KNIFE_TAU = 0.05        # |g_ref| <= KNIFE_TAU * rms(g_ref): the sign of an AdamW step may differ
-KNIFE_FRAC = 0.02       # at most this share of a vector may differ by more than UPDATE_TOL * scale
-UPDATE_TOL = 0.10
+UPDATE_TOL = 0.10       # an update may differ by this share of a step (plus the quotient's allowance)
+GRAD_NOISE = 0.01       # gradient accuracy the allowance assumes, in units of rms(g_ref) ...
+NOISE_SIGMAS = 8.0      # ... and how many sigmas of it an element may use (an element's noise follows the
+                        # magnitudes in its own row and column, not the rms over the whole subset)
+OFF_FRAC = 0.02         # at most this share of a vector may differ by more than UPDATE_TOL * step
 
 
 def max_abs_over_norm(a, b):
@@ -59,28 +64,39 @@ def gate_vector(got, ref, what="gradient", tol=TENSOR_TOL):
     return a, b
 
 
-def knife_edge(g_ref, tau=KNIFE_TAU):
-    """Elements whose reference gradient is small enough for bf16 noise to turn its sign."""
+def grad_rel(g_ref):
+    """|g_ref| in units of its rms: how far each element's gradient is from the noise floor."""
     g = np.asarray(g_ref, dtype=np.float64)
     rms = float(np.sqrt(np.mean(g * g))) if g.size else 0.0
-    return np.abs(g) <= tau * rms
+    return np.abs(g) / max(rms, 1e-300)
 
 
-def gate_update(d_got, d_ref, scale, knife, what="update", tol=TENSOR_TOL):
+def step_allowance(grel):
+    """What one AdamW step of an element may differ by, in steps: UPDATE_TOL plus the relative
+    error of its gradient, at most a full step the other way."""
+    noise = NOISE_SIGMAS * GRAD_NOISE
+    return np.where(grel <= noise, 2.2, UPDATE_TOL + noise / np.maximum(grel, noise))
+
+
+def gate_update(d_got, d_ref, scale, allow, what="update", tol=TENSOR_TOL):
     """d_got, d_ref: change of the trained values over the step(s); scale: size of one full step
-    (the learning rate for AdamW); knife: boolean mask of knife-edge candidates.  Returns
-    (share of elements off by more than UPDATE_TOL * scale, relative l2 of the others)."""
+    (the learning rate for AdamW); allow: per element what it may differ by, in steps
+    (step_allowance, summed over the steps the compared change accumulates).  Returns (share of
+    elements off by more than UPDATE_TOL * scale, relative l2 of the others)."""
     d_got = np.asarray(d_got, dtype=np.float64)
     d_ref = np.asarray(d_ref, dtype=np.float64)
     assert d_got.shape == d_ref.shape
     assert np.linalg.norm(d_ref) > 0, f"{what}: the reference did not move"
-    off = np.abs(d_got - d_ref) > UPDATE_TOL * scale
+    err = np.abs(d_got - d_ref) / scale
+    worst = int(np.argmax(err - allow))
+    assert err[worst] <= allow[worst], (
+        f"{what}: element {worst} differs by {err[worst]:.3f} steps, allowed {allow[worst]:.3f}; "
+        f"{int((err > allow).sum())} such elements")
+    off = err > UPDATE_TOL
     share = float(off.mean()) if off.size else 0.0
-    assert share < KNIFE_FRAC, f"{what}: {share:.2%} of the elements differ by more than {UPDATE_TOL} x step"
-    assert knife[off].all(), (f"{what}: {int((off & ~knife).sum())} elements differ by more than "
-                              f"{UPDATE_TOL} x step although their gradient is not near zero")
+    assert share < OFF_FRAC, f"{what}: {share:.2%} of the elements differ by more than {UPDATE_TOL} x step"
     r = rel_l2(d_got[~off], d_ref[~off])
-    assert r <= tol, f"{what}: relative l2 {r:.3e} > {tol} outside the knife-edge elements"
+    assert r <= tol, f"{what}: relative l2 {r:.3e} > {tol} over the elements within {UPDATE_TOL} x step"
     return share, r
 
 
@@ -134,7 +150,11 @@ class Pair:
                          for r, hr in zip(ranges, head_ranges)]
         else:
             self.reps = [O.Replica(self.ocfg, self.theta, r, **okw) for r in ranges]
-        self.knife = [np.zeros(len(r.idx), bool) for r in self.reps]   # knife-edge candidates so far
+        # per replica and trained element: largest |g_ref| / rms(g_ref) over its steps so far
+        self.grel = [np.zeros(len(r.idx)) for r in self.reps]
+        # ... and the allowances of its steps since the last outer sync, summed (tests/_harness.py
+        # gate_update); an outer step carries mu of it on in the momentum
+        self.allow_acc = [np.zeros(len(r.idx)) for r in self.reps]
         self.seed = seed
 
     def tokens(self, k, rnd, step, B, S):
@@ -156,7 +176,8 @@ class Pair:
         sub_before = rep.theta_sub.astype(np.float64)
         loss_gpu, _ = self.gpu_step(k, tok)
         loss_ref = rep.local_step(self.theta, tok if oracle_tok is None else oracle_tok, self.adam)
-        self.knife[k] |= knife_edge(rep.last_grad)
+        self.grel[k] = np.maximum(self.grel[k], grad_rel(rep.last_grad))
+        self.allow_acc[k] += step_allowance(self.grel[k])
         g_gpu = self.ctx.ppu_get_subset_grads(k)
         after = self.ctx.ppu_get_params(k)[rep.idx].astype(np.float64)
         m_gpu, v_gpu, t_gpu = self.ctx.ppu_get_subset_state(k)
@@ -170,7 +191,7 @@ class Pair:
             assert rec["w_err"] <= TENSOR_TOL, rec
             rec["upd_off"], rec["upd_l2"] = gate_update(
                 after - before, rep.theta_sub.astype(np.float64) - sub_before, self.adam.lr,
-                self.knife[k], "AdamW update")
+                step_allowance(self.grel[k]), "AdamW update")
             gate_adam_state(m_gpu, v_gpu, t_gpu, rep)
         return rec
 

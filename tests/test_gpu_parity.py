@@ -2,7 +2,7 @@
 
 Tolerances: losses 1e-3 relative; subset gradients and updated weights 2e-2 in
 max-abs over l2-norm (bf16 products, fp32 accumulation) and, so that the gate can fail at any
-vector length, 2e-2 in relative l2 for gradients and AdamW moments and the knife-edge rule of
+vector length, 2e-2 in relative l2 for gradients and AdamW moments and the per-element allowance of
 tests/_harness.py for updates; frozen parameters, the trained index set and positions no
 replica trains are bit-exact.
 """
@@ -42,23 +42,27 @@ def _run_round(P: Pair, B, S, H, rnd=0, order=None, check=True):
     return report
 
 
-def _gate_outer(P: Pair, replicas, th_before, th_gpu, buf_before, buf_gpu, th_ref_before, buf_ref_before, m):
+def _gate_outer(P: Pair, replicas, th_before, th_gpu, buf_before, buf_gpu, th_ref_before, buf_ref_before, m,
+                mask=None):
     """The outer step on the positions some listed replica trains: the change of the global
-    parameters and of the momentum against the oracle's, knife-edge elements of the inner AdamW
-    steps excepted (their end values may differ by a whole inner step)."""
+    parameters and of the momentum against the oracle's, with the allowance of
+    tests/_harness.py for elements whose inner gradients are near the noise floor."""
     tr = m > 0
     if not tr.any():
         return
-    knife = np.zeros(len(m), bool)
+    allow = np.zeros(len(m))                # the most lenient owner decides
     for k in replicas:
-        knife[P.reps[k].idx] |= P.knife[k]
+        idx = P.reps[k].idx
+        allow[idx] = np.maximum(allow[idx], P.allow_acc[k])
+        synced = np.ones(len(idx), bool) if mask is None else mask[idx]
+        P.allow_acc[k][synced] *= P.outer.momentum      # what the momentum carries into later rounds
     scale = P.outer.lr * (1.0 + P.outer.momentum) * P.adam.lr
     assert max_abs_over_norm(th_gpu[tr], P.theta[tr]) <= TENSOR_TOL
     assert max_abs_over_norm(buf_gpu[tr], P.buf[tr]) <= TENSOR_TOL
     gate_update(th_gpu[tr].astype(np.float64) - th_before[tr], P.theta[tr] - th_ref_before[tr], scale,
-                knife[tr], "outer step on theta")
+                allow[tr], "outer step on theta")
     gate_update(buf_gpu[tr].astype(np.float64) - buf_before[tr], P.buf[tr] - buf_ref_before[tr],
-                P.adam.lr, knife[tr], "outer momentum")
+                P.adam.lr, allow[tr], "outer momentum")
 
 
 def _check_outer(P: Pair, replicas):
@@ -255,7 +259,7 @@ def _check_outer_group(P: Pair, replicas, group, n_groups):
     still = ~mask | (m == 0)
     assert np.array_equal(th_gpu[still], theta_before[still])
     assert np.array_equal(buf_gpu[still], buf_before[still])
-    _gate_outer(P, replicas, theta_before, th_gpu, buf_before, buf_gpu, th_ref_before, buf_ref_before, m)
+    _gate_outer(P, replicas, theta_before, th_gpu, buf_before, buf_gpu, th_ref_before, buf_ref_before, m, mask)
     assert np.array_equal(P.ctx.ppu_get_working_bf16(), bf16_bits(th_gpu))
     for k in replicas:
         now = P.ctx.ppu_get_params(k)
@@ -278,15 +282,10 @@ def test_streaming_sync_by_layer_groups():
     try:
         order = [(k, h) for k in range(4) for h in range(2)]
         for k, h in order:
-            tok = P.tokens(k, 0, h, 4, 64)
-            P.gpu_step(k, tok)
-            P.reps[k].local_step(P.theta, tok, P.adam)
+            P.step_and_gate(k, P.tokens(k, 0, h, 4, 64))
         _check_outer_group(P, [0, 1, 2, 3], 0, 2)          # layers 0-1
         for k in range(4):                                  # replicas go on from mixed parameters
-            tok = P.tokens(k, 1, 0, 4, 64)
-            loss_gpu, _ = P.gpu_step(k, tok)
-            loss_ref = P.reps[k].local_step(P.theta, tok, P.adam)
-            assert abs(loss_gpu - loss_ref) <= LOSS_RTOL * abs(loss_ref)
+            P.step_and_gate(k, P.tokens(k, 1, 0, 4, 64))
         _check_outer_group(P, [0, 1, 3], 1, 2)              # layers 2-3, replica 2 sits out
         _check_outer_group(P, [0, 1, 2, 3], 2, 2)           # embeddings + final norm: nothing trained
         _check_outer_group(P, [0, 1, 2, 3], 0, 4)           # a finer grouping: layer 0 alone
