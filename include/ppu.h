@@ -21,6 +21,10 @@
  *    asynchronous unless the call returns a host value.
  *  - There is no CPU fallback: without a CUDA device every compute call
  *    fails with PPU_ECUDA.
+ *  - Kernel attributes and device properties are cached per device, so contexts
+ *    on several devices of one process work; a context belongs to the device
+ *    that was current when it was created, and that device must be current in
+ *    every later call on it.
  *
  * Canonical parameter vector (fp32, length ppu_param_count): E[V,d]; then for
  * each layer ln1_g[d], ln1_b[d], W_q[d,d], W_k[d,d], W_v[d,d], W_o[d,d],
@@ -68,17 +72,34 @@ typedef enum {
   PPU_SUBSET_EXPLICIT = 2    /* ranges[k][l] = {lo, hi} given by the caller              */
 } ppu_subset_mode;
 
-/* Which parameters replica k trains (the set I_k^train of Algorithm 1).  In
- * every mode the set is, per layer l, the rows [lo,hi) of W_in and the columns
- * [lo,hi) of W_out; everything else is frozen on every replica.  Replica k
- * uses slice index n = k mod n_slices (Section 2.2.1); n_replicas must be a
- * multiple of n_slices.  lo and hi must be multiples of 8. */
+/* Which parameters replica k trains (the set I_k^train of Algorithm 1).  The set has up to
+ * three parts:
+ *  (a) per layer l, the rows [lo,hi) of W_in and the columns [lo,hi) of W_out (mode, n_slices,
+ *      layer_stride, ranges) - the MLP slicing of Section 2.2.1.  Replica k uses slice index
+ *      n = k mod n_slices; n_replicas must be a multiple of n_slices; lo and hi are multiples
+ *      of 8;
+ *  (b) the rows of W_q, W_k and W_v of a range of heads [h_lo,h_hi) in every layer - the
+ *      columns W_{Q,K,V}[:, H_n] of the MLP + attention-head slicing of Section 2.2.1 (W_o is
+ *      never sliced).  head_ranges gives the range per replica; otherwise n_head_slices > 0
+ *      gives replica k the head group k mod n_head_slices (n_head a multiple of n_head_slices,
+ *      n_replicas a multiple of it too); otherwise all heads when train_non_mlp is set, none
+ *      when it is not;
+ *  (c) with train_non_mlp = 1, every parameter Section 2.2.1 never slices: the embedding (tied
+ *      to the output head), W_o and the gains and shifts of all normalisation layers.  This is
+ *      what the paper's runs train on every node; 0 freezes them on every node.
+ * Everything else is frozen on that replica.  The packed order of a replica's trained values
+ * (ppu_subset_index) is: per trained layer the W_in rows block, then the W_out columns block;
+ * then the positions of (b) and (c) in the order of the canonical vector.  AdamW's weight decay
+ * applies to matrices, not to the gains and shifts of the normalisation layers. */
 typedef struct {
   int32_t n_replicas;    /* K */
   int32_t mode;          /* ppu_subset_mode */
   int32_t n_slices;      /* N (FFN_SLICE: d_ff % (8 N) == 0) */
   int32_t layer_stride;  /* FFN_LAYERS only */
   const int32_t* ranges; /* HOST, EXPLICIT only: [n_replicas][n_layer][2] */
+  int32_t train_non_mlp; /* part (c), and the default of part (b) */
+  int32_t n_head_slices; /* part (b): 0 = not sliced */
+  const int32_t* head_ranges; /* HOST, optional: [n_replicas][2] = {h_lo, h_hi} */
 } ppu_subset_spec;
 
 typedef struct ppu_ctx ppu_ctx;
@@ -93,6 +114,8 @@ typedef struct {
   int64_t launches_last_sync;  /* kernels enqueued by the most recent outer sync       */
   double flops_fwd, flops_dgrad, flops_wgrad; /* executed matmul FLOPs of the last step */
   double outer_bytes;          /* algorithmic bytes of the last outer sync             */
+  int64_t saved_bytes_last_step; /* activation bytes the last step's forward pass kept for
+                                    its backward pass (nothing below the lowest trained layer) */
 } ppu_stats_t;
 
 /* Bytes of device memory a context needs.  bytes: HOST out. */
@@ -154,9 +177,12 @@ int ppu_tensor_count(const ppu_ctx* ctx, int32_t* n);
 /* name: HOST buffer of name_cap bytes; shape: HOST int64[2] (unused dims = 1). */
 int ppu_tensor_info(const ppu_ctx* ctx, int32_t index, char* name, int32_t name_cap,
                     int64_t* offset, int32_t* ndim, int64_t* shape);
-/* Sets the global parameters theta^(t) (canonical vector), refreshes the bf16
- * copy and restarts every replica from them.  Optimizer state is untouched. */
-int ppu_set_params(ppu_ctx* ctx, const float* theta, int64_t n);
+/* replica = -1: sets the global parameters theta^(t) (canonical vector), refreshes the bf16
+ * copy and restarts every replica from them.  replica >= 0: sets that replica's own values
+ * theta_k on its trained positions from the canonical vector given (other positions of the
+ * vector are not read); the global parameters and the other replicas are untouched.
+ * Optimizer state is untouched in both forms. */
+int ppu_set_params(ppu_ctx* ctx, int replica, const float* theta, int64_t n);
 /* replica >= 0: theta_k (global vector with the replica's subset overlaid);
  * replica = -1: the global parameters. */
 int ppu_get_params(ppu_ctx* ctx, int replica, float* theta, int64_t n);
@@ -174,22 +200,48 @@ int ppu_get_subset_grads(ppu_ctx* ctx, int replica, float* grads, int64_t n);
 /* AdamW moments and step count of a replica; any out pointer may be null. */
 int ppu_get_subset_state(ppu_ctx* ctx, int replica, float* m, float* v, int32_t* step,
                          int64_t n);
+/* Restores them (checkpoint resume): m and v in the packed order, length ppu_subset_count;
+ * either may be null to leave it as it is; step >= 0. */
+int ppu_set_subset_state(ppu_ctx* ctx, int replica, const float* m, const float* v, int32_t step,
+                         int64_t n);
+/* Device address of replica k's packed trained values (fp32, ppu_subset_count elements, inside
+ * the caller's arena).  For a multi-GPU exchange step: each GPU steps its own replicas, the
+ * owners' packed values are copied into the same replica's buffer on the other GPUs (plain
+ * device-to-device copies or a collective on these local buffers), and every GPU then runs
+ * the same ppu_outer_sync.  dev_ptr: HOST out. */
+int ppu_replica_values(ppu_ctx* ctx, int replica, void** dev_ptr, int64_t* n);
 int ppu_set_adam_lr(ppu_ctx* ctx, float lr);
 int ppu_sync(ppu_ctx* ctx);   /* waits for the stream; reports PPU_ETOKEN / PPU_ETIMEOUT */
 int ppu_stats(ppu_ctx* ctx, ppu_stats_t* out);
 const char* ppu_last_error(void);
 
-/* Per-kernel-class device timing.  While enabled, every GEMM and attention launch of a local
- * step is bracketed by CUDA events on the context's stream (up to a fixed pool; launches
+/* Per-kernel-class device timing.  While enabled, the launches of a local step and of an outer
+ * sync are bracketed by CUDA events on the context's stream (up to a fixed pool; launches
  * beyond it are not recorded).  ppu_profile_read waits for the stream, sums the recorded
- * intervals and their executed FLOPs since the last read, and empties the pool. */
+ * intervals and their algorithmic work since the last read, and empties the pool.  work is in
+ * FLOPs for the GEMM and attention classes and in algorithmic bytes for the others. */
+enum {
+  PPU_CLS_GEMM = 0,   /* every tcgen05 (or SIMT) GEMM launch                       */
+  PPU_CLS_ATTN = 1,   /* attention forward + backward                              */
+  PPU_CLS_LN = 2,     /* LayerNorm forward, backward, gain/shift gradients         */
+  PPU_CLS_XENT = 3,   /* fused cross-entropy                                       */
+  PPU_CLS_ADAMW = 4,  /* AdamW on the subset                                       */
+  PPU_CLS_OUTER = 5,  /* outer sweep                                               */
+  PPU_CLS_OTHER = 6,  /* embedding gather / scatter, residency moves, reductions   */
+  PPU_CLS_COUNT = 8
+};
 typedef struct {
-  double gemm_ms, gemm_flops;   /* tcgen05 (or SIMT) GEMM launches              */
-  double attn_ms, attn_flops;   /* attention forward + backward launches        */
-  int64_t gemm_launches, attn_launches, dropped;
+  double ms[PPU_CLS_COUNT], work[PPU_CLS_COUNT];
+  int64_t launches[PPU_CLS_COUNT];
+  int64_t dropped;
 } ppu_profile_t;
 int ppu_profile_enable(ppu_ctx* ctx, int enable);
 int ppu_profile_read(ppu_ctx* ctx, ppu_profile_t* out);
+
+/* Test hook: which kernels the context's steps use.  gemm: 0 = tcgen05 tiles, 1 = plain SIMT
+ * check kernel.  attention: 0 = tcgen05 kernels where the shape allows, 1 = SIMT check
+ * kernels.  The default is 0, 0; production code has no reason to call this. */
+int ppu_set_backends(ppu_ctx* ctx, int gemm, int attention);
 
 /* Failure-detection self-test.  Every wait inside the tcgen05 kernels is bounded: when a
  * barrier is not signalled within the limit the kernel sets an error word, releases what it
@@ -219,9 +271,8 @@ int ppu_gemm(const void* A, int64_t lda, int a_kmajor, const void* B, int64_t ld
  * batch*seq; q at column 0, k at d, v at 2d; head j at columns j*d_h).  Forward
  * writes U[T,d] bf16 and lse[batch, n_head, seq] fp32 (log-sum-exp of the scaled
  * scores).  Backward reads them plus dU[T,d] bf16 and writes dqkv[T,3d] bf16;
- * scratch is fp32 [batch*n_head*seq].  backend: 0 = tcgen05 / TMEM kernels,
- * 1 = plain SIMT check kernel, 2 = mma.sync kernels (0 and 2 need d_head 64 or 128).
- * All pointers DEVICE. */
+ * scratch is fp32 [batch*n_head*seq].  backend: 0 = tcgen05 / TMEM kernels (d_head 64 or
+ * 128), 1 = plain SIMT check kernel.  All pointers DEVICE. */
 int ppu_attention_fwd(const void* qkv, void* U, float* lse, int batch, int seq, int n_head,
                       int d_head, int backend, void* cuda_stream);
 int ppu_attention_bwd(const void* qkv, const void* U, const float* lse, const void* dU,

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libppu.so")
 SOURCES = ["ppu_api.cu", "ppu_step.cu", "elementwise.cu", "optim.cu", "gemm_simt.cu",
-           "gemm_tc.cu", "gemm_tc_pair.cu", "attention_simt.cu", "attention_mma.cu", "attention_tc.cu", "attention_static.cu", "wait_probe.cu"]
+           "gemm_tc.cu", "gemm_tc_pair.cu", "attention_simt.cu", "attention_tc.cu", "attention_static.cu", "wait_probe.cu"]
 FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
          "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

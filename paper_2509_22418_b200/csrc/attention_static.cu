@@ -5,6 +5,7 @@
 // that is handed fixed buffers and nothing else.  ppu_attention_bwd needs a per-row scratch
 // vector (delta = rowsum(dU * U)); this variant keeps that vector in a fixed array that lives
 // in the library image instead of asking the caller for it.
+#include <mutex>
 #include "../../include/ppu.h"
 #include "common.cuh"
 
@@ -17,6 +18,7 @@ __device__ __align__(256) float g_static_delta[PPU_STATIC_SCRATCH_FLOATS];
 
 constexpr int MAX_DEVICES = 64;
 float* g_delta_ptr[MAX_DEVICES] = {};   // device address of g_static_delta, per device
+std::mutex g_delta_lock;                // two threads may make the first call on a device at once
 
 // In host code `g_static_delta` is only a handle; the address a kernel can use has to be asked
 // for, once per device, with that device current.
@@ -25,6 +27,7 @@ int static_scratch(float** out) {
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return ppu_fail(PPU_ECUDA, "cudaGetDevice failed: %s", cudaGetErrorString(e));
   if (dev < 0 || dev >= MAX_DEVICES) return ppu_fail(PPU_ECUDA, "device index %d not supported", dev);
+  std::lock_guard<std::mutex> lk(g_delta_lock);
   if (!g_delta_ptr[dev]) {
     float* p = nullptr;
     e = cudaGetSymbolAddress((void**)&p, g_static_delta);
@@ -55,13 +58,12 @@ extern "C" int ppu_attention_bwd_static(const void* qkv, const void* U, const fl
   cudaStream_t st = (cudaStream_t)cuda_stream;
   // Every row the kernels read from the scratch is written first by the same call, so nothing
   // left over from an earlier call is ever used and no clearing is needed.
-  if (backend == 0 || backend == 2) {
-    if (!attn_mma_supported(seq, d_head))
+  if (backend < 0 || backend > 1) return ppu_fail(PPU_EINVAL, "unknown attention backend %d", backend);
+  if (backend == 0) {
+    if (!attn_tc_supported(seq, d_head))
       return ppu_fail(PPU_ESHAPE, "shape not covered by the tensor-core attention");
-    rc = backend == 0 ? launch_attn_bwd_tc((const bf16*)qkv, (const bf16*)U, lse, (const bf16*)dU,
-                                           (bf16*)dqkv, scratch, batch, seq, n_head, d_head, nullptr, st)
-                      : launch_attn_bwd_mma((const bf16*)qkv, (const bf16*)U, lse, (const bf16*)dU,
-                                            (bf16*)dqkv, scratch, batch, seq, n_head, d_head, st);
+    rc = launch_attn_bwd_tc((const bf16*)qkv, (const bf16*)U, lse, (const bf16*)dU, (bf16*)dqkv, scratch,
+                            batch, seq, n_head, d_head, nullptr, st);
   } else {
     rc = launch_attn_bwd_simt((const bf16*)qkv, (const bf16*)U, lse, (const bf16*)dU, (bf16*)dqkv,
                               scratch, batch, seq, n_head, d_head, st);

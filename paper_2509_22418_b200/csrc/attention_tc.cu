@@ -890,27 +890,36 @@ bool encode3d(CUtensorMap* map, const bf16* base, int cols, int S, int B, int64_
              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int sm_count() {
-  static int n_sm = 0;
-  if (n_sm == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-    if (n_sm <= 0) n_sm = 148;
+int sm_count() { return ppu_sm_count(); }
+
+// delta[b, head, s] = sum over the head's columns of dU * U: one warp per (token, head)
+__global__ void attn_delta_kernel(const bf16* __restrict__ U, const bf16* __restrict__ dU,
+                                  float* __restrict__ delta, int S, int h, int dh, int64_t rows) {
+  const int64_t w = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (w >= rows * h) return;
+  const int64_t tok = w / h;
+  const int head = (int)(w % h);
+  const bf16* u = U + tok * (int64_t)h * dh + head * dh;
+  const bf16* g = dU + tok * (int64_t)h * dh + head * dh;
+  float s = 0.f;
+  for (int e = lane * 2; e < dh; e += 64) {
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(u + e));
+    const float2 bq = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(g + e));
+    s += a.x * bq.x + a.y * bq.y;
   }
-  return n_sm;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if (lane == 0) delta[((tok / S) * h + head) * S + (int)(tok % S)] = s;
 }
-template <typename K>
-bool set_smem(K kernel, int bytes) {
-  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
-}
+
 constexpr int EXTRA = 1024 + 256;   // alignment slack + barriers
 
 template <int DH>
 int fwd_t(const bf16* qkv, bf16* U, float* lse, int B, int S, int h, int* flags, cudaStream_t st) {
   constexpr int SM = 7 * 128 * DH * 2 + 2 * 128 * 8 + 256 + FWD_ALIGN_SLACK;
-  static bool ok = set_smem(attn_fwd_tc_kernel<DH>, SM);
-  if (!ok) return -2;
+  static PerDeviceFlag attr;
+  if (!ppu_set_smem_once(attr, attn_fwd_tc_kernel<DH>, SM)) return -2;
   CUtensorMap m;
   if (!encode3d(&m, qkv, 3 * h * DH, S, B, 3 * (int64_t)h * DH, 128)) return -3;
   AttnParams p{}; p.U = U; p.lse_out = lse; p.S = S; p.h = h; p.B = B; p.flags = flags;
@@ -924,8 +933,8 @@ int bwd_t(const bf16* qkv, const float* lse, const bf16* dU, bf16* dqkv, const f
           int S, int h, int* flags, cudaStream_t st, const float2* inv_rope) {
   constexpr int SM_DQ = 7 * 128 * DH * 2 + EXTRA;
   constexpr int SM_KV = 6 * 128 * DH * 2 + 3 * 2 * 128 * 4 + EXTRA;
-  static bool ok = set_smem(attn_dq_tc_kernel<DH>, SM_DQ) && set_smem(attn_dkv_tc_kernel<DH>, SM_KV);
-  if (!ok) return -2;
+  static PerDeviceFlag attr_dq, attr_kv;
+  if (!ppu_set_smem_once(attr_dq, attn_dq_tc_kernel<DH>, SM_DQ) || !ppu_set_smem_once(attr_kv, attn_dkv_tc_kernel<DH>, SM_KV)) return -2;
   const int d = h * DH;
   CUtensorMap mQKV, mG;
   if (!encode3d(&mQKV, qkv, 3 * d, S, B, 3 * (int64_t)d, 128) || !encode3d(&mG, dU, d, S, B, d, 128))
@@ -941,6 +950,13 @@ int bwd_t(const bf16* qkv, const float* lse, const bf16* dU, bf16* dqkv, const f
 }  // namespace
 
 bool attn_tc_supported(int S, int dh) { return (dh == 64 || dh == 128) && S >= 1; }
+
+void launch_attn_delta(const bf16* U, const bf16* dU, float* delta, int B, int S, int h, int dh,
+                       cudaStream_t st) {
+  const int64_t rows = (int64_t)B * S;
+  const int64_t warps = rows * h;
+  attn_delta_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, st>>>(U, dU, delta, S, h, dh, rows);
+}
 
 int launch_attn_fwd_tc(const bf16* qkv, bf16* U, float* lse, int B, int S, int h, int dh, int* flags,
                        cudaStream_t st) {

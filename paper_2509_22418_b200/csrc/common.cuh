@@ -13,7 +13,7 @@ enum { PPU_FLAG_TOKEN = 0, PPU_FLAG_TIMEOUT = 1, PPU_FLAG_COUNT = 8 };
 enum GemmEpilogue {
   EPI_STORE_BF16 = 0,  // C bf16
   EPI_STORE_F32 = 1,   // C fp32
-  EPI_GELU_DUAL = 2,   // C bf16 = acc (pre-activation), C2 bf16 = gelu(acc)
+  EPI_GELU_DUAL = 2,   // C bf16 = acc (pre-activation; skipped when C is null), C2 bf16 = gelu(acc)
   EPI_RESID_F32 = 3,   // C fp32 = aux fp32 + acc (residual stream)
   EPI_DGELU = 4,       // C bf16 = acc * gelu'(aux bf16)
   EPI_ROPE_BF16 = 5,   // C bf16 = acc with rotary positions applied to the columns < rope_cols
@@ -57,11 +57,6 @@ int launch_attn_fwd_simt(const bf16* qkv, bf16* U, float* lse, int B, int S, int
                          cudaStream_t st);
 int launch_attn_bwd_simt(const bf16* qkv, const bf16* U, const float* lse, const bf16* dU,
                          bf16* dqkv, float* scratch, int B, int S, int h, int dh, cudaStream_t st);
-int launch_attn_fwd_mma(const bf16* qkv, bf16* U, float* lse, int B, int S, int h, int dh,
-                        cudaStream_t st);
-int launch_attn_bwd_mma(const bf16* qkv, const bf16* U, const float* lse, const bf16* dU,
-                        bf16* dqkv, float* scratch, int B, int S, int h, int dh, cudaStream_t st);
-bool attn_mma_supported(int S, int dh);
 // tcgen05 attention (TMEM accumulators, TMA operands); flags: device error words or null
 bool attn_tc_supported(int S, int dh);
 int launch_attn_fwd_tc(const bf16* qkv, bf16* U, float* lse, int B, int S, int h, int dh, int* flags,
@@ -73,6 +68,24 @@ int launch_attn_bwd_tc(const bf16* qkv, const bf16* U, const float* lse, const b
 // delta[b,h,s] = sum_e dU * U of the head's slice
 void launch_attn_delta(const bf16* U, const bf16* dU, float* delta, int B, int S, int h, int dh,
                        cudaStream_t st);
+
+// ---- per-device caches -------------------------------------------------------
+// Kernel attributes (dynamic shared-memory limits) and device properties are per device; a
+// process may hold contexts on several.  Lookups are idempotent, so two threads that race on
+// the first use of a device at worst both perform the same query.
+constexpr int PPU_MAX_DEVICES = 64;
+int ppu_current_device();                 // index of the current device, clamped to the table
+int ppu_sm_count();                       // SMs of the current device (read once per device)
+struct PerDeviceFlag { bool done[PPU_MAX_DEVICES] = {}; };
+template <typename Kernel>
+inline bool ppu_set_smem_once(PerDeviceFlag& f, Kernel kernel, int bytes) {
+  const int dev = ppu_current_device();
+  if (f.done[dev]) return true;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess)
+    return false;
+  f.done[dev] = true;
+  return true;
+}
 
 // ---- bandwidth-bound kernels -------------------------------------------------
 void launch_embed(const int32_t* tok, const bf16* E16, float* x, int T, int d, int V, int* flags,
@@ -93,20 +106,40 @@ void launch_xent(bf16* logits, const int32_t* tok, float* row_loss, int B, int S
 void launch_loss_reduce(const float* row_loss, int T, float inv_count, float* out, cudaStream_t st);
 void launch_cast_bf16(const float* src, bf16* dst, int64_t n, cudaStream_t st);
 
-// One trained block of a replica: rows [lo,hi) of W_in then columns [lo,hi) of W_out,
+// rows of E that a batch touches: dE[tok[t], :] += g[t, :] over all t in ascending order of t
+// (one warp owns all occurrences of an id, so the sum has a fixed order and needs no atomics)
+void launch_embed_grad(const int32_t* tok, const float* g, float* dE, int T, int d, int V,
+                       cudaStream_t st);
+// dgamma[c] = sum_t dy[t,c] * xhat[t,c], dbeta[c] = sum_t dy[t,c], in two stages with a fixed
+// order; partial: fp32 scratch [2 * ceil(T / 32) * d]
+void launch_ln_param_grad(const bf16* dy, const float* x, const float2* stats, float* dgamma,
+                          float* dbeta, float* partial, int T, int d, cudaStream_t st);
+
+// One trained FFN block of a replica: rows [lo,hi) of W_in then columns [lo,hi) of W_out,
 // packed back to back at `packed_off` of the replica's packed arrays.
 struct SliceSeg {
   int64_t win_off, wout_off;   // offsets of the layer's W_in / W_out in the canonical vector
   int64_t packed_off;          // start of this layer's block in the packed arrays
   int32_t lo, hi;
 };
+// One contiguous run of the canonical vector that a replica trains outside the FFNs (a whole
+// tensor, or the rows of W_q / W_k / W_v of its heads), packed at `packed_off`.
+struct DenseSeg {
+  int64_t canon_off, len, packed_off;   // len is a multiple of 8
+  int32_t decay;                        // 1: AdamW's weight decay applies (matrices)
+  int32_t pad;
+};
 
 struct AdamHyper { float lr, beta1, beta2, eps, wd, bc1, bc2; };
 
-// AdamW over the packed subset; n_partials gradient buffers (stride grad_stride) are summed in order.
+// AdamW over the packed FFN blocks; n_partials gradient buffers (stride grad_stride) are summed in order.
 void launch_adamw(const SliceSeg* segs, int n_seg, float* master, float* m, float* v,
                   const float* grad, int n_partials, int64_t grad_stride, bf16* w16, int d, int F,
                   int64_t n_total, AdamHyper hp, cudaStream_t st);
+// AdamW over the packed dense runs; the gradient of packed element j is grad[j - grad_shift]
+void launch_adamw_dense(const DenseSeg* segs, int n_seg, float* master, float* m, float* v,
+                        const float* grad, int64_t grad_shift, bf16* w16, int64_t n_total,
+                        AdamHyper hp, cudaStream_t st);
 // packed fp32 <-> canonical vectors
 void launch_slices_gather(const SliceSeg* segs, int n_seg, const float* theta, float* packed,
                           int d, int F, int64_t n_total, cudaStream_t st);
@@ -114,24 +147,37 @@ void launch_slices_gather(const SliceSeg* segs, int n_seg, const float* theta, f
 void launch_slices_to_w16(const SliceSeg* segs, int n_seg, const float* packed, const float* theta,
                           bf16* w16, int from_packed, int d, int F, int64_t n_total,
                           cudaStream_t st);
-void launch_slices_scatter_f32(const SliceSeg* segs, int n_seg, const float* packed, float* dense,
-                               int d, int F, int64_t n_total, cudaStream_t st);
+// the same two moves for the dense runs: mode 0 packed = theta, 1 w16 = bf16(packed), 2 w16 = bf16(theta)
+void launch_dense_move(const DenseSeg* segs, int n_seg, float* packed, const float* theta, bf16* w16,
+                       int mode, int64_t n_total, cudaStream_t st);
 
-// Outer sync tables.  Owner o is one listed replica's trained block of one layer: hidden
-// units [lo,hi); its packed W_in block starts at master + in_off, its W_out block at
-// master + out_off.  For every group of 8 hidden units of every layer, unit_begin/unit_owner
-// (CSR) list the owners that contain the group, in the order the replicas were listed.
+// Outer sync tables.  The canonical vector is cut into runs ("segments") that are uniform in
+// how their owners are found:
+//   kind 0  a run outside the FFN matrices; every owner in [ob, oe) of `dense_owner` trains the
+//           whole run, its value of canonical position i is master[i + shift];
+//   kind 1  (part of) a layer's W_in, kind 2 (part of) its W_out: the owners of a hidden unit are
+//           listed per group of 8 units in unit_begin / unit_owner (CSR over layer * F/8 + unit/8).
+// Work is dealt to blocks in chunks of OUTER_CHUNK elements of one segment.
+constexpr int OUTER_CHUNK = 1 << 16;
+struct OuterSeg {
+  int64_t start, len;        // run of the canonical vector (multiples of 4)
+  int64_t base;              // kinds 1, 2: canonical offset of the whole matrix
+  int32_t kind, layer;
+  int32_t ob, oe;            // kind 0: owners
+};
+struct OuterChunk { int32_t seg; int32_t pad; int64_t off; };   // chunk = elements [off, off + OUTER_CHUNK) of the segment
+struct DenseOwner { float* master; int64_t shift; };
+// a listed replica's trained block of one layer: hidden units [lo,hi); packed W_in block at
+// master + in_off, W_out block at master + out_off
 struct OuterOwner { float* master; int64_t in_off, out_off; int32_t lo, hi; };
 struct OuterTables {
-  const OuterOwner* owners;      // device
+  const OuterSeg* segs;          // device
+  const OuterChunk* chunks;      // device
+  const DenseOwner* dense_owner; // device
   const int32_t* unit_begin;     // device [L * F/8 + 1]
-  const int32_t* unit_owner;     // device
-  int64_t P, e_size, layer_size, win_rel, wout_rel;  // canonical geometry
-  int32_t L, d, F;
+  const OuterOwner* unit_owner;  // device, owners inline
+  int32_t d, F;
 };
-// Segments of the canonical vector the outer sweep works through: 0-3 quarters of E, then three
-// per layer (non-FFN block, W_in, W_out), then the final LayerNorm.  The sweep covers segments
-// [seg_lo, seg_lo + seg_count).
-inline int outer_segments(int n_layer) { return 4 + 3 * n_layer + 1; }
+// sweeps chunks [chunk_lo, chunk_lo + n_chunks)
 void launch_outer(const OuterTables& t, float* theta, float* buf, bf16* w16, float lr, float mu,
-                  int seg_lo, int seg_count, cudaStream_t st);
+                  int chunk_lo, int n_chunks, cudaStream_t st);

@@ -391,7 +391,132 @@ __global__ void cast_bf16_kernel(const float* __restrict__ src, bf16* __restrict
   }
 }
 
+// ---- gradient of the embedding rows a batch touches -----------------------------------------
+// dE[id, :] += sum over the positions t with tok[t] == id, in ascending t, of g[t, :].  One warp
+// per position: the warp of an id's first occurrence gathers all of them (ids are compared after
+// the same clamping the forward gather applies), every other warp leaves at once - so each row
+// of dE has one writer and a fixed summation order.
+__global__ void __launch_bounds__(256)
+embed_grad_kernel(const int32_t* __restrict__ tok, const float* __restrict__ g, float* __restrict__ dE,
+                  int T, int d, int V) {
+  const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (t >= T) return;
+  auto clampv = [V](int id) { return id < 0 ? 0 : (id >= V ? V - 1 : id); };
+  const int id = clampv(tok[t]);
+  bool seen = false;
+  for (int j = lane; j < t && !seen; j += 32) seen = clampv(tok[j]) == id;
+  if (__any_sync(0xffffffffu, seen)) return;
+  float* row = dE + (int64_t)id * d;
+  for (int c0 = 0; c0 < d; c0 += 512) {          // 512 columns at a time: four float4 per lane
+    float4 acc[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int c = c0 + 4 * (lane + 32 * i);
+      acc[i] = c < d ? *reinterpret_cast<const float4*>(row + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    for (int j0 = t & ~31; j0 < T; j0 += 32) {
+      const int j = j0 + lane;
+      const bool hit = j >= t && j < T && clampv(tok[j]) == id;
+      unsigned mask = __ballot_sync(0xffffffffu, hit);
+      while (mask) {
+        const int src = j0 + __ffs(mask) - 1;
+        mask &= mask - 1;
+        const float* gr = g + (int64_t)src * d;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int c = c0 + 4 * (lane + 32 * i);
+          if (c < d) {
+            const float4 v = *reinterpret_cast<const float4*>(gr + c);
+            acc[i].x += v.x; acc[i].y += v.y; acc[i].z += v.z; acc[i].w += v.w;
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int c = c0 + 4 * (lane + 32 * i);
+      if (c < d) *reinterpret_cast<float4*>(row + c) = acc[i];
+    }
+  }
+}
+
+// ---- LayerNorm gain / shift gradients: column sums over the tokens, two stages -------------
+// stage 1: block b sums rows [32 b, 32 b + 32) for every column -> partial[b][0][c] (dy * xhat),
+// partial[b][1][c] (dy); stage 2: one thread per column adds the partials in order of b.
+constexpr int LNP_ROWS = 32;
+__global__ void __launch_bounds__(256)
+ln_param_partial_kernel(const bf16* __restrict__ dy, const float* __restrict__ x,
+                        const float2* __restrict__ stats, float* __restrict__ partial, int T, int d) {
+  const int r0 = blockIdx.x * LNP_ROWS;
+  const int r1 = r0 + LNP_ROWS < T ? r0 + LNP_ROWS : T;
+  float* pg = partial + (int64_t)blockIdx.x * 2 * d;
+  float* pb = pg + d;
+  for (int c = 8 * threadIdx.x; c < d; c += 8 * 256) {
+    float sg[8] = {}, sb[8] = {};
+    for (int t = r0; t < r1; ++t) {
+      const float2 st = stats[t];
+      float f[8];
+      unpack8(*reinterpret_cast<const uint4*>(dy + (int64_t)t * d + c), f);
+      const float4 xa = *reinterpret_cast<const float4*>(x + (int64_t)t * d + c);
+      const float4 xb = *reinterpret_cast<const float4*>(x + (int64_t)t * d + c + 4);
+      const float xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        sg[j] += f[j] * ((xv[j] - st.x) * st.y);
+        sb[j] += f[j];
+      }
+    }
+    *reinterpret_cast<float4*>(pg + c) = make_float4(sg[0], sg[1], sg[2], sg[3]);
+    *reinterpret_cast<float4*>(pg + c + 4) = make_float4(sg[4], sg[5], sg[6], sg[7]);
+    *reinterpret_cast<float4*>(pb + c) = make_float4(sb[0], sb[1], sb[2], sb[3]);
+    *reinterpret_cast<float4*>(pb + c + 4) = make_float4(sb[4], sb[5], sb[6], sb[7]);
+  }
+}
+__global__ void __launch_bounds__(128)
+ln_param_final_kernel(const float* __restrict__ partial, float* __restrict__ dgamma,
+                      float* __restrict__ dbeta, int n_blocks, int d) {
+  const int c = blockIdx.x * 128 + threadIdx.x;
+  if (c >= d) return;
+  float sg = 0.f, sb = 0.f;
+  for (int b = 0; b < n_blocks; ++b) {
+    sg += partial[(int64_t)b * 2 * d + c];
+    sb += partial[(int64_t)b * 2 * d + d + c];
+  }
+  dgamma[c] = sg;
+  dbeta[c] = sb;
+}
+
 }  // namespace
+
+int ppu_current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= PPU_MAX_DEVICES) dev = 0;
+  return dev;
+}
+
+int ppu_sm_count() {
+  static int n_sm[PPU_MAX_DEVICES] = {};
+  const int dev = ppu_current_device();
+  if (n_sm[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 1;
+    n_sm[dev] = n;
+  }
+  return n_sm[dev];
+}
+
+void launch_embed_grad(const int32_t* tok, const float* g, float* dE, int T, int d, int V,
+                       cudaStream_t st) {
+  embed_grad_kernel<<<(unsigned)((T + 7) / 8), 256, 0, st>>>(tok, g, dE, T, d, V);
+}
+
+void launch_ln_param_grad(const bf16* dy, const float* x, const float2* stats, float* dgamma,
+                          float* dbeta, float* partial, int T, int d, cudaStream_t st) {
+  const int nb = (T + LNP_ROWS - 1) / LNP_ROWS;
+  ln_param_partial_kernel<<<nb, 256, 0, st>>>(dy, x, stats, partial, T, d);
+  ln_param_final_kernel<<<(d + 127) / 128, 128, 0, st>>>(partial, dgamma, dbeta, nb, d);
+}
 
 void launch_embed(const int32_t* tok, const bf16* E16, float* x, int T, int d, int V, int* flags,
                   cudaStream_t st) {
@@ -455,7 +580,7 @@ void launch_cast_bf16(const float* src, bf16* dst, int64_t n, cudaStream_t st) {
   const int64_t n8 = n / 8;
   const int threads = 256;
   int64_t blocks = (n8 + threads - 1) / threads;
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks > (int64_t)ppu_sm_count() * 16) blocks = (int64_t)ppu_sm_count() * 16;
   if (blocks < 1) blocks = 1;
   cast_bf16_kernel<<<(unsigned)blocks, threads, 0, st>>>(src, dst, n8);
 }

@@ -171,8 +171,10 @@ __device__ __forceinline__ void drain_tile(const TcParams& p, int m0, int n0, in
           uint32_t o[16];
 #pragma unroll
           for (int j = 0; j < 16; ++j) o[j] = pack2_bf16(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
-          st_v8((bf16*)p.C + ci, o);
-          st_v8((bf16*)p.C + ci + 16, o + 8);
+          if (p.C) {       // (the pre-activation store of EPI_GELU_DUAL is optional)
+            st_v8((bf16*)p.C + ci, o);
+            st_v8((bf16*)p.C + ci + 16, o + 8);
+          }
           if (p.epilogue == EPI_DELTA_BF16) {
             // the product uses the stored (rounded) values, as the attention kernels will
 #pragma unroll
@@ -262,7 +264,7 @@ __device__ __forceinline__ void drain_tile(const TcParams& p, int m0, int n0, in
             o[0] = make_float4(f[0], f[1], f[2], f[3]);
             o[1] = make_float4(f[4], f[5], f[6], f[7]);
           } else {
-            *reinterpret_cast<uint4*>((bf16*)p.C + ci + 8 * j) = pack8_bf16(f);
+            if (p.C) *reinterpret_cast<uint4*>((bf16*)p.C + ci + 8 * j) = pack8_bf16(f);
             if (p.epilogue == EPI_GELU_DUAL) {
 #pragma unroll
               for (int q = 0; q < 8; ++q) f[q] = gelu_dev(f[q]);

@@ -61,7 +61,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
         case EPI_STORE_BF16: ((bf16*)g.C)[ci] = __float2bfloat16_rn(a); break;
         case EPI_STORE_F32: ((float*)g.C)[ci] = a; break;
         case EPI_GELU_DUAL:
-          ((bf16*)g.C)[ci] = __float2bfloat16_rn(a);
+          if (g.C) ((bf16*)g.C)[ci] = __float2bfloat16_rn(a);
           ((bf16*)g.C2)[ci] = __float2bfloat16_rn(gelu_f(a));
           if (g.C3 && n >= g.c3_lo && n < g.c3_hi)
             ((bf16*)g.C3)[(int64_t)m * g.ldc3 + (n - g.c3_lo)] = __float2bfloat16_rn(gelu_f(a));

@@ -9,6 +9,8 @@
 //
 // Every mbarrier wait is bounded: on expiry the CTA raises a shared abort flag and a device
 // error word, all roles leave their loops, tensor memory is released and the kernel returns.
+#include <mutex>
+#include <unordered_map>
 #include "gemm_epilogue.cuh"
 
 namespace tc {
@@ -176,8 +178,37 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
 }  // namespace
 
 namespace gemm_tc_detail {
+// Tensor maps are cached per (address, leading dimension, order, extents, box): a training step
+// issues the same few hundred products every time, and encoding is a driver call.
+namespace mapcache {
+struct MapKey {
+  const void* base; long long ld; int kmajor, rows, K, box_rows;
+  bool operator==(const MapKey& o) const {
+    return base == o.base && ld == o.ld && kmajor == o.kmajor && rows == o.rows && K == o.K && box_rows == o.box_rows;
+  }
+};
+struct MapKeyHash {
+  size_t operator()(const MapKey& k) const {
+    size_t h = std::hash<const void*>()(k.base);
+    auto mix = [&h](size_t v) { h ^= v + 0x9e3779b97f4a7c15ull + (h << 6) + (h >> 2); };
+    mix((size_t)k.ld); mix((size_t)k.kmajor); mix((size_t)k.rows); mix((size_t)k.K); mix((size_t)k.box_rows);
+    return h;
+  }
+};
+std::unordered_map<MapKey, CUtensorMap, MapKeyHash> g_maps;
+std::mutex g_maps_lock;
+constexpr size_t MAP_CACHE_LIMIT = 1 << 16;
+}  // namespace mapcache
+using namespace mapcache;
+
 bool encode_map(CUtensorMap* map, const bf16* base, long long ld, bool kmajor, int rows, int K,
                 int box_rows) {
+  const MapKey key{base, ld, kmajor ? 1 : 0, rows, K, box_rows};
+  {
+    std::lock_guard<std::mutex> lk(g_maps_lock);
+    auto it = g_maps.find(key);
+    if (it != g_maps.end()) { *map = it->second; return true; }
+  }
   // kmajor: memory is [rows, K] (inner = K).  else: memory is [K, rows] (inner = rows).
   cuuint64_t gdim[2];
   cuuint64_t gstride[1] = {(cuuint64_t)ld * 2};
@@ -193,7 +224,11 @@ bool encode_map(CUtensorMap* map, const bf16* base, long long ld, bool kmajor, i
   CUresult r = tc::g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)base, gdim, gstride, box,
                         estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
+  if (r != CUDA_SUCCESS) return false;
+  std::lock_guard<std::mutex> lk(g_maps_lock);
+  if (g_maps.size() >= MAP_CACHE_LIMIT) g_maps.clear();
+  g_maps.emplace(key, *map);
+  return true;
 }
 
 // launch parameters common to every tile shape (tile counts and split-K are set by the launcher)
@@ -221,13 +256,8 @@ namespace {
 template <int BN, bool A_K, bool B_K>
 int launch_t(const GemmArgs& g, cudaStream_t st) {
   using C = Cfg<BN>;
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(gemm_tc_kernel<BN, A_K, B_K>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess)
-      return -1;
-    attr_done = true;
-  }
+  static PerDeviceFlag attr;
+  if (!ppu_set_smem_once(attr, gemm_tc_kernel<BN, A_K, B_K>, C::SMEM)) return -1;
   CUtensorMap mapA, mapB;
   if (!encode_map(&mapA, g.A, g.lda, A_K, g.M, g.K, BM)) return -2;
   if (!encode_map(&mapB, g.B, g.ldb, B_K, g.N, g.K, BN)) return -2;
@@ -238,13 +268,7 @@ int launch_t(const GemmArgs& g, cudaStream_t st) {
   p.splits = g.splits < 1 ? 1 : (g.splits > k_blocks ? k_blocks : g.splits);
   p.split_stride = g.split_stride;
   const int tiles = p.tiles_m * p.tiles_n * p.splits;
-  static int n_sm = 0;
-  if (n_sm == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-    if (n_sm <= 0) n_sm = 148;
-  }
+  const int n_sm = ppu_sm_count();
   const int grid = tiles < n_sm ? tiles : n_sm;
   gemm_tc_kernel<BN, A_K, B_K><<<grid, GEMM_THREADS, C::SMEM, st>>>(mapA, mapB, p);
   return cudaGetLastError() == cudaSuccess ? 0 : -3;
@@ -275,7 +299,7 @@ namespace {
 // the SM-pair kernel on 256 x 256 tiles is chosen for this product
 bool picks_pair256(const GemmArgs& g) {
   const long long tiles_pair = (long long)((g.M + 255) / 256) * ((g.N + 255) / 256);
-  return g.tile_shape == 2 || (g.tile_shape == 0 && g.splits <= 1 && g.M > 128 && g.N > 128 && tiles_pair >= 74);
+  return g.tile_shape == 2 || (g.tile_shape == 0 && g.splits <= 1 && g.M > 128 && g.N > 128 && tiles_pair >= ppu_sm_count() / 2);
 }
 }  // namespace
 
@@ -300,12 +324,12 @@ int launch_gemm_tc(const GemmArgs& g, cudaStream_t st) {
   // Wide tiles when the grid still fills the machine; narrow ones for small outputs.
   // SM pairs on 256 x 256 tiles when those still fill the machine and the product is not split.
   // (256 x 128 pair tiles would fill the last wave of the N = 2048 products better - 512 tiles
-  // instead of 256 on 74 pairs - but their narrower instruction measured 25 % slower, so they are
+  // instead of 256 on the 74 pairs of a B200 - but their narrower instruction measured 25 % slower, so they are
   // never chosen here; tile_shape 3 keeps them testable.)
   if ((g.tile_shape == 2 || g.tile_shape == 3) && g.splits > 1) return -4;
   if (g.tile_shape == 3) return launch_gemm_tc_pair(g, make_params(g), 128, st);
   if (picks_pair256(g)) return launch_gemm_tc_pair(g, make_params(g), 256, st);
   const long long tiles256 = (long long)((g.M + BM - 1) / BM) * ((g.N + 255) / 256) * (g.splits > 1 ? g.splits : 1);
-  if (g.N > 128 && tiles256 >= 148) return launch_bn<256>(g, st);
+  if (g.N > 128 && tiles256 >= ppu_sm_count()) return launch_bn<256>(g, st);
   return launch_bn<128>(g, st);
 }

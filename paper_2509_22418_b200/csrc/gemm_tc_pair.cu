@@ -25,7 +25,7 @@ using namespace gemm_tc_detail;
 
 // The pair's tile is 256 rows x BN columns, BN = 256 or 128.  The narrow tile is for outputs whose
 // 256-wide tiling leaves the last wave of SM pairs half empty (N = 2048 with 8192 rows: 256 tiles
-// on 74 pairs).
+// on the 74 SM pairs of a B200).
 // A stage holds PAIR_KH slabs of 64 k: the issuing thread stalls while the tensor pipe is busy, so
 // a barrier wait per 64 k (four instructions) is not hidden behind the products; one per 128 k is.
 constexpr int PAIR_KH = 2;
@@ -233,13 +233,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
 
 template <int PAIR_BN, bool A_K, bool B_K>
 int launch_pair_t(const GemmArgs& g, const TcParams& p0, cudaStream_t st) {
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(gemm_tc_pair_kernel<PAIR_BN, A_K, B_K>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             PairCfg<PAIR_BN>::SMEM) != cudaSuccess)
-      return -1;
-    attr_done = true;
-  }
+  static PerDeviceFlag attr;
+  if (!ppu_set_smem_once(attr, gemm_tc_pair_kernel<PAIR_BN, A_K, B_K>, PairCfg<PAIR_BN>::SMEM)) return -1;
   CUtensorMap mapA, mapB;
   if (!encode_map(&mapA, g.A, g.lda, A_K, g.M, g.K, 128)) return -2;
   if (!encode_map(&mapB, g.B, g.ldb, B_K, g.N, g.K, PAIR_BN / 2)) return -2;
@@ -248,13 +243,7 @@ int launch_pair_t(const GemmArgs& g, const TcParams& p0, cudaStream_t st) {
   p.tiles_n = (g.N + PAIR_BN - 1) / PAIR_BN;
   p.splits = 1; p.split_stride = 0;
   const int tiles = p.tiles_m * p.tiles_n;
-  static int n_sm = 0;
-  if (n_sm == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-    if (n_sm <= 0) n_sm = 148;
-  }
+  const int n_sm = ppu_sm_count();
   const int pairs = tiles < n_sm / 2 ? tiles : n_sm / 2;
   gemm_tc_pair_kernel<PAIR_BN, A_K, B_K><<<2 * pairs, GEMM_THREADS, PairCfg<PAIR_BN>::SMEM, st>>>(mapA, mapB, p);
   return cudaGetLastError() == cudaSuccess ? 0 : -3;

@@ -86,6 +86,26 @@ static int build_ranges(const ppu_model_cfg* c, const ppu_subset_spec* s,
   } else {
     return ppu_fail(PPU_ESUBSET, "unknown subset mode %d", s->mode);
   }
+  // heads whose query / key / value rows are trained, and the never-sliced rest
+  const int h = c->n_head;
+  if (s->train_non_mlp != 0 && s->train_non_mlp != 1)
+    return ppu_fail(PPU_ESUBSET, "train_non_mlp must be 0 or 1");
+  if (s->n_head_slices < 0 || (s->n_head_slices > 0 && (h % s->n_head_slices || K % s->n_head_slices)))
+    return ppu_fail(PPU_ESUBSET, "n_head and n_replicas must be multiples of n_head_slices");
+  for (int k = 0; k < K; ++k) {
+    ReplicaState& r = reps[k];
+    r.rest = s->train_non_mlp == 1;
+    if (s->head_ranges) {
+      r.h_lo = s->head_ranges[2 * k]; r.h_hi = s->head_ranges[2 * k + 1];
+      if (r.h_lo < 0 || r.h_hi < r.h_lo || r.h_hi > h)
+        return ppu_fail(PPU_ESUBSET, "replica %d: bad head range [%d,%d)", k, r.h_lo, r.h_hi);
+    } else if (s->n_head_slices > 0) {
+      const int per = h / s->n_head_slices;
+      r.h_lo = (k % s->n_head_slices) * per; r.h_hi = r.h_lo + per;
+    } else if (r.rest) {
+      r.h_lo = 0; r.h_hi = h;
+    }
+  }
   return PPU_OK;
 }
 
@@ -128,27 +148,55 @@ static void build_geometry(ppu_ctx* c) {
   }
   add("lnf_g", c->off_lnfg, 1, d, 1);
   add("lnf_b", c->off_lnfb, 1, d, 1);
-  // packed subset tables
-  c->max_sub = 0;
+  // packed subset tables: FFN blocks first, then the dense runs in canonical order
+  const int dh = (int)(d / c->cfg.n_head);
+  c->max_ffn = c->max_dense = 0;
+  c->min_lowest = L;
+  c->any_rest = false;
   for (auto& r2 : c->reps) {
-    r2.segs.clear(); r2.seg_layer.clear(); r2.n_sub = 0; r2.lowest = -1;
+    r2.segs.clear(); r2.seg_layer.clear(); r2.dense.clear();
+    r2.n_ffn = r2.n_dense = r2.n_sub = 0; r2.lowest = -1;
     for (int l = 0; l < L; ++l) {
       if (r2.hi[l] <= r2.lo[l]) continue;
       if (r2.lowest < 0) r2.lowest = l;
       SliceSeg s;
       const int64_t b = c->e_size + l * c->layer_size;
       s.win_off = b + c->rel_win; s.wout_off = b + c->rel_wout;
-      s.packed_off = r2.n_sub; s.lo = r2.lo[l]; s.hi = r2.hi[l];
+      s.packed_off = r2.n_ffn; s.lo = r2.lo[l]; s.hi = r2.hi[l];
       r2.segs.push_back(s); r2.seg_layer.push_back(l);
-      r2.n_sub += 2 * (int64_t)(s.hi - s.lo) * d;
+      r2.n_ffn += 2 * (int64_t)(s.hi - s.lo) * d;
     }
-    if (r2.n_sub > c->max_sub) c->max_sub = r2.n_sub;
+    int64_t at = r2.n_ffn;
+    auto run = [&](int64_t off, int64_t len, int decay) {
+      if (len <= 0) return;
+      DenseSeg s; s.canon_off = off; s.len = len; s.packed_off = at; s.decay = decay; s.pad = 0;
+      r2.dense.push_back(s);
+      at += len;
+    };
+    const int64_t r0 = (int64_t)r2.h_lo * dh * d, rn = (int64_t)(r2.h_hi - r2.h_lo) * dh * d;
+    if (r2.rest) run(0, c->e_size, 1);
+    for (int l = 0; l < L && r2.deep(); ++l) {
+      const int64_t b = c->e_size + l * c->layer_size;
+      if (r2.rest) { run(b + c->rel_ln1g, d, 0); run(b + c->rel_ln1b, d, 0); }
+      for (int q = 0; q < 3; ++q) run(b + c->rel_wq + q * d * d + r0, rn, 1);
+      if (r2.rest) { run(b + c->rel_wo, d * d, 1); run(b + c->rel_ln2g, d, 0); run(b + c->rel_ln2b, d, 0); }
+    }
+    if (r2.rest) { run(c->off_lnfg, d, 0); run(c->off_lnfb, d, 0); }
+    r2.n_dense = at - r2.n_ffn;
+    r2.n_sub = at;
+    if (r2.deep()) r2.lowest = 0;
+    if (r2.n_ffn > c->max_ffn) c->max_ffn = r2.n_ffn;
+    if (r2.n_dense > c->max_dense) c->max_dense = r2.n_dense;
+    if (r2.lowest >= 0 && r2.lowest < c->min_lowest) c->min_lowest = r2.lowest;
+    c->any_rest = c->any_rest || r2.rest;
   }
+  c->max_ffn = (c->max_ffn + 63) & ~(int64_t)63;
   c->wmax.assign(L, 0);
   for (auto& r2 : c->reps)
     for (int l = 0; l < L; ++l) c->wmax[l] = std::max(c->wmax[l], (int)(r2.hi[l] - r2.lo[l]));
   // The subset products have few output tiles when slices are narrow: cut their reduction over
-  // tokens so that about one wave of CTAs works on them.  One factor for the whole context.
+  // tokens so that about one wave of CTAs works on them.  One factor for the whole context
+  // (148 SMs assumed: the factor only balances work, any value gives the same sums in order).
   int64_t min_tiles = 1 << 30;
   for (auto& r2 : c->reps)
     for (auto& s : r2.segs) {
@@ -173,26 +221,39 @@ static size_t carve(ppu_ctx* c, uint8_t* base) {
   c->theta = (float*)take(c->P * 4);
   c->buf = (float*)take(c->P * 4);
   c->w16 = (bf16*)take(c->P * 2);
+  size_t unit_entries = 0;
   for (auto& r : c->reps) {
     r.master = (float*)take(r.n_sub * 4);
     r.m = (float*)take(r.n_sub * 4);
     r.v = (float*)take(r.n_sub * 4);
     r.d_segs = (SliceSeg*)take(sizeof(SliceSeg) * (r.segs.size() + 1));
+    r.d_dense = (DenseSeg*)take(sizeof(DenseSeg) * (r.dense.size() + 1));
+    for (auto& s : r.segs) unit_entries += (size_t)(s.hi - s.lo) / 8;
   }
-  c->max_sub = (c->max_sub + 63) & ~(int64_t)63;
-  c->grad = (float*)take(c->max_sub * 4 * c->wgrad_splits);
+  c->grad = (float*)take((c->max_ffn * c->wgrad_splits + c->max_dense) * 4);
   c->loss = (float*)take(sizeof(float) * (c->K + 1));
   c->flags = (int*)take(sizeof(int) * PPU_FLAG_COUNT);
   c->rope_cs = (float2*)take(sizeof(float2) * c->cfg.max_seq * (d / h / 2));
   c->tok_stage = (int32_t*)take(sizeof(int32_t) * T);
-  c->d_owners = (OuterOwner*)take(sizeof(OuterOwner) * ((size_t)c->K * L + 1));
+  // outer-sync tables: a layer's dense block splits at most at every head boundary of W_q/k/v
+  c->cap_oseg = 8 + (size_t)L * (16 + 6 * (size_t)(h + 1));
+  c->cap_ochunk = (size_t)(c->P / OUTER_CHUNK) + c->cap_oseg + 8;
+  c->cap_downer = c->cap_oseg * (size_t)c->K + 1;
+  c->cap_uowner = unit_entries + 1;
+  c->d_oseg = (OuterSeg*)take(sizeof(OuterSeg) * c->cap_oseg);
+  c->d_ochunk = (OuterChunk*)take(sizeof(OuterChunk) * c->cap_ochunk);
+  c->d_downer = (DenseOwner*)take(sizeof(DenseOwner) * c->cap_downer);
   c->d_unit_begin = (int32_t*)take(sizeof(int32_t) * ((size_t)L * (F / 8) + 1));
-  c->d_unit_owner = (int32_t*)take(sizeof(int32_t) * ((size_t)c->K * L * (F / 8) + 1));
+  c->d_unit_owner = (OuterOwner*)take(sizeof(OuterOwner) * c->cap_uowner);
   c->state_bytes = off;
+  // Activations kept for the backward pass, per layer.  Layers below the lowest layer that any
+  // replica's backward pass reaches run forward only: they share one set of buffers (two for
+  // the residual stream, which alternates) and keep no pre-activation at all.
   c->acts.assign(L, LayerActs());
-  for (int l = 0; l < L; ++l) {
-    LayerActs& a = c->acts[l];
-    a.x = (float*)take(T * d * 4);
+  const int first_kept = c->min_lowest < L ? c->min_lowest : L;
+  LayerActs shared = LayerActs();
+  float* shared_x[2] = {nullptr, nullptr};
+  auto layer_set = [&](LayerActs& a) {
     a.x1 = (float*)take(T * d * 4);
     a.st1 = (float2*)take(T * 8);
     a.st2 = (float2*)take(T * 8);
@@ -200,6 +261,23 @@ static size_t carve(ppu_ctx* c, uint8_t* base) {
     a.U = (bf16*)take(T * d * 2);
     a.lse = (float*)take(T * h * 4);
     a.b = (bf16*)take(T * d * 2);
+  };
+  if (first_kept > 0) {
+    layer_set(shared);
+    shared_x[0] = (float*)take(T * d * 4);
+    shared_x[1] = (float*)take(T * d * 4);
+  }
+  for (int l = 0; l < L; ++l) {
+    LayerActs& a = c->acts[l];
+    if (l < first_kept) {
+      a = shared;
+      a.x = shared_x[l & 1];
+      a.Hd = nullptr;
+      a.As = nullptr;
+      continue;
+    }
+    a.x = (float*)take(T * d * 4);
+    layer_set(a);
     a.Hd = (bf16*)take(T * F * 2);
     a.As = (bf16*)take(T * (int64_t)c->wmax[l] * 2);
   }
@@ -216,6 +294,7 @@ static size_t carve(ppu_ctx* c, uint8_t* base) {
   c->dqkv = (bf16*)take(T * 3 * d * 2);
   c->attn_scratch = (float*)take(T * h * 4);
   c->row_loss = (float*)take(T * 4);
+  c->ln_partial = c->any_rest ? (float*)take((size_t)2 * ((T + 31) / 32) * d * 4) : nullptr;
   c->act_bytes = off - c->state_bytes;
   return off;
 }
@@ -230,6 +309,16 @@ static int init_ctx(ppu_ctx* c, const ppu_model_cfg* cfg, const ppu_subset_spec*
   c->adam_lr = cfg->adam_lr;
   build_geometry(c);
   return PPU_OK;
+}
+
+// every replica's packed values <- the global parameters (Algorithm 1 line 6)
+static void ppu_restart_replicas(ppu_ctx* c) {
+  for (auto& r : c->reps) {
+    launch_slices_gather(r.d_segs, (int)r.segs.size(), c->theta, r.master, c->cfg.d_model,
+                         c->cfg.d_ff, r.n_ffn, c->stream);
+    launch_dense_move(r.d_dense, (int)r.dense.size(), r.master, c->theta, nullptr, 0, r.n_dense,
+                      c->stream);
+  }
 }
 
 extern "C" int ppu_query_bytes(const ppu_model_cfg* cfg, const ppu_subset_spec* spec, size_t* bytes) {
@@ -261,11 +350,7 @@ extern "C" int ppu_create(const ppu_model_cfg* cfg, const ppu_subset_spec* spec,
   c->arena = (uint8_t*)arena;
   c->arena_bytes = need;
   c->stream = (cudaStream_t)cuda_stream;
-  const char* e = getenv("PPU_GEMM");
-  c->gemm_backend = (e && !strcmp(e, "simt")) ? 1 : 0;
-  e = getenv("PPU_ATTN");
-  c->attn_backend = (e && !strcmp(e, "simt")) ? 1 : (e && !strcmp(e, "mma")) ? 2 : 0;
-  if (c->gemm_backend == 0 && gemm_tc_init() != 0) {
+  if (gemm_tc_init() != 0) {
     delete c;
     return ppu_fail(PPU_ECUDA, "cuTensorMapEncodeTiled not available from the driver");
   }
@@ -300,15 +385,17 @@ extern "C" int ppu_create(const ppu_model_cfg* cfg, const ppu_subset_spec* spec,
       }
     CREATE_OK(cudaMemcpyAsync(c->rope_cs, cs.data(), cs.size() * sizeof(float2),
                               cudaMemcpyHostToDevice, st));
-    for (auto& r : c->reps)
+    for (auto& r : c->reps) {
       if (!r.segs.empty())
         CREATE_OK(cudaMemcpyAsync(r.d_segs, r.segs.data(), r.segs.size() * sizeof(SliceSeg),
                                   cudaMemcpyHostToDevice, st));
+      if (!r.dense.empty())
+        CREATE_OK(cudaMemcpyAsync(r.d_dense, r.dense.data(), r.dense.size() * sizeof(DenseSeg),
+                                  cudaMemcpyHostToDevice, st));
+    }
     CREATE_OK(cudaStreamSynchronize(st));
   }
-  for (auto& r : c->reps)
-    launch_slices_gather(r.d_segs, (int)r.segs.size(), c->theta, r.master, c->cfg.d_model,
-                         c->cfg.d_ff, r.n_sub, st);
+  ppu_restart_replicas(c);
   CREATE_OK(cudaStreamSynchronize(st));
   CREATE_OK(cudaGetLastError());
 #undef CREATE_OK
@@ -358,14 +445,43 @@ extern "C" int ppu_tensor_info(const ppu_ctx* ctx, int32_t index, char* name, in
   return PPU_OK;
 }
 
-extern "C" int ppu_set_params(ppu_ctx* c, const float* theta, int64_t n) {
+// Moves between a canonical host vector and a replica's packed host array (the order of
+// ppu_subset_index).  to_packed: packed <- theta on the trained positions; else the reverse.
+static void host_pack(const ppu_ctx* c, const ReplicaState& r, float* theta, float* packed, bool to_packed) {
+  const int64_t d = c->cfg.d_model, F = c->cfg.d_ff;
+  auto mv = [&](float* canon, float* pk, size_t n) {
+    if (to_packed) memcpy(pk, canon, n * 4); else memcpy(canon, pk, n * 4);
+  };
+  for (const auto& s : r.segs) {
+    const int w = s.hi - s.lo;
+    float* p = packed + s.packed_off;
+    mv(theta + s.win_off + (int64_t)s.lo * d, p, (size_t)w * d);
+    p += (int64_t)w * d;
+    for (int64_t row = 0; row < d; ++row) mv(theta + s.wout_off + row * F + s.lo, p + row * w, (size_t)w);
+  }
+  for (const auto& s : r.dense) mv(theta + s.canon_off, packed + s.packed_off, (size_t)s.len);
+}
+
+extern "C" int ppu_set_params(ppu_ctx* c, int replica, const float* theta, int64_t n) {
   NEED_CTX(c);
   if (!theta || n != c->P) return ppu_fail(PPU_EINVAL, "theta null or wrong length");
+  if (replica < -1 || replica >= c->K) return ppu_fail(PPU_EINVAL, "replica out of range");
+  if (replica >= 0) {
+    ReplicaState& r = c->reps[replica];
+    if (r.n_sub == 0) return PPU_OK;
+    std::vector<float> packed(r.n_sub);
+    host_pack(c, r, const_cast<float*>(theta), packed.data(), true);
+    CUDA_OK(cudaStreamSynchronize(c->stream));
+    CUDA_OK(cudaMemcpy(r.master, packed.data(), r.n_sub * 4, cudaMemcpyHostToDevice));
+    if (c->resident == replica) {       // lay the new values over the working copy again
+      c->resident = -2;                 // neither the global values nor any replica's
+      ppu_make_resident(c, replica);
+    }
+    return PPU_OK;
+  }
   CUDA_OK(cudaMemcpyAsync(c->theta, theta, n * 4, cudaMemcpyHostToDevice, c->stream));
   launch_cast_bf16(c->theta, c->w16, c->P, c->stream);
-  for (auto& r : c->reps)
-    launch_slices_gather(r.d_segs, (int)r.segs.size(), c->theta, r.master, c->cfg.d_model,
-                         c->cfg.d_ff, r.n_sub, c->stream);
+  ppu_restart_replicas(c);
   c->resident = -1;
   CUDA_OK(cudaStreamSynchronize(c->stream));
   CUDA_OK(cudaGetLastError());
@@ -376,27 +492,15 @@ extern "C" int ppu_get_params(ppu_ctx* c, int replica, float* theta, int64_t n) 
   NEED_CTX(c);
   if (!theta || n != c->P) return ppu_fail(PPU_EINVAL, "theta null or wrong length");
   if (replica < -1 || replica >= c->K) return ppu_fail(PPU_EINVAL, "replica out of range");
-  if (replica < 0) {
-    CUDA_OK(cudaMemcpyAsync(theta, c->theta, n * 4, cudaMemcpyDeviceToHost, c->stream));
-    CUDA_OK(cudaStreamSynchronize(c->stream));
-    return PPU_OK;
-  }
-  // global vector first, then the replica's packed subset is laid over it on the host
-  ReplicaState& r = c->reps[replica];
   CUDA_OK(cudaMemcpyAsync(theta, c->theta, n * 4, cudaMemcpyDeviceToHost, c->stream));
   CUDA_OK(cudaStreamSynchronize(c->stream));
+  if (replica < 0) return PPU_OK;
+  // the replica's packed subset is laid over the global vector on the host
+  ReplicaState& r = c->reps[replica];
   if (r.n_sub == 0) return PPU_OK;
   std::vector<float> packed(r.n_sub);
   CUDA_OK(cudaMemcpy(packed.data(), r.master, r.n_sub * 4, cudaMemcpyDeviceToHost));
-  const int64_t d = c->cfg.d_model, F = c->cfg.d_ff;
-  for (const auto& s : r.segs) {
-    const int w = s.hi - s.lo;
-    const float* p = packed.data() + s.packed_off;
-    memcpy(theta + s.win_off + (int64_t)s.lo * d, p, (size_t)w * d * 4);
-    p += (int64_t)w * d;
-    for (int64_t row = 0; row < d; ++row)
-      memcpy(theta + s.wout_off + row * F + s.lo, p + row * w, (size_t)w * 4);
-  }
+  host_pack(c, r, theta, packed.data(), false);
   return PPU_OK;
 }
 
@@ -442,22 +546,28 @@ extern "C" int ppu_subset_index(const ppu_ctx* c, int replica, int64_t* index, i
     for (int64_t row = 0; row < d; ++row)
       for (int col = 0; col < w; ++col) index[j++] = s.wout_off + row * F + s.lo + col;
   }
+  for (const auto& s : r.dense)
+    for (int64_t i = 0; i < s.len; ++i) index[j++] = s.canon_off + i;
   return PPU_OK;
 }
 extern "C" int ppu_get_subset_grads(ppu_ctx* c, int replica, float* grads, int64_t n) {
   NEED_CTX(c);
   NEED_REPLICA(c, replica);
   if (c->last_stepped != replica) return ppu_fail(PPU_ESTATE, "gradients belong to replica %d", c->last_stepped);
-  if (!grads || n != c->reps[replica].n_sub) return ppu_fail(PPU_EINVAL, "grads null or wrong length");
-  CUDA_OK(cudaMemcpyAsync(grads, c->grad, n * 4, cudaMemcpyDeviceToHost, c->stream));
+  const ReplicaState& r = c->reps[replica];
+  if (!grads || n != r.n_sub) return ppu_fail(PPU_EINVAL, "grads null or wrong length");
   CUDA_OK(cudaStreamSynchronize(c->stream));
-  if (c->last_partials > 1) {   // add the split-K partials in the order the optimizer kernel uses
-    std::vector<float> part(n);
+  if (r.n_ffn) CUDA_OK(cudaMemcpy(grads, c->grad, r.n_ffn * 4, cudaMemcpyDeviceToHost));
+  if (c->last_partials > 1 && r.n_ffn) {   // add the split-K partials in the order the optimizer kernel uses
+    std::vector<float> part(r.n_ffn);
     for (int q = 1; q < c->last_partials; ++q) {
-      CUDA_OK(cudaMemcpy(part.data(), c->grad + (int64_t)q * c->max_sub, n * 4, cudaMemcpyDeviceToHost));
-      for (int64_t i = 0; i < n; ++i) grads[i] += part[i];
+      CUDA_OK(cudaMemcpy(part.data(), c->grad + (int64_t)q * c->max_ffn, r.n_ffn * 4, cudaMemcpyDeviceToHost));
+      for (int64_t i = 0; i < r.n_ffn; ++i) grads[i] += part[i];
     }
   }
+  if (r.n_dense)
+    CUDA_OK(cudaMemcpy(grads + r.n_ffn, c->grad + c->max_ffn * c->wgrad_splits, r.n_dense * 4,
+                       cudaMemcpyDeviceToHost));
   return PPU_OK;
 }
 extern "C" int ppu_get_subset_state(ppu_ctx* c, int replica, float* m, float* v, int32_t* step,
@@ -470,6 +580,35 @@ extern "C" int ppu_get_subset_state(ppu_ctx* c, int replica, float* m, float* v,
   if (v) CUDA_OK(cudaMemcpyAsync(v, r.v, n * 4, cudaMemcpyDeviceToHost, c->stream));
   CUDA_OK(cudaStreamSynchronize(c->stream));
   if (step) *step = r.step;
+  return PPU_OK;
+}
+extern "C" int ppu_set_subset_state(ppu_ctx* c, int replica, const float* m, const float* v,
+                                    int32_t step, int64_t n) {
+  NEED_CTX(c);
+  NEED_REPLICA(c, replica);
+  ReplicaState& r = c->reps[replica];
+  if ((m || v) && n != r.n_sub) return ppu_fail(PPU_EINVAL, "wrong length");
+  if (step < 0) return ppu_fail(PPU_EINVAL, "negative step count");
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  if (m && n) CUDA_OK(cudaMemcpy(r.m, m, n * 4, cudaMemcpyHostToDevice));
+  if (v && n) CUDA_OK(cudaMemcpy(r.v, v, n * 4, cudaMemcpyHostToDevice));
+  r.step = step;
+  return PPU_OK;
+}
+extern "C" int ppu_replica_values(ppu_ctx* c, int replica, void** dev_ptr, int64_t* n) {
+  NEED_CTX(c);
+  NEED_REPLICA(c, replica);
+  if (!dev_ptr || !n) return ppu_fail(PPU_EINVAL, "null out pointer");
+  *dev_ptr = c->reps[replica].master;
+  *n = c->reps[replica].n_sub;
+  return PPU_OK;
+}
+extern "C" int ppu_set_backends(ppu_ctx* c, int gemm, int attention) {
+  NEED_CTX(c);
+  if (gemm < 0 || gemm > 1 || attention < 0 || attention > 1)
+    return ppu_fail(PPU_EINVAL, "backends are 0 (tcgen05) or 1 (SIMT check kernels)");
+  c->gemm_backend = gemm;
+  c->attn_backend = attention;
   return PPU_OK;
 }
 extern "C" int ppu_set_adam_lr(ppu_ctx* c, float lr) {
@@ -496,6 +635,7 @@ extern "C" int ppu_stats(ppu_ctx* c, ppu_stats_t* out) {
   out->flops_dgrad = c->flops_dgrad;
   out->flops_wgrad = c->flops_wgrad;
   out->outer_bytes = c->outer_bytes;
+  out->saved_bytes_last_step = c->saved_bytes;
   return PPU_OK;
 }
 
@@ -525,11 +665,11 @@ extern "C" int ppu_gemm(const void* A, int64_t lda, int a_kmajor, const void* B,
 extern "C" int ppu_attention_fwd(const void* qkv, void* U, float* lse, int batch, int seq,
                                  int n_head, int d_head, int backend, void* cuda_stream) {
   if (!qkv || !U || !lse) return ppu_fail(PPU_EINVAL, "null operand");
+  if (backend < 0 || backend > 1) return ppu_fail(PPU_EINVAL, "unknown attention backend %d", backend);
   int rc;
-  if (backend == 0 || backend == 2) {
-    if (!attn_mma_supported(seq, d_head)) return ppu_fail(PPU_ESHAPE, "shape not covered by the tensor-core attention");
-    rc = backend == 0 ? launch_attn_fwd_tc((const bf16*)qkv, (bf16*)U, lse, batch, seq, n_head, d_head, nullptr, (cudaStream_t)cuda_stream)
-                      : launch_attn_fwd_mma((const bf16*)qkv, (bf16*)U, lse, batch, seq, n_head, d_head, (cudaStream_t)cuda_stream);
+  if (backend == 0) {
+    if (!attn_tc_supported(seq, d_head)) return ppu_fail(PPU_ESHAPE, "shape not covered by the tensor-core attention");
+    rc = launch_attn_fwd_tc((const bf16*)qkv, (bf16*)U, lse, batch, seq, n_head, d_head, nullptr, (cudaStream_t)cuda_stream);
   } else {
     rc = launch_attn_fwd_simt((const bf16*)qkv, (bf16*)U, lse, batch, seq, n_head, d_head, (cudaStream_t)cuda_stream);
   }
@@ -541,11 +681,11 @@ extern "C" int ppu_attention_bwd(const void* qkv, const void* U, const float* ls
                                  void* dqkv, float* scratch, int batch, int seq, int n_head,
                                  int d_head, int backend, void* cuda_stream) {
   if (!qkv || !U || !lse || !dU || !dqkv || !scratch) return ppu_fail(PPU_EINVAL, "null operand");
+  if (backend < 0 || backend > 1) return ppu_fail(PPU_EINVAL, "unknown attention backend %d", backend);
   int rc;
-  if (backend == 0 || backend == 2) {
-    if (!attn_mma_supported(seq, d_head)) return ppu_fail(PPU_ESHAPE, "shape not covered by the tensor-core attention");
-    rc = backend == 0 ? launch_attn_bwd_tc((const bf16*)qkv, (const bf16*)U, lse, (const bf16*)dU, (bf16*)dqkv, scratch, batch, seq, n_head, d_head, nullptr, (cudaStream_t)cuda_stream)
-                      : launch_attn_bwd_mma((const bf16*)qkv, (const bf16*)U, lse, (const bf16*)dU, (bf16*)dqkv, scratch, batch, seq, n_head, d_head, (cudaStream_t)cuda_stream);
+  if (backend == 0) {
+    if (!attn_tc_supported(seq, d_head)) return ppu_fail(PPU_ESHAPE, "shape not covered by the tensor-core attention");
+    rc = launch_attn_bwd_tc((const bf16*)qkv, (const bf16*)U, lse, (const bf16*)dU, (bf16*)dqkv, scratch, batch, seq, n_head, d_head, nullptr, (cudaStream_t)cuda_stream);
   } else {
     rc = launch_attn_bwd_simt((const bf16*)qkv, (const bf16*)U, lse, (const bf16*)dU, (bf16*)dqkv, scratch, batch, seq, n_head, d_head, (cudaStream_t)cuda_stream);
   }

@@ -31,41 +31,41 @@ int ppu_make_resident(ppu_ctx* c, int k) {
   const int d = c->cfg.d_model, F = c->cfg.d_ff;
   if (c->resident >= 0) {
     ReplicaState& r = c->reps[c->resident];
-    launch_slices_to_w16(r.d_segs, (int)r.segs.size(), nullptr, c->theta, c->w16, 0, d, F, r.n_sub,
+    EvScope ev(c, PPU_CLS_OTHER, 6.0 * (double)r.n_sub);
+    launch_slices_to_w16(r.d_segs, (int)r.segs.size(), nullptr, c->theta, c->w16, 0, d, F, r.n_ffn,
                          c->stream);
-    c->launches++;
+    launch_dense_move(r.d_dense, (int)r.dense.size(), nullptr, c->theta, c->w16, 2, r.n_dense, c->stream);
+    c->launches += (r.segs.empty() ? 0 : 1) + (r.dense.empty() ? 0 : 1);
   }
   if (k >= 0) {
     ReplicaState& r = c->reps[k];
-    launch_slices_to_w16(r.d_segs, (int)r.segs.size(), r.master, nullptr, c->w16, 1, d, F, r.n_sub,
+    EvScope ev(c, PPU_CLS_OTHER, 6.0 * (double)r.n_sub);
+    launch_slices_to_w16(r.d_segs, (int)r.segs.size(), r.master, nullptr, c->w16, 1, d, F, r.n_ffn,
                          c->stream);
-    c->launches++;
+    launch_dense_move(r.d_dense, (int)r.dense.size(), r.master, nullptr, c->w16, 1, r.n_dense, c->stream);
+    c->launches += (r.segs.empty() ? 0 : 1) + (r.dense.empty() ? 0 : 1);
   }
   c->resident = k;
   return PPU_OK;
 }
 
-namespace {
-
 constexpr size_t EV_POOL_PAIRS = 16384;
 
-// Brackets one launch with events when profiling is on.
-struct EvScope {
-  ppu_ctx* c; int slot = -1;
-  EvScope(ppu_ctx* ctx, int cls, double flops) : c(ctx) {
-    if (!c->profiling) return;
-    if (c->ev_recs.size() >= EV_POOL_PAIRS) { c->ev_dropped++; return; }
-    slot = (int)c->ev_recs.size();
-    if (c->ev_pool.size() < 2 * (size_t)(slot + 1)) {
-      cudaEvent_t a, b;
-      if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { slot = -1; return; }
-      c->ev_pool.push_back(a); c->ev_pool.push_back(b);
-    }
-    c->ev_recs.push_back({cls, flops});
-    cudaEventRecord(c->ev_pool[2 * slot], c->stream);
+EvScope::EvScope(ppu_ctx* ctx, int cls, double work) : c(ctx) {
+  if (!c->profiling) return;
+  if (c->ev_recs.size() >= EV_POOL_PAIRS) { c->ev_dropped++; return; }
+  slot = (int)c->ev_recs.size();
+  if (c->ev_pool.size() < 2 * (size_t)(slot + 1)) {
+    cudaEvent_t a, b;
+    if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { slot = -1; return; }
+    c->ev_pool.push_back(a); c->ev_pool.push_back(b);
   }
-  ~EvScope() { if (slot >= 0) cudaEventRecord(c->ev_pool[2 * slot + 1], c->stream); }
-};
+  c->ev_recs.push_back({cls, work});
+  cudaEventRecord(c->ev_pool[2 * slot], c->stream);
+}
+EvScope::~EvScope() { if (slot >= 0) cudaEventRecord(c->ev_pool[2 * slot + 1], c->stream); }
+
+namespace {
 
 struct Sched {
   ppu_ctx* c;
@@ -77,7 +77,19 @@ struct Sched {
     dh = d / h; L = c->cfg.n_layer;
   }
   const bf16* W(int l, int64_t rel) const { return c->w16 + c->e_size + (int64_t)l * c->layer_size + rel; }
-  const float* Pf(int l, int64_t rel) const { return c->theta + c->e_size + (int64_t)l * c->layer_size + rel; }
+  int64_t canon(int l, int64_t rel) const { return c->e_size + (int64_t)l * c->layer_size + rel; }
+  // fp32 LayerNorm gain / shift as the replica sees it: its own value where it trains them
+  const float* lnp(const ReplicaState* rep, int64_t off) const {
+    if (rep && rep->rest) {
+      const int64_t po = rep->packed_of(off);
+      if (po >= 0) return rep->master + po;
+    }
+    return c->theta + off;
+  }
+  // where the gradient of the dense run starting at canonical offset `off` goes
+  float* gdense(const ReplicaState& r, int64_t off) const {
+    return c->grad + c->max_ffn * c->wgrad_splits + (r.packed_of(off) - r.n_ffn);
+  }
 
   void gemm(const bf16* A, int64_t lda, int ak, const bf16* Bm, int64_t ldb, int bk, int M, int N,
             int K, int epi, void* C, int64_t ldc, void* C2, const void* aux, int64_t ldaux,
@@ -90,30 +102,50 @@ struct Sched {
     g.ldaux = ldaux; g.flags = c->flags; g.splits = splits; g.split_stride = split_stride;
     g.rope_S = S; g.rope_dh = dh; g.rope_cols = rope_cols;
     g.C3 = C3; g.ldc3 = ldc3; g.c3_lo = c3_lo; g.c3_hi = c3_hi;
-    EvScope ev(c, 0, 2.0 * M * N * (double)K);
+    EvScope ev(c, PPU_CLS_GEMM, 2.0 * M * N * (double)K);
     rc = c->gemm_backend == 1 ? launch_gemm_simt(g, c->stream) : launch_gemm_tc(g, c->stream);
     c->launches++;
     if (flop_counter) *flop_counter += 2.0 * M * N * (double)K;
   }
+  // weight gradient dW[M,N] = X^T Y over the tokens: X [T, >=M] and Y [T, >=N] token-major, fp32 out
+  void wgrad(const bf16* X, int64_t ldx, const bf16* Y, int64_t ldy, int M, int N, float* out, int64_t ldo) {
+    gemm(X, ldx, 0, Y, ldy, 0, M, N, T, EPI_STORE_F32, out, ldo, nullptr, nullptr, 0, &c->flops_wgrad);
+  }
+  void ln_fwd(const float* x, const float* g, const float* b, bf16* y, float2* st) {
+    EvScope ev(c, PPU_CLS_LN, 6.0 * T * (double)d);
+    launch_ln_fwd(x, g, b, y, st, T, d, c->cfg.ln_eps, c->stream);
+    c->launches++;
+  }
+  void ln_bwd(const bf16* dy, const float* x, const float2* st, const float* gamma, const float* gin) {
+    EvScope ev(c, PPU_CLS_LN, (gin ? 16.0 : 12.0) * T * (double)d);
+    launch_ln_bwd(dy, x, st, gamma, gin, c->g, c->g16, T, d, c->stream);
+    c->launches++;
+  }
+  void ln_param_grad(const ReplicaState& r, const bf16* dy, const float* x, const float2* st,
+                     int64_t off_g, int64_t off_b) {
+    EvScope ev(c, PPU_CLS_LN, 6.0 * T * (double)d);
+    launch_ln_param_grad(dy, x, st, gdense(r, off_g), gdense(r, off_b), c->ln_partial, T, d, c->stream);
+    c->launches += 2;
+  }
   // split-K partial buffers the subset weight-gradient products of this step write
   int partials() const { const int kb = (T + 63) / 64; return c->wgrad_splits < kb ? c->wgrad_splits : kb; }
-  // 0: tcgen05 kernels, 2: mma.sync kernels (both need d_h 64 or 128), 1: SIMT
-  int attn_kind() const {
-    if (c->attn_backend == 0 && attn_tc_supported(S, dh)) return 0;
-    if (c->attn_backend != 1 && attn_mma_supported(S, dh)) return 2;
-    return 1;
-  }
+  // 0: tcgen05 kernels (d_h 64 or 128), 1: SIMT
+  int attn_kind() const { return (c->attn_backend == 0 && attn_tc_supported(S, dh)) ? 0 : 1; }
 
   // Forward pass over all parameters (Appendix C.1 forward equations), saving what the
-  // restricted backward needs.
-  void forward(const int32_t* tok, const ReplicaState* rep = nullptr) {
+  // restricted backward needs: nothing of the layers below the replica's lowest trained layer.
+  void forward(const int32_t* tok, const ReplicaState* rep, bool keep) {
     cudaStream_t st = c->stream;
-    launch_embed(tok, c->w16, c->acts[0].x, T, d, V, c->flags, st); c->launches++;
+    c->saved_bytes = 0;
+    const int lowest = (keep && rep && rep->lowest >= 0) ? rep->lowest : L;   // evaluation keeps nothing
+    {
+      EvScope ev(c, PPU_CLS_OTHER, 6.0 * T * (double)d);
+      launch_embed(tok, c->w16, c->acts[0].x, T, d, V, c->flags, st); c->launches++;
+    }
     for (int l = 0; l < L && !rc; ++l) {
       LayerActs& a = c->acts[l];
       float* x_next = (l + 1 < L) ? c->acts[l + 1].x : c->x_last;
-      launch_ln_fwd(a.x, Pf(l, c->rel_ln1g), Pf(l, c->rel_ln1b), c->a16, a.st1, T, d, c->cfg.ln_eps, st);
-      c->launches++;
+      ln_fwd(a.x, lnp(rep, canon(l, c->rel_ln1g)), lnp(rep, canon(l, c->rel_ln1b)), c->a16, a.st1);
       if (c->gemm_backend == 0) {   // rotary positions applied in the projection's epilogue
         gemm(c->a16, d, 1, W(l, c->rel_wq), d, 1, T, 3 * d, d, EPI_ROPE_BF16, a.qkv, 3 * d, nullptr,
              c->rope_cs, 0, &c->flops_fwd, 1, 0, 2 * d);
@@ -124,55 +156,64 @@ struct Sched {
       }
       {
         const double fl = 4.0 * B * h * dh * 0.5 * S * (double)(S + 1);
-        EvScope ev(c, 1, fl);
-        const int kind = attn_kind();
-        if (kind == 0) rc |= launch_attn_fwd_tc(a.qkv, a.U, a.lse, B, S, h, dh, c->flags, st);
-        else if (kind == 2) rc |= launch_attn_fwd_mma(a.qkv, a.U, a.lse, B, S, h, dh, st);
+        EvScope ev(c, PPU_CLS_ATTN, fl);
+        if (attn_kind() == 0) rc |= launch_attn_fwd_tc(a.qkv, a.U, a.lse, B, S, h, dh, c->flags, st);
         else rc |= launch_attn_fwd_simt(a.qkv, a.U, a.lse, B, S, h, dh, st);
         c->launches++;
         c->flops_fwd += fl;
       }
       gemm(a.U, d, 1, W(l, c->rel_wo), d, 1, T, d, d, EPI_RESID_F32, a.x1, d, nullptr, a.x, d,
            &c->flops_fwd);
-      launch_ln_fwd(a.x1, Pf(l, c->rel_ln2g), Pf(l, c->rel_ln2b), a.b, a.st2, T, d, c->cfg.ln_eps, st);
-      c->launches++;
-      // gelu(Hd) goes to a buffer shared by all layers; only the replica's own columns are kept
+      ln_fwd(a.x1, lnp(rep, canon(l, c->rel_ln2g)), lnp(rep, canon(l, c->rel_ln2b)), a.b, a.st2);
+      // gelu(Hd) goes to a buffer shared by all layers; only the replica's own columns are kept,
+      // and the pre-activation only where the backward pass will come
+      const bool kept = l >= lowest;
       const int lo = rep ? rep->lo[l] : 0, hi = rep ? rep->hi[l] : 0;
-      gemm(a.b, d, 1, W(l, c->rel_win), d, 1, T, F, d, EPI_GELU_DUAL, a.Hd, F, c->A_tmp, nullptr, 0,
-           &c->flops_fwd, 1, 0, 0, hi > lo ? a.As : nullptr, hi - lo, lo, hi);
+      gemm(a.b, d, 1, W(l, c->rel_win), d, 1, T, F, d, EPI_GELU_DUAL, kept ? a.Hd : nullptr, F, c->A_tmp,
+           nullptr, 0, &c->flops_fwd, 1, 0, 0, (kept && hi > lo) ? a.As : nullptr, hi - lo, lo, hi);
       gemm(c->A_tmp, F, 1, W(l, c->rel_wout), F, 1, T, d, F, EPI_RESID_F32, x_next, d, nullptr, a.x1, d,
            &c->flops_fwd);
+      if (kept)   // x, x1, both statistics, qkv, U, lse, b, Hd and the trained columns of gelu(Hd)
+        c->saved_bytes += (int64_t)T * (4 * d + 4 * d + 16 + 6 * d + 2 * d + 4 * h + 2 * d + 2 * (int64_t)F + 2 * (hi - lo));
     }
-    launch_ln_fwd(c->x_last, c->theta + c->off_lnfg, c->theta + c->off_lnfb, c->f16, c->stf, T, d,
-                  c->cfg.ln_eps, st);
-    c->launches++;
+    ln_fwd(c->x_last, lnp(rep, c->off_lnfg), lnp(rep, c->off_lnfb), c->f16, c->stf);
     gemm(c->f16, d, 1, c->w16, d, 1, T, V, d, EPI_STORE_BF16, c->logits, V, nullptr, nullptr, 0,
          &c->flops_fwd);
   }
 
   void loss(const int32_t* tok, int write_grad, float* out) {
     cudaStream_t st = c->stream;
-    launch_xent(c->logits, tok, c->row_loss, B, S, V, write_grad, st); c->launches++;
+    {
+      EvScope ev(c, PPU_CLS_XENT, (write_grad ? 4.0 : 2.0) * T * (double)V);
+      launch_xent(c->logits, tok, c->row_loss, B, S, V, write_grad, st); c->launches++;
+    }
     launch_loss_reduce(c->row_loss, T, 1.f / (float)((int64_t)B * (S - 1)), out, st); c->launches++;
   }
 
-  // Restricted backward (Appendix C.1): input gradients through every slice and head down to
-  // the lowest trained layer, weight gradients only for the replica's own hidden-unit range.
-  void backward(const ReplicaState& r) {
+  // Restricted backward (Appendix C.1): input gradients through every FFN slice and every head,
+  // weight gradients only for what the replica trains - its hidden-unit range per layer, the
+  // query / key / value rows of its heads, and (paper's MLP-only and MLP + head slicing) the
+  // parameters that are never sliced.  When only FFN slices are trained the pass stops at the
+  // lowest trained layer, where only that slice's part is computed.
+  void backward(const ReplicaState& r, const int32_t* tok) {
     if (r.lowest < 0) return;
     cudaStream_t st = c->stream;
-    // output head (tied embedding is frozen: no weight gradient)
+    const bool deep = r.deep();
+    const int kind = attn_kind();
+    // output head: dE (tied embedding) = dlogits^T f when the embedding is trained
+    if (r.rest) wgrad(c->logits, V, c->f16, d, V, d, gdense(r, 0), d);
     gemm(c->logits, V, 1, c->w16, d, 0, T, d, V, EPI_STORE_BF16, c->t16, d, nullptr, nullptr, 0,
          &c->flops_dgrad);
-    launch_ln_bwd(c->t16, c->x_last, c->stf, c->theta + c->off_lnfg, nullptr, c->g, c->g16, T, d, st);
-    c->launches++;
+    if (r.rest) ln_param_grad(r, c->t16, c->x_last, c->stf, c->off_lnfg, c->off_lnfb);
+    ln_bwd(c->t16, c->x_last, c->stf, lnp(&r, c->off_lnfg), nullptr);
     int seg = (int)r.segs.size() - 1;
     for (int l = L - 1; l >= r.lowest && !rc; --l) {
       LayerActs& a = c->acts[l];
       const bool trained = seg >= 0 && r.seg_layer[seg] == l;
       const SliceSeg* s = trained ? &r.segs[seg] : nullptr;
       const int w = trained ? s->hi - s->lo : 0;
-      if (l == r.lowest) {
+      const bool cut = !deep && l == r.lowest;
+      if (cut) {
         // only this replica's slice: dA_n = G V_n, through the activation, then both products
         gemm(c->g16, d, 1, W(l, c->rel_wout) + s->lo, F, 0, T, w, d, EPI_DGELU, c->dHd + s->lo, F,
              nullptr, a.Hd + s->lo, F, &c->flops_dgrad);
@@ -183,20 +224,21 @@ struct Sched {
       if (trained) {
         // dW_in[lo:hi,:] = dHd[:,lo:hi]^T b      dW_out[:,lo:hi] = g^T A[:,lo:hi]
         gemm(c->dHd + s->lo, F, 0, a.b, d, 0, w, d, T, EPI_STORE_F32, c->grad + s->packed_off, d,
-             nullptr, nullptr, 0, &c->flops_wgrad, partials(), c->max_sub);
+             nullptr, nullptr, 0, &c->flops_wgrad, partials(), c->max_ffn);
         gemm(c->g16, d, 0, a.As, w, 0, d, w, T, EPI_STORE_F32,
              c->grad + s->packed_off + (int64_t)w * d, w, nullptr, nullptr, 0, &c->flops_wgrad,
-             partials(), c->max_sub);
+             partials(), c->max_ffn);
         --seg;
       }
-      if (l == r.lowest) break;
+      if (cut) break;
       gemm(c->dHd, F, 1, W(l, c->rel_win), d, 0, T, d, F, EPI_STORE_BF16, c->t16, d, nullptr,
            nullptr, 0, &c->flops_dgrad);
-      launch_ln_bwd(c->t16, a.x1, a.st2, Pf(l, c->rel_ln2g), c->g, c->g, c->g16, T, d, st);
-      c->launches++;
+      if (r.rest) ln_param_grad(r, c->t16, a.x1, a.st2, canon(l, c->rel_ln2g), canon(l, c->rel_ln2b));
+      ln_bwd(c->t16, a.x1, a.st2, lnp(&r, canon(l, c->rel_ln2g)), c->g);
+      // dW_o = g1^T U
+      if (r.rest) wgrad(c->g16, d, a.U, d, d, d, gdense(r, canon(l, c->rel_wo)), d);
       // dU = g1 W_O^T; where the tile shape allows, its epilogue also forms delta = rowsum(dU * U)
       // per (token, head) for the attention backward
-      const int kind = attn_kind();
       bool delta_fused = false;
       if (kind == 0 && c->gemm_backend == 0) {
         GemmArgs q;
@@ -213,21 +255,38 @@ struct Sched {
              0, &c->flops_dgrad);
       {
         const double fl = 10.0 * B * h * dh * 0.5 * S * (double)(S + 1);
-        EvScope ev(c, 1, fl);
+        EvScope ev(c, PPU_CLS_ATTN, fl);
         if (kind == 0)   // rotates dq, dk back on the way out (the output drain overlaps the next item's products)
           rc |= launch_attn_bwd_tc(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, c->flags, st,
                                    c->rope_cs, delta_fused);
-        else if (kind == 2)
-          rc |= launch_attn_bwd_mma(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, st);
         else
           rc |= launch_attn_bwd_simt(a.qkv, a.U, a.lse, c->t16, c->dqkv, c->attn_scratch, B, S, h, dh, st);
         c->launches += (kind == 1 ? 2 : 3) - (delta_fused ? 1 : 0);
         c->flops_dgrad += fl;
         if (kind != 0) { launch_rope(c->dqkv, c->rope_cs, B, S, h, dh, 1, st); c->launches++; }
       }
+      if (r.h_hi > r.h_lo) {
+        // dW_{q,k,v}[rows of the trained heads] = dqkv[:, those columns]^T a, with a = LN1(x) formed
+        // again from the saved block input (it is not kept by the forward pass)
+        ln_fwd(a.x, lnp(&r, canon(l, c->rel_ln1g)), lnp(&r, canon(l, c->rel_ln1b)), c->a16, a.st1);
+        const int rows = (r.h_hi - r.h_lo) * dh, r0 = r.h_lo * dh;
+        if (rows == d) {    // every head: W_q, W_k, W_v are adjacent, one product
+          wgrad(c->dqkv, 3 * d, c->a16, d, 3 * d, d, gdense(r, canon(l, c->rel_wq)), d);
+        } else {
+          for (int q = 0; q < 3; ++q)
+            wgrad(c->dqkv + q * d + r0, 3 * d, c->a16, d, rows, d,
+                  gdense(r, canon(l, c->rel_wq) + (int64_t)q * d * d + (int64_t)r0 * d), d);
+        }
+      }
+      if (l == 0 && !r.rest) break;      // nothing below needs the input gradient
       gemm(c->dqkv, 3 * d, 1, W(l, c->rel_wq), d, 0, T, d, 3 * d, EPI_STORE_BF16, c->t16, d, nullptr,
            nullptr, 0, &c->flops_dgrad);
-      launch_ln_bwd(c->t16, a.x, a.st1, Pf(l, c->rel_ln1g), c->g, c->g, c->g16, T, d, st);
+      if (r.rest) ln_param_grad(r, c->t16, a.x, a.st1, canon(l, c->rel_ln1g), canon(l, c->rel_ln1b));
+      ln_bwd(c->t16, a.x, a.st1, lnp(&r, canon(l, c->rel_ln1g)), c->g);
+    }
+    if (r.rest && !rc) {   // input embedding: the rows the batch used, added to the head's part
+      EvScope ev(c, PPU_CLS_OTHER, 12.0 * T * (double)d);
+      launch_embed_grad(tok, c->g, gdense(r, 0), T, d, V, st);
       c->launches++;
     }
   }
@@ -254,9 +313,9 @@ extern "C" int ppu_local_step(ppu_ctx* c, int replica, const int32_t* tokens, in
   c->flops_fwd = c->flops_dgrad = c->flops_wgrad = 0;
   ppu_make_resident(c, replica);
   Sched s(c, batch, seq);
-  s.forward(tokens, &r);
+  s.forward(tokens, &r, true);
   s.loss(tokens, 1, c->loss + replica);
-  s.backward(r);
+  s.backward(r, tokens);
   if (s.rc) return ppu_fail(PPU_ECUDA, "kernel launch failed in local step (%d)", s.rc);
   r.step += 1;
   if (r.n_sub > 0) {
@@ -266,9 +325,12 @@ extern "C" int ppu_local_step(ppu_ctx* c, int replica, const int32_t* tokens, in
     hp.bc1 = (float)(1.0 - std::pow((double)hp.beta1, (double)r.step));
     hp.bc2 = (float)(1.0 - std::pow((double)hp.beta2, (double)r.step));
     c->last_partials = s.partials();
-    launch_adamw(r.d_segs, (int)r.segs.size(), r.master, r.m, r.v, c->grad, c->last_partials, c->max_sub, c->w16,
-                 c->cfg.d_model, c->cfg.d_ff, r.n_sub, hp, c->stream);
-    c->launches++;
+    EvScope ev(c, PPU_CLS_ADAMW, 30.0 * (double)r.n_sub + 4.0 * (c->last_partials - 1) * (double)r.n_ffn);
+    launch_adamw(r.d_segs, (int)r.segs.size(), r.master, r.m, r.v, c->grad, c->last_partials, c->max_ffn, c->w16,
+                 c->cfg.d_model, c->cfg.d_ff, r.n_ffn, hp, c->stream);
+    launch_adamw_dense(r.d_dense, (int)r.dense.size(), r.master, r.m, r.v, c->grad + c->max_ffn * c->wgrad_splits,
+                       r.n_ffn, c->w16, r.n_dense, hp, c->stream);
+    c->launches += (r.segs.empty() ? 0 : 1) + (r.dense.empty() ? 0 : 1);
   }
   r.stepped = true;
   c->last_stepped = replica;
@@ -309,7 +371,7 @@ extern "C" int ppu_eval_loss(ppu_ctx* c, int replica, const int32_t* tokens, int
   if (!loss_out) return ppu_fail(PPU_EINVAL, "loss_out is null");
   ppu_make_resident(c, replica);
   Sched s(c, batch, seq);
-  s.forward(tokens);
+  s.forward(tokens, replica >= 0 ? &c->reps[replica] : nullptr, false);
   s.loss(tokens, 0, c->loss + c->K);
   if (s.rc) return ppu_fail(PPU_ECUDA, "kernel launch failed in evaluation (%d)", s.rc);
   float v = 0.f;
@@ -321,6 +383,111 @@ extern "C" int ppu_eval_loss(ppu_ctx* c, int replica, const int32_t* tokens, int
 }
 
 namespace {
+// Builds the outer-sync tables for a list of replicas: the segments of the canonical vector with
+// their owners, the chunk list the kernel walks, and the per-hidden-unit owner lists of the FFN
+// matrices.  Segments never straddle a layer (or the embedding / final-norm) boundary, so a
+// streaming-sync group is a contiguous range of chunks.
+int build_outer_tables(ppu_ctx* c, const std::vector<int32_t>& list) {
+  const int L = c->cfg.n_layer, F = c->cfg.d_ff, d = c->cfg.d_model;
+  const int64_t fd = (int64_t)F * d;
+  std::vector<OuterSeg> segs;
+  std::vector<DenseOwner> downers;
+  // dense runs of the listed replicas, as (start, end, master, shift) events
+  struct Run { int64_t lo, hi; float* master; int64_t shift; };
+  std::vector<Run> runs;
+  for (int k : list) {
+    const ReplicaState& r = c->reps[k];
+    for (const auto& s : r.dense) runs.push_back({s.canon_off, s.canon_off + s.len, r.master, s.packed_off - s.canon_off});
+  }
+  // cuts [lo, hi) of the canonical vector at every run boundary and lists each piece's owners;
+  // neighbouring pieces with the same owners and shifts are joined
+  auto add_dense = [&](int64_t lo, int64_t hi, int layer) {
+    std::vector<int64_t> cuts = {lo, hi};
+    for (const auto& r : runs) {
+      if (r.lo > lo && r.lo < hi) cuts.push_back(r.lo);
+      if (r.hi > lo && r.hi < hi) cuts.push_back(r.hi);
+    }
+    std::sort(cuts.begin(), cuts.end());
+    cuts.erase(std::unique(cuts.begin(), cuts.end()), cuts.end());
+    std::vector<DenseOwner> prev; bool have_prev = false;
+    for (size_t i = 0; i + 1 < cuts.size(); ++i) {
+      std::vector<DenseOwner> own;
+      for (const auto& r : runs)
+        if (r.lo <= cuts[i] && r.hi >= cuts[i + 1]) own.push_back({r.master, r.shift});
+      const bool same = have_prev && own.size() == prev.size() &&
+                        std::equal(own.begin(), own.end(), prev.begin(), [](const DenseOwner& a, const DenseOwner& b) {
+                          return a.master == b.master && a.shift == b.shift; });
+      if (same) { segs.back().len += cuts[i + 1] - cuts[i]; continue; }
+      OuterSeg sg; sg.start = cuts[i]; sg.len = cuts[i + 1] - cuts[i]; sg.base = 0; sg.kind = 0; sg.layer = layer;
+      sg.ob = (int32_t)downers.size();
+      downers.insert(downers.end(), own.begin(), own.end());
+      sg.oe = (int32_t)downers.size();
+      segs.push_back(sg);
+      prev = own; have_prev = true;
+    }
+  };
+  std::vector<int> layer_seg_begin(L + 2, 0);
+  add_dense(0, c->e_size, -1);
+  for (int l = 0; l < L; ++l) {
+    layer_seg_begin[l] = (int)segs.size();
+    const int64_t base = c->e_size + (int64_t)l * c->layer_size;
+    add_dense(base, base + c->rel_win, l);
+    OuterSeg sg; sg.layer = l; sg.ob = sg.oe = 0; sg.len = fd;
+    sg.start = sg.base = base + c->rel_win; sg.kind = 1; segs.push_back(sg);
+    sg.start = sg.base = base + c->rel_wout; sg.kind = 2; segs.push_back(sg);
+  }
+  layer_seg_begin[L] = (int)segs.size();
+  add_dense(c->off_lnfg, c->P, -1);
+  layer_seg_begin[L + 1] = (int)segs.size();
+  // chunk list; chunk index where every layer begins
+  std::vector<OuterChunk> chunks;
+  std::vector<int> seg_chunk_begin(segs.size() + 1, 0);
+  for (size_t i = 0; i < segs.size(); ++i) {
+    seg_chunk_begin[i] = (int)chunks.size();
+    for (int64_t off = 0; off < segs[i].len; off += OUTER_CHUNK) chunks.push_back({(int32_t)i, 0, off});
+  }
+  seg_chunk_begin[segs.size()] = (int)chunks.size();
+  c->layer_chunk_begin.assign(L + 2, 0);
+  for (int l = 0; l <= L + 1; ++l) c->layer_chunk_begin[l] = seg_chunk_begin[layer_seg_begin[l]];
+  c->chunks_e = c->layer_chunk_begin[0];
+  c->n_chunks = (int)chunks.size();
+  // owners of every group of 8 hidden units, in the order the replicas were listed
+  std::vector<std::vector<OuterOwner>> per_group((size_t)L * (F / 8));
+  for (int k : list) {
+    const ReplicaState& r = c->reps[k];
+    for (size_t i = 0; i < r.segs.size(); ++i) {
+      const SliceSeg& s = r.segs[i];
+      OuterOwner o;
+      o.master = r.master; o.in_off = s.packed_off;
+      o.out_off = s.packed_off + (int64_t)(s.hi - s.lo) * d; o.lo = s.lo; o.hi = s.hi;
+      const int l = r.seg_layer[i];
+      for (int u8 = s.lo / 8; u8 < s.hi / 8; ++u8) per_group[(size_t)l * (F / 8) + u8].push_back(o);
+    }
+  }
+  std::vector<int32_t> begin(per_group.size() + 1, 0);
+  std::vector<OuterOwner> flat;
+  for (size_t gi = 0; gi < per_group.size(); ++gi) {
+    begin[gi] = (int32_t)flat.size();
+    flat.insert(flat.end(), per_group[gi].begin(), per_group[gi].end());
+  }
+  begin[per_group.size()] = (int32_t)flat.size();
+  if (segs.size() > c->cap_oseg || chunks.size() > c->cap_ochunk || downers.size() > c->cap_downer ||
+      flat.size() > c->cap_uowner)
+    return ppu_fail(PPU_ESTATE, "outer-sync tables larger than the arena reserved for them");
+  // the previous sync's kernel may still be reading the tables
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  CUDA_OK(cudaMemcpy(c->d_oseg, segs.data(), segs.size() * sizeof(OuterSeg), cudaMemcpyHostToDevice));
+  CUDA_OK(cudaMemcpy(c->d_ochunk, chunks.data(), chunks.size() * sizeof(OuterChunk), cudaMemcpyHostToDevice));
+  if (!downers.empty())
+    CUDA_OK(cudaMemcpy(c->d_downer, downers.data(), downers.size() * sizeof(DenseOwner), cudaMemcpyHostToDevice));
+  CUDA_OK(cudaMemcpy(c->d_unit_begin, begin.data(), begin.size() * 4, cudaMemcpyHostToDevice));
+  if (!flat.empty())
+    CUDA_OK(cudaMemcpy(c->d_unit_owner, flat.data(), flat.size() * sizeof(OuterOwner), cudaMemcpyHostToDevice));
+  c->h_oseg = segs;
+  c->cached_sync_list = list;
+  return PPU_OK;
+}
+
 // Outer step over the listed replicas on one group of positions (group < 0: every position).
 int outer_sync_impl(ppu_ctx* c, const int32_t* replicas, int n, int group, int n_groups) {
   if (!c) return ppu_fail(PPU_EINVAL, "ctx is null");
@@ -338,75 +505,53 @@ int outer_sync_impl(ppu_ctx* c, const int32_t* replicas, int n, int group, int n
     }
   }
   const int64_t launches0 = c->launches;
+  if (list != c->cached_sync_list || c->n_chunks == 0) {
+    const int rc = build_outer_tables(c, list);
+    if (rc) return rc;
+  }
   // layers [l0, l1) and, for the last group, the embeddings and the final LayerNorm
   const bool all = group < 0, tail = all || group == n_groups;
   const int per = all ? L : L / n_groups;
   const int l0 = all ? 0 : (tail ? L : group * per), l1 = all ? L : (tail ? L : l0 + per);
+  // positions swept and (owner, owned position) pairs inside the swept range
+  const int64_t lo_pos = c->e_size + (int64_t)l0 * c->layer_size, hi_pos = c->e_size + (int64_t)l1 * c->layer_size;
+  auto inside = [&](int64_t pos) { return (pos >= lo_pos && pos < hi_pos) || (tail && (pos < c->e_size || pos >= c->off_lnfg)); };
   double owned = 0;
   for (int k : list) {
     const ReplicaState& r = c->reps[k];
     for (size_t i = 0; i < r.segs.size(); ++i)
       if (r.seg_layer[i] >= l0 && r.seg_layer[i] < l1) owned += 2.0 * (double)(r.segs[i].hi - r.segs[i].lo) * d;
-  }
-  if (list != c->cached_sync_list || list.empty()) {
-    std::vector<OuterOwner> owners;
-    std::vector<std::vector<int32_t>> per_group((size_t)L * (F / 8));
-    for (int k : list) {
-      const ReplicaState& r = c->reps[k];
-      for (size_t i = 0; i < r.segs.size(); ++i) {
-        const SliceSeg& s = r.segs[i];
-        OuterOwner o;
-        o.master = r.master; o.in_off = s.packed_off;
-        o.out_off = s.packed_off + (int64_t)(s.hi - s.lo) * d; o.lo = s.lo; o.hi = s.hi;
-        const int32_t id = (int32_t)owners.size();
-        owners.push_back(o);
-        const int l = r.seg_layer[i];
-        for (int u8 = s.lo / 8; u8 < s.hi / 8; ++u8) per_group[(size_t)l * (F / 8) + u8].push_back(id);
-      }
-    }
-    std::vector<int32_t> begin(per_group.size() + 1, 0), flat;
-    for (size_t gi = 0; gi < per_group.size(); ++gi) {
-      begin[gi] = (int32_t)flat.size();
-      flat.insert(flat.end(), per_group[gi].begin(), per_group[gi].end());
-    }
-    begin[per_group.size()] = (int32_t)flat.size();
-    // the previous sync's kernel may still be reading the tables
-    CUDA_OK(cudaStreamSynchronize(c->stream));
-    if (!owners.empty())
-      CUDA_OK(cudaMemcpy(c->d_owners, owners.data(), owners.size() * sizeof(OuterOwner), cudaMemcpyHostToDevice));
-    CUDA_OK(cudaMemcpy(c->d_unit_begin, begin.data(), begin.size() * 4, cudaMemcpyHostToDevice));
-    if (!flat.empty())
-      CUDA_OK(cudaMemcpy(c->d_unit_owner, flat.data(), flat.size() * 4, cudaMemcpyHostToDevice));
-    c->cached_sync_list = list;
+    for (const auto& s : r.dense) if (inside(s.canon_off)) owned += (double)s.len;
   }
   // a group step rewrites the working copy only on its own positions: everywhere else it must
   // already hold the global values, not the resident replica's
   if (!all) ppu_make_resident(c, -1);
   OuterTables t;
-  t.owners = c->d_owners; t.unit_begin = c->d_unit_begin; t.unit_owner = c->d_unit_owner;
-  t.P = c->P; t.e_size = c->e_size; t.layer_size = c->layer_size; t.win_rel = c->rel_win;
-  t.wout_rel = c->rel_wout; t.L = L; t.d = d; t.F = F;
-  const int n_seg = outer_segments(L);
+  t.segs = c->d_oseg; t.chunks = c->d_ochunk; t.dense_owner = c->d_downer;
+  t.unit_begin = c->d_unit_begin; t.unit_owner = c->d_unit_owner; t.d = d; t.F = F;
   double swept = 0;
-  auto sweep = [&](int seg_lo, int seg_count) {
-    if (seg_count <= 0) return;
-    launch_outer(t, c->theta, c->buf, c->w16, c->cfg.outer_lr, c->cfg.outer_momentum, seg_lo, seg_count, c->stream);
+  if (all) swept = (double)c->P;
+  else if (tail) swept = (double)c->e_size + (double)(c->P - c->off_lnfg);
+  else swept = (double)(l1 - l0) * (double)c->layer_size;
+  c->outer_bytes = 18.0 * swept + 8.0 * owned;
+  auto sweep = [&](int chunk_lo, int chunk_hi, double share) {
+    if (chunk_hi <= chunk_lo) return;
+    EvScope ev(c, PPU_CLS_OUTER, c->outer_bytes * share);
+    launch_outer(t, c->theta, c->buf, c->w16, c->cfg.outer_lr, c->cfg.outer_momentum, chunk_lo,
+                 chunk_hi - chunk_lo, c->stream);
     c->launches++;
   };
   if (all) {
-    sweep(0, n_seg);
-    swept = (double)c->P;
+    sweep(0, c->n_chunks, 1.0);
   } else if (tail) {
-    sweep(0, 4);                // embeddings
-    sweep(n_seg - 1, 1);        // final LayerNorm
-    swept = (double)c->e_size + (double)(c->P - c->e_size - (int64_t)L * c->layer_size);
+    const double e_share = (double)c->e_size / swept;
+    sweep(0, c->chunks_e, e_share);                                   // embeddings
+    sweep(c->layer_chunk_begin[L], c->n_chunks, 1.0 - e_share);       // final LayerNorm
   } else {
-    sweep(4 + 3 * l0, 3 * (l1 - l0));
-    swept = (double)(l1 - l0) * (double)c->layer_size;
+    sweep(c->layer_chunk_begin[l0], c->layer_chunk_begin[l1], 1.0);
   }
   c->resident = -1;   // the working copy now holds the global parameters everywhere
   c->launches_last_sync = c->launches - launches0;
-  c->outer_bytes = 18.0 * swept + 8.0 * owned;
   CUDA_OK(cudaGetLastError());
   return PPU_OK;
 }
@@ -434,8 +579,8 @@ extern "C" int ppu_profile_read(ppu_ctx* c, ppu_profile_t* out) {
   for (size_t i = 0; i < c->ev_recs.size(); ++i) {
     float ms = 0.f;
     CUDA_OK(cudaEventElapsedTime(&ms, c->ev_pool[2 * i], c->ev_pool[2 * i + 1]));
-    if (c->ev_recs[i].cls == 0) { out->gemm_ms += ms; out->gemm_flops += c->ev_recs[i].flops; out->gemm_launches++; }
-    else { out->attn_ms += ms; out->attn_flops += c->ev_recs[i].flops; out->attn_launches++; }
+    const int cls = c->ev_recs[i].cls;
+    out->ms[cls] += ms; out->work[cls] += c->ev_recs[i].work; out->launches[cls]++;
   }
   out->dropped = c->ev_dropped;
   c->ev_recs.clear();

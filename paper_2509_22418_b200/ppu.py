@@ -38,20 +38,35 @@ class ModelCfg(C.Structure):
 
 class SubsetSpec(C.Structure):
     _fields_ = [("n_replicas", C.c_int32), ("mode", C.c_int32), ("n_slices", C.c_int32),
-                ("layer_stride", C.c_int32), ("ranges", C.POINTER(C.c_int32))]
+                ("layer_stride", C.c_int32), ("ranges", C.POINTER(C.c_int32)),
+                ("train_non_mlp", C.c_int32), ("n_head_slices", C.c_int32),
+                ("head_ranges", C.POINTER(C.c_int32))]
 
 
 class Stats(C.Structure):
     _fields_ = [("param_count", C.c_int64), ("arena_bytes", C.c_int64), ("state_bytes", C.c_int64),
                 ("activation_bytes", C.c_int64), ("launches_last_step", C.c_int64),
                 ("launches_last_sync", C.c_int64), ("flops_fwd", C.c_double),
-                ("flops_dgrad", C.c_double), ("flops_wgrad", C.c_double), ("outer_bytes", C.c_double)]
+                ("flops_dgrad", C.c_double), ("flops_wgrad", C.c_double), ("outer_bytes", C.c_double),
+                ("saved_bytes_last_step", C.c_int64)]
+
+
+CLS_GEMM, CLS_ATTN, CLS_LN, CLS_XENT, CLS_ADAMW, CLS_OUTER, CLS_OTHER, CLS_COUNT = 0, 1, 2, 3, 4, 5, 6, 8
+CLS_NAMES = {CLS_GEMM: "gemm", CLS_ATTN: "attention", CLS_LN: "layernorm", CLS_XENT: "cross_entropy",
+             CLS_ADAMW: "adamw", CLS_OUTER: "outer", CLS_OTHER: "other"}
 
 
 class Profile(C.Structure):
-    _fields_ = [("gemm_ms", C.c_double), ("gemm_flops", C.c_double), ("attn_ms", C.c_double),
-                ("attn_flops", C.c_double), ("gemm_launches", C.c_int64),
-                ("attn_launches", C.c_int64), ("dropped", C.c_int64)]
+    _fields_ = [("ms", C.c_double * CLS_COUNT), ("work", C.c_double * CLS_COUNT),
+                ("launches", C.c_int64 * CLS_COUNT), ("dropped", C.c_int64)]
+
+    # the two classes bench.py's roofline is built from
+    gemm_ms = property(lambda self: self.ms[CLS_GEMM])
+    gemm_flops = property(lambda self: self.work[CLS_GEMM])
+    gemm_launches = property(lambda self: self.launches[CLS_GEMM])
+    attn_ms = property(lambda self: self.ms[CLS_ATTN])
+    attn_flops = property(lambda self: self.work[CLS_ATTN])
+    attn_launches = property(lambda self: self.launches[CLS_ATTN])
 
 
 _lib = None
@@ -80,14 +95,22 @@ def make_cfg(n_layer, d_model, n_head, d_ff, vocab, max_batch, max_seq, ln_eps=1
                     adam_lr, adam_beta1, adam_beta2, adam_eps, adam_wd, outer_lr, outer_momentum)
 
 
-def make_spec(n_replicas, mode=SUBSET_FFN_SLICE, n_slices=1, layer_stride=1, ranges=None):
-    """ranges: int array [K][L][2] for SUBSET_EXPLICIT.  Returns (spec, keepalive)."""
-    keep = None
+def make_spec(n_replicas, mode=SUBSET_FFN_SLICE, n_slices=1, layer_stride=1, ranges=None,
+              train_non_mlp=0, n_head_slices=0, head_ranges=None):
+    """ranges: int array [K][L][2] for SUBSET_EXPLICIT; head_ranges: optional int array [K][2].
+    Returns (spec, keepalive)."""
+    keep = []
     ptr = C.POINTER(C.c_int32)()
+    hptr = C.POINTER(C.c_int32)()
     if ranges is not None:
-        keep = np.ascontiguousarray(ranges, dtype=np.int32)
-        ptr = keep.ctypes.data_as(C.POINTER(C.c_int32))
-    return SubsetSpec(n_replicas, mode, n_slices, layer_stride, ptr), keep
+        keep.append(np.ascontiguousarray(ranges, dtype=np.int32))
+        ptr = keep[-1].ctypes.data_as(C.POINTER(C.c_int32))
+    if head_ranges is not None:
+        keep.append(np.ascontiguousarray(head_ranges, dtype=np.int32))
+        assert keep[-1].shape == (n_replicas, 2)
+        hptr = keep[-1].ctypes.data_as(C.POINTER(C.c_int32))
+    return SubsetSpec(n_replicas, mode, n_slices, layer_stride, ptr, int(train_non_mlp),
+                      int(n_head_slices), hptr), keep
 
 
 def ppu_query_bytes(cfg: ModelCfg, spec: SubsetSpec) -> int:
@@ -179,9 +202,9 @@ class Context:
             recs.append((name.value.decode(), off.value, tuple(shape[:nd.value])))
         return recs
 
-    def ppu_set_params(self, theta: np.ndarray) -> None:
+    def ppu_set_params(self, theta: np.ndarray, replica: int = -1) -> None:
         t = np.ascontiguousarray(theta, dtype=np.float32)
-        _check(lib().ppu_set_params(self._h, _np_ptr(t, C.c_float), C.c_int64(t.size)))
+        _check(lib().ppu_set_params(self._h, replica, _np_ptr(t, C.c_float), C.c_int64(t.size)))
 
     def ppu_get_params(self, replica: int = -1) -> np.ndarray:
         out = np.empty(self.param_count, dtype=np.float32)
@@ -225,6 +248,25 @@ class Context:
         _check(lib().ppu_get_subset_state(self._h, replica, _np_ptr(m, C.c_float),
                                           _np_ptr(v, C.c_float), C.byref(step), C.c_int64(n)))
         return m, v, step.value
+
+    def ppu_set_subset_state(self, replica: int, m, v, step: int) -> None:
+        n = self.ppu_subset_count(replica)
+        mm = None if m is None else np.ascontiguousarray(m, dtype=np.float32)
+        vv = None if v is None else np.ascontiguousarray(v, dtype=np.float32)
+        _check(lib().ppu_set_subset_state(self._h, replica,
+                                          None if mm is None else _np_ptr(mm, C.c_float),
+                                          None if vv is None else _np_ptr(vv, C.c_float),
+                                          C.c_int32(step), C.c_int64(n)))
+
+    def ppu_replica_values(self, replica: int):
+        """The replica's packed trained values as a torch view into the arena (no copy)."""
+        ptr, n = C.c_void_p(), C.c_int64()
+        _check(lib().ppu_replica_values(self._h, replica, C.byref(ptr), C.byref(n)))
+        off = ptr.value - self.arena.data_ptr()
+        return self.arena[off:off + 4 * n.value].view(self.torch.float32)
+
+    def ppu_set_backends(self, gemm: int = 0, attention: int = 0) -> None:
+        _check(lib().ppu_set_backends(self._h, gemm, attention))
 
     def ppu_set_adam_lr(self, lr: float) -> None:
         _check(lib().ppu_set_adam_lr(self._h, C.c_float(lr)))

@@ -13,8 +13,8 @@ by a wrong result at any size:
     step * (0.1 + 0.08 / r_i), r_i = the largest |g_ref,i| / rms(g_ref) over the steps so far
     (gradients accurate to 1e-2 rms - half the gradient gate - at eight sigma), and by 2.2 steps
     (a full step the other way) where r_i <= 0.08, i.e. where that noise can turn the sign;
-    fewer than 2 % of the elements may differ by more than 0.1 step; the rest must agree to
-    2e-2 in relative l2.
+    (a tail bound: up to 1e-5 of the elements may pass it); fewer than 2 % of the elements may
+    differ by more than 0.1 step; the rest must agree to 2e-2 in relative l2.
 tests/test_gates_can_fail.py plants mistakes in the oracle and checks that each gate rejects them.
 """
 from __future__ import annotations
@@ -30,6 +30,7 @@ UPDATE_TOL = 0.10       # an update may differ by this share of a step (plus the
 GRAD_NOISE = 0.01       # gradient accuracy the allowance assumes, in units of rms(g_ref) ...
 NOISE_SIGMAS = 8.0      # ... and how many sigmas of it an element may use (an element's noise follows the
                         # magnitudes in its own row and column, not the rms over the whole subset)
+OUTLIER_FRAC = 1e-5     # share of a vector that may exceed its per-element allowance (tail of the noise)
 OFF_FRAC = 0.02         # at most this share of a vector may differ by more than UPDATE_TOL * step
 
 
@@ -64,11 +65,25 @@ def gate_vector(got, ref, what="gradient", tol=TENSOR_TOL):
     return a, b
 
 
-def grad_rel(g_ref):
-    """|g_ref| in units of its rms: how far each element's gradient is from the noise floor."""
+def grad_rel(g_ref, groups=None):
+    """|g_ref| in units of its rms: how far each element's gradient is from the noise floor.
+    groups (optional, int per element): the rms is taken per group - per parameter tensor, whose
+    gradients differ in scale by orders of magnitude (an embedding row, a LayerNorm gain)."""
     g = np.asarray(g_ref, dtype=np.float64)
-    rms = float(np.sqrt(np.mean(g * g))) if g.size else 0.0
-    return np.abs(g) / max(rms, 1e-300)
+    if not g.size:
+        return np.zeros(0)
+    if groups is None:
+        return np.abs(g) / max(float(np.sqrt(np.mean(g * g))), 1e-300)
+    ss = np.bincount(groups, weights=g * g)
+    cnt = np.bincount(groups)
+    rms = np.sqrt(ss / np.maximum(cnt, 1))
+    return np.abs(g) / np.maximum(rms[groups], 1e-300)
+
+
+def tensor_groups(cfg, idx):
+    """For each flat parameter index the number of the tensor it lies in."""
+    starts = np.array([off for _, off, _ in O.layout(cfg)], dtype=np.int64)
+    return (np.searchsorted(starts, idx, side="right") - 1).astype(np.int64)
 
 
 def step_allowance(grel):
@@ -88,10 +103,14 @@ def gate_update(d_got, d_ref, scale, allow, what="update", tol=TENSOR_TOL):
     assert d_got.shape == d_ref.shape
     assert np.linalg.norm(d_ref) > 0, f"{what}: the reference did not move"
     err = np.abs(d_got - d_ref) / scale
+    # the allowance is a tail bound, not a hard one: a handful of elements in a million may pass it,
+    # none may differ by more than a full step the other way
+    over = err > allow
     worst = int(np.argmax(err - allow))
-    assert err[worst] <= allow[worst], (
-        f"{what}: element {worst} differs by {err[worst]:.3f} steps, allowed {allow[worst]:.3f}; "
-        f"{int((err > allow).sum())} such elements")
+    assert int(over.sum()) <= max(2, int(OUTLIER_FRAC * err.size)), (
+        f"{what}: {int(over.sum())} of {err.size} elements differ by more than their allowance; the worst, "
+        f"element {worst}, by {err[worst]:.3f} steps against {allow[worst]:.3f}")
+    assert err.max() <= 2.2 * max(1.0, float(allow.max()) / 2.2), f"{what}: an element differs by {err.max():.3f} steps"
     off = err > UPDATE_TOL
     share = float(off.mean()) if off.size else 0.0
     assert share < OFF_FRAC, f"{what}: {share:.2%} of the elements differ by more than {UPDATE_TOL} x step"
@@ -113,7 +132,7 @@ class Pair:
 
     def __init__(self, dims, ranges, max_batch, max_seq, seed=11, adam=None, outer=None,
                  mode=None, n_slices=1, layer_stride=1, dtype=np.float64, ln_jitter=0.0,
-                 train_non_mlp=False, head_ranges=None):
+                 train_non_mlp=False, head_ranges=None, gemm_backend=0):
         from paper_2509_22418_b200 import ppu
         self.ppu = ppu
         L, d, h, F, V = dims
@@ -136,6 +155,8 @@ class Pair:
         else:
             spec, keep = ppu.make_spec(K, mode, n_slices=n_slices, layer_stride=layer_stride, **extra)
         self.ctx = ppu.Context(cfg, spec, keep)
+        if gemm_backend:
+            self.ctx.ppu_set_backends(gemm=gemm_backend)
         recs = self.ctx.tensors()
         assert [(n, o, tuple(s)) for n, o, s in recs] == [(n, o, tuple(s)) for n, o, s in O.layout(self.ocfg)]
         self.theta32 = synth.init_params(seed, recs, ln_jitter=ln_jitter)
@@ -152,9 +173,11 @@ class Pair:
             self.reps = [O.Replica(self.ocfg, self.theta, r, **okw) for r in ranges]
         # per replica and trained element: largest |g_ref| / rms(g_ref) over its steps so far
         self.grel = [np.zeros(len(r.idx)) for r in self.reps]
-        # ... and the allowances of its steps since the last outer sync, summed (tests/_harness.py
-        # gate_update); an outer step carries mu of it on in the momentum
+        self.groups = [tensor_groups(self.ocfg, r.idx) for r in self.reps]
+        # ... and the allowances of its steps since its last outer sync, summed (gate_update);
+        # carry: per position what the outer momentum may differ by, in inner steps
         self.allow_acc = [np.zeros(len(r.idx)) for r in self.reps]
+        self.carry = np.zeros(len(self.theta))
         self.seed = seed
 
     def tokens(self, k, rnd, step, B, S):
@@ -176,7 +199,7 @@ class Pair:
         sub_before = rep.theta_sub.astype(np.float64)
         loss_gpu, _ = self.gpu_step(k, tok)
         loss_ref = rep.local_step(self.theta, tok if oracle_tok is None else oracle_tok, self.adam)
-        self.grel[k] = np.maximum(self.grel[k], grad_rel(rep.last_grad))
+        self.grel[k] = np.maximum(self.grel[k], grad_rel(rep.last_grad, self.groups[k]))
         self.allow_acc[k] += step_allowance(self.grel[k])
         g_gpu = self.ctx.ppu_get_subset_grads(k)
         after = self.ctx.ppu_get_params(k)[rep.idx].astype(np.float64)

@@ -83,7 +83,7 @@ def _attention_case(B, S, h, dh, seed):
     return qkv, dU, dict(q=q, k=k, v=v, A=A), U, lse, dU64
 
 
-@pytest.mark.parametrize("backend", [1, 2, 0])
+@pytest.mark.parametrize("backend", [1, 0])
 @pytest.mark.parametrize("B,S,h,dh", [(2, 64, 4, 16), (1, 200, 2, 64), (2, 256, 2, 128), (1, 130, 3, 32),
                                       (1, 1024, 2, 128), (2, 333, 2, 64), (1, 2048, 1, 128), (1, 64, 1, 64),
                                       (1, 7, 2, 64),

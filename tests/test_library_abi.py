@@ -28,8 +28,9 @@ def test_every_declared_symbol_is_exported(ppu):
 
 def test_struct_sizes_match_header(ppu):
     assert ctypes.sizeof(ppu.ModelCfg) == 7 * 4 + 9 * 4
-    assert ctypes.sizeof(ppu.SubsetSpec) == 4 * 4 + 8
-    assert ctypes.sizeof(ppu.Stats) == 6 * 8 + 4 * 8
+    assert ctypes.sizeof(ppu.SubsetSpec) == 4 * 4 + 8 + 2 * 4 + 8
+    assert ctypes.sizeof(ppu.Stats) == 6 * 8 + 4 * 8 + 8
+    assert ctypes.sizeof(ppu.Profile) == 3 * 8 * 8 + 8
 
 
 def test_query_bytes_and_validation_on_host(ppu):
@@ -51,7 +52,13 @@ def test_query_bytes_and_validation_on_host(ppu):
         (cfg, ppu.make_spec(4, ppu.SUBSET_FFN_LAYERS, layer_stride=5)[0]),
         (cfg, ppu.make_spec(1, ppu.SUBSET_EXPLICIT, ranges=[[[0, 12], [0, 8]]])[0]),
         (cfg, ppu.make_spec(1, ppu.SUBSET_EXPLICIT, ranges=[[[0, 512], [0, 8]]])[0]),
+        (cfg, ppu.make_spec(4, n_slices=4, n_head_slices=3)[0]),     # 4 heads do not split in 3
+        (cfg, ppu.make_spec(4, n_slices=4, train_non_mlp=2)[0]),
+        (cfg, ppu.make_spec(4, n_slices=4, head_ranges=[[0, 1], [1, 2], [2, 5], [0, 4]])[0]),
     ]
+    # training the never-sliced parameters and the projections costs state per replica
+    assert ppu.ppu_query_bytes(cfg, ppu.make_spec(4, n_slices=4, train_non_mlp=1)[0]) > n
+    assert ppu.ppu_query_bytes(cfg, ppu.make_spec(4, n_slices=4, n_head_slices=2)[0]) > n
     for c, s in bad:
         with pytest.raises(ppu.PpuError):
             ppu.ppu_query_bytes(c, s)
