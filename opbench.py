@@ -1,7 +1,11 @@
-"""Single-kernel timing driver: python -m paper_2509_22418_b200.opbench <op> [options]
+"""Single-kernel timing driver: python opbench.py <op> [options]
 
   gemm  --m M --n N --k K [--a-mn] [--b-mn] [--f32]   one GEMM through ppu_gemm
   attn  --batch B --seq S --heads H --dh D             attention forward + backward
+  path  --layers L [--batch B --seq S] [--replicas K]  local steps + one outer sync of a model with
+                                                       the 1.3B-class layer shape but only L layers
+                                                       (a few GB: the small case for profiler
+                                                       captures of the bandwidth-bound kernels)
 Times with CUDA events on the launching stream after warm-up; operands are sized by the caller
 (keep them above the 126 MB L2 if DRAM behaviour matters).  Also the target of profiler runs.
 """
@@ -10,12 +14,12 @@ import sys
 
 import torch
 
-from . import build, ppu
+from paper_2509_22418_b200 import build, ppu, synth
 
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["gemm", "attn"])
+    ap.add_argument("op", choices=["gemm", "attn", "path"])
     ap.add_argument("--m", type=int, default=8192)
     ap.add_argument("--n", type=int, default=8192)
     ap.add_argument("--k", type=int, default=2048)
@@ -28,6 +32,9 @@ def main():
     ap.add_argument("--dh", type=int, default=128)
     ap.add_argument("--backend", type=int, default=0, help="attention: 0 tcgen05, 1 SIMT, 2 mma.sync; gemm: 0 tcgen05 (shape chosen), 1 SIMT, "
                          "2 tcgen05 one CTA per tile, 3 tcgen05 SM pairs 256 x 256, 4 SM pairs 256 x 128")
+    ap.add_argument("--layers", type=int, default=4)
+    ap.add_argument("--replicas", type=int, default=4)
+    ap.add_argument("--train-non-mlp", action="store_true")
     ap.add_argument("--iters", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     a = ap.parse_args()
@@ -48,7 +55,31 @@ def main():
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) / a.iters
 
-    if a.op == "gemm":
+    if a.op == "path":
+        d, F, V = a.heads * a.dh, 4 * a.heads * a.dh, 32768
+        K = a.replicas
+        cfg = ppu.make_cfg(a.layers, d, a.heads, F, V, a.batch, a.seq, adam_lr=3e-4, adam_beta2=0.99)
+        spec, keep = ppu.make_spec(K, n_slices=K, train_non_mlp=int(a.train_non_mlp))
+        ctx = ppu.Context(cfg, spec, keep)
+        ctx.ppu_set_params(synth.init_params(0, ctx.tensors()))
+        toks = [torch.from_numpy(synth.tokens(0, k, 0, 0, a.batch, a.seq, V)).cuda() for k in range(K)]
+        ctx.ppu_profile_enable(True)
+        for it in range(a.warmup + a.iters):
+            if it == a.warmup:
+                ctx.ppu_profile_read()
+            for k in range(K):
+                ctx.ppu_local_step(k, toks[k])
+            ctx.ppu_outer_sync(list(range(K)))
+        prof = ctx.ppu_profile_read()
+        for cls, name in ppu.CLS_NAMES.items():
+            if prof.launches[cls]:
+                tensor = cls in (ppu.CLS_GEMM, ppu.CLS_ATTN)
+                rate = prof.work[cls] / (prof.ms[cls] * 1e-3) / (1e12 if tensor else 1e9)
+                print(f"{name:14s} {prof.launches[cls]:6d} launches {prof.ms[cls]:9.3f} ms  "
+                      f"{rate:9.1f} {'TFLOP/s' if tensor else 'GB/s'}")
+        print(f"arena {ctx.ppu_stats().arena_bytes / 2**30:.2f} GiB")
+        ctx.close()
+    elif a.op == "gemm":
         A = torch.randn((a.k, a.m) if a.a_mn else (a.m, a.k), generator=g).to(dev).bfloat16()
         B = torch.randn((a.k, a.n) if a.b_mn else (a.n, a.k), generator=g).to(dev).bfloat16()
         ms = timed(lambda: ppu.ppu_gemm(A, not a.a_mn, B, not a.b_mn, a.m, a.n, a.k, out_f32=a.f32,

@@ -132,7 +132,7 @@ class Pair:
 
     def __init__(self, dims, ranges, max_batch, max_seq, seed=11, adam=None, outer=None,
                  mode=None, n_slices=1, layer_stride=1, dtype=np.float64, ln_jitter=0.0,
-                 train_non_mlp=False, head_ranges=None, gemm_backend=0):
+                 train_non_mlp=False, head_ranges=None, gemm_backend=0, oracle_replicas=None):
         from paper_2509_22418_b200 import ppu
         self.ppu = ppu
         L, d, h, F, V = dims
@@ -166,17 +166,23 @@ class Pair:
         okw = {}
         if train_non_mlp:
             okw["train_non_mlp"] = True
-        if head_ranges is not None:
-            self.reps = [O.Replica(self.ocfg, self.theta, r, head_range=tuple(hr), **okw)
-                         for r, hr in zip(ranges, head_ranges)]
-        else:
-            self.reps = [O.Replica(self.ocfg, self.theta, r, **okw) for r in ranges]
+        # oracle_replicas: build the oracle's state only for these (the others are None) - at the
+        # largest shapes the oracle follows a sample of the replicas
+        want = set(range(K)) if oracle_replicas is None else set(oracle_replicas)
+        self.reps = []
+        for k, r in enumerate(ranges):
+            if k not in want:
+                self.reps.append(None)
+            elif head_ranges is not None:
+                self.reps.append(O.Replica(self.ocfg, self.theta, r, head_range=tuple(head_ranges[k]), **okw))
+            else:
+                self.reps.append(O.Replica(self.ocfg, self.theta, r, **okw))
         # per replica and trained element: largest |g_ref| / rms(g_ref) over its steps so far
-        self.grel = [np.zeros(len(r.idx)) for r in self.reps]
-        self.groups = [tensor_groups(self.ocfg, r.idx) for r in self.reps]
+        self.grel = [None if r is None else np.zeros(len(r.idx)) for r in self.reps]
+        self.groups = [None if r is None else tensor_groups(self.ocfg, r.idx) for r in self.reps]
         # ... and the allowances of its steps since its last outer sync, summed (gate_update);
         # carry: per position what the outer momentum may differ by, in inner steps
-        self.allow_acc = [np.zeros(len(r.idx)) for r in self.reps]
+        self.allow_acc = [None if r is None else np.zeros(len(r.idx)) for r in self.reps]
         self.carry = np.zeros(len(self.theta))
         self.seed = seed
 
@@ -190,15 +196,21 @@ class Pair:
         loss = self.ctx.ppu_loss(k)
         return loss, t
 
-    def step_and_gate(self, k, tok, oracle_tok=None, check=True):
+    def step_and_gate(self, k, tok, oracle_tok=None, check=True, oracle_grad=None):
         """One local step of replica k on both sides, every per-step gate applied.  oracle_tok:
-        the batch the oracle sees when it differs from the library's (a batch of identical
-        sequences has the loss and gradient of one of them).  Returns a record of the numbers."""
+        the batch the oracle sees when it differs from the library's (a batch made of copies of
+        a few sequences has the loss and gradient of those sequences).  oracle_grad = (loss, dense
+        full gradient) of the oracle for this batch at the replica's current parameters, when
+        several replicas share one full backward pass (the replica takes its own entries:
+        Algorithm 1 line 9).  Returns a record of the numbers."""
         rep = self.reps[k]
         before = self.ctx.ppu_get_params(k)[rep.idx].astype(np.float64)
         sub_before = rep.theta_sub.astype(np.float64)
         loss_gpu, _ = self.gpu_step(k, tok)
-        loss_ref = rep.local_step(self.theta, tok if oracle_tok is None else oracle_tok, self.adam)
+        if oracle_grad is not None:
+            loss_ref = rep.apply_gradient(oracle_grad[0], oracle_grad[1][rep.idx], self.adam)
+        else:
+            loss_ref = rep.local_step(self.theta, tok if oracle_tok is None else oracle_tok, self.adam)
         self.grel[k] = np.maximum(self.grel[k], grad_rel(rep.last_grad, self.groups[k]))
         self.allow_acc[k] += step_allowance(self.grel[k])
         g_gpu = self.ctx.ppu_get_subset_grads(k)
@@ -220,3 +232,107 @@ class Pair:
 
     def close(self):
         self.ctx.close()
+
+
+# ---- rounds and outer steps against the oracle ---------------------------------------------
+def run_round(P, B, S, H, rnd=0, order=None, check=True):
+    """H local steps on every replica; after every step the loss, the subset gradient, the AdamW
+    update and moments are gated against the oracle, and frozen parameters must keep their bits."""
+    K = P.K
+    report = []
+    theta0_gpu = P.ctx.ppu_get_params(-1)
+    order = order or [(k, h) for k in range(K) for h in range(H)]
+    for k, h in order:
+        tok = P.tokens(k, rnd, h, B, S)
+        rec = P.step_and_gate(k, tok, check=check)
+        rec["h"] = h
+        report.append(rec)
+        if check:
+            th_gpu = P.ctx.ppu_get_params(k)
+            idx = P.reps[k].idx
+            # frozen parameters: exactly the bits that were loaded
+            mask = np.ones(len(th_gpu), bool)
+            mask[idx] = False
+            assert np.array_equal(th_gpu[mask], theta0_gpu[mask])
+            # the trained positions moved (an update that rounds to nothing is a rare accident)
+            assert (th_gpu[idx] != theta0_gpu[idx]).mean() > 0.999
+    return report
+
+
+def gate_outer(P, replicas, th_before, th_gpu, buf_before, buf_gpu, th_ref_before, buf_ref_before, m,
+                mask=None):
+    """The outer step on the positions some listed replica trains: the change of the global
+    parameters and of the momentum against the oracle's, with the allowance of
+    tests/_harness.py for elements whose inner gradients are near the noise floor."""
+    tr = m > 0
+    if not tr.any():
+        return
+    mu = P.outer.momentum
+    allow = np.zeros(len(m))                # the most lenient owner decides
+    for k in replicas:
+        idx = P.reps[k].idx
+        allow[idx] = np.maximum(allow[idx], P.allow_acc[k])
+        synced = np.ones(len(idx), bool) if mask is None else mask[idx]
+        P.allow_acc[k][synced] = 0.0
+    # (relative l2 at twice the per-step tolerance: the outer change adds up the inner steps' errors)
+    # the momentum buffer carries earlier rounds' differences on: err(buf) <= mu err(buf_old) + err(Delta),
+    # err(theta step) <= lr_out ((1 + mu) err(Delta) + mu^2 err(buf_old))
+    allow_buf = allow + mu * P.carry
+    allow_th = allow + mu * mu / (1.0 + mu) * P.carry
+    P.carry = np.where(tr, allow_buf, P.carry)
+    scale = P.outer.lr * (1.0 + mu) * P.adam.lr
+    assert max_abs_over_norm(th_gpu[tr], P.theta[tr]) <= TENSOR_TOL
+    assert max_abs_over_norm(buf_gpu[tr], P.buf[tr]) <= TENSOR_TOL
+    gate_update(th_gpu[tr].astype(np.float64) - th_before[tr], P.theta[tr] - th_ref_before[tr], scale,
+                allow_th[tr], "outer step on theta", 2 * TENSOR_TOL)
+    gate_update(buf_gpu[tr].astype(np.float64) - buf_before[tr], P.buf[tr] - buf_ref_before[tr],
+                P.adam.lr, allow_buf[tr], "outer momentum", 2 * TENSOR_TOL)
+
+
+def check_outer(P, replicas):
+    theta_before = P.ctx.ppu_get_params(-1)
+    buf_before = P.ctx.ppu_get_outer_momentum()
+    P.ctx.ppu_outer_sync(replicas)
+    P.ctx.ppu_sync()
+    th_gpu = P.ctx.ppu_get_params(-1)
+    buf_gpu = P.ctx.ppu_get_outer_momentum()
+    th_ref_before, buf_ref_before = P.theta, P.buf
+    P.theta, P.buf, m = O.outer_sync(P.theta, P.buf, [P.reps[k] for k in replicas], P.outer)
+    assert np.array_equal(th_gpu[m == 0], theta_before[m == 0])       # untouched bits
+    assert np.array_equal(buf_gpu[m == 0], buf_before[m == 0])
+    gate_outer(P, replicas, theta_before, th_gpu, buf_before, buf_gpu, th_ref_before, buf_ref_before, m)
+    # working copy is the bf16 rounding of the new parameters; replicas restart from them
+    assert np.array_equal(P.ctx.ppu_get_working_bf16(), bf16_bits(th_gpu))
+    for k in replicas:
+        assert np.array_equal(P.ctx.ppu_get_params(k), th_gpu)
+    return th_gpu
+
+
+def check_outer_group(P, replicas, group, n_groups):
+    """One streaming-sync step on a group of layers against the oracle's masked outer step."""
+    theta_before = P.ctx.ppu_get_params(-1)
+    buf_before = P.ctx.ppu_get_outer_momentum()
+    local_before = {k: P.ctx.ppu_get_params(k) for k in replicas}
+    P.ctx.ppu_outer_sync_group(replicas, group, n_groups)
+    P.ctx.ppu_sync()
+    th_gpu = P.ctx.ppu_get_params(-1)
+    buf_gpu = P.ctx.ppu_get_outer_momentum()
+    mask = O.sync_group_mask(P.ocfg, group, n_groups)
+    th_ref_before, buf_ref_before = P.theta, P.buf
+    P.theta, P.buf, m = O.outer_sync(P.theta, P.buf, [P.reps[k] for k in replicas], P.outer, mask=mask)
+    # outside the group, and where no listed replica trains: the same bits as before
+    still = ~mask | (m == 0)
+    assert np.array_equal(th_gpu[still], theta_before[still])
+    assert np.array_equal(buf_gpu[still], buf_before[still])
+    gate_outer(P, replicas, theta_before, th_gpu, buf_before, buf_gpu, th_ref_before, buf_ref_before, m, mask)
+    assert np.array_equal(P.ctx.ppu_get_working_bf16(), bf16_bits(th_gpu))
+    for k in replicas:
+        now = P.ctx.ppu_get_params(k)
+        idx = P.reps[k].idx
+        inside = np.zeros(len(now), bool)
+        inside[idx] = mask[idx]
+        assert np.array_equal(now[inside], th_gpu[inside])                     # restarted in the group
+        assert np.array_equal(now[~inside], np.where(mask, th_gpu, local_before[k])[~inside])   # kept elsewhere
+        assert max_abs_over_norm(now[idx], P.reps[k].theta_sub) <= TENSOR_TOL
+
+

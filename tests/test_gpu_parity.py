@@ -12,83 +12,10 @@ import numpy as np
 import pytest
 
 from oracle import ppu_oracle as O
-from tests._harness import (LOSS_RTOL, TENSOR_TOL, Pair, bf16_bits, gate_update, gate_vector,
-                            max_abs_over_norm, rel_l2)
+from tests._harness import (LOSS_RTOL, TENSOR_TOL, Pair, bf16_bits, check_outer, check_outer_group,
+                            gate_update, gate_vector, max_abs_over_norm, rel_l2, run_round)
 
 pytestmark = pytest.mark.gpu
-
-
-def _run_round(P: Pair, B, S, H, rnd=0, order=None, check=True):
-    """H local steps on every replica; after every step the loss, the subset gradient, the AdamW
-    update and moments are gated against the oracle, and frozen parameters must keep their bits."""
-    K = P.K
-    report = []
-    theta0_gpu = P.ctx.ppu_get_params(-1)
-    order = order or [(k, h) for k in range(K) for h in range(H)]
-    for k, h in order:
-        tok = P.tokens(k, rnd, h, B, S)
-        rec = P.step_and_gate(k, tok, check=check)
-        rec["h"] = h
-        report.append(rec)
-        if check:
-            th_gpu = P.ctx.ppu_get_params(k)
-            idx = P.reps[k].idx
-            # frozen parameters: exactly the bits that were loaded
-            mask = np.ones(len(th_gpu), bool)
-            mask[idx] = False
-            assert np.array_equal(th_gpu[mask], theta0_gpu[mask])
-            # the trained positions moved (an update that rounds to nothing is a rare accident)
-            assert (th_gpu[idx] != theta0_gpu[idx]).mean() > 0.999
-    return report
-
-
-def _gate_outer(P: Pair, replicas, th_before, th_gpu, buf_before, buf_gpu, th_ref_before, buf_ref_before, m,
-                mask=None):
-    """The outer step on the positions some listed replica trains: the change of the global
-    parameters and of the momentum against the oracle's, with the allowance of
-    tests/_harness.py for elements whose inner gradients are near the noise floor."""
-    tr = m > 0
-    if not tr.any():
-        return
-    mu = P.outer.momentum
-    allow = np.zeros(len(m))                # the most lenient owner decides
-    for k in replicas:
-        idx = P.reps[k].idx
-        allow[idx] = np.maximum(allow[idx], P.allow_acc[k])
-        synced = np.ones(len(idx), bool) if mask is None else mask[idx]
-        P.allow_acc[k][synced] = 0.0
-    # (relative l2 at twice the per-step tolerance: the outer change adds up the inner steps' errors)
-    # the momentum buffer carries earlier rounds' differences on: err(buf) <= mu err(buf_old) + err(Delta),
-    # err(theta step) <= lr_out ((1 + mu) err(Delta) + mu^2 err(buf_old))
-    allow_buf = allow + mu * P.carry
-    allow_th = allow + mu * mu / (1.0 + mu) * P.carry
-    P.carry = np.where(tr, allow_buf, P.carry)
-    scale = P.outer.lr * (1.0 + mu) * P.adam.lr
-    assert max_abs_over_norm(th_gpu[tr], P.theta[tr]) <= TENSOR_TOL
-    assert max_abs_over_norm(buf_gpu[tr], P.buf[tr]) <= TENSOR_TOL
-    gate_update(th_gpu[tr].astype(np.float64) - th_before[tr], P.theta[tr] - th_ref_before[tr], scale,
-                allow_th[tr], "outer step on theta", 2 * TENSOR_TOL)
-    gate_update(buf_gpu[tr].astype(np.float64) - buf_before[tr], P.buf[tr] - buf_ref_before[tr],
-                P.adam.lr, allow_buf[tr], "outer momentum", 2 * TENSOR_TOL)
-
-
-def _check_outer(P: Pair, replicas):
-    theta_before = P.ctx.ppu_get_params(-1)
-    buf_before = P.ctx.ppu_get_outer_momentum()
-    P.ctx.ppu_outer_sync(replicas)
-    P.ctx.ppu_sync()
-    th_gpu = P.ctx.ppu_get_params(-1)
-    buf_gpu = P.ctx.ppu_get_outer_momentum()
-    th_ref_before, buf_ref_before = P.theta, P.buf
-    P.theta, P.buf, m = O.outer_sync(P.theta, P.buf, [P.reps[k] for k in replicas], P.outer)
-    assert np.array_equal(th_gpu[m == 0], theta_before[m == 0])       # untouched bits
-    assert np.array_equal(buf_gpu[m == 0], buf_before[m == 0])
-    _gate_outer(P, replicas, theta_before, th_gpu, buf_before, buf_gpu, th_ref_before, buf_ref_before, m)
-    # working copy is the bf16 rounding of the new parameters; replicas restart from them
-    assert np.array_equal(P.ctx.ppu_get_working_bf16(), bf16_bits(th_gpu))
-    for k in replicas:
-        assert np.array_equal(P.ctx.ppu_get_params(k), th_gpu)
-    return th_gpu
 
 
 @pytest.mark.parametrize("gemm", [0, 1], ids=["tc", "simt"])
@@ -102,12 +29,12 @@ def test_tiny_config_full_protocol(gemm):
     try:
         for k in range(4):      # the trained index set is exact
             assert np.array_equal(P.ctx.ppu_subset_index(k), P.reps[k].idx)
-        rep = _run_round(P, 4, 64, 3)
+        rep = run_round(P, 4, 64, 3)
         print("\n".join(str(r) for r in rep))
-        _check_outer(P, [0, 1, 2, 3])
+        check_outer(P, [0, 1, 2, 3])
         # second round continues from the merged parameters with the kept AdamW state
-        rep = _run_round(P, 4, 64, 1, rnd=1)
-        _check_outer(P, [0, 1, 2, 3])
+        rep = run_round(P, 4, 64, 1, rnd=1)
+        check_outer(P, [0, 1, 2, 3])
     finally:
         P.close()
 
@@ -129,15 +56,15 @@ def test_ragged_model_mixed_subsets(gemm):
         for k in range(4):
             assert np.array_equal(P.ctx.ppu_subset_index(k), P.reps[k].idx)
         order = [(k, h) for h in range(2) for k in range(4)]     # interleaved replicas
-        rep = _run_round(P, 3, 80, 2, order=order)
+        rep = run_round(P, 3, 80, 2, order=order)
         print("\n".join(str(r) for r in rep))
-        _check_outer(P, [0, 1, 3])          # replica 2 sits this round out
+        check_outer(P, [0, 1, 3])          # replica 2 sits this round out
         # replica 2 was not listed: it keeps its own values of its subset
         th2 = P.ctx.ppu_get_params(2)
         assert max_abs_over_norm(th2[P.reps[2].idx], P.reps[2].theta_sub) <= TENSOR_TOL
         # shorter batch than the maximum, then everyone joins
-        _run_round(P, 2, 48, 1, rnd=1)
-        _check_outer(P, [0, 1, 2, 3])
+        run_round(P, 2, 48, 1, rnd=1)
+        check_outer(P, [0, 1, 2, 3])
     finally:
         P.close()
 
@@ -148,8 +75,8 @@ def test_wide_rows_use_the_register_layernorm():
         ranges = [O.slice_ranges(O.Model(*dims), 2, k) for k in range(2)]
         P = Pair(dims, ranges, B, S, seed=6)
         try:
-            _run_round(P, B, S, 2)
-            _check_outer(P, [0, 1])
+            run_round(P, B, S, 2)
+            check_outer(P, [0, 1])
         finally:
             P.close()
 
@@ -163,7 +90,7 @@ def test_run_to_run_and_interleaving_determinism():
                   [(k, h) for h in range(2) for k in (3, 1, 0, 2)]):
         P = Pair(dims, ranges, 4, 64, seed=3)
         try:
-            _run_round(P, 4, 64, 2, order=order, check=False)
+            run_round(P, 4, 64, 2, order=order, check=False)
             P.ctx.ppu_outer_sync([0, 1, 2, 3])
             outs.append((P.ctx.ppu_get_params(-1), P.ctx.ppu_get_outer_momentum()))
         finally:
@@ -181,7 +108,7 @@ def test_whole_layer_subsets_and_eval_loss():
     try:
         for k in range(2):
             assert np.array_equal(P.ctx.ppu_subset_index(k), P.reps[k].idx)
-        _run_round(P, 2, 32, 2)
+        run_round(P, 2, 32, 2)
         tok = P.tokens(0, 9, 9, 2, 32)
         t = torch.from_numpy(tok).cuda()
         for k in (-1, 0, 1):
@@ -189,7 +116,7 @@ def test_whole_layer_subsets_and_eval_loss():
             ref, _ = O.forward(P.ocfg, th, tok, keep=False)
             got = P.ctx.ppu_eval_loss(k, t)
             assert abs(got - ref) <= LOSS_RTOL * ref
-        _check_outer(P, [0, 1])
+        check_outer(P, [0, 1])
     finally:
         P.close()
 
@@ -248,34 +175,6 @@ def test_host_entry_point_and_argument_errors():
         ppu.ppu_query_bytes(cfg, spec)
 
 
-def _check_outer_group(P: Pair, replicas, group, n_groups):
-    """One streaming-sync step on a group of layers against the oracle's masked outer step."""
-    theta_before = P.ctx.ppu_get_params(-1)
-    buf_before = P.ctx.ppu_get_outer_momentum()
-    local_before = {k: P.ctx.ppu_get_params(k) for k in replicas}
-    P.ctx.ppu_outer_sync_group(replicas, group, n_groups)
-    P.ctx.ppu_sync()
-    th_gpu = P.ctx.ppu_get_params(-1)
-    buf_gpu = P.ctx.ppu_get_outer_momentum()
-    mask = O.sync_group_mask(P.ocfg, group, n_groups)
-    th_ref_before, buf_ref_before = P.theta, P.buf
-    P.theta, P.buf, m = O.outer_sync(P.theta, P.buf, [P.reps[k] for k in replicas], P.outer, mask=mask)
-    # outside the group, and where no listed replica trains: the same bits as before
-    still = ~mask | (m == 0)
-    assert np.array_equal(th_gpu[still], theta_before[still])
-    assert np.array_equal(buf_gpu[still], buf_before[still])
-    _gate_outer(P, replicas, theta_before, th_gpu, buf_before, buf_gpu, th_ref_before, buf_ref_before, m, mask)
-    assert np.array_equal(P.ctx.ppu_get_working_bf16(), bf16_bits(th_gpu))
-    for k in replicas:
-        now = P.ctx.ppu_get_params(k)
-        idx = P.reps[k].idx
-        inside = np.zeros(len(now), bool)
-        inside[idx] = mask[idx]
-        assert np.array_equal(now[inside], th_gpu[inside])                     # restarted in the group
-        assert np.array_equal(now[~inside], np.where(mask, th_gpu, local_before[k])[~inside])   # kept elsewhere
-        assert max_abs_over_norm(now[idx], P.reps[k].theta_sub) <= TENSOR_TOL
-
-
 def test_streaming_sync_by_layer_groups():
     """Appendix "Streaming Synchronization": the outer step taken on one group of layers at a time,
     with local steps in between; a group that no replica trains (embeddings, final norm) moves
@@ -288,12 +187,12 @@ def test_streaming_sync_by_layer_groups():
         order = [(k, h) for k in range(4) for h in range(2)]
         for k, h in order:
             P.step_and_gate(k, P.tokens(k, 0, h, 4, 64))
-        _check_outer_group(P, [0, 1, 2, 3], 0, 2)          # layers 0-1
+        check_outer_group(P, [0, 1, 2, 3], 0, 2)          # layers 0-1
         for k in range(4):                                  # replicas go on from mixed parameters
             P.step_and_gate(k, P.tokens(k, 1, 0, 4, 64))
-        _check_outer_group(P, [0, 1, 3], 1, 2)              # layers 2-3, replica 2 sits out
-        _check_outer_group(P, [0, 1, 2, 3], 2, 2)           # embeddings + final norm: nothing trained
-        _check_outer_group(P, [0, 1, 2, 3], 0, 4)           # a finer grouping: layer 0 alone
+        check_outer_group(P, [0, 1, 3], 1, 2)              # layers 2-3, replica 2 sits out
+        check_outer_group(P, [0, 1, 2, 3], 2, 2)           # embeddings + final norm: nothing trained
+        check_outer_group(P, [0, 1, 2, 3], 0, 4)           # a finer grouping: layer 0 alone
         with pytest.raises(P.ppu.PpuError):
             P.ctx.ppu_outer_sync_group([0], 0, 3)           # 4 layers do not split into 3 groups
         with pytest.raises(P.ppu.PpuError):
@@ -312,9 +211,9 @@ def test_layernorm_gains_and_shifts_away_from_their_initial_values():
         try:
             g = P.theta32[[o for n, o, s in P.ctx.tensors() if n.endswith("ln1_g")][0]:][:8]
             assert np.abs(g - 1).max() > 0.05          # the inputs really are perturbed
-            rep = _run_round(P, B, S, 2)
+            rep = run_round(P, B, S, 2)
             print("\n".join(str(r) for r in rep))
-            _check_outer(P, [0, 1])
+            check_outer(P, [0, 1])
         finally:
             P.close()
 
@@ -340,7 +239,7 @@ def test_adamw_arithmetic_with_visible_epsilon_and_decay():
                 assert 0.05 < np.median(np.abs(rep.last_grad)) / P.adam.eps < 20
                 gate_vector(after - before, rep.theta_sub - sub_before, "AdamW update, all elements")
                 print(rec)
-        _check_outer(P, [0, 2])
+        check_outer(P, [0, 2])
     finally:
         P.close()
 
@@ -362,7 +261,7 @@ def _paper_scheme_round(dims, B, S, K, N, head_slices, seed, H=2, explicit_heads
     try:
         for k in range(K):      # the trained index set, in the packed order, is exact
             assert np.array_equal(P.ctx.ppu_subset_index(k), P.reps[k].idx)
-        rep = _run_round(P, B, S, H)
+        rep = run_round(P, B, S, H)
         print("\n".join(str(r) for r in rep))
         import torch
         tok = P.tokens(0, 9, 9, B, S)
@@ -371,9 +270,9 @@ def _paper_scheme_round(dims, B, S, K, N, head_slices, seed, H=2, explicit_heads
             ref, _ = O.forward(P.ocfg, th, tok, keep=False)
             got = P.ctx.ppu_eval_loss(k, torch.from_numpy(tok).cuda())
             assert abs(got - ref) <= LOSS_RTOL * ref
-        _check_outer(P, list(range(K)))
-        _run_round(P, B, S, 1, rnd=1)
-        _check_outer(P, list(range(K - 1)))            # one replica sits the second sync out
+        check_outer(P, list(range(K)))
+        run_round(P, B, S, 1, rnd=1)
+        check_outer(P, list(range(K - 1)))            # one replica sits the second sync out
         return P.ocfg
     finally:
         P.close()
@@ -408,8 +307,8 @@ def test_head_slices_with_everything_else_frozen():
     try:
         for k in range(3):
             assert np.array_equal(P.ctx.ppu_subset_index(k), P.reps[k].idx)
-        _run_round(P, 2, 96, 2)
-        _check_outer(P, [0, 1, 2])
+        run_round(P, 2, 96, 2)
+        check_outer(P, [0, 1, 2])
     finally:
         P.close()
 
