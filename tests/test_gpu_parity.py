@@ -366,3 +366,49 @@ def test_checkpoint_save_destroy_restore_continues_bit_exactly():
         assert np.array_equal(x, y)
     for x, y in zip(want[2:], got[2:]):
         assert np.array_equal(x, y)
+
+
+def test_exchange_step_two_emulated_gpus_equal_one_gpu_bit_for_bit():
+    """Algorithm 1 line 14 across GPUs: replica k is stepped by GPU k mod 2, the owners' end values
+    are copied into the other GPU's buffers, and both run the same outer step.  Two contexts on
+    this one GPU play the two GPUs, one after the other; their global parameters, momentum and
+    working copy must equal, bit for bit, those of one context that stepped all four replicas.
+    (The collective itself is covered by the two-rank CPU test of the exchange.)"""
+    from paper_2509_22418_b200 import dist as pd, ppu, synth
+    import torch
+    dims, B, S, K = (2, 64, 4, 256, 512), 4, 64, 4
+
+    def build():
+        spec, keep = ppu.make_spec(K, n_slices=2, train_non_mlp=1, n_head_slices=2)   # m = 2 and m = 4 positions
+        c = ppu.Context(ppu.make_cfg(*dims, B, S), spec, keep)
+        c.ppu_set_params(synth.init_params(5, c.tensors(), ln_jitter=0.1))
+        return c
+
+    def tok(k, rnd, h):
+        return torch.from_numpy(synth.tokens(5, k, rnd, h, B, S, dims[4])).cuda()
+
+    one, two = build(), [build(), build()]
+    try:
+        for rnd in range(2):
+            for k in range(K):
+                for h in range(2):
+                    one.ppu_local_step(k, tok(k, rnd, h))
+                    two[pd.owner_rank(k, 2)].ppu_local_step(k, tok(k, rnd, h))
+            one.ppu_outer_sync(list(range(K)))
+            for c in two:
+                c.ppu_sync()
+            pd.exchange_between_contexts(two, K)
+            for c in two:
+                c.ppu_outer_sync(list(range(K)))
+            want = (one.ppu_get_params(-1), one.ppu_get_outer_momentum(), one.ppu_get_working_bf16())
+            assert (want[0] != synth.init_params(5, one.tensors(), ln_jitter=0.1)).mean() > 0.9
+            for c in two:
+                got = (c.ppu_get_params(-1), c.ppu_get_outer_momentum(), c.ppu_get_working_bf16())
+                for x, y in zip(want, got):
+                    assert np.array_equal(x, y)
+                for k in range(K):
+                    assert np.array_equal(c.ppu_get_params(k), want[0])
+    finally:
+        one.close()
+        for c in two:
+            c.close()
