@@ -179,5 +179,5 @@ struct OuterTables {
   int32_t d, F;
 };
 // sweeps chunks [chunk_lo, chunk_lo + n_chunks)
-void launch_outer(const OuterTables& t, float* theta, float* buf, bf16* w16, float lr, float mu,
+void launch_outer(const OuterTables& t, int kind, float* theta, float* buf, bf16* w16, float lr, float mu,
                   int chunk_lo, int n_chunks, cudaStream_t st);

@@ -226,15 +226,16 @@ __device__ __forceinline__ void outer_chunk(const OuterTables& t, const OuterSeg
   }
 }
 
-__global__ void __launch_bounds__(OUTER_THREADS)
-outer_kernel(OuterTables t, float* __restrict__ theta, float* __restrict__ buf,
-             bf16* __restrict__ w16, float lr, float mu, int chunk_lo, int n_chunks) {
+// One kernel per segment kind (no kind branches inside, three resident blocks per SM); each walks
+// its own chunk list.
+template <int KIND>
+__global__ void __launch_bounds__(OUTER_THREADS, 3)
+outer_kernel(OuterTables t, const OuterChunk* __restrict__ chunks, float* __restrict__ theta,
+             float* __restrict__ buf, bf16* __restrict__ w16, float lr, float mu, int n_chunks) {
   for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
-    const OuterChunk ch = t.chunks[chunk_lo + c];
+    const OuterChunk ch = chunks[c];
     const OuterSeg sg = t.segs[ch.seg];
-    if (sg.kind == 0) outer_chunk<0>(t, sg, ch.off, theta, buf, w16, lr, mu);
-    else if (sg.kind == 1) outer_chunk<1>(t, sg, ch.off, theta, buf, w16, lr, mu);
-    else outer_chunk<2>(t, sg, ch.off, theta, buf, w16, lr, mu);
+    outer_chunk<KIND>(t, sg, ch.off, theta, buf, w16, lr, mu);
   }
 }
 
@@ -296,11 +297,14 @@ void launch_dense_move(const DenseSeg* segs, int n_seg, float* packed, const flo
   dense_move_kernel<<<seg_grid(n_total, n_seg), 256, 0, st>>>(segs, packed, theta, w16, mode);
 }
 
-void launch_outer(const OuterTables& t, float* theta, float* buf, bf16* w16, float lr, float mu,
+void launch_outer(const OuterTables& t, int kind, float* theta, float* buf, bf16* w16, float lr, float mu,
                   int chunk_lo, int n_chunks, cudaStream_t st) {
   if (n_chunks <= 0) return;
   // three resident blocks per SM; a chunk gives every thread 16 float4 per array
   int grid = ppu_sm_count() * 3;
   if (grid > n_chunks) grid = n_chunks;
-  outer_kernel<<<grid, OUTER_THREADS, 0, st>>>(t, theta, buf, w16, lr, mu, chunk_lo, n_chunks);
+  const OuterChunk* ch = t.chunks + chunk_lo;
+  if (kind == 0) outer_kernel<0><<<grid, OUTER_THREADS, 0, st>>>(t, ch, theta, buf, w16, lr, mu, n_chunks);
+  else if (kind == 1) outer_kernel<1><<<grid, OUTER_THREADS, 0, st>>>(t, ch, theta, buf, w16, lr, mu, n_chunks);
+  else outer_kernel<2><<<grid, OUTER_THREADS, 0, st>>>(t, ch, theta, buf, w16, lr, mu, n_chunks);
 }

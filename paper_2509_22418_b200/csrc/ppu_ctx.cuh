@@ -89,8 +89,11 @@ struct ppu_ctx {
   int32_t* d_unit_begin = nullptr; OuterOwner* d_unit_owner = nullptr;
   size_t cap_oseg = 0, cap_ochunk = 0, cap_downer = 0, cap_uowner = 0;
   std::vector<OuterSeg> h_oseg;
-  std::vector<int> layer_chunk_begin;          // chunk index where layer l's segments begin; [L] = final norm
-  int n_chunks = 0, chunks_e = 0;              // total; chunks of E come first
+  // per segment kind: where its chunk list starts in the device array, and inside that list the
+  // index where layer l's chunks begin ([L]: final norm, [L + 1]: end; E's chunks precede layer 0)
+  int kind_chunk_base[3] = {0, 0, 0};
+  std::vector<int> layer_chunk_begin[3];
+  int n_chunks = 0;
   std::vector<int32_t> cached_sync_list;
   // per-class event timing
   bool profiling = false;

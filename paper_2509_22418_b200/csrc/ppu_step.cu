@@ -439,17 +439,21 @@ int build_outer_tables(ppu_ctx* c, const std::vector<int32_t>& list) {
   layer_seg_begin[L] = (int)segs.size();
   add_dense(c->off_lnfg, c->P, -1);
   layer_seg_begin[L + 1] = (int)segs.size();
-  // chunk list; chunk index where every layer begins
+  // chunk lists, one per segment kind (each kind has its own kernel), all in canonical order; for
+  // every kind the index where each layer's chunks begin ([L]: the final norm, [L + 1]: the end)
   std::vector<OuterChunk> chunks;
-  std::vector<int> seg_chunk_begin(segs.size() + 1, 0);
-  for (size_t i = 0; i < segs.size(); ++i) {
-    seg_chunk_begin[i] = (int)chunks.size();
-    for (int64_t off = 0; off < segs[i].len; off += OUTER_CHUNK) chunks.push_back({(int32_t)i, 0, off});
+  for (int kind = 0; kind < 3; ++kind) {
+    c->kind_chunk_base[kind] = (int)chunks.size();
+    c->layer_chunk_begin[kind].assign(L + 2, 0);
+    int l_next = 0;
+    for (size_t i = 0; i < segs.size(); ++i) {
+      while (l_next <= L + 1 && (int)i >= layer_seg_begin[l_next])
+        c->layer_chunk_begin[kind][l_next++] = (int)chunks.size() - c->kind_chunk_base[kind];
+      if (segs[i].kind != kind) continue;
+      for (int64_t off = 0; off < segs[i].len; off += OUTER_CHUNK) chunks.push_back({(int32_t)i, 0, off});
+    }
+    while (l_next <= L + 1) c->layer_chunk_begin[kind][l_next++] = (int)chunks.size() - c->kind_chunk_base[kind];
   }
-  seg_chunk_begin[segs.size()] = (int)chunks.size();
-  c->layer_chunk_begin.assign(L + 2, 0);
-  for (int l = 0; l <= L + 1; ++l) c->layer_chunk_begin[l] = seg_chunk_begin[layer_seg_begin[l]];
-  c->chunks_e = c->layer_chunk_begin[0];
   c->n_chunks = (int)chunks.size();
   // owners of every group of 8 hidden units, in the order the replicas were listed
   std::vector<std::vector<OuterOwner>> per_group((size_t)L * (F / 8));
@@ -534,21 +538,34 @@ int outer_sync_impl(ppu_ctx* c, const int32_t* replicas, int n, int group, int n
   else if (tail) swept = (double)c->e_size + (double)(c->P - c->off_lnfg);
   else swept = (double)(l1 - l0) * (double)c->layer_size;
   c->outer_bytes = 18.0 * swept + 8.0 * owned;
-  auto sweep = [&](int chunk_lo, int chunk_hi, double share) {
-    if (chunk_hi <= chunk_lo) return;
-    EvScope ev(c, PPU_CLS_OUTER, c->outer_bytes * share);
-    launch_outer(t, c->theta, c->buf, c->w16, c->cfg.outer_lr, c->cfg.outer_momentum, chunk_lo,
-                 chunk_hi - chunk_lo, c->stream);
-    c->launches++;
-  };
-  if (all) {
-    sweep(0, c->n_chunks, 1.0);
-  } else if (tail) {
-    const double e_share = (double)c->e_size / swept;
-    sweep(0, c->chunks_e, e_share);                                   // embeddings
-    sweep(c->layer_chunk_begin[L], c->n_chunks, 1.0 - e_share);       // final LayerNorm
-  } else {
-    sweep(c->layer_chunk_begin[l0], c->layer_chunk_begin[l1], 1.0);
+  {
+    EvScope ev(c, PPU_CLS_OUTER, c->outer_bytes);     // brackets all launches of this sync
+    if (all) {
+      // E's chunks precede layer 0 in the kind-0 list: index 0 is the start of E
+      for (int kind = 0; kind < 3; ++kind) {
+        const int n = (kind < 2 ? c->kind_chunk_base[kind + 1] : c->n_chunks) - c->kind_chunk_base[kind];
+        if (n <= 0) continue;
+        launch_outer(t, kind, c->theta, c->buf, c->w16, c->cfg.outer_lr, c->cfg.outer_momentum,
+                     c->kind_chunk_base[kind], n, c->stream);
+        c->launches++;
+      }
+    } else if (tail) {
+      // embeddings (the kind-0 chunks before layer 0) and the final LayerNorm
+      launch_outer(t, 0, c->theta, c->buf, c->w16, c->cfg.outer_lr, c->cfg.outer_momentum,
+                   c->kind_chunk_base[0], c->layer_chunk_begin[0][0], c->stream);
+      launch_outer(t, 0, c->theta, c->buf, c->w16, c->cfg.outer_lr, c->cfg.outer_momentum,
+                   c->kind_chunk_base[0] + c->layer_chunk_begin[0][L],
+                   c->layer_chunk_begin[0][L + 1] - c->layer_chunk_begin[0][L], c->stream);
+      c->launches += 2;
+    } else {
+      for (int kind = 0; kind < 3; ++kind) {
+        const int lo = c->layer_chunk_begin[kind][l0], hi = c->layer_chunk_begin[kind][l1];
+        if (hi <= lo) continue;
+        launch_outer(t, kind, c->theta, c->buf, c->w16, c->cfg.outer_lr, c->cfg.outer_momentum,
+                     c->kind_chunk_base[kind] + lo, hi - lo, c->stream);
+        c->launches++;
+      }
+    }
   }
   c->resident = -1;   // the working copy now holds the global parameters everywhere
   c->launches_last_sync = c->launches - launches0;

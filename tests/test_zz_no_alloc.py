@@ -51,3 +51,23 @@ def test_static_scratch_rejects_sizes_beyond_its_limit():
                                             C.c_void_p(qkv.data_ptr()), too_many, 64, 1, 64, 0,
                                             C.c_void_p(st))
     assert rc == -2 and b"exceeds" in ppu.lib().ppu_last_error()
+
+
+def test_static_scratch_against_the_oracle():
+    """The same entry point against the CPU oracle's attention backward (Appendix C.1, MHA), so
+    that this file stands on its own."""
+    import torch
+    from oracle import ppu_oracle as O
+    from paper_2509_22418_b200 import ppu
+    from tests.test_gpu_ops import _attention_case
+    B, S, h, dh = 2, 200, 2, 64
+    qkv, dU, L, U_ref, lse_ref, dU64 = _attention_case(B, S, h, dh, seed=77)
+    U, lse = ppu.ppu_attention_fwd(qkv, B, S, h, dh, backend=0)
+    dq, dk, dv = O._attention_bwd(O.Model(1, h * dh, h, 8, 8), L, dU64.reshape(B, S, h * dh), None)
+    got = ppu.ppu_attention_bwd_static(qkv, U, lse, dU, B, S, h, dh, backend=0)
+    torch.cuda.synchronize()
+    g = got.float().cpu().numpy()
+    d = h * dh
+    for name, a, ref in (("dq", g[:, :d], dq), ("dk", g[:, d:2 * d], dk), ("dv", g[:, 2 * d:], dv)):
+        ref = ref.reshape(B * S, d)
+        assert np.abs(a - ref).max() <= 2e-2 * np.abs(ref).max(), name
