@@ -170,6 +170,17 @@ struct DenseOwner { float* master; int64_t shift; };
 // a listed replica's trained block of one layer: hidden units [lo,hi); packed W_in block at
 // master + in_off, W_out block at master + out_off
 struct OuterOwner { float* master; int64_t in_off, out_off; int32_t lo, hi; };
+// Division by a fixed divisor d < 2^16 as multiply-high and shift: with 2^shift < d <= 2^(shift+1)
+// and mul = floor(2^(32 + shift) / d) + 1, floor(n / d) = (n * mul) >> (32 + shift) for every
+// n < 2^28 (the sweep divides element offsets inside one weight matrix).
+struct FastDiv { uint32_t mul, shift; };
+inline FastDiv make_fast_div(uint32_t d) {
+  FastDiv f; f.shift = 0;
+  while ((1u << f.shift) < d) ++f.shift;          // 2^shift >= d
+  if (f.shift > 0) --f.shift;                     // 2^shift < d <= 2^(shift + 1): mul fits 32 bits
+  f.mul = (uint32_t)((((uint64_t)1 << (32 + f.shift)) / d) + 1);
+  return f;
+}
 struct OuterTables {
   const OuterSeg* segs;          // device
   const OuterChunk* chunks;      // device
@@ -177,6 +188,7 @@ struct OuterTables {
   const int32_t* unit_begin;     // device [L * F/8 + 1]
   const OuterOwner* unit_owner;  // device, owners inline
   int32_t d, F;
+  FastDiv div_d, div_F;
 };
 // sweeps chunks [chunk_lo, chunk_lo + n_chunks)
 void launch_outer(const OuterTables& t, int kind, float* theta, float* buf, bf16* w16, float lr, float mu,

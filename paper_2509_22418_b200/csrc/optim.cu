@@ -139,15 +139,21 @@ constexpr int OUTER_THREADS = 256;
 
 __device__ __forceinline__ void outer_update(float4& th, float4& bu, const float4& total, int count,
                                              float lr, float mu) {
-  const float m = count > 0 ? (float)count : 1.f;
+  // (a division by m = 1 or by the stand-in for m = 0 changes nothing and is skipped: the sweep
+  // runs at the power-capped SM clock and is sensitive to its instruction count)
   float* pt = &th.x; float* pb = &bu.x; const float* pd = &total.x;
 #pragma unroll
   for (int e = 0; e < 4; ++e) {
-    const float g = -(pd[e] / m);
+    const float g = count > 1 ? -(pd[e] / (float)count) : -pd[e];
     const float b = mu * pb[e] + g;
     pt[e] = pt[e] - lr * (g + mu * b);
     pb[e] = b;
   }
+}
+
+// n / divisor for n < 2^31 with the divisor's precomputed multiplier and shift
+__device__ __forceinline__ uint32_t fast_div(uint32_t n, FastDiv f) {
+  return (uint32_t)(((uint64_t)n * f.mul) >> 32) >> f.shift;
 }
 
 template <int KIND>
@@ -198,8 +204,8 @@ __device__ __forceinline__ void outer_chunk(const OuterTables& t, const OuterSeg
       } else {
         const uint32_t rel = rel0 + 4u * e;
         uint32_t unit, inner;
-        if (KIND == 1) { unit = rel / (uint32_t)t.d; inner = rel - unit * (uint32_t)t.d; }
-        else { inner = rel / (uint32_t)t.F; unit = rel - inner * (uint32_t)t.F; }
+        if (KIND == 1) { unit = fast_div(rel, t.div_d); inner = rel - unit * (uint32_t)t.d; }
+        else { inner = fast_div(rel, t.div_F); unit = rel - inner * (uint32_t)t.F; }
         const int ob = ub[unit >> 3], oe = ub[(unit >> 3) + 1];
         for (int o = ob; o < oe; ++o) {
           const OuterOwner ow = t.unit_owner[o];

@@ -533,6 +533,7 @@ int outer_sync_impl(ppu_ctx* c, const int32_t* replicas, int n, int group, int n
   OuterTables t;
   t.segs = c->d_oseg; t.chunks = c->d_ochunk; t.dense_owner = c->d_downer;
   t.unit_begin = c->d_unit_begin; t.unit_owner = c->d_unit_owner; t.d = d; t.F = F;
+  t.div_d = make_fast_div((uint32_t)d); t.div_F = make_fast_div((uint32_t)F);
   double swept = 0;
   if (all) swept = (double)c->P;
   else if (tail) swept = (double)c->e_size + (double)(c->P - c->off_lnfg);
