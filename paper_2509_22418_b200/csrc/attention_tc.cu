@@ -628,10 +628,14 @@ attn_dq_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_const
 // S^T into bf16 P^T and then dP^T into bf16 dS^T, each written back over the first half of the
 // thread's own accumulator columns, and dV += P^T dU, dK += dS^T Q take those as A operands
 // straight from tensor memory.  The tensor-memory budget (two 128-column accumulators for dV and
-// dK plus the two score buffers) leaves no room to double-buffer the scores, so the slab is
-// pipelined in halves instead: one thread issues S^T and dP^T, a second one dV and dK;
-// S^T of slab i+1 may start as soon as dV of slab i has consumed P^T (while the row threads are
-// still forming dS^T), and dP^T of slab i+1 as soon as dK of slab i is done.
+// dK plus the two score buffers) leaves no room to double-buffer the scores, and with one score
+// buffer S^T -> P^T -> dV -> next S^T is a serial chain that leaves the tensor pipe idle while
+// the row threads work.  So the chain is split by query half: S^T and dV are issued per half
+// (64-column / 64-deep products) with their own barriers, S^T of slab i+1's half h may start
+// as soon as dV of slab i's half h has consumed that half's P^T, and the two row groups drift
+// half a period apart - one group's exponentials run under the other's products.  One thread
+// issues S^T and dP^T, a second one dV and dK; dP^T of slab i+1 may start as soon as dK of
+// slab i is done.
 // Work items of the dk/dv kernel: 128 keys of one head of one sequence, heavy (first key block)
 // first; qb of the item is its key block.
 __device__ __forceinline__ bool work_item_kv(int k, int n_batch, int h, int nq, WorkItem& w) {
@@ -656,24 +660,29 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
   // per-query statistics of a slab, staged one slab ahead: [slab % 3][lse * log2e | delta][128]
   float* row_stat = reinterpret_cast<float*>(smem + (2 + 2 * NS) * QT);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (2 + 2 * NS) * QT + 3 * 2 * 128 * 4);
-  enum { KV_FULL = 0, KV_EMPTY, QG_FULL, QG_EMPTY = QG_FULL + NS, S_FULL = QG_EMPTY + NS, DP_FULL, P_FULL, DS_FULL,
-         TS_EMPTY, TP_EMPTY, OUT_FULL, ACC_EMPTY, NBAR };
+  // S_FULL, P_FULL and TS_EMPTY exist per query half of the slab (= per row group)
+  enum { KV_FULL = 0, KV_EMPTY, QG_FULL, QG_EMPTY = QG_FULL + NS, S_FULL = QG_EMPTY + NS, DP_FULL = S_FULL + 2,
+         P_FULL, DS_FULL = P_FULL + 2, TS_EMPTY, TP_EMPTY = TS_EMPTY + 2, OUT_FULL, ACC_EMPTY, NBAR };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar0 = smem_u32(bars);
   auto B = [&](int i) { return bar0 + 8u * i; };
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int d = p.h * DH, S = p.S, nq = (S + 127) / 128;
-  // row thread (grp, row) fetches the statistic `grp` of query `row` of query block qblk
+  // Row thread (grp, row) stages one statistic of one of its own group's 64 queries of query block
+  // qblk: threads 0-63 the log-sum-exp, threads 64-127 delta.  A group reads only what its own
+  // threads staged, so its hand-over needs no one but itself.
   auto fetch_stat = [&](const WorkItem& w, int qblk, int grp, int row) -> float {
-    const int q = qblk * 128 + row;
+    const int q = qblk * 128 + 64 * grp + (row & 63);
     const int64_t i = ((int64_t)w.b * p.h + w.head) * S + (q < S ? q : S - 1);
-    return grp == 0 ? __ldg(p.lse + i) * LOG2E : __ldg(p.delta + i);
+    return row < 64 ? __ldg(p.lse + i) * LOG2E : __ldg(p.delta + i);
   };
+  // where that value goes inside a staging slot laid out [lse | delta][128 queries]
+  auto stat_slot = [](int grp, int row) { return (row >> 6) * 128 + 64 * grp + (row & 63); };
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NBAR; ++i) mbar_init(B(i), 1);
-    mbar_init(B(P_FULL), 8); mbar_init(B(DS_FULL), 8); mbar_init(B(ACC_EMPTY), 8);
+    mbar_init(B(P_FULL), 4); mbar_init(B(P_FULL + 1), 4); mbar_init(B(DS_FULL), 8); mbar_init(B(ACC_EMPTY), 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -683,7 +692,7 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
     WorkItem w0;
     if (work_item_kv(0, p.B, p.h, nq, w0)) {
       const int g0 = (warp - 2) >> 2, r0 = (warp & 3) * 32 + lane;
-      row_stat[g0 * 128 + r0] = fetch_stat(w0, w0.qb, g0, r0);
+      row_stat[stat_slot(g0, r0)] = fetch_stat(w0, w0.qb, g0, r0);
     }
   }
   tc_fence_before();
@@ -718,7 +727,7 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc_s = make_idesc(128, 128, false, false);
+      constexpr uint32_t idesc_s = make_idesc(128, 128, false, false), idesc_h = make_idesc(128, 64, false, false);
       const uint32_t k_lo = klo(Ks), v_lo = klo(Vs);
       WorkItem w; uint32_t c = 0; bool ok = true;
       for (int k = 0; ok && work_item_kv(k, p.B, p.h, nq, w); ++k) {
@@ -728,13 +737,19 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
           const uint32_t Qst = Rs + st * 2 * QT, Gst = Qst + QT;
           if (!mbar_wait(B(QG_FULL + st), (c / NS) & 1, abort_flag, p.flags)) { ok = false; break; }
           const uint32_t q_lo = klo(Qst), g_lo = klo(Gst);
-          // S^T overwrites P^T of the previous slab: wait until dV has consumed it
-          if (c > 0 && !mbar_wait(B(TS_EMPTY), prev, abort_flag, p.flags)) { ok = false; break; }
-          tc_fence_after();
+          // S^T is formed per query half (64-column products), each half as soon as dV has consumed
+          // that half's P^T of the previous slab: the two row groups then work out of phase, and
+          // one group's exponentials overlap the other's products
 #pragma unroll
-          for (int ks = 0; ks < DH / 16; ++ks)
-            umma_lo(tS, k_lo + kstep<128>(ks), q_lo + kstep<128>(ks), idesc_s, ks > 0);
-          umma_commit(B(S_FULL));
+          for (int hh = 0; hh < 2; ++hh) {
+            if (c > 0 && !mbar_wait(B(TS_EMPTY + hh), prev, abort_flag, p.flags)) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int ks = 0; ks < DH / 16; ++ks)
+              umma_lo(tS + 64 * hh, k_lo + kstep<128>(ks), q_lo + 512u * hh + kstep<128>(ks), idesc_h, ks > 0);
+            umma_commit(B(S_FULL + hh));
+          }
+          if (!ok) break;
           // dP^T overwrites dS^T of the previous slab: wait until dK has consumed it
           if (c > 0 && !mbar_wait(B(TP_EMPTY), prev, abort_flag, p.flags)) { ok = false; break; }
           tc_fence_after();
@@ -758,13 +773,17 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
           const uint32_t Qst = Rs + st * 2 * QT, Gst = Qst + QT;
           if (!mbar_wait(B(QG_FULL + st), (c / NS) & 1, abort_flag, p.flags)) { ok = false; break; }
           const uint32_t gmn_lo = mlo<128>(Gst), qmn_lo = mlo<128>(Qst);
-          if (!mbar_wait(B(P_FULL), ph, abort_flag, p.flags)) { ok = false; break; }
-          tc_fence_after();
           // group g's 64 queries sit in the first 32 columns of its own half of the accumulator
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks)
-            umma_ts_lo(tV, tS + (ks >> 2) * 64 + (ks & 3) * 8, gmn_lo + mstep(ks), idesc_o, (it > 0 || ks > 0));
-          umma_commit(B(TS_EMPTY));
+          for (int hh = 0; hh < 2; ++hh) {
+            if (!mbar_wait(B(P_FULL + hh), ph, abort_flag, p.flags)) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int ks = 4 * hh; ks < 4 * hh + 4; ++ks)
+              umma_ts_lo(tV, tS + hh * 64 + (ks & 3) * 8, gmn_lo + mstep(ks), idesc_o, (it > 0 || ks > 0));
+            umma_commit(B(TS_EMPTY + hh));
+          }
+          if (!ok) break;
           if (!mbar_wait(B(DS_FULL), ph, abort_flag, p.flags)) { ok = false; break; }
           tc_fence_after();
 #pragma unroll
@@ -799,7 +818,7 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
         const float next_stat = it + 1 < n ? fetch_stat(w, kb + it + 1, grp, row)
                                            : (have_next ? fetch_stat(wn, wn.qb, grp, row) : 0.f);
         // ---- P^T from S^T
-        if (!mbar_wait(B(S_FULL), ph, abort_flag, p.flags)) { ok = false; break; }
+        if (!mbar_wait(B(S_FULL + grp), ph, abort_flag, p.flags)) { ok = false; break; }
         tc_fence_after();
         uint32_t rs[64], pk[32];
         tmem_ld32(tS + lane_off + 64 * grp, rs);
@@ -822,10 +841,10 @@ attn_dkv_tc_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
         tmem_st32(tS + lane_off + 64 * grp, pk);
         tmem_st_wait();
         tc_fence_before();
-        // next slab's statistics: written before this arrival, they are visible to every thread
-        // that later sees the next slab's S^T (which is issued only after dV of this slab)
-        if (more) row_stat[(((cs + 1) % 3) * 2 + grp) * 128 + row] = next_stat;
-        warp_arrive(B(P_FULL));
+        // next slab's statistics: written before this arrival, they are visible to every thread of
+        // the group that later sees its half of the next slab's S^T (issued only after this half's dV)
+        if (more) row_stat[((cs + 1) % 3) * 256 + stat_slot(grp, row)] = next_stat;
+        warp_arrive(B(P_FULL + grp));
         // ---- dS^T from dP^T
         if (!mbar_wait(B(DP_FULL), ph, abort_flag, p.flags)) { ok = false; break; }
         tc_fence_after();

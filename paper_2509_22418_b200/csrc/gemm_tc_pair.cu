@@ -244,7 +244,12 @@ int launch_pair_t(const GemmArgs& g, const TcParams& p0, cudaStream_t st) {
   p.splits = 1; p.split_stride = 0;
   const int tiles = p.tiles_m * p.tiles_n;
   const int n_sm = ppu_sm_count();
-  const int pairs = tiles < n_sm / 2 ? tiles : n_sm / 2;
+  // as many pairs as give every pair the same number of tiles: 256 tiles on 74 pairs take four
+  // waves whether 74 or 64 pairs work on them, and on a power-capped part the idle SMs' share of
+  // the budget raises the clock of the busy ones
+  const int max_pairs = n_sm / 2;
+  const int waves = (tiles + max_pairs - 1) / max_pairs;
+  const int pairs = tiles < max_pairs ? tiles : (tiles + waves - 1) / waves;
   gemm_tc_pair_kernel<PAIR_BN, A_K, B_K><<<2 * pairs, GEMM_THREADS, PairCfg<PAIR_BN>::SMEM, st>>>(mapA, mapB, p);
   return cudaGetLastError() == cudaSuccess ? 0 : -3;
 }
