@@ -210,6 +210,12 @@ int ppu_set_subset_state(ppu_ctx* ctx, int replica, const float* m, const float*
  * device-to-device copies or a collective on these local buffers), and every GPU then runs
  * the same ppu_outer_sync.  dev_ptr: HOST out. */
 int ppu_replica_values(ppu_ctx* ctx, int replica, void** dev_ptr, int64_t* n);
+/* Debug aid: every sub-buffer the context carves out of the arena (parameters, each replica's
+ * packed arrays, every activation and scratch buffer) is followed by a 256-byte guard block
+ * filled at creation with a fixed pattern that no kernel may write.  This call waits for the
+ * stream, reads all guard blocks back and reports how many were modified (n_bad: HOST out);
+ * PPU_ESTATE if any was - an out-of-bounds write by one of the kernels. */
+int ppu_check_guards(ppu_ctx* ctx, int64_t* n_bad);
 int ppu_set_adam_lr(ppu_ctx* ctx, float lr);
 int ppu_sync(ppu_ctx* ctx);   /* waits for the stream; reports PPU_ETOKEN / PPU_ETIMEOUT */
 int ppu_stats(ppu_ctx* ctx, ppu_stats_t* out);

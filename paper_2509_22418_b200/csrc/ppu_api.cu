@@ -210,9 +210,13 @@ static void build_geometry(ppu_ctx* c) {
 // Carves the arena.  With base == nullptr only the sizes are computed.
 static size_t carve(ppu_ctx* c, uint8_t* base) {
   size_t off = 0;
+  // every sub-buffer is followed by a guard block that no kernel may touch (ppu_check_guards)
+  c->guards.clear();
   auto take = [&](size_t bytes) -> uint8_t* {
     uint8_t* p = base ? base + off : nullptr;
     off += (bytes + 255) & ~(size_t)255;
+    c->guards.push_back(off);
+    off += PPU_GUARD_BYTES;
     return p;
   };
   const int64_t d = c->cfg.d_model, F = c->cfg.d_ff, V = c->cfg.vocab;
@@ -364,6 +368,7 @@ extern "C" int ppu_create(const ppu_model_cfg* cfg, const ppu_subset_spec* spec,
     }                                                                                  \
   } while (0)
   CREATE_OK(cudaMemsetAsync(c->arena, 0, c->state_bytes, st));
+  for (size_t g : c->guards) CREATE_OK(cudaMemsetAsync(c->arena + g, PPU_GUARD_BYTE, PPU_GUARD_BYTES, st));
   // LayerNorm gains start at one
   {
     std::vector<float> ones(c->cfg.d_model, 1.f);
@@ -609,6 +614,25 @@ extern "C" int ppu_set_backends(ppu_ctx* c, int gemm, int attention) {
     return ppu_fail(PPU_EINVAL, "backends are 0 (tcgen05) or 1 (SIMT check kernels)");
   c->gemm_backend = gemm;
   c->attn_backend = attention;
+  return PPU_OK;
+}
+extern "C" int ppu_check_guards(ppu_ctx* c, int64_t* n_bad) {
+  NEED_CTX(c);
+  if (!n_bad) return ppu_fail(PPU_EINVAL, "n_bad is null");
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  // the guards are gathered with one strided copy each into a host array, then compared
+  std::vector<uint8_t> host(c->guards.size() * PPU_GUARD_BYTES);
+  for (size_t i = 0; i < c->guards.size(); ++i)
+    CUDA_OK(cudaMemcpyAsync(host.data() + i * PPU_GUARD_BYTES, c->arena + c->guards[i], PPU_GUARD_BYTES,
+                            cudaMemcpyDeviceToHost, c->stream));
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  int64_t bad = 0; size_t first = 0;
+  for (size_t i = 0; i < c->guards.size(); ++i)
+    for (int b = 0; b < PPU_GUARD_BYTES; ++b)
+      if (host[i * PPU_GUARD_BYTES + b] != PPU_GUARD_BYTE) { if (!bad) first = i; ++bad; break; }
+  *n_bad = bad;
+  if (bad) return ppu_fail(PPU_ESTATE, "%lld guard blocks overwritten (first: the one after sub-buffer %zu of the arena)",
+                           (long long)bad, first);
   return PPU_OK;
 }
 extern "C" int ppu_set_adam_lr(ppu_ctx* c, float lr) {

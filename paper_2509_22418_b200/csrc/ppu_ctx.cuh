@@ -6,6 +6,10 @@
 #include "../../include/ppu.h"
 #include "common.cuh"
 
+// guard block after every sub-buffer of the arena
+constexpr int PPU_GUARD_BYTES = 256;
+constexpr int PPU_GUARD_BYTE = 0xA5;
+
 struct TensorRec { std::string name; int64_t offset; int ndim; int64_t shape[2]; };
 
 struct ReplicaState {
@@ -68,6 +72,7 @@ struct ppu_ctx {
   // arena
   uint8_t* arena = nullptr;
   size_t arena_bytes = 0, state_bytes = 0, act_bytes = 0;
+  std::vector<size_t> guards;   // arena offsets of the guard blocks
   float *theta = nullptr, *buf = nullptr;
   bf16* w16 = nullptr;
   float* grad = nullptr;        // [wgrad_splits][max_ffn] partials of the FFN blocks, then [max_dense]

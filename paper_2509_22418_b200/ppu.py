@@ -268,6 +268,11 @@ class Context:
     def ppu_set_backends(self, gemm: int = 0, attention: int = 0) -> None:
         _check(lib().ppu_set_backends(self._h, gemm, attention))
 
+    def ppu_check_guards(self) -> int:
+        n = C.c_int64()
+        _check(lib().ppu_check_guards(self._h, C.byref(n)))
+        return n.value
+
     def ppu_set_adam_lr(self, lr: float) -> None:
         _check(lib().ppu_set_adam_lr(self._h, C.c_float(lr)))
 

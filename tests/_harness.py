@@ -231,7 +231,14 @@ class Pair:
         return rec
 
     def close(self):
-        self.ctx.close()
+        import sys
+        try:
+            # no kernel wrote outside its buffers (guard blocks between all sub-buffers of the arena);
+            # skipped while another failure is propagating, so that it is not replaced
+            if sys.exc_info()[0] is None:
+                assert self.ctx.ppu_check_guards() == 0
+        finally:
+            self.ctx.close()
 
 
 # ---- rounds and outer steps against the oracle ---------------------------------------------

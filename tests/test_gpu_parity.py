@@ -412,3 +412,29 @@ def test_exchange_step_two_emulated_gpus_equal_one_gpu_bit_for_bit():
         one.close()
         for c in two:
             c.close()
+
+
+def test_guard_blocks_detect_a_stray_write():
+    """The guard blocks between the arena's sub-buffers are intact after steps and a sync, and a
+    byte written into one from the host side of the test (through the arena tensor) is reported."""
+    import torch
+    from paper_2509_22418_b200 import ppu, synth
+    dims, B, S = (2, 64, 4, 256, 512), 4, 64
+    spec, keep = ppu.make_spec(4, n_slices=4, train_non_mlp=1)
+    ctx = ppu.Context(ppu.make_cfg(*dims, B, S), spec, keep)
+    try:
+        ctx.ppu_set_params(synth.init_params(1, ctx.tensors()))
+        for k in range(4):
+            ctx.ppu_local_step(k, torch.from_numpy(synth.tokens(1, k, 0, 0, B, S, dims[4])).cuda())
+        ctx.ppu_outer_sync([0, 1, 2, 3])
+        assert ctx.ppu_check_guards() == 0
+        # theta (P fp32 values, padded to 256 bytes) is the first sub-buffer: its guard follows it
+        base = ((ctx.arena.data_ptr() + 255) & ~255) - ctx.arena.data_ptr()
+        first_guard = base + ((ctx.param_count * 4 + 255) & ~255)
+        assert int(ctx.arena[first_guard]) == 0xA5
+        ctx.arena[first_guard + 7] = 0
+        with pytest.raises(ppu.PpuError) as ei:
+            ctx.ppu_check_guards()
+        assert ei.value.code == -5
+    finally:
+        ctx.close()
