@@ -325,6 +325,9 @@ def main():
     ap.add_argument("--impl", default="ppu", choices=["ppu", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="leave out the round and sweep objects")
+    ap.add_argument("--exchange", action="store_true",
+                    help="N > 1: one set of K replicas dealt over the GPUs (replica k on GPU k mod N) with the real "
+                         "exchange step before the outer sync, instead of N independent sets")
     args = ap.parse_args()
     w = WORKLOADS[args.workload]
     if args.sweep:
@@ -353,8 +356,16 @@ def main():
     ctx = ppu.Context(cfg, spec, keep, device=f"cuda:{local}")
     ctx.ppu_set_params(synth.init_params(SEED + rank, ctx.tensors()))
     n_tok = args.warmup + args.steps
-    group = pdist.replica_group(K, world, rank)       # this rank's replicas (global ids)
-    host_tok = [synth.tokens(SEED, group[i % K], 0, i, B, S, V) for i in range(n_tok)]
+    exchange = args.exchange and world > 1
+    if exchange:
+        # one model on all GPUs (same parameters everywhere), replica k stepped by GPU k mod world
+        ctx.ppu_set_params(synth.init_params(SEED, ctx.tensors()))
+        mine = pdist.my_replicas(K, world, rank)
+        group = list(range(K))
+    else:
+        mine = list(range(K))
+        group = pdist.replica_group(K, world, rank)   # this rank's replicas (global ids)
+    host_tok = [synth.tokens(SEED, group[mine[i % len(mine)]], 0, i, B, S, V) for i in range(n_tok)]
     pinned = [torch.from_numpy(t).pin_memory() for t in host_tok]
     dev_tok = [t.to(ctx.device) for t in pinned]
     torch.cuda.synchronize()
@@ -365,9 +376,13 @@ def main():
 
     def region(use_host, profile):
         """warm-up, then `steps` local steps and one outer sync between two events."""
+        rep_of = lambda i: mine[i % len(mine)]
         for i in range(args.warmup):
-            ctx.ppu_local_step(i % K, dev_tok[i])
-        ctx.ppu_outer_sync(sorted({i % K for i in range(args.warmup)}))
+            ctx.ppu_local_step(rep_of(i), dev_tok[i])
+        if exchange:
+            pdist.outer_sync_all_gpus(ctx, K, world, rank)
+        else:
+            ctx.ppu_outer_sync(sorted({rep_of(i) for i in range(args.warmup)}))
         ctx.ppu_sync()
         if profile:
             ctx.ppu_profile_enable(True)
@@ -378,11 +393,14 @@ def main():
         for j in range(args.steps):
             i = args.warmup + j
             if use_host:
-                ctx.ppu_local_step_host(i % K, host_tok[i])
+                ctx.ppu_local_step_host(rep_of(i), host_tok[i])
             else:
-                ctx.ppu_local_step(i % K, dev_tok[i])
+                ctx.ppu_local_step(rep_of(i), dev_tok[i])
         e1.record()
-        ctx.ppu_outer_sync(sorted({(args.warmup + j) % K for j in range(args.steps)}))
+        if exchange:     # all-gather of the replicas' end values, then the same outer step on every GPU
+            pdist.outer_sync_all_gpus(ctx, K, world, rank)
+        else:
+            ctx.ppu_outer_sync(sorted({rep_of(args.warmup + j) for j in range(args.steps)}))
         e2.record()
         barrier()
         prof = ctx.ppu_profile_read() if profile else None
@@ -420,7 +438,9 @@ def main():
         metric="local-step tokens/s", value=tokens / (total_ms * 1e-3), unit="tokens/s",
         n_gpus=world, steps=args.steps, warmup=args.warmup, ms_per_step=total_ms / args.steps,
         higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
-        config=workload_config(args.workload, w),
+        config=dict(workload_config(args.workload, w),
+                    multi_gpu=("one set of replicas dealt over the GPUs, exchange step before the outer sync"
+                               if exchange else "replicas only: every GPU runs its own independent set")),
         local_step_ms=steps_ms / args.steps,
         outer_sync=dict(ms=outer_ms, algorithmic_bytes=st.outer_bytes,
                         gbs=st.outer_bytes / (outer_ms * 1e-3) / 1e9, peak_gbs=pk["hbm"],
