@@ -9,15 +9,15 @@ What it computes, all in numpy (float64 unless a dtype is passed), following
 "Partial Parameter Updates for Efficient Distributed Training":
 
 * the decoder forward pass on all parameters and the loss of Eq. 2.2;
-* the gradient of Algorithm 1 line 9 in two ways: the definition (full
+* the masked gradient of Algorithm 1 in two ways: the definition (full
   backward, then mask to the trainable index set) and the restricted backward
   of Appendix C.1 (weight gradients only for the trained FFN slice and, under
   head slicing, for the trained heads' query / key / value projections; input
   gradients through every slice and head; nothing below the lowest trained
   layer when only FFN slices are trained);
-* the inner AdamW update on the subset (Algorithm 1 line 10, Section 3.1);
+* the inner AdamW update on the subset (Algorithm 1, the inner update, Section 3.1);
 * per-node deltas, the count vector m, the count-normalised average and the
-  outer Nesterov step (Algorithm 1 lines 12-15, Eq. 2.4-2.5);
+  outer Nesterov step (Algorithm 1, the outer step, Eq. 2.4-2.5);
 * the closed-form parameter and FLOP counts of Table 1 and Appendix C.2.
 
 numpy's matmul is the only library primitive used as a step.  There is no
@@ -480,7 +480,7 @@ def count_vector(n_total: int, index_sets) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------
-# inner optimizer (Algorithm 1 line 10; AdamW, Section 3.1)
+# inner optimizer (Algorithm 1, the inner update; AdamW, Section 3.1)
 # --------------------------------------------------------------------------
 def adamw_update(p, g, m, v, t, hp: AdamW, decay=None):
     """One decoupled-weight-decay Adam step on arrays of equal shape; t is the
@@ -522,7 +522,7 @@ class Replica:
         return th
 
     def gradient(self, theta_global, tokens, mode="restricted"):
-        """g_k[I_train] of Algorithm 1 line 9, in the order of self.idx: by the
+        """g_k[I_train], the masked gradient of Algorithm 1, in the order of self.idx: by the
         definition (mode "masked_full": the full gradient, then the mask) or by
         the restricted backward of Appendix C.1."""
         th = self.materialise(theta_global)
@@ -553,7 +553,7 @@ class Replica:
         return loss, g
 
     def apply_gradient(self, loss, g, hp: AdamW):
-        """Algorithm 1 line 10 for a gradient g[I_train] that is already known (several
+        """The inner update of Algorithm 1 for a gradient g[I_train] that is already known (several
         nodes that start from the same parameters and see the same batch share one full
         backward pass: each takes its own entries of it)."""
         self.t += 1
@@ -568,7 +568,7 @@ class Replica:
 
 
 # --------------------------------------------------------------------------
-# outer synchronisation (Algorithm 1 lines 12-15; Eq. 2.4-2.5)
+# outer synchronisation (Algorithm 1, the outer step; Eq. 2.4-2.5)
 # --------------------------------------------------------------------------
 def sync_group_mask(cfg: Model, group: int, n_groups: int) -> np.ndarray:
     """Positions synchronised together under streaming synchronisation by layers
