@@ -6,9 +6,9 @@
  * forward pass of a pre-LayerNorm causal decoder over all parameters,
  * back-propagates activation gradients down to its lowest trained layer,
  * forms weight gradients only for its own fixed parameter subset, applies
- * AdamW to that subset (Algorithm 1, lines 8-10), and the replicas are
+ * AdamW to that subset (Algorithm 1, the local step), and the replicas are
  * periodically merged by a count-normalised average of their deltas followed
- * by an outer Nesterov step (Algorithm 1, lines 12-15).
+ * by an outer Nesterov step (Algorithm 1, the outer step).
  *
  * Conventions
  *  - Every function returns PPU_OK (0) or a negative ppu_status.  Nothing
@@ -129,7 +129,7 @@ int ppu_create(const ppu_model_cfg* cfg, const ppu_subset_spec* spec, void* aren
                size_t arena_bytes, void* cuda_stream, ppu_ctx** out);
 int ppu_destroy(ppu_ctx* ctx);
 
-/* Algorithm 1 lines 8-10 for one replica: forward on all parameters, restricted
+/* The local step of Algorithm 1 for one replica: forward on all parameters, restricted
  * backward (Appendix C.1), AdamW on I_k^train; the replica's step count grows by
  * one.  tokens: DEVICE int32 [batch, seq], kept alive by the caller until the
  * stream has passed the call.  Ids outside [0, vocab) are clamped and reported
@@ -141,7 +141,7 @@ int ppu_local_step(ppu_ctx* ctx, int replica, const int32_t* tokens, int batch, 
 int ppu_local_step_host(ppu_ctx* ctx, int replica, const int32_t* tokens_host, int batch,
                         int seq, double* loss_out);
 
-/* Algorithm 1 lines 12-15 over the listed replicas (HOST array, no duplicates):
+/* The outer step of Algorithm 1 over the listed replicas (HOST array, no duplicates):
  * Delta[i] = sum_k (theta_k[i] - theta[i]) / m[i] with m counted over the list
  * and Delta = 0 where m = 0; pseudo-gradient g = -Delta; buf = mu buf + g;
  * theta -= eta (g + mu buf).  Sweeps every parameter, refreshes the bf16 working

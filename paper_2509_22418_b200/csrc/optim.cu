@@ -1,6 +1,6 @@
-// Optimizer-side kernels: AdamW over a replica's packed subset (Algorithm 1 line 10), moves
+// Optimizer-side kernels: AdamW over a replica's packed subset (Algorithm 1, the inner update), moves
 // between the packed subset arrays and the canonical vectors, and the outer synchronisation
-// sweep (Algorithm 1 lines 12-15).  All are HBM-bound: float4 accesses, grids sized from the
+// sweep (Algorithm 1, the outer step).  All are HBM-bound: float4 accesses, grids sized from the
 // SM count of the current device.
 #include "common.cuh"
 
@@ -125,7 +125,7 @@ dense_move_kernel(const DenseSeg* __restrict__ segs, float* packed, const float*
 }
 
 // ---------------------------------------------------------------------------------------------
-// Outer sweep (Algorithm 1 lines 12-15): Delta = sum over owners (theta_k - theta) / m, 0 where
+// Outer sweep (Algorithm 1, the outer step): Delta = sum over owners (theta_k - theta) / m, 0 where
 // m = 0; g = -Delta; buf = mu buf + g; theta -= lr (g + mu buf); the bf16 copy is refreshed and
 // every owner restarts from the new value (line 6).
 //

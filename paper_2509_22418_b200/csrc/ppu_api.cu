@@ -315,7 +315,7 @@ static int init_ctx(ppu_ctx* c, const ppu_model_cfg* cfg, const ppu_subset_spec*
   return PPU_OK;
 }
 
-// every replica's packed values <- the global parameters (Algorithm 1 line 6)
+// every replica's packed values <- the global parameters (Algorithm 1, the replica reset)
 static void ppu_restart_replicas(ppu_ctx* c) {
   for (auto& r : c->reps) {
     launch_slices_gather(r.d_segs, (int)r.segs.size(), c->theta, r.master, c->cfg.d_model,

@@ -1,4 +1,4 @@
-// Step scheduler: enqueues the kernels of one local step (Algorithm 1 lines 8-10) and of the
+// Step scheduler: enqueues the kernels of one local step (the inner loop body of Algorithm 1) and of the
 // outer synchronisation (lines 12-15) on the context's stream.  No host synchronisation
 // happens inside a local step.
 #include <algorithm>

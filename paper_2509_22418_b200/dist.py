@@ -2,7 +2,7 @@
 
 Between outer syncs the replicas of Algorithm 1 never exchange data, so G GPUs run G disjoint
 sets of replicas with no data-path collective.  Every H steps the paper all-reduces the sparse
-deltas and divides by the count vector m (Algorithm 1 line 14, Eq. 2.4).  Here that exchange
+deltas and divides by the count vector m (Algorithm 1, the count-normalised average, Eq. 2.4).  Here that exchange
 step is an all-gather of the replicas' end values: replica k lives on GPU k mod G, every GPU
 holds a buffer for every replica's packed trained values (ppu_replica_values), the owners'
 values are gathered into those buffers, and every GPU then runs the same ppu_outer_sync over
@@ -77,7 +77,7 @@ def exchange_replica_values(values, world: int, rank: int, group=None):
 
 
 def outer_sync_all_gpus(ctx, n_replicas: int, world: int, rank: int, group=None):
-    """The exchange step followed by the outer step (Algorithm 1 lines 12-15) on every GPU.
+    """The exchange step followed by the outer step of Algorithm 1 on every GPU.
     ctx: this rank's ppu.Context holding all n_replicas replicas, of which it stepped
     my_replicas(n_replicas, world, rank).  Returns the bytes received."""
     ctx.ppu_sync()                       # the local steps that produced the values have finished

@@ -202,7 +202,7 @@ class Pair:
         a few sequences has the loss and gradient of those sequences).  oracle_grad = (loss, dense
         full gradient) of the oracle for this batch at the replica's current parameters, when
         several replicas share one full backward pass (the replica takes its own entries:
-        Algorithm 1 line 9).  Returns a record of the numbers."""
+        Algorithm 1, the masked gradient).  Returns a record of the numbers."""
         rep = self.reps[k]
         before = self.ctx.ppu_get_params(k)[rep.idx].astype(np.float64)
         sub_before = rep.theta_sub.astype(np.float64)

@@ -13,7 +13,7 @@ parameters trained.
 
 1.3B-class (4 x 2048 tokens = 4 copies of one sequence).  One full backward pass of the oracle
 from the initial parameters serves every replica that starts from them on that batch - each
-takes its own entries (Algorithm 1 line 9: the masked full gradient) and applies its own AdamW
+takes its own entries (the masked full gradient of Algorithm 1) and applies its own AdamW
 step:
   * subset-fraction sweep: FFN fractions 1, 1/2, 1/4, 1/8, 1/32 and the whole-layer variant
     (every 4th block, replicas 0 and 3), gated on up to 20M sampled positions per variant;
@@ -223,6 +223,6 @@ def test_1p3b_round_protocol_eight_replicas_two_steps_and_outer_sync(shared_1p3b
         assert (th_new[ffn] != theta0[ffn]).mean() > 0.99
         assert np.array_equal(P.ctx.ppu_get_working_bf16(), bf16_bits(th_new))
         for k in (0, 7):
-            assert np.array_equal(P.ctx.ppu_get_params(k), th_new)       # replicas restart (Algorithm 1 line 6)
+            assert np.array_equal(P.ctx.ppu_get_params(k), th_new)       # replicas restart (Algorithm 1, the replica reset)
     finally:
         P.close()

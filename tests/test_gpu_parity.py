@@ -369,7 +369,7 @@ def test_checkpoint_save_destroy_restore_continues_bit_exactly():
 
 
 def test_exchange_step_two_emulated_gpus_equal_one_gpu_bit_for_bit():
-    """Algorithm 1 line 14 across GPUs: replica k is stepped by GPU k mod 2, the owners' end values
+    """Algorithm 1, the count-normalised average across GPUs: replica k is stepped by GPU k mod 2, the owners' end values
     are copied into the other GPU's buffers, and both run the same outer step.  Two contexts on
     this one GPU play the two GPUs, one after the other; their global parameters, momentum and
     working copy must equal, bit for bit, those of one context that stepped all four replicas.

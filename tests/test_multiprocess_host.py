@@ -1,6 +1,6 @@
 """Host-side logic of the N > 1 path with two gloo ranks on CPU: disjoint replica groups, the
 max-over-ranks reduction of step times that bench.py reports, and the exchange step of the
-outer sync (Algorithm 1 line 14): every rank ends up with every owner's end values."""
+outer sync (Algorithm 1, the count-normalised average): every rank ends up with every owner's end values."""
 import os
 import socket
 
