@@ -267,8 +267,9 @@ int ppu_wait_probe(int limit, void* cuda_stream);
  * multiples of 8.  out_f32: C is fp32, else bf16.  backend: 0 = tcgen05 tiles,
  * shape chosen from the problem size as the training step does; 1 = plain SIMT
  * check kernel; 2 = tcgen05, one CTA per 128-row tile; 3 = tcgen05, one SM pair
- * (cta_group::2) per 256 x 256 tile; 4 = the same per 256 x 128 tile.  All
- * pointers DEVICE.  Asynchronous on stream. */
+ * (cta_group::2) per 256 x 256 tile, a half-empty last wave of tiles worked as
+ * 128-column halves; 4 = one SM pair per 256 x 128 tile; 5 = as 3 with whole
+ * tiles only.  All pointers DEVICE.  Asynchronous on stream. */
 int ppu_gemm(const void* A, int64_t lda, int a_kmajor, const void* B, int64_t ldb,
              int b_kmajor, void* C, int64_t ldc, int out_f32, int M, int N, int K,
              int backend, void* cuda_stream);

@@ -30,8 +30,9 @@ def main():
     ap.add_argument("--seq", type=int, default=2048)
     ap.add_argument("--heads", type=int, default=16)
     ap.add_argument("--dh", type=int, default=128)
-    ap.add_argument("--backend", type=int, default=0, help="attention: 0 tcgen05, 1 SIMT, 2 mma.sync; gemm: 0 tcgen05 (shape chosen), 1 SIMT, "
-                         "2 tcgen05 one CTA per tile, 3 tcgen05 SM pairs 256 x 256, 4 SM pairs 256 x 128")
+    ap.add_argument("--backend", type=int, default=0, help="attention: 0 tcgen05, 1 SIMT; gemm: 0 tcgen05 (shape chosen), 1 SIMT, "
+                         "2 tcgen05 one CTA per tile, 3 tcgen05 SM pairs 256 x 256, 4 SM pairs 256 x 128, "
+                         "5 as 3 on whole tiles only")
     ap.add_argument("--layers", type=int, default=4)
     ap.add_argument("--replicas", type=int, default=4)
     ap.add_argument("--train-non-mlp", action="store_true")

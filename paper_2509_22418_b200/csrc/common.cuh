@@ -41,7 +41,8 @@ struct GemmArgs {
   // EPI_ROPE_BF16: aux is the (cos, sin) table [rope_S][rope_dh / 2]; row m is position m % rope_S
   int rope_S = 0, rope_dh = 0, rope_cols = 0;
   // tcgen05 tile shape: 0 chosen from the problem size, 1 one CTA per 128-row tile, 2 an SM pair
-  // per 256 x 256 tile, 3 an SM pair per 256 x 128 tile (tests force each)
+  // per 256 x 256 tile, 3 an SM pair per 256 x 128 tile, 4 as 2 without cutting the tiles of a
+  // half-empty last wave in two (tests force each)
   int tile_shape = 0;
 };
 

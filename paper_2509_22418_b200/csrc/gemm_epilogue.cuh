@@ -74,6 +74,8 @@ struct TcParams {
   const void* aux; long long ldaux;
   int* flags;
   int tiles_m, tiles_n;
+  int tail_from;   // SM-pair kernel: tiles from this index on are worked as two 128-column halves
+  int n_fastest;   // SM-pair kernel: consecutive tile indices walk along N (else along M)
   int splits; long long split_stride;
   int wide;   // every output / auxiliary row start is 32-byte aligned: use 32-byte accesses
   int rope_S, rope_dh, rope_cols;
@@ -88,15 +90,16 @@ int launch_gemm_tc_pair(const GemmArgs& g, const TcParams& p, int bn, cudaStream
 // Drains rows [m0 + 32 quarter, +32) x columns [n0 + half BN/2, + BN/2) of the accumulator at
 // TMEM column t_acc through registers into global memory, applying the epilogue p.epilogue.
 // One row per lane; `sp` is the split-K slice (offsets the output by sp * split_stride).
-template <int BN>
-__device__ __forceinline__ void drain_tile(const TcParams& p, int m0, int n0, int sp, uint32_t t_acc,
-                                           int quarter, int half, int lane) {
+// (drain_cols: the same for an explicit range [c_begin, c_end) of the tile's columns, both
+// multiples of 32)
+__device__ __forceinline__ void drain_cols(const TcParams& p, int m0, int n0, int sp, uint32_t t_acc,
+                                           int quarter, int c_begin, int c_end, int lane) {
   const int m = m0 + quarter * 32 + lane;
   const bool row_ok = m < p.M;
   const uint32_t t_row = t_acc + ((uint32_t)(quarter * 32) << 16);
   float head_dot = 0.f;   // EPI_DELTA_BF16: running sum over the current head's columns
 #pragma unroll 1
-  for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
+  for (int c0 = c_begin; c0 < c_end; c0 += 32) {
     const int nb = n0 + c0;
     if (nb >= p.N) break;                  // warp-uniform
     uint32_t r[32];
@@ -279,6 +282,12 @@ __device__ __forceinline__ void drain_tile(const TcParams& p, int m0, int n0, in
       }
     }
   }
+}
+
+template <int BN>
+__device__ __forceinline__ void drain_tile(const TcParams& p, int m0, int n0, int sp, uint32_t t_acc,
+                                           int quarter, int half, int lane) {
+  drain_cols(p, m0, n0, sp, t_acc, quarter, half * (BN / 2), (half + 1) * (BN / 2), lane);
 }
 
 }  // namespace gemm_tc_detail

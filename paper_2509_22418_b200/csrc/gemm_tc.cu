@@ -236,7 +236,7 @@ TcParams make_params(const GemmArgs& g) {
   TcParams p;
   p.M = g.M; p.N = g.N; p.K = g.K; p.epilogue = g.epilogue;
   p.C = g.C; p.ldc = g.ldc; p.C2 = g.C2; p.aux = g.aux; p.ldaux = g.ldaux; p.flags = g.flags;
-  p.tiles_m = p.tiles_n = 0; p.splits = 1; p.split_stride = 0;
+  p.tiles_m = p.tiles_n = 0; p.tail_from = 1 << 30; p.n_fastest = 0; p.splits = 1; p.split_stride = 0;
   p.C3 = g.C3; p.ldc3 = g.ldc3; p.c3_lo = g.c3_lo; p.c3_hi = g.c3_hi;
   p.rope_S = g.rope_S > 0 ? g.rope_S : 1; p.rope_dh = g.rope_dh > 0 ? g.rope_dh : 2; p.rope_cols = g.rope_cols;
   const bool f32 = g.epilogue == EPI_STORE_F32 || g.epilogue == EPI_RESID_F32;
@@ -299,7 +299,7 @@ namespace {
 // the SM-pair kernel on 256 x 256 tiles is chosen for this product
 bool picks_pair256(const GemmArgs& g) {
   const long long tiles_pair = (long long)((g.M + 255) / 256) * ((g.N + 255) / 256);
-  return g.tile_shape == 2 || (g.tile_shape == 0 && g.splits <= 1 && g.M > 128 && g.N > 128 && tiles_pair >= ppu_sm_count() / 2);
+  return g.tile_shape == 2 || g.tile_shape == 4 || (g.tile_shape == 0 && g.splits <= 1 && g.M > 128 && g.N > 128 && tiles_pair >= ppu_sm_count() / 2);
 }
 }  // namespace
 
@@ -323,10 +323,11 @@ int launch_gemm_tc(const GemmArgs& g, cudaStream_t st) {
     return -4;
   // Wide tiles when the grid still fills the machine; narrow ones for small outputs.
   // SM pairs on 256 x 256 tiles when those still fill the machine and the product is not split.
-  // (256 x 128 pair tiles would fill the last wave of the N = 2048 products better - 512 tiles
-  // instead of 256 on the 74 pairs of a B200 - but their narrower instruction measured 25 % slower, so they are
-  // never chosen here; tile_shape 3 keeps them testable.)
-  if ((g.tile_shape == 2 || g.tile_shape == 3) && g.splits > 1) return -4;
+  // (256 x 128 pair tiles throughout would fill the last wave of the N = 2048 products better -
+  // 512 tiles instead of 256 on the 74 pairs of a B200 - but the narrower product measured 25 %
+  // slower, so only a half-empty last wave is worked that way, inside the 256-wide kernel;
+  // tile_shape 3 keeps the narrow kernel testable, 4 is the 256-wide kernel without narrow units.)
+  if (g.tile_shape >= 2 && g.splits > 1) return -4;
   if (g.tile_shape == 3) return launch_gemm_tc_pair(g, make_params(g), 128, st);
   if (picks_pair256(g)) return launch_gemm_tc_pair(g, make_params(g), 256, st);
   const long long tiles256 = (long long)((g.M + BM - 1) / BM) * ((g.N + 255) / 256) * (g.splits > 1 ? g.splits : 1);

@@ -25,7 +25,10 @@ using namespace gemm_tc_detail;
 
 // The pair's tile is 256 rows x BN columns, BN = 256 or 128.  The narrow tile is for outputs whose
 // 256-wide tiling leaves the last wave of SM pairs half empty (N = 2048 with 8192 rows: 256 tiles
-// on the 74 SM pairs of a B200).
+// on the 74 SM pairs of a B200: three full waves and 34 tiles).  The 256-wide kernel can work the
+// tiles from index p.tail_from on as two 128-column halves each, so that the 34 leftover tiles
+// become 68 units on 74 pairs: the narrow product runs at about 0.7 of the wide one's rate, so
+// the last wave takes 0.7 of a tile's time instead of a whole one.
 // A stage holds PAIR_KH slabs of 64 k: the issuing thread stalls while the tensor pipe is busy, so
 // a barrier wait per 64 k (four instructions) is not hidden behind the products; one per 128 k is.
 constexpr int PAIR_KH = 2;
@@ -83,10 +86,31 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
       : "memory");
 }
 
+// one unit of work of a pair: rows [m0, m0 + 256) x columns [n0, n0 + bn)
+struct PairUnit { int m0, n0, bn; };
+template <int PAIR_BN>
+__device__ __forceinline__ PairUnit pair_unit(const TcParams& p, int u) {
+  PairUnit w;
+  int tile = u, half = 0;
+  w.bn = PAIR_BN;
+  if (PAIR_BN == 256 && u >= p.tail_from) {
+    const int v = u - p.tail_from;
+    tile = p.tail_from + (v >> 1); half = v & 1; w.bn = 128;
+  }
+  // consecutive tiles (which the pairs work on at the same time) walk along the smaller operand:
+  // the rows of A they share then stay in L2 while B is swept, or the other way round
+  const int row = p.n_fastest ? tile / p.tiles_n : tile % p.tiles_m;
+  const int col = p.n_fastest ? tile % p.tiles_n : tile / p.tiles_m;
+  w.m0 = row * 256;
+  w.n0 = col * PAIR_BN + half * 128;
+  return w;
+}
+
+// mapB2: B with a box of 64 rows (the narrow units of a K-major B); otherwise a copy of mapB
 template <int PAIR_BN, bool A_K, bool B_K>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
-                    const TcParams p) {
+                    const __grid_constant__ CUtensorMap mapB2, const TcParams p) {
   using PC = PairCfg<PAIR_BN>;
   constexpr int ST = PC::STAGES, PAIR_STAGE_BYTES = PC::STAGE_BYTES, HALF_BYTES = PC::A_HALF, B_SLAB = PC::B_SLAB;
   extern __shared__ uint8_t smem_raw[];
@@ -126,6 +150,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
 
   const int n_pairs = gridDim.x >> 1, pair = blockIdx.x >> 1;
   const int num_tiles = p.tiles_m * p.tiles_n;
+  const int num_units = num_tiles + (PAIR_BN == 256 && num_tiles > p.tail_from ? num_tiles - p.tail_from : 0);
   const int k_blocks = (p.K + PAIR_KH * BK - 1) / (PAIR_KH * BK);
 
   if (warp == 0) {
@@ -133,16 +158,20 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
       // ---------------- TMA producer (both CTAs) ----------------
       int s = 0; uint32_t ph = 0;
       bool ok = true;
-      for (int tile = pair; tile < num_tiles && ok; tile += n_pairs) {
-        const int m0 = (tile % p.tiles_m) * 256 + (int)rank * 128;
-        const int n0 = (tile / p.tiles_m) * PAIR_BN + (int)rank * (PAIR_BN / 2);
+      for (int u = pair; u < num_units && ok; u += n_pairs) {
+        const PairUnit w = pair_unit<PAIR_BN>(p, u);
+        const int m0 = w.m0 + (int)rank * 128;
+        const int n0 = w.n0 + (int)rank * (w.bn / 2);
+        const bool narrow = w.bn != PAIR_BN;
+        const int b_slab = narrow ? B_SLAB / 2 : B_SLAB;          // this CTA's bn/2 rows of B, 64 k
+        const CUtensorMap* mB = narrow ? &mapB2 : &mapB;
         for (int kb = 0; kb < k_blocks; ++kb) {
           ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.flags);
           if (!ok) break;
           const uint32_t a_dst = smem_u32(smem + s * PAIR_STAGE_BYTES);
           const uint32_t b_dst = a_dst + HALF_BYTES;
           const uint32_t fb = map_to_rank(full_bar(s), 0);
-          if (leader) mbar_expect_tx(full_bar(s), 2 * PAIR_STAGE_BYTES);
+          if (leader) mbar_expect_tx(full_bar(s), 2 * (HALF_BYTES + PAIR_KH * b_slab));
           // (k past the end of the reduction reads zeros)
 #pragma unroll
           for (int kh = 0; kh < PAIR_KH; ++kh) {
@@ -154,11 +183,11 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
               tma_load_2d_pair(a_dst + kh * SLAB_BYTES + 8192, &mapA, fb, m0 + 64, k0);
             }
             if (B_K) {
-              tma_load_2d_pair(b_dst + kh * B_SLAB, &mapB, fb, k0, n0);
+              tma_load_2d_pair(b_dst + kh * b_slab, mB, fb, k0, n0);
             } else {
 #pragma unroll
               for (int i = 0; i < PAIR_BN / 128; ++i)
-                tma_load_2d_pair(b_dst + kh * B_SLAB + i * 8192, &mapB, fb, n0 + 64 * i, k0);
+                if (i < w.bn / 128) tma_load_2d_pair(b_dst + kh * b_slab + i * 8192, &mapB, fb, n0 + 64 * i, k0);
             }
           }
           if (++s == ST) { s = 0; ph ^= 1u; }
@@ -168,12 +197,14 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
   } else if (warp == 1) {
     if (lane == 0 && leader) {
       // ---------------- MMA issuer (leader CTA only) ----------------
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_K ? 0u : 1u) << 15) |
-                             ((B_K ? 0u : 1u) << 16) | ((uint32_t)(PAIR_BN >> 3) << 17) |
-                             ((uint32_t)(256 >> 4) << 24);
+      const uint32_t idesc0 = (1u << 4) | (1u << 7) | (1u << 10) | ((A_K ? 0u : 1u) << 15) |
+                              ((B_K ? 0u : 1u) << 16) | ((uint32_t)(256 >> 4) << 24);
       int s = 0; uint32_t ph = 0;
       int acc = 0; uint32_t acc_ph = 0;
-      for (int tile = pair; tile < num_tiles; tile += n_pairs) {
+      for (int u = pair; u < num_units; u += n_pairs) {
+        const PairUnit w = pair_unit<PAIR_BN>(p, u);
+        const uint32_t idesc = idesc0 | ((uint32_t)(w.bn >> 3) << 17);
+        const uint32_t b_slab = w.bn != PAIR_BN ? B_SLAB / 2 : B_SLAB;
         if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.flags)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * PAIR_BN);
@@ -187,7 +218,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
 #pragma unroll
           for (int k = 0; k < PAIR_KH * (BK / UMMA_K); ++k) {
             const uint32_t kh = (uint32_t)(k / (BK / UMMA_K)), kk = (uint32_t)(k % (BK / UMMA_K));
-            const uint32_t slab = kh * SLAB_BYTES, slab_b = kh * B_SLAB;
+            const uint32_t slab = kh * SLAB_BYTES, slab_b = kh * b_slab;
             const uint64_t adesc = A_K ? make_desc(a_addr + slab + kk * 32, 16, 1024) : make_desc(a_addr + slab + kk * 2048, 8192, 1024);
             const uint64_t bdesc = B_K ? make_desc(b_addr + slab_b + kk * 32, 16, 1024) : make_desc(b_addr + slab_b + kk * 2048, 8192, 1024);
             umma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
@@ -205,12 +236,13 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     const int quarter = warp & 3;
     const int half = (warp - 2) >> 2;
     int acc = 0; uint32_t acc_ph = 0;
-    for (int tile = pair; tile < num_tiles; tile += n_pairs) {
-      const int m0 = (tile % p.tiles_m) * 256 + (int)rank * 128;
-      const int n0 = (tile / p.tiles_m) * PAIR_BN;
+    for (int u = pair; u < num_units; u += n_pairs) {
+      const PairUnit w = pair_unit<PAIR_BN>(p, u);
+      const int m0 = w.m0 + (int)rank * 128;
       if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.flags)) break;
       tc_fence_after();
-      drain_tile<PAIR_BN>(p, m0, n0, 0, tmem_base + (uint32_t)(acc * PAIR_BN), quarter, half, lane);
+      drain_cols(p, m0, w.n0, 0, tmem_base + (uint32_t)(acc * PAIR_BN), quarter, half * (w.bn / 2),
+                 (half + 1) * (w.bn / 2), lane);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_rank(tempty_bar(acc), 0));
@@ -235,13 +267,18 @@ template <int PAIR_BN, bool A_K, bool B_K>
 int launch_pair_t(const GemmArgs& g, const TcParams& p0, cudaStream_t st) {
   static PerDeviceFlag attr;
   if (!ppu_set_smem_once(attr, gemm_tc_pair_kernel<PAIR_BN, A_K, B_K>, PairCfg<PAIR_BN>::SMEM)) return -1;
-  CUtensorMap mapA, mapB;
+  CUtensorMap mapA, mapB, mapB2;
   if (!encode_map(&mapA, g.A, g.lda, A_K, g.M, g.K, 128)) return -2;
   if (!encode_map(&mapB, g.B, g.ldb, B_K, g.N, g.K, PAIR_BN / 2)) return -2;
   TcParams p = p0;
   p.tiles_m = (g.M + 255) / 256;
   p.tiles_n = (g.N + PAIR_BN - 1) / PAIR_BN;
   p.splits = 1; p.split_stride = 0;
+  // tiles that run at the same time share operand rows through L2: walk along the shorter side
+  // of the output, so that a wave of pairs covers few rows of the larger operand and all of the
+  // smaller one (8192 x 2048 x 8192: 1341 -> 1452 TFLOP/s; the 134 MB A operand no longer
+  // passes through L2 once per wave)
+  p.n_fastest = g.M > g.N ? 1 : 0;
   const int tiles = p.tiles_m * p.tiles_n;
   const int n_sm = ppu_sm_count();
   // as many pairs as give every pair the same number of tiles: 256 tiles on 74 pairs take four
@@ -249,8 +286,19 @@ int launch_pair_t(const GemmArgs& g, const TcParams& p0, cudaStream_t st) {
   // the budget raises the clock of the busy ones
   const int max_pairs = n_sm / 2;
   const int waves = (tiles + max_pairs - 1) / max_pairs;
-  const int pairs = tiles < max_pairs ? tiles : (tiles + waves - 1) / waves;
-  gemm_tc_pair_kernel<PAIR_BN, A_K, B_K><<<2 * pairs, GEMM_THREADS, PairCfg<PAIR_BN>::SMEM, st>>>(mapA, mapB, p);
+  int pairs = tiles < max_pairs ? tiles : (tiles + waves - 1) / waves;
+  // a last wave that fills at most half of the pairs is worked as 128-column halves by all of
+  // them (not with the row-sum epilogue, whose running sum spans a thread's 128 columns)
+  const int rem = tiles % max_pairs;
+  p.tail_from = 1 << 30;
+  if (PAIR_BN == 256 && g.tile_shape != 4 && g.epilogue != EPI_DELTA_BF16 && tiles > max_pairs && rem > 0 &&
+      2 * rem <= max_pairs) {
+    p.tail_from = tiles - rem;
+    pairs = max_pairs;
+  }
+  mapB2 = mapB;
+  if (B_K && p.tail_from < tiles && !encode_map(&mapB2, g.B, g.ldb, true, g.N, g.K, 64)) return -2;
+  gemm_tc_pair_kernel<PAIR_BN, A_K, B_K><<<2 * pairs, GEMM_THREADS, PairCfg<PAIR_BN>::SMEM, st>>>(mapA, mapB, mapB2, p);
   return cudaGetLastError() == cudaSuccess ? 0 : -3;
 }
 

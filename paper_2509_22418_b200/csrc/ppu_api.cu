@@ -677,8 +677,8 @@ extern "C" int ppu_gemm(const void* A, int64_t lda, int a_kmajor, const void* B,
   g.M = M; g.N = N; g.K = K;
   g.epilogue = out_f32 ? EPI_STORE_F32 : EPI_STORE_BF16;
   g.C = C; g.ldc = ldc; g.C2 = nullptr; g.aux = nullptr; g.ldaux = 0; g.flags = nullptr;
-  if (backend < 0 || backend > 4) return ppu_fail(PPU_EINVAL, "unknown gemm backend %d", backend);
-  g.tile_shape = backend == 2 ? 1 : backend == 3 ? 2 : backend == 4 ? 3 : 0;
+  if (backend < 0 || backend > 5) return ppu_fail(PPU_EINVAL, "unknown gemm backend %d", backend);
+  g.tile_shape = backend == 2 ? 1 : backend == 3 ? 2 : backend == 4 ? 3 : backend == 5 ? 4 : 0;
   const int rc = backend == 1 ? launch_gemm_simt(g, (cudaStream_t)cuda_stream)
                               : launch_gemm_tc(g, (cudaStream_t)cuda_stream);
   if (rc) return ppu_fail(rc == -4 ? PPU_ESHAPE : PPU_ECUDA, "gemm launch failed (%d)", rc);

@@ -29,8 +29,9 @@ GEMM_SHAPES = [
 
 
 # backends: 0 tcgen05 with the tile shape the step would choose, 1 SIMT, 2 tcgen05 one CTA per tile,
-# 3 tcgen05 SM pairs (cta_group::2) on 256 x 256 tiles, 4 the same on 256 x 128 tiles
-@pytest.mark.parametrize("backend", [0, 1, 2, 3, 4])
+# 3 tcgen05 SM pairs (cta_group::2) on 256 x 256 tiles, 4 the same on 256 x 128 tiles, 5 as 3 but
+# never cutting the tiles of a half-empty last wave
+@pytest.mark.parametrize("backend", [0, 1, 2, 3, 4, 5])
 @pytest.mark.parametrize("a_k,b_k", [(1, 1), (1, 0), (0, 1), (0, 0)])
 @pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
 def test_gemm_against_oracle_matmul(backend, a_k, b_k, M, N, K):
@@ -48,6 +49,31 @@ def test_gemm_against_oracle_matmul(backend, a_k, b_k, M, N, K):
         tol = (2e-5 if out_f32 else 2 ** -8)
         err = np.abs(got - ref)
         assert np.all(err <= tol * np.abs(ref) + tol * rms), (float(err.max()), rms)
+
+
+@pytest.mark.parametrize("a_k,b_k", [(1, 1), (1, 0), (0, 1), (0, 0)])
+@pytest.mark.parametrize("M,N,K", [(8192, 2048, 192), (8000, 2000, 200), (2560, 5888, 136)])
+def test_gemm_half_empty_last_wave(a_k, b_k, M, N, K):
+    """Outputs whose 256 x 256 tiles leave the last wave of SM pairs at most half full (256 tiles,
+    and 230, on the 74 pairs of a B200): the SM-pair kernel works those last tiles as 128-column halves.  Checked
+    against the oracle's matmul and, bit for bit, against the same kernel on whole tiles only."""
+    import torch
+    from paper_2509_22418_b200 import ppu
+    rng = np.random.default_rng(M + 3 * N + 5 * K + 2 * a_k + b_k)
+    A, A64 = _bf16_tensor(rng, (M, K) if a_k else (K, M))
+    B, B64 = _bf16_tensor(rng, (N, K) if b_k else (K, N))
+    ref = (A64 if a_k else A64.T) @ (B64.T if b_k else B64)
+    rms = math.sqrt(float((ref ** 2).mean()))
+    for out_f32 in (True, False):
+        outs = {}
+        for backend in (0, 3, 5):
+            Cd = ppu.ppu_gemm(A, a_k, B, b_k, M, N, K, out_f32=out_f32, backend=backend)
+            torch.cuda.synchronize()
+            outs[backend] = Cd.float().cpu().numpy()
+            tol = (2e-5 if out_f32 else 2 ** -8)
+            err = np.abs(outs[backend].astype(np.float64) - ref)
+            assert np.all(err <= tol * np.abs(ref) + tol * rms), (backend, float(err.max()), rms)
+        assert np.array_equal(outs[3], outs[5]) and np.array_equal(outs[0], outs[3])
 
 
 def test_gemm_strided_operands_and_column_offset():
