@@ -304,70 +304,94 @@ __global__ void rope_kernel(bf16* __restrict__ qkv, const float2* __restrict__ c
   *p = pack8(f);
 }
 
-// ---- fused cross-entropy: one block per token row, row held in registers ----
-// Reads the logits once; writes dlogits = (softmax - onehot) / count in place.
+// ---- fused cross-entropy: a persistent block per SM walks token rows, row held in registers ----
+// Reads the logits once; writes dlogits = (softmax - onehot) / count in place.  The next row's
+// loads are issued before the current row's reductions and exponentials, so that they (and the
+// current row's stores) overlap the arithmetic instead of following it.
 constexpr int XE_THREADS = 1024;
 template <int NCH>
-__global__ void __launch_bounds__(XE_THREADS)
+__global__ void __launch_bounds__(XE_THREADS, 1)
 xent_kernel(bf16* __restrict__ logits, const int32_t* __restrict__ tok,
-            float* __restrict__ row_loss, int S, int V, float inv_count, int write_grad) {
+            float* __restrict__ row_loss, int T, int S, int V, float inv_count, int write_grad) {
   __shared__ float red[XE_THREADS / 32];
-  const int64_t t = blockIdx.x;
-  const int s = (int)(t % S);
-  uint4* rowp = reinterpret_cast<uint4*>(logits + t * V);
   const int nvec = V / 8;
-  if (s == S - 1) {  // no next token: no loss, zero gradient
-    if (write_grad)
-      for (int i = threadIdx.x; i < nvec; i += XE_THREADS) rowp[i] = make_uint4(0, 0, 0, 0);
-    if (threadIdx.x == 0) row_loss[t] = 0.f;
-    return;
-  }
-  int target = tok[t + 1];
-  target = target < 0 ? 0 : (target >= V ? V - 1 : target);
-  float v[NCH][8];
-  float mx = -INFINITY;
+  uint4 nxt[NCH];
+  auto load_row = [&](int64_t row) {
+    const uint4* rp = reinterpret_cast<const uint4*>(logits + row * V);
 #pragma unroll
-  for (int c = 0; c < NCH; ++c) {
-    const int i = threadIdx.x + c * XE_THREADS;
-    if (i < nvec) {
-      unpack8(rowp[i], v[c]);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) mx = fmaxf(mx, v[c][j]);
+    for (int c = 0; c < NCH; ++c) {
+      const int i = threadIdx.x + c * XE_THREADS;
+      if (i < nvec) nxt[c] = rp[i];
     }
-  }
-  mx = block_max<XE_THREADS / 32>(mx, red);
-  float sum = 0.f;
+  };
+  int64_t t = blockIdx.x;
+  if (t < T) load_row(t);
+  for (; t < T; t += gridDim.x) {
+    const int s = (int)(t % S);
+    uint4* rowp = reinterpret_cast<uint4*>(logits + t * V);
+    float v[NCH][8];
+    float mx = -INFINITY;
 #pragma unroll
-  for (int c = 0; c < NCH; ++c) {
-    const int i = threadIdx.x + c * XE_THREADS;
-    if (i < nvec) {
+    for (int c = 0; c < NCH; ++c) {
+      const int i = threadIdx.x + c * XE_THREADS;
+      if (i < nvec) {
+        unpack8(nxt[c], v[c]);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        v[c][j] = __expf(v[c][j] - mx);
-        sum += v[c][j];
+        for (int j = 0; j < 8; ++j) mx = fmaxf(mx, v[c][j]);
       }
     }
-  }
-  sum = block_sum<XE_THREADS / 32>(sum, red);
-  const float inv = 1.f / sum;
-  if (threadIdx.x == 0) {
-    const float zt = __bfloat162float(logits[t * V + target]);
-    row_loss[t] = logf(sum) + mx - zt;
-  }
-  if (!write_grad) return;
-  __syncthreads();  // the target logit is read before anyone overwrites the row
+    if (t + gridDim.x < T) load_row(t + gridDim.x);
+    if (s == S - 1) {  // no next token: no loss, zero gradient (block-uniform)
+      if (write_grad)
+        for (int i = threadIdx.x; i < nvec; i += XE_THREADS) rowp[i] = make_uint4(0, 0, 0, 0);
+      if (threadIdx.x == 0) row_loss[t] = 0.f;
+      continue;
+    }
+    int target = tok[t + 1];
+    target = target < 0 ? 0 : (target >= V ? V - 1 : target);
+    // the thread that holds the target logit takes it from its registers
+    const int oc = (target >> 3) / XE_THREADS, oj = target & 7;
+    const bool owner = (target >> 3) % XE_THREADS == (int)threadIdx.x;
+    float zt = 0.f;
+    if (owner) {
 #pragma unroll
-  for (int c = 0; c < NCH; ++c) {
-    const int i = threadIdx.x + c * XE_THREADS;
-    if (i < nvec) {
-      float f[8];
+      for (int c = 0; c < NCH; ++c)
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        float p = v[c][j] * inv;
-        if (8 * i + j == target) p -= 1.f;
-        f[j] = p * inv_count;
+        for (int j = 0; j < 8; ++j)
+          if (c == oc && j == oj) zt = v[c][j];
+    }
+    mx = block_max<XE_THREADS / 32>(mx, red);
+    float sum = 0.f;
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      const int i = threadIdx.x + c * XE_THREADS;
+      if (i < nvec) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          v[c][j] = __expf(v[c][j] - mx);
+          sum += v[c][j];
+        }
       }
-      rowp[i] = pack8(f);
+    }
+    sum = block_sum<XE_THREADS / 32>(sum, red);
+    const float inv = 1.f / sum;
+    if (owner) row_loss[t] = logf(sum) + mx - zt;
+    if (!write_grad) continue;
+    const float scale = inv * inv_count;
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      const int i = threadIdx.x + c * XE_THREADS;
+      if (i < nvec) {
+        float f[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) f[j] = v[c][j] * scale;
+        if (owner && c == oc) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (j == oj) f[j] = (v[c][j] * inv - 1.f) * inv_count;
+        }
+        rowp[i] = pack8(f);
+      }
     }
   }
 }
@@ -562,14 +586,15 @@ void launch_xent(bf16* logits, const int32_t* tok, float* row_loss, int B, int S
   const int T = B * S;
   const float inv_count = 1.f / (float)((int64_t)B * (S - 1));
   const int nch = (V / 8 + XE_THREADS - 1) / XE_THREADS;
+  const int grid = T < ppu_sm_count() ? T : ppu_sm_count();
   if (nch <= 1)
-    xent_kernel<1><<<T, XE_THREADS, 0, st>>>(logits, tok, row_loss, S, V, inv_count, write_grad);
+    xent_kernel<1><<<grid, XE_THREADS, 0, st>>>(logits, tok, row_loss, T, S, V, inv_count, write_grad);
   else if (nch <= 2)
-    xent_kernel<2><<<T, XE_THREADS, 0, st>>>(logits, tok, row_loss, S, V, inv_count, write_grad);
+    xent_kernel<2><<<grid, XE_THREADS, 0, st>>>(logits, tok, row_loss, T, S, V, inv_count, write_grad);
   else if (nch <= 4)
-    xent_kernel<4><<<T, XE_THREADS, 0, st>>>(logits, tok, row_loss, S, V, inv_count, write_grad);
+    xent_kernel<4><<<grid, XE_THREADS, 0, st>>>(logits, tok, row_loss, T, S, V, inv_count, write_grad);
   else
-    xent_kernel<8><<<T, XE_THREADS, 0, st>>>(logits, tok, row_loss, S, V, inv_count, write_grad);
+    xent_kernel<8><<<grid, XE_THREADS, 0, st>>>(logits, tok, row_loss, T, S, V, inv_count, write_grad);
 }
 
 void launch_loss_reduce(const float* row_loss, int T, float inv_count, float* out, cudaStream_t st) {
