@@ -112,7 +112,8 @@ void launch_cast_bf16(const float* src, bf16* dst, int64_t n, cudaStream_t st);
 void launch_embed_grad(const int32_t* tok, const float* g, float* dE, int T, int d, int V,
                        cudaStream_t st);
 // dgamma[c] = sum_t dy[t,c] * xhat[t,c], dbeta[c] = sum_t dy[t,c], in two stages with a fixed
-// order; partial: fp32 scratch [2 * ceil(T / 32) * d]
+// order; partial: fp32 scratch [2 * ln_param_partial_blocks(T) * d]
+int ln_param_partial_blocks(int T);
 void launch_ln_param_grad(const bf16* dy, const float* x, const float2* stats, float* dgamma,
                           float* dbeta, float* partial, int T, int d, cudaStream_t st);
 
@@ -139,8 +140,8 @@ void launch_adamw(const SliceSeg* segs, int n_seg, float* master, float* m, floa
                   int64_t n_total, AdamHyper hp, cudaStream_t st);
 // AdamW over the packed dense runs; the gradient of packed element j is grad[j - grad_shift]
 void launch_adamw_dense(const DenseSeg* segs, int n_seg, float* master, float* m, float* v,
-                        const float* grad, int64_t grad_shift, bf16* w16, int64_t n_total,
-                        AdamHyper hp, cudaStream_t st);
+                        const float* grad, int64_t grad_shift, bf16* w16, int64_t packed_base,
+                        int64_t n_total, AdamHyper hp, cudaStream_t st);
 // packed fp32 <-> canonical vectors
 void launch_slices_gather(const SliceSeg* segs, int n_seg, const float* theta, float* packed,
                           int d, int F, int64_t n_total, cudaStream_t st);
@@ -148,9 +149,10 @@ void launch_slices_gather(const SliceSeg* segs, int n_seg, const float* theta, f
 void launch_slices_to_w16(const SliceSeg* segs, int n_seg, const float* packed, const float* theta,
                           bf16* w16, int from_packed, int d, int F, int64_t n_total,
                           cudaStream_t st);
-// the same two moves for the dense runs: mode 0 packed = theta, 1 w16 = bf16(packed), 2 w16 = bf16(theta)
+// the same two moves for the dense runs, which fill packed positions [packed_base, packed_base +
+// n_total): mode 0 packed = theta, 1 w16 = bf16(packed), 2 w16 = bf16(theta)
 void launch_dense_move(const DenseSeg* segs, int n_seg, float* packed, const float* theta, bf16* w16,
-                       int mode, int64_t n_total, cudaStream_t st);
+                       int mode, int64_t packed_base, int64_t n_total, cudaStream_t st);
 
 // Outer sync tables.  The canonical vector is cut into runs ("segments") that are uniform in
 // how their owners are found:

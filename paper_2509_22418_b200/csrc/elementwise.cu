@@ -465,10 +465,11 @@ embed_grad_kernel(const int32_t* __restrict__ tok, const float* __restrict__ g, 
   }
 }
 
+constexpr int LNP_ROWS = 16;
 // ---- LayerNorm gain / shift gradients: column sums over the tokens, two stages -------------
-// stage 1: block b sums rows [32 b, 32 b + 32) for every column -> partial[b][0][c] (dy * xhat),
-// partial[b][1][c] (dy); stage 2: one thread per column adds the partials in order of b.
-constexpr int LNP_ROWS = 32;
+// stage 1: block b sums rows [16 b, 16 b + 16) for every column -> partial[b][0][c] (dy * xhat),
+// partial[b][1][c] (dy); stage 2: a block takes 32 columns, each of its 32 warps adds a 32nd of
+// the partials in order of b, and the 32 sums are added in order - a fixed order throughout.
 __global__ void __launch_bounds__(256)
 ln_param_partial_kernel(const bf16* __restrict__ dy, const float* __restrict__ x,
                         const float2* __restrict__ stats, float* __restrict__ partial, int T, int d) {
@@ -478,6 +479,7 @@ ln_param_partial_kernel(const bf16* __restrict__ dy, const float* __restrict__ x
   float* pb = pg + d;
   for (int c = 8 * threadIdx.x; c < d; c += 8 * 256) {
     float sg[8] = {}, sb[8] = {};
+#pragma unroll 4
     for (int t = r0; t < r1; ++t) {
       const float2 st = stats[t];
       float f[8];
@@ -497,18 +499,31 @@ ln_param_partial_kernel(const bf16* __restrict__ dy, const float* __restrict__ x
     *reinterpret_cast<float4*>(pb + c + 4) = make_float4(sb[4], sb[5], sb[6], sb[7]);
   }
 }
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(1024)
 ln_param_final_kernel(const float* __restrict__ partial, float* __restrict__ dgamma,
                       float* __restrict__ dbeta, int n_blocks, int d) {
-  const int c = blockIdx.x * 128 + threadIdx.x;
-  if (c >= d) return;
+  __shared__ float sh[2][32][32];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int c = blockIdx.x * 32 + lane;
+  const int per = (n_blocks + 31) / 32;
+  const int b0 = w * per, b1 = b0 + per < n_blocks ? b0 + per : n_blocks;
   float sg = 0.f, sb = 0.f;
-  for (int b = 0; b < n_blocks; ++b) {
-    sg += partial[(int64_t)b * 2 * d + c];
-    sb += partial[(int64_t)b * 2 * d + d + c];
+  if (c < d) {
+#pragma unroll 8
+    for (int b = b0; b < b1; ++b) {
+      sg += partial[(int64_t)b * 2 * d + c];
+      sb += partial[(int64_t)b * 2 * d + d + c];
+    }
   }
-  dgamma[c] = sg;
-  dbeta[c] = sb;
+  sh[0][w][lane] = sg; sh[1][w][lane] = sb;
+  __syncthreads();
+  if (w == 0 && c < d) {
+    float tg = 0.f, tb = 0.f;
+#pragma unroll
+    for (int q = 0; q < 32; ++q) { tg += sh[0][q][lane]; tb += sh[1][q][lane]; }
+    dgamma[c] = tg;
+    dbeta[c] = tb;
+  }
 }
 
 }  // namespace
@@ -535,11 +550,13 @@ void launch_embed_grad(const int32_t* tok, const float* g, float* dE, int T, int
   embed_grad_kernel<<<(unsigned)((T + 7) / 8), 256, 0, st>>>(tok, g, dE, T, d, V);
 }
 
+int ln_param_partial_blocks(int T) { return (T + LNP_ROWS - 1) / LNP_ROWS; }
+
 void launch_ln_param_grad(const bf16* dy, const float* x, const float2* stats, float* dgamma,
                           float* dbeta, float* partial, int T, int d, cudaStream_t st) {
-  const int nb = (T + LNP_ROWS - 1) / LNP_ROWS;
+  const int nb = ln_param_partial_blocks(T);
   ln_param_partial_kernel<<<nb, 256, 0, st>>>(dy, x, stats, partial, T, d);
-  ln_param_final_kernel<<<(d + 127) / 128, 128, 0, st>>>(partial, dgamma, dbeta, nb, d);
+  ln_param_final_kernel<<<(d + 31) / 32, 1024, 0, st>>>(partial, dgamma, dbeta, nb, d);
 }
 
 void launch_embed(const int32_t* tok, const bf16* E16, float* x, int T, int d, int V, int* flags,

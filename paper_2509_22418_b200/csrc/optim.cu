@@ -67,25 +67,46 @@ adamw_kernel(const SliceSeg* __restrict__ segs, float* __restrict__ master, floa
   }
 }
 
+// The dense runs of a replica are contiguous in its packed arrays (positions [base, base + n)) but
+// of very different lengths (a LayerNorm vector, the embedding), so the kernels that walk them
+// cut the packed range into equal chunks instead of giving every run the same number of blocks:
+// a block finds the run its chunk starts in by bisection and steps to the next run where a
+// float4 lies past the current one's end.  f(run, offset inside the run, packed position).
+constexpr int64_t DENSE_CHUNK = 16384;
+template <class F>
+__device__ __forceinline__ void dense_walk(const DenseSeg* __restrict__ segs, int n_seg, int64_t base,
+                                           int64_t n, F f) {
+  for (int64_t p0 = base + blockIdx.x * DENSE_CHUNK; p0 < base + n; p0 += (int64_t)gridDim.x * DENSE_CHUNK) {
+    const int64_t p1 = p0 + DENSE_CHUNK < base + n ? p0 + DENSE_CHUNK : base + n;
+    int lo = 0, hi = n_seg - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (segs[mid].packed_off <= p0) lo = mid; else hi = mid - 1;
+    }
+    int si = lo;
+    DenseSeg s = segs[si];
+    for (int64_t p = p0 + 4 * threadIdx.x; p < p1; p += 4 * blockDim.x) {
+      while (p >= s.packed_off + s.len) s = segs[++si];
+      f(s, p - s.packed_off, p);
+    }
+  }
+}
+
 __global__ void __launch_bounds__(256)
-adamw_dense_kernel(const DenseSeg* __restrict__ segs, float* __restrict__ master,
-                   float* __restrict__ m, float* __restrict__ v, const float* __restrict__ grad,
-                   int64_t grad_shift, bf16* __restrict__ w16, AdamHyper hp) {
-  const DenseSeg s = segs[blockIdx.y];
-  const float wd = s.decay ? hp.wd : 0.f;
-  for (int64_t j = 4 * (blockIdx.x * (int64_t)blockDim.x + threadIdx.x); j < s.len;
-       j += 4 * (int64_t)gridDim.x * blockDim.x) {
-    const int64_t pj = s.packed_off + j;
+adamw_dense_kernel(const DenseSeg* __restrict__ segs, int n_seg, int64_t base, int64_t n,
+                   float* __restrict__ master, float* __restrict__ m, float* __restrict__ v,
+                   const float* __restrict__ grad, int64_t grad_shift, bf16* __restrict__ w16, AdamHyper hp) {
+  dense_walk(segs, n_seg, base, n, [&](const DenseSeg& s, int64_t j, int64_t pj) {
     const float4 g = *reinterpret_cast<const float4*>(grad + (pj - grad_shift));
     float4 p = *reinterpret_cast<float4*>(master + pj);
     float4 mm = *reinterpret_cast<float4*>(m + pj);
     float4 vv = *reinterpret_cast<float4*>(v + pj);
-    adamw4(p, mm, vv, g, hp, wd);
+    adamw4(p, mm, vv, g, hp, s.decay ? hp.wd : 0.f);
     *reinterpret_cast<float4*>(master + pj) = p;
     *reinterpret_cast<float4*>(m + pj) = mm;
     *reinterpret_cast<float4*>(v + pj) = vv;
     store_bf16x4(w16 + s.canon_off + j, p);
-  }
+  });
 }
 
 // mode 0: packed = theta[subset]; 1: w16[subset] = bf16(packed); 2: w16[subset] = bf16(theta);
@@ -112,22 +133,20 @@ slice_move_kernel(const SliceSeg* __restrict__ segs, float* packed, float* dense
 }
 
 __global__ void __launch_bounds__(256)
-dense_move_kernel(const DenseSeg* __restrict__ segs, float* packed, const float* theta, bf16* w16,
-                  int mode) {
-  const DenseSeg s = segs[blockIdx.y];
-  for (int64_t j = 4 * (blockIdx.x * (int64_t)blockDim.x + threadIdx.x); j < s.len;
-       j += 4 * (int64_t)gridDim.x * blockDim.x) {
-    const int64_t ci = s.canon_off + j, pj = s.packed_off + j;
+dense_move_kernel(const DenseSeg* __restrict__ segs, int n_seg, int64_t base, int64_t n, float* packed,
+                  const float* theta, bf16* w16, int mode) {
+  dense_walk(segs, n_seg, base, n, [&](const DenseSeg& s, int64_t j, int64_t pj) {
+    const int64_t ci = s.canon_off + j;
     if (mode == 0) *reinterpret_cast<float4*>(packed + pj) = *reinterpret_cast<const float4*>(theta + ci);
     else if (mode == 1) store_bf16x4(w16 + ci, *reinterpret_cast<const float4*>(packed + pj));
     else store_bf16x4(w16 + ci, *reinterpret_cast<const float4*>(theta + ci));
-  }
+  });
 }
 
 // ---------------------------------------------------------------------------------------------
 // Outer sweep (Algorithm 1, the outer step): Delta = sum over owners (theta_k - theta) / m, 0 where
 // m = 0; g = -Delta; buf = mu buf + g; theta -= lr (g + mu buf); the bf16 copy is refreshed and
-// every owner restarts from the new value (line 6).
+// every owner restarts from the new value.
 //
 // A persistent grid walks a list of chunks (OUTER_CHUNK elements of one segment each), so the
 // decoding of "which tensor, which owners" is uniform per block and chunk, and segments of any
@@ -272,12 +291,17 @@ void launch_adamw(const SliceSeg* segs, int n_seg, float* master, float* m, floa
                                                          grad_stride, w16, d, F, hp);
 }
 
+static unsigned dense_grid(int64_t n) {
+  const int64_t chunks = (n + DENSE_CHUNK - 1) / DENSE_CHUNK, cap = (int64_t)ppu_sm_count() * 8;
+  return (unsigned)(chunks < cap ? chunks : cap);
+}
+
 void launch_adamw_dense(const DenseSeg* segs, int n_seg, float* master, float* m, float* v,
-                        const float* grad, int64_t grad_shift, bf16* w16, int64_t n_total,
-                        AdamHyper hp, cudaStream_t st) {
-  if (n_seg == 0) return;
-  adamw_dense_kernel<<<seg_grid(n_total, n_seg), 256, 0, st>>>(segs, master, m, v, grad, grad_shift,
-                                                               w16, hp);
+                        const float* grad, int64_t grad_shift, bf16* w16, int64_t packed_base,
+                        int64_t n_total, AdamHyper hp, cudaStream_t st) {
+  if (n_seg == 0 || n_total <= 0) return;
+  adamw_dense_kernel<<<dense_grid(n_total), 256, 0, st>>>(segs, n_seg, packed_base, n_total, master, m, v,
+                                                          grad, grad_shift, w16, hp);
 }
 
 static void slice_move(const SliceSeg* segs, int n_seg, float* packed, float* dense, bf16* w16,
@@ -298,9 +322,10 @@ void launch_slices_to_w16(const SliceSeg* segs, int n_seg, const float* packed, 
 }
 
 void launch_dense_move(const DenseSeg* segs, int n_seg, float* packed, const float* theta, bf16* w16,
-                       int mode, int64_t n_total, cudaStream_t st) {
-  if (n_seg == 0) return;
-  dense_move_kernel<<<seg_grid(n_total, n_seg), 256, 0, st>>>(segs, packed, theta, w16, mode);
+                       int mode, int64_t packed_base, int64_t n_total, cudaStream_t st) {
+  if (n_seg == 0 || n_total <= 0) return;
+  dense_move_kernel<<<dense_grid(n_total), 256, 0, st>>>(segs, n_seg, packed_base, n_total, packed, theta,
+                                                         w16, mode);
 }
 
 void launch_outer(const OuterTables& t, int kind, float* theta, float* buf, bf16* w16, float lr, float mu,

@@ -298,7 +298,7 @@ static size_t carve(ppu_ctx* c, uint8_t* base) {
   c->dqkv = (bf16*)take(T * 3 * d * 2);
   c->attn_scratch = (float*)take(T * h * 4);
   c->row_loss = (float*)take(T * 4);
-  c->ln_partial = c->any_rest ? (float*)take((size_t)2 * ((T + 31) / 32) * d * 4) : nullptr;
+  c->ln_partial = c->any_rest ? (float*)take((size_t)2 * ln_param_partial_blocks(T) * d * 4) : nullptr;
   c->act_bytes = off - c->state_bytes;
   return off;
 }
@@ -320,7 +320,7 @@ static void ppu_restart_replicas(ppu_ctx* c) {
   for (auto& r : c->reps) {
     launch_slices_gather(r.d_segs, (int)r.segs.size(), c->theta, r.master, c->cfg.d_model,
                          c->cfg.d_ff, r.n_ffn, c->stream);
-    launch_dense_move(r.d_dense, (int)r.dense.size(), r.master, c->theta, nullptr, 0, r.n_dense,
+    launch_dense_move(r.d_dense, (int)r.dense.size(), r.master, c->theta, nullptr, 0, r.n_ffn, r.n_dense,
                       c->stream);
   }
 }

@@ -34,7 +34,7 @@ int ppu_make_resident(ppu_ctx* c, int k) {
     EvScope ev(c, PPU_CLS_OTHER, 6.0 * (double)r.n_sub);
     launch_slices_to_w16(r.d_segs, (int)r.segs.size(), nullptr, c->theta, c->w16, 0, d, F, r.n_ffn,
                          c->stream);
-    launch_dense_move(r.d_dense, (int)r.dense.size(), nullptr, c->theta, c->w16, 2, r.n_dense, c->stream);
+    launch_dense_move(r.d_dense, (int)r.dense.size(), nullptr, c->theta, c->w16, 2, r.n_ffn, r.n_dense, c->stream);
     c->launches += (r.segs.empty() ? 0 : 1) + (r.dense.empty() ? 0 : 1);
   }
   if (k >= 0) {
@@ -42,7 +42,7 @@ int ppu_make_resident(ppu_ctx* c, int k) {
     EvScope ev(c, PPU_CLS_OTHER, 6.0 * (double)r.n_sub);
     launch_slices_to_w16(r.d_segs, (int)r.segs.size(), r.master, nullptr, c->w16, 1, d, F, r.n_ffn,
                          c->stream);
-    launch_dense_move(r.d_dense, (int)r.dense.size(), r.master, nullptr, c->w16, 1, r.n_dense, c->stream);
+    launch_dense_move(r.d_dense, (int)r.dense.size(), r.master, nullptr, c->w16, 1, r.n_ffn, r.n_dense, c->stream);
     c->launches += (r.segs.empty() ? 0 : 1) + (r.dense.empty() ? 0 : 1);
   }
   c->resident = k;
@@ -329,7 +329,7 @@ extern "C" int ppu_local_step(ppu_ctx* c, int replica, const int32_t* tokens, in
     launch_adamw(r.d_segs, (int)r.segs.size(), r.master, r.m, r.v, c->grad, c->last_partials, c->max_ffn, c->w16,
                  c->cfg.d_model, c->cfg.d_ff, r.n_ffn, hp, c->stream);
     launch_adamw_dense(r.d_dense, (int)r.dense.size(), r.master, r.m, r.v, c->grad + c->max_ffn * c->wgrad_splits,
-                       r.n_ffn, c->w16, r.n_dense, hp, c->stream);
+                       r.n_ffn, c->w16, r.n_ffn, r.n_dense, hp, c->stream);
     c->launches += (r.segs.empty() ? 0 : 1) + (r.dense.empty() ? 0 : 1);
   }
   r.stepped = true;
