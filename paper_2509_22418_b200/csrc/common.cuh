@@ -156,15 +156,18 @@ void launch_dense_move(const DenseSeg* segs, int n_seg, float* packed, const flo
 
 // Outer sync tables.  The canonical vector is cut into runs ("segments") that are uniform in
 // how their owners are found:
-//   kind 0  a run outside the FFN matrices; every owner in [ob, oe) of `dense_owner` trains the
-//           whole run, its value of canonical position i is master[i + shift];
-//   kind 1  (part of) a layer's W_in, kind 2 (part of) its W_out: the owners of a hidden unit are
+//   kind 0  a run that is contiguous in its owners' packed arrays too - anything outside the FFN
+//           matrices, and the rows of a W_in between two slice boundaries; every owner in
+//           [ob, oe) of `dense_owner` trains the whole run, its value of canonical position i
+//           is master[i + shift];
+//   kind 2  a layer's W_out, of which a replica trains columns: the owners of a hidden unit are
 //           listed per group of 8 units in unit_begin / unit_owner (CSR over layer * F/8 + unit/8).
+// (There is no kind 1: W_in had a kind of its own until its rows were swept as dense runs.)
 // Work is dealt to blocks in chunks of OUTER_CHUNK elements of one segment.
 constexpr int OUTER_CHUNK = 1 << 16;
 struct OuterSeg {
   int64_t start, len;        // run of the canonical vector (multiples of 4)
-  int64_t base;              // kinds 1, 2: canonical offset of the whole matrix
+  int64_t base;              // kind 2: canonical offset of the whole matrix
   int32_t kind, layer;
   int32_t ob, oe;            // kind 0: owners
 };

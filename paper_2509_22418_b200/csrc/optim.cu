@@ -184,8 +184,12 @@ __device__ __forceinline__ void outer_chunk(const OuterTables& t, const OuterSeg
   float* th_p = theta + sg.start + off;
   float* bu_p = buf + sg.start + off;
   bf16* w_p = w16 + sg.start + off;
-  // element index of the chunk's first float inside its matrix (kinds 1, 2)
+  // element index of the chunk's first float inside its matrix (kind 2)
   const uint32_t rel0 = KIND ? (uint32_t)(sg.start + off - sg.base) : 0u;
+  // kind 0: the common owner counts are none and one; the single owner's record is read once
+  const int n_own = KIND == 0 ? sg.oe - sg.ob : 0;
+  DenseOwner own0{nullptr, 0};
+  if (KIND == 0 && n_own == 1) own0 = t.dense_owner[sg.ob];
   const int32_t* ub = KIND ? t.unit_begin + (int64_t)sg.layer * (t.F / 8) : nullptr;
   for (uint32_t e0 = threadIdx.x; e0 < n4; e0 += OUTER_U * OUTER_THREADS) {
     float4 th[OUTER_U], bu[OUTER_U];
@@ -206,31 +210,38 @@ __device__ __forceinline__ void outer_chunk(const OuterTables& t, const OuterSeg
       const float4 old = th[k];
       if (KIND == 0) {
         const int64_t ci = sg.start + off + 4 * (int64_t)e;
-        for (int o = sg.ob; o < sg.oe; ++o) {
-          const DenseOwner ow = t.dense_owner[o];
-          const float4 v = __ldcs(reinterpret_cast<const float4*>(ow.master + ci + ow.shift));
-          total.x += v.x - old.x; total.y += v.y - old.y; total.z += v.z - old.z; total.w += v.w - old.w;
-          ++count;
+        if (n_own == 1) {
+          const float4 v = __ldcs(reinterpret_cast<const float4*>(own0.master + ci + own0.shift));
+          total.x = v.x - old.x; total.y = v.y - old.y; total.z = v.z - old.z; total.w = v.w - old.w;
+          count = 1;
+        } else {
+          for (int o = sg.ob; o < sg.oe; ++o) {
+            const DenseOwner ow = t.dense_owner[o];
+            const float4 v = __ldcs(reinterpret_cast<const float4*>(ow.master + ci + ow.shift));
+            total.x += v.x - old.x; total.y += v.y - old.y; total.z += v.z - old.z; total.w += v.w - old.w;
+            ++count;
+          }
         }
         outer_update(th[k], bu[k], total, count, lr, mu);
         __stcs(reinterpret_cast<float4*>(th_p) + e, th[k]);
         __stcs(reinterpret_cast<float4*>(bu_p) + e, bu[k]);
         store_bf16x4(w_p + 4 * (int64_t)e, th[k]);
-        for (int o = sg.ob; o < sg.oe; ++o) {      // the owners restart from the new parameters
-          const DenseOwner ow = t.dense_owner[o];
-          *reinterpret_cast<float4*>(ow.master + ci + ow.shift) = th[k];
+        // the owners restart from the new parameters
+        if (n_own == 1) {
+          *reinterpret_cast<float4*>(own0.master + ci + own0.shift) = th[k];
+        } else {
+          for (int o = sg.ob; o < sg.oe; ++o) {
+            const DenseOwner ow = t.dense_owner[o];
+            *reinterpret_cast<float4*>(ow.master + ci + ow.shift) = th[k];
+          }
         }
       } else {
         const uint32_t rel = rel0 + 4u * e;
-        uint32_t unit, inner;
-        if (KIND == 1) { unit = fast_div(rel, t.div_d); inner = rel - unit * (uint32_t)t.d; }
-        else { inner = fast_div(rel, t.div_F); unit = rel - inner * (uint32_t)t.F; }
+        const uint32_t inner = fast_div(rel, t.div_F), unit = rel - inner * (uint32_t)t.F;
         const int ob = ub[unit >> 3], oe = ub[(unit >> 3) + 1];
         for (int o = ob; o < oe; ++o) {
           const OuterOwner ow = t.unit_owner[o];
-          const float* p = KIND == 1
-                               ? ow.master + ow.in_off + (int64_t)((int)unit - ow.lo) * t.d + inner
-                               : ow.master + ow.out_off + (int64_t)inner * (ow.hi - ow.lo) + ((int)unit - ow.lo);
+          const float* p = ow.master + ow.out_off + (int64_t)inner * (ow.hi - ow.lo) + ((int)unit - ow.lo);
           const float4 v = __ldcs(reinterpret_cast<const float4*>(p));
           total.x += v.x - old.x; total.y += v.y - old.y; total.z += v.z - old.z; total.w += v.w - old.w;
           ++count;
@@ -241,9 +252,7 @@ __device__ __forceinline__ void outer_chunk(const OuterTables& t, const OuterSeg
         store_bf16x4(w_p + 4 * (int64_t)e, th[k]);
         for (int o = ob; o < oe; ++o) {
           const OuterOwner ow = t.unit_owner[o];
-          float* p = KIND == 1
-                         ? ow.master + ow.in_off + (int64_t)((int)unit - ow.lo) * t.d + inner
-                         : ow.master + ow.out_off + (int64_t)inner * (ow.hi - ow.lo) + ((int)unit - ow.lo);
+          float* p = ow.master + ow.out_off + (int64_t)inner * (ow.hi - ow.lo) + ((int)unit - ow.lo);
           *reinterpret_cast<float4*>(p) = th[k];
         }
       }
@@ -336,6 +345,5 @@ void launch_outer(const OuterTables& t, int kind, float* theta, float* buf, bf16
   if (grid > n_chunks) grid = n_chunks;
   const OuterChunk* ch = t.chunks + chunk_lo;
   if (kind == 0) outer_kernel<0><<<grid, OUTER_THREADS, 0, st>>>(t, ch, theta, buf, w16, lr, mu, n_chunks);
-  else if (kind == 1) outer_kernel<1><<<grid, OUTER_THREADS, 0, st>>>(t, ch, theta, buf, w16, lr, mu, n_chunks);
-  else outer_kernel<2><<<grid, OUTER_THREADS, 0, st>>>(t, ch, theta, buf, w16, lr, mu, n_chunks);
+  else if (kind == 2) outer_kernel<2><<<grid, OUTER_THREADS, 0, st>>>(t, ch, theta, buf, w16, lr, mu, n_chunks);
 }

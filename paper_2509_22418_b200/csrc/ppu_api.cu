@@ -239,8 +239,9 @@ static size_t carve(ppu_ctx* c, uint8_t* base) {
   c->flags = (int*)take(sizeof(int) * PPU_FLAG_COUNT);
   c->rope_cs = (float2*)take(sizeof(float2) * c->cfg.max_seq * (d / h / 2));
   c->tok_stage = (int32_t*)take(sizeof(int32_t) * T);
-  // outer-sync tables: a layer's dense block splits at most at every head boundary of W_q/k/v
-  c->cap_oseg = 8 + (size_t)L * (16 + 6 * (size_t)(h + 1));
+  // outer-sync tables: a layer's dense block splits at most at every head boundary of W_q/k/v and
+  // at both ends of every replica's W_in rows
+  c->cap_oseg = 8 + (size_t)L * (16 + 6 * (size_t)(h + 1) + 2 * (size_t)c->K + 2);
   c->cap_ochunk = (size_t)(c->P / OUTER_CHUNK) + c->cap_oseg + 8;
   c->cap_downer = c->cap_oseg * (size_t)c->K + 1;
   c->cap_uowner = unit_entries + 1;

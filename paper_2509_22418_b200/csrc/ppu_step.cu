@@ -398,6 +398,12 @@ int build_outer_tables(ppu_ctx* c, const std::vector<int32_t>& list) {
   for (int k : list) {
     const ReplicaState& r = c->reps[k];
     for (const auto& s : r.dense) runs.push_back({s.canon_off, s.canon_off + s.len, r.master, s.packed_off - s.canon_off});
+    // a replica's rows [lo, hi) of a W_in are one contiguous run of the canonical vector and of
+    // its packed array alike, so W_in is swept like the runs outside the FFNs
+    for (const auto& s : r.segs) {
+      const int64_t lo = s.win_off + (int64_t)s.lo * d, hi = s.win_off + (int64_t)s.hi * d;
+      runs.push_back({lo, hi, r.master, s.packed_off - lo});
+    }
   }
   // cuts [lo, hi) of the canonical vector at every run boundary and lists each piece's owners;
   // neighbouring pieces with the same owners and shifts are joined
@@ -431,9 +437,8 @@ int build_outer_tables(ppu_ctx* c, const std::vector<int32_t>& list) {
   for (int l = 0; l < L; ++l) {
     layer_seg_begin[l] = (int)segs.size();
     const int64_t base = c->e_size + (int64_t)l * c->layer_size;
-    add_dense(base, base + c->rel_win, l);
+    add_dense(base, base + c->rel_wout, l);           // attention, LayerNorm and W_in
     OuterSeg sg; sg.layer = l; sg.ob = sg.oe = 0; sg.len = fd;
-    sg.start = sg.base = base + c->rel_win; sg.kind = 1; segs.push_back(sg);
     sg.start = sg.base = base + c->rel_wout; sg.kind = 2; segs.push_back(sg);
   }
   layer_seg_begin[L] = (int)segs.size();
