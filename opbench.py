@@ -36,6 +36,7 @@ def main():
     ap.add_argument("--layers", type=int, default=4)
     ap.add_argument("--replicas", type=int, default=4)
     ap.add_argument("--train-non-mlp", action="store_true")
+    ap.add_argument("--head-slices", type=int, default=0, help="path: MLP + head slicing with this many head groups")
     ap.add_argument("--iters", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     a = ap.parse_args()
@@ -60,7 +61,7 @@ def main():
         d, F, V = a.heads * a.dh, 4 * a.heads * a.dh, 32768
         K = a.replicas
         cfg = ppu.make_cfg(a.layers, d, a.heads, F, V, a.batch, a.seq, adam_lr=3e-4, adam_beta2=0.99)
-        spec, keep = ppu.make_spec(K, n_slices=K, train_non_mlp=int(a.train_non_mlp))
+        spec, keep = ppu.make_spec(K, n_slices=K, train_non_mlp=int(a.train_non_mlp), n_head_slices=a.head_slices)
         ctx = ppu.Context(cfg, spec, keep)
         ctx.ppu_set_params(synth.init_params(0, ctx.tensors()))
         toks = [torch.from_numpy(synth.tokens(0, k, 0, 0, a.batch, a.seq, V)).cuda() for k in range(K)]
