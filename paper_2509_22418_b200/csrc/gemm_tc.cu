@@ -301,7 +301,11 @@ namespace {
 // (2048 x 2048 x 8192, 64 tiles: 0.053 ms against 0.092; 512 x 2048 x 8192, 16 tiles: equal)
 bool picks_pair256(const GemmArgs& g) {
   const long long tiles_pair = (long long)((g.M + 255) / 256) * ((g.N + 255) / 256);
-  return g.tile_shape == 2 || g.tile_shape == 4 || (g.tile_shape == 0 && g.splits <= 1 && g.M > 128 && g.N > 128 && tiles_pair >= 16);
+  // (a split product needs as many 128-k blocks as slices, or the pair kernel would write fewer
+  // partial outputs than the caller adds up)
+  const bool split_ok = g.splits <= 1 || g.splits <= (g.K + 127) / 128;
+  return split_ok && (g.tile_shape == 2 || g.tile_shape == 4 ||
+                      (g.tile_shape == 0 && g.M > 128 && g.N > 128 && tiles_pair >= 16));
 }
 }  // namespace
 
@@ -329,7 +333,7 @@ int launch_gemm_tc(const GemmArgs& g, cudaStream_t st) {
   // 512 tiles instead of 256 on the 74 pairs of a B200 - but the narrower product measured 25 %
   // slower, so only a half-empty last wave is worked that way, inside the 256-wide kernel;
   // tile_shape 3 keeps the narrow kernel testable, 4 is the 256-wide kernel without narrow units.)
-  if (g.tile_shape >= 2 && g.splits > 1) return -4;
+  if (g.splits > 1 && (g.tile_shape == 3 || g.epilogue != EPI_STORE_F32)) return -4;
   if (g.tile_shape == 3) return launch_gemm_tc_pair(g, make_params(g), 128, st);
   if (picks_pair256(g)) return launch_gemm_tc_pair(g, make_params(g), 256, st);
   const long long tiles256 = (long long)((g.M + BM - 1) / BM) * ((g.N + 255) / 256) * (g.splits > 1 ? g.splits : 1);

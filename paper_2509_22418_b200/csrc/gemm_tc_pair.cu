@@ -87,12 +87,18 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 }
 
 // one unit of work of a pair: rows [m0, m0 + 256) x columns [n0, n0 + bn)
-struct PairUnit { int m0, n0, bn; };
+// (kb0, kb1: the unit's range of 128-k blocks; sp: its split-K slice)
+struct PairUnit { int m0, n0, bn, sp, kb0, kb1; };
 template <int PAIR_BN>
-__device__ __forceinline__ PairUnit pair_unit(const TcParams& p, int u) {
+__device__ __forceinline__ PairUnit pair_unit(const TcParams& p, int u, int num_tiles, int k_blocks) {
   PairUnit w;
   int tile = u, half = 0;
-  w.bn = PAIR_BN;
+  w.bn = PAIR_BN; w.sp = 0; w.kb0 = 0; w.kb1 = k_blocks;
+  if (p.splits > 1) {          // split-K products have whole tiles only
+    w.sp = u / num_tiles; tile = u - w.sp * num_tiles;
+    w.kb0 = (int)((long long)w.sp * k_blocks / p.splits);
+    w.kb1 = (int)((long long)(w.sp + 1) * k_blocks / p.splits);
+  }
   if (PAIR_BN == 256 && u >= p.tail_from) {
     const int v = u - p.tail_from;
     tile = p.tail_from + (v >> 1); half = v & 1; w.bn = 128;
@@ -150,8 +156,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
 
   const int n_pairs = gridDim.x >> 1, pair = blockIdx.x >> 1;
   const int num_tiles = p.tiles_m * p.tiles_n;
-  const int num_units = num_tiles + (PAIR_BN == 256 && num_tiles > p.tail_from ? num_tiles - p.tail_from : 0);
   const int k_blocks = (p.K + PAIR_KH * BK - 1) / (PAIR_KH * BK);
+  const int num_units = p.splits > 1 ? num_tiles * p.splits
+                                     : num_tiles + (PAIR_BN == 256 && num_tiles > p.tail_from ? num_tiles - p.tail_from : 0);
 
   if (warp == 0) {
     if (lane == 0) {
@@ -159,13 +166,13 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
       int s = 0; uint32_t ph = 0;
       bool ok = true;
       for (int u = pair; u < num_units && ok; u += n_pairs) {
-        const PairUnit w = pair_unit<PAIR_BN>(p, u);
+        const PairUnit w = pair_unit<PAIR_BN>(p, u, num_tiles, k_blocks);
         const int m0 = w.m0 + (int)rank * 128;
         const int n0 = w.n0 + (int)rank * (w.bn / 2);
         const bool narrow = w.bn != PAIR_BN;
         const int b_slab = narrow ? B_SLAB / 2 : B_SLAB;          // this CTA's bn/2 rows of B, 64 k
         const CUtensorMap* mB = narrow ? &mapB2 : &mapB;
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.flags);
           if (!ok) break;
           const uint32_t a_dst = smem_u32(smem + s * PAIR_STAGE_BYTES);
@@ -202,14 +209,14 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
       int s = 0; uint32_t ph = 0;
       int acc = 0; uint32_t acc_ph = 0;
       for (int u = pair; u < num_units; u += n_pairs) {
-        const PairUnit w = pair_unit<PAIR_BN>(p, u);
+        const PairUnit w = pair_unit<PAIR_BN>(p, u, num_tiles, k_blocks);
         const uint32_t idesc = idesc0 | ((uint32_t)(w.bn >> 3) << 17);
         const uint32_t b_slab = w.bn != PAIR_BN ? B_SLAB / 2 : B_SLAB;
         if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.flags)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * PAIR_BN);
         bool ok = true;
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           ok = mbar_wait(full_bar(s), ph, abort_flag, p.flags);
           if (!ok) break;
           tc_fence_after();
@@ -221,7 +228,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             const uint32_t slab = kh * SLAB_BYTES, slab_b = kh * b_slab;
             const uint64_t adesc = A_K ? make_desc(a_addr + slab + kk * 32, 16, 1024) : make_desc(a_addr + slab + kk * 2048, 8192, 1024);
             const uint64_t bdesc = B_K ? make_desc(b_addr + slab_b + kk * 32, 16, 1024) : make_desc(b_addr + slab_b + kk * 2048, 8192, 1024);
-            umma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            umma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb > w.kb0 || k > 0) ? 1u : 0u);
           }
           umma_commit_pair(empty_bar(s));        // both CTAs' slots are free once these MMAs have read them
           if (++s == ST) { s = 0; ph ^= 1u; }
@@ -237,11 +244,11 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     const int half = (warp - 2) >> 2;
     int acc = 0; uint32_t acc_ph = 0;
     for (int u = pair; u < num_units; u += n_pairs) {
-      const PairUnit w = pair_unit<PAIR_BN>(p, u);
+      const PairUnit w = pair_unit<PAIR_BN>(p, u, num_tiles, k_blocks);
       const int m0 = w.m0 + (int)rank * 128;
       if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.flags)) break;
       tc_fence_after();
-      drain_cols(p, m0, w.n0, 0, tmem_base + (uint32_t)(acc * PAIR_BN), quarter, half * (w.bn / 2),
+      drain_cols(p, m0, w.n0, w.sp, tmem_base + (uint32_t)(acc * PAIR_BN), quarter, half * (w.bn / 2),
                  (half + 1) * (w.bn / 2), lane);
       tc_fence_before();
       __syncwarp();
@@ -273,13 +280,17 @@ int launch_pair_t(const GemmArgs& g, const TcParams& p0, cudaStream_t st) {
   TcParams p = p0;
   p.tiles_m = (g.M + 255) / 256;
   p.tiles_n = (g.N + PAIR_BN - 1) / PAIR_BN;
-  p.splits = 1; p.split_stride = 0;
+  // split-K (fp32 partial outputs sp * split_stride apart, summed by the consumer): each unit of
+  // work is a whole tile over a slice of the 128-k blocks
+  const int k_blocks = (g.K + PAIR_KH * BK - 1) / (PAIR_KH * BK);
+  p.splits = g.splits < 1 ? 1 : (g.splits > k_blocks ? k_blocks : g.splits);
+  p.split_stride = g.split_stride;
   // tiles that run at the same time share operand rows through L2: walk along the shorter side
   // of the output, so that a wave of pairs covers few rows of the larger operand and all of the
   // smaller one (8192 x 2048 x 8192: 1341 -> 1452 TFLOP/s; the 134 MB A operand no longer
   // passes through L2 once per wave)
   p.n_fastest = g.M > g.N ? 1 : 0;
-  const int tiles = p.tiles_m * p.tiles_n;
+  const int tiles = p.tiles_m * p.tiles_n * p.splits;
   const int n_sm = ppu_sm_count();
   // as many pairs as give every pair the same number of tiles: 256 tiles on 74 pairs take four
   // waves whether 74 or 64 pairs work on them, and on a power-capped part the idle SMs' share of
@@ -291,7 +302,7 @@ int launch_pair_t(const GemmArgs& g, const TcParams& p0, cudaStream_t st) {
   // them (not with the row-sum epilogue, whose running sum spans a thread's 128 columns)
   const int rem = tiles % max_pairs;
   p.tail_from = 1 << 30;
-  if (PAIR_BN == 256 && g.tile_shape != 4 && g.epilogue != EPI_DELTA_BF16 && tiles > max_pairs && rem > 0 &&
+  if (PAIR_BN == 256 && p.splits == 1 && g.tile_shape != 4 && g.epilogue != EPI_DELTA_BF16 && tiles > max_pairs && rem > 0 &&
       2 * rem <= max_pairs) {
     p.tail_from = tiles - rem;
     pairs = max_pairs;

@@ -205,6 +205,19 @@ static void build_geometry(ppu_ctx* c) {
     }
   c->wgrad_splits = 1;
   while (min_tiles * c->wgrad_splits * 2 <= 148 && c->wgrad_splits < 8) c->wgrad_splits *= 2;
+  // Slices wide enough for the SM-pair kernel (16 tiles of 256 x 256 or more) are cut so that
+  // the 74 pairs are filled once: 32 tiles (a 1024-wide slice at d = 2048) run as two slices.
+  int64_t min_pair_tiles = 1 << 30;
+  for (auto& r2 : c->reps)
+    for (auto& s : r2.segs) {
+      const int64_t t = (int64_t)((s.hi - s.lo + 255) / 256) * ((d + 255) / 256);
+      if (t < min_pair_tiles) min_pair_tiles = t;
+    }
+  if (min_pair_tiles >= 16 && min_pair_tiles < (1 << 30)) {
+    c->wgrad_splits = (int)(74 / min_pair_tiles);
+    if (c->wgrad_splits < 1) c->wgrad_splits = 1;
+    if (c->wgrad_splits > 8) c->wgrad_splits = 8;
+  }
 }
 
 // Carves the arena.  With base == nullptr only the sizes are computed.
