@@ -46,7 +46,7 @@ OUTER = dict(lr=0.7, momentum=0.9)
 SEED = 1234
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant GEMM kernel (SM-pair
 # kernel, 128-k stages); set to None whenever that kernel changes after the capture
-GEMM_TRAFFIC_BYTES = 183.8e6
+GEMM_TRAFFIC_BYTES = 182.0e6
 
 
 def peaks():
